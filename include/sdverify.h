@@ -1,0 +1,190 @@
+/*
+ * sdverify — batched verification of a draft token tree on one B200.
+ *
+ * Hyper-Bagel (arXiv 2509.18824) accelerates next-token prediction by
+ * speculative decoding: a light draft model proposes several tokens and the
+ * target model validates all of them in one parallel pass (Sec. 1), which
+ * trades the memory-access bottleneck of autoregressive decoding for a
+ * computational one; the target's outputs are unchanged (Sec. 4.1).  This
+ * library is that validation pass, split into its four data-parallel parts:
+ *
+ *   sd_verify_attention  attention of every tree node over the cached prefix
+ *                        KV and over its own ancestors' KV (per layer)
+ *   sd_lmhead_argmax     target's greedy token at every tree node
+ *   sd_accept_tree       longest root path whose drafts the target confirms
+ *   sd_compact_kv        accepted nodes' KV appended to the cache (all layers)
+ *
+ * Conventions common to every call
+ *   - "dev" pointers are device memory on the current CUDA device, "host"
+ *     pointers are ordinary host memory.  The caller owns every buffer; the
+ *     library allocates nothing and frees nothing.
+ *   - bf16 tensors are passed as void* / uint16 bit patterns.
+ *   - Calls enqueue work on `stream` (a cudaStream_t passed as void*) and
+ *     return without synchronising.
+ *   - Host-detectable problems (null or misaligned pointers, unsupported
+ *     shapes, workspace too small) return a negative sd_status before anything
+ *     is launched.  Problems only visible on the device (bad parent array,
+ *     block-table entry out of range, an expired bounded wait) store the first
+ *     error code into *dev_status (int32, dev, must be 0 on entry) and the
+ *     kernel finishes normally; outputs are unspecified in that case.
+ *   - Same inputs give bit-identical outputs from run to run.
+ *   - All dev pointers must be 16-byte aligned.
+ *
+ * Layouts
+ *   KV cache of one layer, K and V each:  bf16 [num_blocks][Hkv][64][D]
+ *       (block = 64 tokens; one (block, head) tile is 16 KiB contiguous)
+ *   logical token t of sequence b lives in block block_table[b][t / 64],
+ *       slot t % 64.  Slots at or beyond len[b] may hold any finite values.
+ *   q, out:            bf16 [B][T_max][Hq][D]
+ *   tree K, tree V:    bf16 [B][T_max][Hkv][D]
+ *   query head h uses KV head h / (Hq / Hkv).
+ *   Node 0 of a tree is the root (the last emitted token, whose KV is not yet
+ *   cached); parents[b][0] = -1 and 0 <= parents[b][i] < i.
+ *
+ * Supported: D = 128, block_size = 64, 1 <= T_max <= 64, Hq % Hkv == 0,
+ * Hq / Hkv <= 8.
+ */
+#ifndef SDVERIFY_H
+#define SDVERIFY_H
+
+#include <stddef.h>
+#include <stdint.h>
+
+#ifdef __cplusplus
+extern "C" {
+#endif
+
+typedef enum {
+    SD_OK = 0,
+    SD_ERR_INVALID_ARG = -1,
+    SD_ERR_INVALID_TREE = -2,
+    SD_ERR_UNSUPPORTED = -3,
+    SD_ERR_WORKSPACE = -4,
+    SD_ERR_CUDA = -5,
+    SD_ERR_TIMEOUT = -6,
+    SD_ERR_BOUNDS = -7
+} sd_status;
+
+/* Paged KV cache of ONE layer (dev memory owned by the caller). */
+typedef struct {
+    void *k;             /* dev bf16 [num_blocks][Hkv][64][D] */
+    void *v;             /* dev bf16 [num_blocks][Hkv][64][D] */
+    int32_t num_blocks;
+} sd_kv_layer;
+
+/* Batch geometry shared by the calls.  Scalars are host values; pointers are
+ * dev arrays owned by the caller. */
+typedef struct {
+    int32_t B;                   /* sequences                                        */
+    int32_t T_max;               /* row stride of per-node arrays; 1..64             */
+    int32_t Hq, Hkv, D;          /* query heads, KV heads, head dim (128)            */
+    int32_t block_size;          /* 64                                               */
+    int32_t max_blocks_per_seq;  /* row stride of block_table                        */
+    const int32_t *block_table;  /* dev [B][max_blocks_per_seq]; covers len+n_nodes  */
+    const int32_t *len;          /* dev [B] cached prefix length of each sequence    */
+    const int32_t *n_nodes;      /* dev [B] nodes in each tree, 1..T_max             */
+    const int32_t *parents;      /* dev [B][T_max]                                   */
+    uint64_t *anc_mask;          /* dev [B][T_max]; bit j of [b][i] set iff node j is
+                                    i itself or an ancestor of i (sd_tree_prepare)   */
+} sd_batch;
+
+/* Library version (major*100 + minor). */
+int sd_version(void);
+
+/* Static, human-readable name of a status code. */
+const char *sd_status_string(sd_status s);
+
+/*
+ * Scratch bytes that sd_verify_attention (for this geometry; only the host
+ * scalars of *geom are read) and sd_lmhead_argmax (for M rows, vocabulary V)
+ * need; the larger of the two.  Pass M = 0 or V = 0 to size for attention
+ * only, geom = NULL for the LM head only.
+ */
+size_t sd_workspace_bytes(const sd_batch *geom, int32_t M, int32_t V);
+
+/*
+ * Ancestor masks of the draft trees (Sec. 1: the speculative tokens are
+ * validated together; a node may attend only to its own root path).
+ * Validates parents (root -1, parent < child, n_nodes in 1..T_max) and fills
+ * batch->anc_mask.  A bad tree stores SD_ERR_INVALID_TREE into *dev_status.
+ */
+sd_status sd_tree_prepare(const sd_batch *batch, int32_t *dev_status, void *stream);
+
+/*
+ * Tree-masked GQA attention of one layer (Sec. 1, batched validation; Sec. 4.1,
+ * results equal the target's own decoding).  For sequence b, node i < n_nodes[b]
+ * and query head h:  out = softmax(scale * q . K^T) V  over the keys
+ * { cached tokens t < len[b] } U { tree nodes j with bit j set in anc_mask[b][i] }.
+ *   q, k_tree, v_tree : dev bf16, layouts above (read only)
+ *   out               : dev bf16 [B][T_max][Hq][D]; rows of nodes >= n_nodes[b] are zeroed
+ *   lse               : dev f32 [B][T_max][Hq] or NULL; natural-log sum of exp of the scaled scores
+ *   workspace         : dev scratch of at least sd_workspace_bytes(batch, 0, 0)
+ * Arithmetic: bf16 inputs, fp32 accumulation, bf16 output (round to nearest even).
+ * Needs batch->anc_mask filled.  Errors: SD_ERR_INVALID_ARG, SD_ERR_UNSUPPORTED,
+ * SD_ERR_WORKSPACE on the host; SD_ERR_BOUNDS (block-table entry outside
+ * [0, num_blocks)) or SD_ERR_TIMEOUT through *dev_status.
+ */
+sd_status sd_verify_attention(const sd_batch *batch, const sd_kv_layer *cache,
+                              const void *q, const void *k_tree, const void *v_tree,
+                              float scale, void *out, float *lse,
+                              void *workspace, size_t workspace_bytes,
+                              int32_t *dev_status, void *stream);
+
+/*
+ * LM-head projection with fused arg-max (Sec. 1 / Sec. 4.1: the target's own
+ * greedy prediction at every speculative position).
+ *   logits[r][v] = sum_k hidden[r][k] * W[v][k]     (never written to memory)
+ *   argmax[r]    = lowest v attaining max_v logits[r][v]
+ *   maxlogit[r]  = that maximum (fp32), optional
+ *   hidden : dev bf16 [M][Hd]      W : dev bf16 [V][Hd]  (row-major, Hd contiguous)
+ *   Hd % 64 == 0, V >= 1, M >= 1
+ *   workspace : dev scratch of at least sd_workspace_bytes(NULL, M, V)
+ * Arithmetic: bf16 products accumulated in fp32.
+ */
+sd_status sd_lmhead_argmax(const void *hidden, const void *W,
+                           int32_t M, int32_t Hd, int32_t V,
+                           int32_t *argmax, float *maxlogit,
+                           void *workspace, size_t workspace_bytes,
+                           int32_t *dev_status, void *stream);
+
+/*
+ * Greedy acceptance (Sec. 1 "validated"; Sec. 4.1 reports the average
+ * acceptance length this step produces).  Node j >= 1 matches when
+ * draft_tok[b][j] == target_argmax[b][parents[b][j]]; a node is valid when
+ * every non-root node on its root path matches; the valid node of greatest
+ * depth wins, the smallest index among equals.
+ *   n_acc[b]    = its depth + 1 (the root always counts)
+ *   path[b][k]  = k-th node from the root, k < n_acc[b]; -1 beyond
+ *   out_tok[b]  = draft tokens of path[b][1..], then target_argmax at the last
+ *                 accepted node (bonus token): n_acc[b] tokens; -1 beyond
+ *   new_len[b]  = len[b] + n_acc[b]
+ * All arrays dev int32: draft_tok, target_argmax, path, out_tok [B][T_max];
+ * n_acc, new_len [B].  A bad parent array stores SD_ERR_INVALID_TREE.
+ */
+sd_status sd_accept_tree(const sd_batch *batch, const int32_t *draft_tok,
+                         const int32_t *target_argmax,
+                         int32_t *n_acc, int32_t *path, int32_t *out_tok, int32_t *new_len,
+                         int32_t *dev_status, void *stream);
+
+/*
+ * KV compaction (Sec. 4.1: the KV cache is the running context).  For every
+ * layer l < L, sequence b and k < n_acc[b]: cache slot len[b] + k (through the
+ * block table) receives tree row path[b][k], all KV heads, K and V, byte for
+ * byte.  Nothing else in any cache changes.  One launch covers all layers.
+ *   layers        : host array [L] of cache descriptors
+ *   k_tree_layers,
+ *   v_tree_layers : host arrays [L] of dev pointers, bf16 [B][T_max][Hkv][D]
+ *   n_acc, path   : dev, as produced by sd_accept_tree
+ * The tree buffers must not alias the caches.  A destination block outside
+ * [0, num_blocks) or a path entry outside [0, T_max) stores SD_ERR_BOUNDS and
+ * skips that row.
+ */
+sd_status sd_compact_kv(const sd_batch *batch, const sd_kv_layer *layers, int32_t L,
+                        const void *const *k_tree_layers, const void *const *v_tree_layers,
+                        const int32_t *n_acc, const int32_t *path,
+                        int32_t *dev_status, void *stream);
+
+#ifdef __cplusplus
+}
+#endif
+#endif /* SDVERIFY_H */

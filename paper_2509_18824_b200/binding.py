@@ -1,0 +1,193 @@
+"""ctypes binding of libsdverify.so: same names as the C header, argument
+marshalling only.  Tensors are torch CUDA tensors (device memory and streams
+are all torch is used for); every step of the computation runs in the
+library's kernels.  There is no CPU fallback: if the shared library cannot be
+loaded, importing this module raises.
+"""
+from __future__ import annotations
+
+import ctypes as C
+import os
+from typing import List, Optional, Sequence
+
+import torch
+
+_HERE = os.path.dirname(os.path.abspath(__file__))
+LIB_PATH = os.path.join(_HERE, "libsdverify.so")
+
+SD_OK = 0
+SD_ERR_INVALID_ARG = -1
+SD_ERR_INVALID_TREE = -2
+SD_ERR_UNSUPPORTED = -3
+SD_ERR_WORKSPACE = -4
+SD_ERR_CUDA = -5
+SD_ERR_TIMEOUT = -6
+SD_ERR_BOUNDS = -7
+
+# kernel launches behind one call (kept in step with the kernels; used for launch accounting)
+KERNELS_PER_ATTENTION = 2      # split-KV partials + merge
+KERNELS_PER_LMHEAD = 2         # tiles + cross-slab reduce
+
+EXPORTS = ["sd_version", "sd_status_string", "sd_workspace_bytes", "sd_tree_prepare",
+           "sd_verify_attention", "sd_lmhead_argmax", "sd_accept_tree", "sd_compact_kv"]
+
+
+class sd_kv_layer(C.Structure):
+    _fields_ = [("k", C.c_void_p), ("v", C.c_void_p), ("num_blocks", C.c_int32)]
+
+
+class sd_batch(C.Structure):
+    _fields_ = [("B", C.c_int32), ("T_max", C.c_int32), ("Hq", C.c_int32), ("Hkv", C.c_int32),
+                ("D", C.c_int32), ("block_size", C.c_int32), ("max_blocks_per_seq", C.c_int32),
+                ("block_table", C.c_void_p), ("len", C.c_void_p), ("n_nodes", C.c_void_p),
+                ("parents", C.c_void_p), ("anc_mask", C.c_void_p)]
+
+
+def _load() -> C.CDLL:
+    if not os.path.exists(LIB_PATH):
+        from . import build as _build          # needs nvcc; raises if it fails
+        _build.build()
+    lib = C.CDLL(LIB_PATH)
+    lib.sd_version.restype = C.c_int
+    lib.sd_status_string.restype = C.c_char_p
+    lib.sd_status_string.argtypes = [C.c_int]
+    lib.sd_workspace_bytes.restype = C.c_size_t
+    lib.sd_workspace_bytes.argtypes = [C.c_void_p, C.c_int32, C.c_int32]
+    lib.sd_tree_prepare.restype = C.c_int
+    lib.sd_tree_prepare.argtypes = [C.c_void_p, C.c_void_p, C.c_void_p]
+    lib.sd_verify_attention.restype = C.c_int
+    lib.sd_verify_attention.argtypes = [C.c_void_p, C.c_void_p, C.c_void_p, C.c_void_p, C.c_void_p,
+                                        C.c_float, C.c_void_p, C.c_void_p, C.c_void_p, C.c_size_t,
+                                        C.c_void_p, C.c_void_p]
+    lib.sd_lmhead_argmax.restype = C.c_int
+    lib.sd_lmhead_argmax.argtypes = [C.c_void_p, C.c_void_p, C.c_int32, C.c_int32, C.c_int32,
+                                     C.c_void_p, C.c_void_p, C.c_void_p, C.c_size_t, C.c_void_p, C.c_void_p]
+    lib.sd_accept_tree.restype = C.c_int
+    lib.sd_accept_tree.argtypes = [C.c_void_p] * 9
+    lib.sd_compact_kv.restype = C.c_int
+    lib.sd_compact_kv.argtypes = [C.c_void_p, C.c_void_p, C.c_int32, C.c_void_p, C.c_void_p,
+                                  C.c_void_p, C.c_void_p, C.c_void_p, C.c_void_p]
+    return lib
+
+
+lib = _load()
+
+
+class SdError(RuntimeError):
+    def __init__(self, code: int):
+        self.code = code
+        super().__init__(sd_status_string(code))
+
+
+def sd_version() -> int:
+    return int(lib.sd_version())
+
+
+def sd_status_string(code: int) -> str:
+    return lib.sd_status_string(int(code)).decode()
+
+
+def _check(code: int) -> None:
+    if code != SD_OK:
+        raise SdError(code)
+
+
+def _ptr(t) -> Optional[int]:
+    if t is None:
+        return None
+    if isinstance(t, int):
+        return t
+    assert t.is_cuda and t.is_contiguous(), "device tensors must be contiguous CUDA tensors"
+    return t.data_ptr()
+
+
+def _stream(stream) -> int:
+    if stream is None:
+        return torch.cuda.current_stream().cuda_stream
+    if isinstance(stream, int):
+        return stream
+    return stream.cuda_stream
+
+
+class Batch:
+    """Owns the device arrays named by the C struct ``sd_batch``."""
+
+    def __init__(self, B, T_max, Hq, Hkv, D, block_table, lens, n_nodes, parents,
+                 block_size=64, device="cuda"):
+        dev = torch.device(device)
+        to = lambda a: torch.as_tensor(a, dtype=torch.int32).contiguous().to(dev)
+        self.B, self.T_max, self.Hq, self.Hkv, self.D = int(B), int(T_max), int(Hq), int(Hkv), int(D)
+        self.block_table = to(block_table).reshape(self.B, -1).contiguous()
+        self.len = to(lens)
+        self.n_nodes = to(n_nodes)
+        self.parents = to(parents).reshape(self.B, self.T_max).contiguous()
+        self.anc_mask = torch.zeros((self.B, self.T_max), dtype=torch.int64, device=dev)
+        self.max_blocks = int(self.block_table.shape[1])
+        self.c = sd_batch(self.B, self.T_max, self.Hq, self.Hkv, self.D, int(block_size), self.max_blocks,
+                          self.block_table.data_ptr(), self.len.data_ptr(), self.n_nodes.data_ptr(),
+                          self.parents.data_ptr(), self.anc_mask.data_ptr())
+
+    @classmethod
+    def of(cls, w, device="cuda") -> "Batch":
+        """From any object carrying B, T_max, Hq, Hkv, D, block_table, len, n_nodes, parents."""
+        return cls(w.B, w.T_max, w.Hq, w.Hkv, w.D, w.block_table, w.len, w.n_nodes, w.parents, device=device)
+
+    def ref(self):
+        return C.byref(self.c)
+
+
+def kv_layer(k_cache: torch.Tensor, v_cache: torch.Tensor) -> sd_kv_layer:
+    return sd_kv_layer(_ptr(k_cache), _ptr(v_cache), int(k_cache.shape[0]))
+
+
+def new_status(device="cuda") -> torch.Tensor:
+    return torch.zeros(1, dtype=torch.int32, device=device)
+
+
+def sd_workspace_bytes(batch: Optional[Batch], M: int = 0, V: int = 0) -> int:
+    return int(lib.sd_workspace_bytes(batch.ref() if batch is not None else None, int(M), int(V)))
+
+
+def sd_tree_prepare(batch: Batch, status: torch.Tensor, stream=None) -> None:
+    _check(lib.sd_tree_prepare(batch.ref(), _ptr(status), _stream(stream)))
+
+
+def sd_verify_attention(batch: Batch, cache: sd_kv_layer, q, k_tree, v_tree, scale: float,
+                        out, lse, workspace, status, stream=None) -> None:
+    _check(lib.sd_verify_attention(batch.ref(), C.byref(cache), _ptr(q), _ptr(k_tree), _ptr(v_tree),
+                                   C.c_float(scale), _ptr(out), _ptr(lse), _ptr(workspace),
+                                   workspace.numel() * workspace.element_size(), _ptr(status),
+                                   _stream(stream)))
+
+
+def sd_lmhead_argmax(hidden, W, argmax, maxlogit, workspace, status, stream=None) -> None:
+    M, Hd = hidden.shape
+    V = W.shape[0]
+    assert W.shape[1] == Hd
+    _check(lib.sd_lmhead_argmax(_ptr(hidden), _ptr(W), int(M), int(Hd), int(V), _ptr(argmax),
+                                _ptr(maxlogit), _ptr(workspace),
+                                workspace.numel() * workspace.element_size(), _ptr(status), _stream(stream)))
+
+
+def sd_accept_tree(batch: Batch, draft_tok, target_argmax, n_acc, path, out_tok, new_len,
+                   status, stream=None) -> None:
+    _check(lib.sd_accept_tree(batch.ref(), _ptr(draft_tok), _ptr(target_argmax), _ptr(n_acc), _ptr(path),
+                              _ptr(out_tok), _ptr(new_len), _ptr(status), _stream(stream)))
+
+
+class LayerSet:
+    """Host arrays of per-layer descriptors for ``sd_compact_kv`` (built once, reused)."""
+
+    def __init__(self, k_caches: Sequence[torch.Tensor], v_caches: Sequence[torch.Tensor],
+                 k_trees: Sequence[torch.Tensor], v_trees: Sequence[torch.Tensor]):
+        L = len(k_caches)
+        self.L = L
+        self.layers = (sd_kv_layer * L)(*[kv_layer(k, v) for k, v in zip(k_caches, v_caches)])
+        self.kt = (C.c_void_p * L)(*[_ptr(t) for t in k_trees])
+        self.vt = (C.c_void_p * L)(*[_ptr(t) for t in v_trees])
+        self._keep = (list(k_caches), list(v_caches), list(k_trees), list(v_trees))
+
+
+def sd_compact_kv(batch: Batch, layers: LayerSet, n_acc, path, status, stream=None) -> None:
+    _check(lib.sd_compact_kv(batch.ref(), layers.layers, layers.L, layers.kt, layers.vt,
+                             _ptr(n_acc), _ptr(path), _ptr(status), _stream(stream)))

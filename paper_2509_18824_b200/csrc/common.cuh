@@ -1,0 +1,46 @@
+// Shared device/host helpers of the sdverify kernels.
+#pragma once
+#include <cuda_runtime.h>
+#include <cuda_bf16.h>
+#include <stdint.h>
+#include "sdverify.h"
+
+namespace sdv {
+
+constexpr int kBlock = 64;     // tokens per KV-cache block
+constexpr int kD = 128;        // head dimension
+constexpr int kMaxT = 64;      // nodes per tree
+
+// first error wins; kernels never trap
+__device__ __forceinline__ void set_status(int32_t* status, int code) {
+    if (status) atomicCAS(status, 0, code);
+}
+
+__device__ __forceinline__ float bf16_bits_to_float(uint16_t b) {
+    return __uint_as_float(((uint32_t)b) << 16);
+}
+__device__ __forceinline__ float bf16lo(uint32_t u) { return __uint_as_float(u << 16); }
+__device__ __forceinline__ float bf16hi(uint32_t u) { return __uint_as_float(u & 0xffff0000u); }
+
+inline bool aligned16(const void* p) { return (reinterpret_cast<uintptr_t>(p) & 15u) == 0; }
+
+inline sd_status cuda_ok(cudaError_t e) { return e == cudaSuccess ? SD_OK : SD_ERR_CUDA; }
+
+// launch-side entry points implemented in the kernel files
+sd_status launch_tree_prepare(const sd_batch& bt, int32_t* dev_status, cudaStream_t st);
+sd_status launch_accept(const sd_batch& bt, const int32_t* draft, const int32_t* target,
+                        int32_t* n_acc, int32_t* path, int32_t* out_tok, int32_t* new_len,
+                        int32_t* dev_status, cudaStream_t st);
+sd_status launch_compact(const sd_batch& bt, const sd_kv_layer* layers, int L,
+                         const void* const* kt, const void* const* vt,
+                         const int32_t* n_acc, const int32_t* path, int32_t* dev_status, cudaStream_t st);
+size_t attention_workspace_bytes(const sd_batch& bt);
+sd_status launch_attention(const sd_batch& bt, const sd_kv_layer& cache, const void* q,
+                           const void* kt, const void* vt, float scale, void* out, float* lse,
+                           void* ws, size_t ws_bytes, int32_t* dev_status, cudaStream_t st);
+size_t lmhead_workspace_bytes(int M, int V);
+sd_status launch_lmhead(const void* hidden, const void* W, int M, int Hd, int V,
+                        int32_t* argmax, float* maxlogit, void* ws, size_t ws_bytes,
+                        int32_t* dev_status, cudaStream_t st);
+
+}  // namespace sdv

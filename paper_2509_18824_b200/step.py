@@ -1,0 +1,142 @@
+"""One whole verify step as a sequence of library calls.
+
+Per layer: tree attention; then once: LM-head arg-max, greedy acceptance and
+KV compaction over all layers.  This file only moves tensors to the device and
+issues the C-ABI calls in order; it computes nothing itself.  (The layers'
+projections, MLPs and norms of a real decoder are outside this library: q,
+tree K/V and the final hidden states are inputs.)
+"""
+from __future__ import annotations
+
+from typing import List, Optional
+
+import numpy as np
+import torch
+
+from . import binding as sd
+
+
+def to_device(a: np.ndarray, device="cuda") -> torch.Tensor:
+    """numpy -> device tensor; bf16 bit patterns (uint16) travel as int16."""
+    if a.dtype == np.uint16:
+        a = a.view(np.int16)
+    return torch.from_numpy(np.ascontiguousarray(a)).to(device)
+
+
+def pinned(a: np.ndarray) -> torch.Tensor:
+    if a.dtype == np.uint16:
+        a = a.view(np.int16)
+    return torch.from_numpy(np.ascontiguousarray(a)).pin_memory()
+
+
+class VerifyStep:
+    """Device-resident state (KV caches, LM-head weights, geometry) plus the
+    per-step inputs and outputs of one batch."""
+
+    def __init__(self, w, device="cuda", layers: Optional[List[int]] = None, keep_host_inputs=False):
+        self.device = torch.device(device)
+        self.w = w
+        self.L = len(w.q)
+        d = self.device
+        self.batch = sd.Batch.of(w, device=d)
+        self.status = sd.new_status(d)
+        # resident state
+        self.k_cache = [to_device(x, d) for x in w.k_cache]
+        self.v_cache = [to_device(x, d) for x in w.v_cache]
+        self.W = to_device(w.W, d) if w.W is not None else None
+        # per-step inputs
+        self.q = [to_device(x, d) for x in w.q]
+        self.k_tree = [to_device(x, d) for x in w.k_tree]
+        self.v_tree = [to_device(x, d) for x in w.v_tree]
+        self.hidden = to_device(w.hidden, d) if w.hidden is not None else None
+        self.draft_tok = to_device(w.draft_tok, d) if w.draft_tok is not None else None
+        # outputs
+        B, T = w.B, w.T_max
+        self.out = [torch.zeros((B, T, w.Hq, w.D), dtype=torch.bfloat16, device=d) for _ in range(self.L)]
+        self.lse = [torch.zeros((B, T, w.Hq), dtype=torch.float32, device=d) for _ in range(self.L)]
+        M = B * T
+        self.argmax = torch.zeros(M, dtype=torch.int32, device=d)
+        self.maxlogit = torch.zeros(M, dtype=torch.float32, device=d)
+        self.n_acc = torch.zeros(B, dtype=torch.int32, device=d)
+        self.path = torch.zeros((B, T), dtype=torch.int32, device=d)
+        self.out_tok = torch.zeros((B, T), dtype=torch.int32, device=d)
+        self.new_len = torch.zeros(B, dtype=torch.int32, device=d)
+        nbytes = sd.sd_workspace_bytes(self.batch, M if self.W is not None else 0, w.V if self.W is not None else 0)
+        self.workspace = torch.empty(max(nbytes, 256), dtype=torch.uint8, device=d)
+        self.caches = [sd.kv_layer(k, v) for k, v in zip(self.k_cache, self.v_cache)]
+        self.layerset = sd.LayerSet(self.k_cache, self.v_cache, self.k_tree, self.v_tree)
+        self.scale = float(w.scale)
+        sd.sd_tree_prepare(self.batch, self.status)
+        # pinned host copies for the end-to-end path
+        self.host = None
+        if keep_host_inputs:
+            self.host = dict(
+                q=[pinned(x) for x in w.q], k_tree=[pinned(x) for x in w.k_tree],
+                v_tree=[pinned(x) for x in w.v_tree], hidden=pinned(w.hidden),
+                draft_tok=pinned(w.draft_tok), parents=pinned(w.parents), n_nodes=pinned(w.n_nodes))
+            self.host_out = dict(
+                n_acc=torch.zeros(B, dtype=torch.int32).pin_memory(),
+                path=torch.zeros((B, T), dtype=torch.int32).pin_memory(),
+                out_tok=torch.zeros((B, T), dtype=torch.int32).pin_memory(),
+                new_len=torch.zeros(B, dtype=torch.int32).pin_memory())
+
+    # -- pieces ---------------------------------------------------------
+    def attention(self, l: int, stream=None):
+        sd.sd_verify_attention(self.batch, self.caches[l], self.q[l], self.k_tree[l], self.v_tree[l],
+                               self.scale, self.out[l], self.lse[l], self.workspace, self.status, stream)
+
+    def lmhead(self, stream=None):
+        sd.sd_lmhead_argmax(self.hidden, self.W, self.argmax, self.maxlogit, self.workspace, self.status, stream)
+
+    def accept(self, target=None, stream=None):
+        sd.sd_accept_tree(self.batch, self.draft_tok, self.argmax if target is None else target,
+                          self.n_acc, self.path, self.out_tok, self.new_len, self.status, stream)
+
+    def compact(self, stream=None):
+        sd.sd_compact_kv(self.batch, self.layerset, self.n_acc, self.path, self.status, stream)
+
+    # -- the whole step -------------------------------------------------
+    def run(self, stream=None):
+        for l in range(self.L):
+            self.attention(l, stream)
+        self.lmhead(stream)
+        self.accept(None, stream)
+        self.compact(stream)
+
+    @property
+    def launches_per_step(self) -> int:
+        """Kernel launches of one run(): per layer the partial and the merge kernel;
+        the LM-head kernels; acceptance; compaction."""
+        return self.L * sd.KERNELS_PER_ATTENTION + sd.KERNELS_PER_LMHEAD + 1 + (self.L + 63) // 64
+
+    def h2d_bytes(self) -> int:
+        h = self.host
+        n = sum(t.numel() * t.element_size() for k in ("q", "k_tree", "v_tree") for t in h[k])
+        return n + sum(h[k].numel() * h[k].element_size() for k in ("hidden", "draft_tok", "parents", "n_nodes"))
+
+    def d2h_bytes(self) -> int:
+        return sum(t.numel() * t.element_size() for t in self.host_out.values())
+
+    def run_from_host(self):
+        """End-to-end step: this step's inputs come from pinned host memory, the
+        accepted tokens go back to the host; caches and weights stay resident."""
+        h = self.host
+        for l in range(self.L):
+            self.q[l].copy_(h["q"][l], non_blocking=True)
+            self.k_tree[l].copy_(h["k_tree"][l], non_blocking=True)
+            self.v_tree[l].copy_(h["v_tree"][l], non_blocking=True)
+        self.hidden.copy_(h["hidden"], non_blocking=True)
+        self.draft_tok.copy_(h["draft_tok"], non_blocking=True)
+        self.batch.parents.copy_(h["parents"], non_blocking=True)
+        self.batch.n_nodes.copy_(h["n_nodes"], non_blocking=True)
+        sd.sd_tree_prepare(self.batch, self.status)
+        self.run()
+        self.host_out["n_acc"].copy_(self.n_acc, non_blocking=True)
+        self.host_out["path"].copy_(self.path, non_blocking=True)
+        self.host_out["out_tok"].copy_(self.out_tok, non_blocking=True)
+        self.host_out["new_len"].copy_(self.new_len, non_blocking=True)
+
+    def check_status(self):
+        code = int(self.status.item())
+        if code != 0:
+            raise sd.SdError(code)

@@ -1,0 +1,51 @@
+"""The C-ABI library loads without a GPU and exports every symbol the header declares."""
+import ctypes
+import os
+import re
+
+ROOT = os.path.dirname(os.path.dirname(os.path.abspath(__file__)))
+
+
+def declared_symbols():
+    text = open(os.path.join(ROOT, "include", "sdverify.h")).read()
+    text = re.sub(r"/\*.*?\*/", "", text, flags=re.S)
+    return sorted(set(re.findall(r"\b(sd_[a-z_0-9]+)\s*\(", text)))
+
+
+def test_library_loads_and_exports_the_header():
+    from paper_2509_18824_b200 import build
+    lib = ctypes.CDLL(build.build())
+    syms = declared_symbols()
+    assert {"sd_verify_attention", "sd_lmhead_argmax", "sd_accept_tree", "sd_compact_kv"} <= set(syms)
+    for s in syms:
+        assert hasattr(lib, s), s
+    lib.sd_status_string.restype = ctypes.c_char_p
+    assert lib.sd_status_string(0) == b"SD_OK"
+    assert lib.sd_status_string(-7) == b"SD_ERR_BOUNDS"
+    assert lib.sd_version() >= 100
+
+
+def test_binding_matches_header():
+    from paper_2509_18824_b200 import binding
+    assert sorted(binding.EXPORTS) == declared_symbols()
+    # host-side argument checks need no GPU: a null geometry is refused before any launch
+    assert binding.lib.sd_tree_prepare(None, None, None) == binding.SD_ERR_INVALID_ARG
+    bt = binding.sd_batch(1, 65, 4, 1, 128, 64, 4, 16, 16, 16, 16, 16)
+    assert binding.lib.sd_tree_prepare(ctypes.byref(bt), 16, None) == binding.SD_ERR_UNSUPPORTED
+    bt = binding.sd_batch(1, 8, 4, 1, 64, 64, 4, 16, 16, 16, 16, 16)
+    assert binding.lib.sd_tree_prepare(ctypes.byref(bt), 16, None) == binding.SD_ERR_UNSUPPORTED
+    bt = binding.sd_batch(1, 8, 4, 1, 128, 64, 4, 16, 16, 8, 16, 16)     # misaligned n_nodes
+    assert binding.lib.sd_tree_prepare(ctypes.byref(bt), 16, None) == binding.SD_ERR_INVALID_ARG
+    assert binding.sd_workspace_bytes(None, 60, 152064) > 0
+
+
+def test_product_code_never_touches_the_checker():
+    pkg = os.path.join(ROOT, "paper_2509_18824_b200")
+    for dirpath, _, files in os.walk(pkg):
+        if "_build" in dirpath:
+            continue
+        for f in files:
+            if f.endswith((".py", ".cu", ".cuh", ".h")):
+                text = open(os.path.join(dirpath, f)).read()
+                assert "import oracle" not in text and "from oracle" not in text, f
+                assert "liboracle" not in text and "sd_oracle" not in text, f

@@ -1,0 +1,292 @@
+"""GPU parity: every library call against the fp64 checker on the same seeded inputs."""
+import numpy as np
+import pytest
+import torch
+
+import oracle
+from paper_2509_18824_b200 import binding as sd
+from paper_2509_18824_b200 import workloads as wl
+from paper_2509_18824_b200.step import VerifyStep, to_device
+from helpers import Tiny, root_path
+from gpu_util import (gpu_attention, check_attention, gpu_lmhead, check_argmax)
+
+pytestmark = pytest.mark.gpu
+
+
+# ------------------------------------------------------------------ trees / accept
+def run_accept(w, draft, target):
+    bt = sd.Batch.of(w)
+    st = sd.new_status()
+    B, T = w.B, w.T_max
+    n_acc = torch.full((B,), -9, dtype=torch.int32, device="cuda")
+    path = torch.full((B, T), -9, dtype=torch.int32, device="cuda")
+    out_tok = torch.full((B, T), -9, dtype=torch.int32, device="cuda")
+    new_len = torch.full((B,), -9, dtype=torch.int32, device="cuda")
+    sd.sd_accept_tree(bt, to_device(draft), to_device(target), n_acc, path, out_tok, new_len, st)
+    torch.cuda.synchronize()
+    return [x.cpu().numpy() for x in (n_acc, path, out_tok, new_len)], int(st.item())
+
+
+@pytest.mark.parametrize("cfg", ["c1", "c2", "c4", "c5", "chain11"])
+def test_accept_bit_exact_random_small_vocab(cfg):
+    w = wl.make_geometry(wl.spec(cfg))
+    g = np.random.default_rng(1)
+    for vocab in (2, 3, 50):
+        draft = g.integers(0, vocab, size=(w.B, w.T_max)).astype(np.int32)
+        target = g.integers(0, vocab, size=(w.B, w.T_max)).astype(np.int32)
+        ref = oracle.accept(oracle.Geometry.of(w), draft, target)
+        got, status = run_accept(w, draft, target)
+        assert status == 0
+        for a, b in zip(got, ref):
+            np.testing.assert_array_equal(a, b)
+
+
+def test_accept_planted_and_ragged_node_counts():
+    w = wl.make_geometry(wl.spec("c5"))
+    g = np.random.default_rng(2)
+    target = g.integers(0, w.V, size=(w.B, w.T_max)).astype(np.int32)
+    wl.plant(w, target, np.arange(w.B) % 7)
+    ref = oracle.accept(oracle.Geometry.of(w), w.draft_tok, target)
+    got, status = run_accept(w, w.draft_tok, target)
+    assert status == 0
+    for a, b in zip(got, ref):
+        np.testing.assert_array_equal(a, b)
+    np.testing.assert_array_equal(got[0], w.planted_len + 1)
+    # fewer nodes than T_max in some sequences
+    w.n_nodes = np.array([60, 1, 33, 2, 59, 17, 60, 5], dtype=np.int32)
+    draft = g.integers(0, 2, size=(w.B, w.T_max)).astype(np.int32)
+    target = g.integers(0, 2, size=(w.B, w.T_max)).astype(np.int32)
+    ref = oracle.accept(oracle.Geometry.of(w), draft, target)
+    got, status = run_accept(w, draft, target)
+    assert status == 0
+    for a, b in zip(got, ref):
+        np.testing.assert_array_equal(a, b)
+
+
+def test_tree_prepare_masks_and_bad_tree_status():
+    w = wl.make_geometry(wl.spec("c4"))
+    bt = sd.Batch.of(w)
+    st = sd.new_status()
+    sd.sd_tree_prepare(bt, st)
+    torch.cuda.synchronize()
+    assert int(st.item()) == 0
+    am = bt.anc_mask.cpu().numpy().view(np.uint64)
+    for b in range(w.B):
+        for i in range(w.T_max):
+            want = sum(1 << j for j in root_path(w.parents[b], i))
+            assert int(am[b, i]) == want
+    bad = wl.make_geometry(wl.spec("c1"))
+    bad.parents = bad.parents.copy(); bad.parents[0, 3] = 5      # parent > child
+    bt = sd.Batch.of(bad)
+    st = sd.new_status()
+    sd.sd_tree_prepare(bt, st)
+    torch.cuda.synchronize()
+    assert int(st.item()) == sd.SD_ERR_INVALID_TREE
+    _, status = run_accept(bad, np.zeros((1, 8), np.int32), np.zeros((1, 8), np.int32))
+    assert status == sd.SD_ERR_INVALID_TREE
+
+
+# ------------------------------------------------------------------ attention
+def tiny128(seed, **kw):
+    kw.setdefault("D", 128)
+    return Tiny(seed, **kw)
+
+
+@pytest.mark.parametrize("lens", [(0, 1), (63, 64), (65, 127), (128, 129), (700, 5), (1023, 1025)])
+def test_attention_edge_lengths_peaked_scores(lens):
+    p = tiny128(sum(lens), B=2, T=8, Hq=8, Hkv=2, lens=lens, gain=4.0)
+    out, lse, status = gpu_attention(p)
+    assert status == 0
+    ref, rlse = oracle.attention(oracle.Geometry.of(p), p.k_cache, p.v_cache, p.q, p.k_tree, p.v_tree, p.scale)
+    check_attention(out, ref, f"lens={lens}")
+    np.testing.assert_allclose(lse, rlse, rtol=2e-3, atol=2e-3)
+
+
+def test_attention_gqa7_wide_trees_and_unused_nodes():
+    g = np.random.default_rng(0)
+    T = 64
+    par = np.stack([np.array([-1] + [int(g.integers(max(0, i - 9), i)) for i in range(1, T)]) for _ in range(3)])
+    p = tiny128(5, B=3, T=T, Hq=14, Hkv=2, lens=(300, 64, 1500), parents=par, gain=3.0)
+    p.n_nodes = np.array([64, 7, 33], dtype=np.int32)
+    out, lse, status = gpu_attention(p)
+    assert status == 0
+    ref, rlse = oracle.attention(oracle.Geometry.of(p), p.k_cache, p.v_cache, p.q, p.k_tree, p.v_tree, p.scale)
+    check_attention(out, ref)
+    for b in range(3):          # rows of unused nodes are zeroed
+        assert (out[b, p.n_nodes[b]:] == 0).all()
+    ok = np.isfinite(rlse)
+    np.testing.assert_allclose(lse[ok], rlse[ok], rtol=2e-3, atol=2e-3)
+
+
+def test_attention_planted_key_large_v_and_bad_block_table():
+    p = tiny128(6, B=1, T=8, Hq=4, Hkv=1, lens=(900,), gain=1.0)
+    # one key with score ~ +30, V rows scaled by 64
+    qv = wl.bf16_bits_to_f32(p.q[0, 5, 2])
+    t_star = 517
+    blk = p.block_table[0, t_star // 64]
+    p.k_cache[blk, 0, t_star % 64] = wl.f32_to_bf16_bits(qv * (30.0 / (p.scale * float(qv @ qv))))
+    p.v_cache[:] = wl.f32_to_bf16_bits(wl.bf16_bits_to_f32(p.v_cache) * 64)
+    p.v_tree[:] = wl.f32_to_bf16_bits(wl.bf16_bits_to_f32(p.v_tree) * 64)
+    out, lse, status = gpu_attention(p)
+    assert status == 0
+    ref, rlse = oracle.attention(oracle.Geometry.of(p), p.k_cache, p.v_cache, p.q, p.k_tree, p.v_tree, p.scale)
+    d = np.abs(out - ref)
+    assert np.sqrt((d ** 2).sum() / (ref ** 2).sum()) <= 2e-2
+    assert abs(rlse[0, 5, 2] - 30.0) < 0.1 and abs(lse[0, 5, 2] - rlse[0, 5, 2]) < 0.05
+    # a block-table entry outside the cache is reported, not dereferenced
+    p.block_table = p.block_table.copy(); p.block_table[0, 3] = p.num_blocks + 100
+    _, _, status = gpu_attention(p)
+    assert status == sd.SD_ERR_BOUNDS
+
+
+@pytest.mark.parametrize("cfg,gain", [("c1", 1.0), ("c1", 45.0), ("c2", 1.0), ("c2", 45.0)])
+def test_attention_configs_full_compare(cfg, gain):
+    w = wl.make(cfg, lmhead=False, q_gain=gain)
+    out, lse, status = gpu_attention(w, layer=0)
+    assert status == 0
+    ref, rlse = oracle.attention(oracle.Geometry.of(w), w.k_cache[0], w.v_cache[0], w.q[0], w.k_tree[0],
+                                 w.v_tree[0], w.scale)
+    mx, mean, rel = check_attention(out, ref, f"{cfg} gain {gain}")
+    np.testing.assert_allclose(lse, rlse, rtol=2e-3, atol=2e-3)
+
+
+def sample_rows(w, n, seed):
+    g = np.random.default_rng(seed)
+    rows = np.stack([g.integers(0, w.B, n), g.integers(0, w.T_max, n), g.integers(0, w.Hq, n)], 1).astype(np.int32)
+    rows[0] = (0, 0, 0)
+    rows[1] = (w.B - 1, w.T_max - 1, w.Hq - 1)
+    return rows
+
+
+@pytest.mark.parametrize("cfg,gain", [("c3", 1.0), ("c3", 45.0), ("c4", 1.0), ("c4", 45.0), ("chain11", 45.0)])
+def test_attention_full_size_sampled_rows(cfg, gain):
+    w = wl.make(cfg, lmhead=False, q_gain=gain)
+    out, lse, status = gpu_attention(w, layer=0)
+    assert status == 0
+    rows = sample_rows(w, 192, 3)
+    ref, rlse = oracle.attention_rows(oracle.Geometry.of(w), w.k_cache[0], w.v_cache[0], w.q[0], w.k_tree[0],
+                                      w.v_tree[0], w.scale, rows)
+    got = out[rows[:, 0], rows[:, 1], rows[:, 2]]
+    check_attention(got, ref, f"{cfg} gain {gain}")
+    np.testing.assert_allclose(lse[rows[:, 0], rows[:, 1], rows[:, 2]], rlse, rtol=2e-3, atol=2e-3)
+    assert np.isfinite(out).all()
+
+
+# ------------------------------------------------------------------ LM head
+@pytest.mark.parametrize("M,Hd,V", [(1, 64, 1), (5, 128, 1000), (8, 256, 1024), (61, 192, 129), (130, 64, 4099)])
+def test_lmhead_small_shapes_crisp(M, Hd, V):
+    g = np.random.default_rng(M + V)
+    h = wl.f32_to_bf16_bits(g.standard_normal((M, Hd)).astype(np.float32))
+    W = wl.f32_to_bf16_bits((g.standard_normal((V, Hd)) / np.sqrt(Hd)).astype(np.float32))
+    am, mx = gpu_lmhead(h, W)
+    ram, t1, t2 = oracle.lmhead(h, W)
+    check_argmax(am, mx, ram, t1, t2)
+
+
+def test_lmhead_exact_ties_lowest_index():
+    g = np.random.default_rng(4)
+    M, Hd, V = 6, 128, 3000
+    h = wl.f32_to_bf16_bits(g.standard_normal((M, Hd)).astype(np.float32))
+    W = wl.f32_to_bf16_bits((0.01 * g.standard_normal((V, Hd))).astype(np.float32))
+    W[[2999, 130, 1500, 131]] = wl.f32_to_bf16_bits(wl.bf16_bits_to_f32(h[2]) * 4)
+    am, mx = gpu_lmhead(h, W)
+    ram, t1, t2 = oracle.lmhead(h, W)
+    assert am[2] == 130 == ram[2]
+    np.testing.assert_array_equal(am, ram)
+
+
+def test_lmhead_c1_and_c2_full():
+    for cfg, gain in (("c1", 1.0), ("c1", 16.0), ("c2", 1.0), ("c2", 60.0)):
+        w = wl.make(cfg, attention=False, hidden_gain=gain)
+        am, mx = gpu_lmhead(w.hidden, w.W)
+        ram, t1, t2 = oracle.lmhead(w.hidden, w.W)
+        in_band, mis_in, mis_out = check_argmax(am, mx, ram, t1, t2, require_all=(gain > 1))
+        print(f"{cfg} gain {gain}: rows {len(am)}, in band {in_band}, mismatches in band {mis_in}, outside {mis_out}")
+
+
+# ------------------------------------------------------------------ compaction
+def test_compact_bit_exact_and_touches_nothing_else():
+    sp = wl.spec("c5"); sp.L = 3; sp.prefix = 250; sp.B = 5
+    w = wl.make_geometry(sp)
+    w.len = np.array([250, 58, 63, 64, 0], dtype=np.int32)     # 58+: crossing a block boundary
+    wl.fill_attention(w)
+    g = np.random.default_rng(5)
+    target = g.integers(0, 5, size=(w.B, w.T_max)).astype(np.int32)
+    wl.plant(w, target, np.array([6, 5, 0, 3, 6]))
+    G = oracle.Geometry.of(w)
+    n_acc, path, _, _ = oracle.accept(G, w.draft_tok, target)
+    bt = sd.Batch.of(w)
+    st = sd.new_status()
+    kc = [to_device(x) for x in w.k_cache]; vc = [to_device(x) for x in w.v_cache]
+    kt = [to_device(x) for x in w.k_tree]; vt = [to_device(x) for x in w.v_tree]
+    ls = sd.LayerSet(kc, vc, kt, vt)
+    sd.sd_compact_kv(bt, ls, to_device(n_acc), to_device(path), st)
+    torch.cuda.synchronize()
+    assert int(st.item()) == 0
+    for l in range(w.L):
+        rk, rv = w.k_cache[l].copy(), w.v_cache[l].copy()
+        oracle.compact(G, rk, rv, w.k_tree[l], w.v_tree[l], n_acc, path)
+        assert not np.array_equal(rk, w.k_cache[l])
+        np.testing.assert_array_equal(kc[l].cpu().numpy().view(np.uint16), rk)
+        np.testing.assert_array_equal(vc[l].cpu().numpy().view(np.uint16), rv)
+
+
+# ------------------------------------------------------------------ the whole step
+def test_chained_step_tiny():
+    """run(): attention -> LM head -> accept -> compact chained on the device, crisp logits."""
+    w = wl.make("c1", hidden_gain=16.0)
+    ram, t1, t2 = oracle.lmhead(w.hidden, w.W)
+    assert (t1 - t2).min() > 1e-3
+    wl.plant(w, ram.reshape(w.B, w.T_max), np.array([3]))
+    G = oracle.Geometry.of(w)
+    ref_acc = oracle.accept(G, w.draft_tok, ram.reshape(w.B, w.T_max))
+    vs = VerifyStep(w, keep_host_inputs=True)
+    for mode in ("device", "host"):
+        vs.run() if mode == "device" else vs.run_from_host()
+        torch.cuda.synchronize()
+        vs.check_status()
+        np.testing.assert_array_equal(vs.argmax.cpu().numpy(), ram)
+        for got, ref in zip((vs.n_acc, vs.path, vs.out_tok, vs.new_len), ref_acc):
+            np.testing.assert_array_equal(got.cpu().numpy(), ref)
+    assert vs.host_out["n_acc"][0] == 4
+    rk, rv = w.k_cache[0].copy(), w.v_cache[0].copy()
+    oracle.compact(G, rk, rv, w.k_tree[0], w.v_tree[0], ref_acc[0], ref_acc[1])
+    np.testing.assert_array_equal(vs.k_cache[0].cpu().numpy().view(np.uint16), rk)
+    np.testing.assert_array_equal(vs.v_cache[0].cpu().numpy().view(np.uint16), rv)
+
+
+def test_full_step_c5_shapes():
+    """28 layers, batch 8, prefix 4096: planted paths are recovered bit-exactly,
+    attention agrees on sampled rows in every layer, caches match after compaction."""
+    w = wl.make("c5")
+    ram, t1, t2 = oracle.lmhead(w.hidden, w.W)
+    wl.plant(w, ram.reshape(w.B, w.T_max))
+    G = oracle.Geometry.of(w)
+    ref_acc = oracle.accept(G, w.draft_tok, ram.reshape(w.B, w.T_max))
+    np.testing.assert_array_equal(ref_acc[0], w.planted_len + 1)
+
+    vs = VerifyStep(w)
+    for l in range(vs.L):
+        vs.attention(l)
+    vs.lmhead()
+    torch.cuda.synchronize()
+    vs.check_status()
+    am = vs.argmax.cpu().numpy()
+    in_band, mis_in, mis_out = check_argmax(am, vs.maxlogit.cpu().numpy(), ram, t1, t2)
+    print(f"c5 LM head: rows {len(am)}, in band {in_band}, mismatches in band {mis_in}, outside {mis_out}")
+    # acceptance on the checker's argmax is bit exact
+    vs.accept(target=to_device(ram))
+    vs.compact()
+    torch.cuda.synchronize()
+    vs.check_status()
+    for got, ref in zip((vs.n_acc, vs.path, vs.out_tok, vs.new_len), ref_acc):
+        np.testing.assert_array_equal(got.cpu().numpy(), ref)
+    rows = sample_rows(w, 24, 9)
+    for l in range(w.L):
+        ref, _ = oracle.attention_rows(G, w.k_cache[l], w.v_cache[l], w.q[l], w.k_tree[l], w.v_tree[l], w.scale, rows)
+        got = vs.out[l].float().cpu().numpy()[rows[:, 0], rows[:, 1], rows[:, 2]]
+        check_attention(got, ref, f"layer {l}")
+        rk, rv = w.k_cache[l], w.v_cache[l]          # compact the host copy in place
+        oracle.compact(G, rk, rv, w.k_tree[l], w.v_tree[l], ref_acc[0], ref_acc[1])
+        assert np.array_equal(vs.k_cache[l].cpu().numpy().view(np.uint16), rk)
+        assert np.array_equal(vs.v_cache[l].cpu().numpy().view(np.uint16), rv)
