@@ -32,8 +32,10 @@ static AttnPlan make_plan(const sd_batch& bt) {
     return p;
 }
 
-// workspace: per (b, kvh, chunk): m[rows], l[rows], acc[rows][D]   (fp32)
-__host__ __device__ static inline size_t partial_stride(const AttnPlan& p) { return (size_t)p.rows * (kD + 2); }
+// workspace: per (b, kvh, chunk): m[rows4], l[rows4], acc[rows][D] (fp32), rows4 = rows rounded
+// up to a multiple of 4 so that every acc row stays 16-byte aligned
+__host__ __device__ static inline size_t rows4(const AttnPlan& p) { return (size_t)((p.rows + 3) & ~3); }
+__host__ __device__ static inline size_t partial_stride(const AttnPlan& p) { return 2 * rows4(p) + (size_t)p.rows * kD; }
 
 size_t attention_workspace_bytes(const sd_batch& bt) {
     AttnPlan p = make_plan(bt);
@@ -182,8 +184,8 @@ attn_partial_kernel(sd_batch bt, sd_kv_layer cache, const uint16_t* __restrict__
     if (row < plan.rows) {
         float* base = ws + ((size_t)(b * bt.Hkv + kvh) * plan.n_chunks + chunk) * partial_stride(plan);
         base[row] = m;
-        base[plan.rows + row] = l;
-        float4* o = reinterpret_cast<float4*>(base + 2 * (size_t)plan.rows + (size_t)row * kD);
+        base[rows4(plan) + row] = l;
+        float4* o = reinterpret_cast<float4*>(base + 2 * rows4(plan) + (size_t)row * kD);
 #pragma unroll
         for (int d = 0; d < kD; d += 4) o[d / 4] = make_float4(acc[d], acc[d + 1], acc[d + 2], acc[d + 3]);
     }
@@ -219,8 +221,8 @@ attn_merge_kernel(sd_batch bt, const float* __restrict__ ws, AttnPlan plan,
         if (!live) continue;
         const float* pc = base + (size_t)c * partial_stride(plan);
         const float w = exp2f(pc[row] - M);
-        den = fmaf(w, pc[plan.rows + row], den);
-        num = fmaf(w, pc[2 * (size_t)plan.rows + (size_t)row * kD + d], num);
+        den = fmaf(w, pc[rows4(plan) + row], den);
+        num = fmaf(w, pc[2 * rows4(plan) + (size_t)row * kD + d], num);
     }
     out[orow * kD + d] = __float2bfloat16(num / den);
     if (lse && d == 0) lse[orow] = (M + log2f(den)) * 0.6931471805599453f;

@@ -1,137 +1,294 @@
-// LM-head projection with fused arg-max: logits never reach memory.
-// Each CTA computes a (rows x vocab) tile of hidden . W^T, keeps only the
-// per-row (max, lowest index) of its vocabulary slab, and a second kernel
-// reduces the slabs.
+// LM-head projection with fused arg-max on the 5th-generation tensor cores.
+//
+// logits^T = W . hidden^T is computed tile by tile with the vocabulary along
+// the MMA M dimension (TMEM lanes) and the hidden rows along N (TMEM columns):
+// every CTA streams its own slab of W exactly once (TMA, 128-byte swizzle)
+// while the small hidden matrix is re-read from L2.  The accumulator never
+// leaves TMEM: the epilogue warps reduce each column over the 128 vocabulary
+// lanes (max + lowest index) and keep a running best per hidden row; only
+// (max, index) pairs per CTA reach memory, and a tiny kernel merges them.
 #include "common.cuh"
+#include "sm100.cuh"
 
 namespace sdv {
+using namespace sm100;
 
-constexpr int kTM = 64;     // rows per CTA
-constexpr int kTN = 128;    // vocabulary entries per CTA
-constexpr int kTK = 32;     // contraction step
+constexpr int kBM = 128;            // vocabulary rows per tile (MMA M)
+constexpr int kLmThreads = 192;     // warps 0-3 epilogue, warp 4 TMA producer, warp 5 MMA issuer
+constexpr int kMaxCols = 512;       // hidden rows per launch (TMEM columns)
+constexpr int kMaxCtas = 256;
+constexpr int kMaxStages = 8;
+constexpr int kSmemBudget = 227 * 1024 - 2048;
+
+struct LmParams {
+    int rows;          // hidden rows handled by this launch (<= 512)
+    int row0;          // index of the first one
+    int Hd, V;
+    int n_parts;       // MMA instructions along N per k-step (1 or 2)
+    int part_n;        // N of each (multiple of 16, <= 256)
+    int n_pad;         // n_parts * part_n
+    int buf_stride;    // TMEM columns per accumulator buffer
+    int acc_bufs;      // 1 or 2 accumulator buffers
+    int tmem_cols;     // allocation (power of two >= 32)
+    int n_tiles;       // vocabulary tiles
+    int stages;
+    int32_t* part_key; // [gridDim.x][kMaxCols] order-preserving integer image of the max logit
+    int32_t* part_idx; // [gridDim.x][kMaxCols]
+};
 
 size_t lmhead_workspace_bytes(int M, int V) {
-    const size_t slabs = (size_t)(V + kTN - 1) / kTN;
-    return (size_t)M * slabs * (sizeof(float) + sizeof(int32_t));
+    (void)M; (void)V;
+    return (size_t)kMaxCtas * kMaxCols * 2 * sizeof(int32_t);
 }
 
-__device__ __forceinline__ void better(float& v, int& i, float v2, int i2) {
-    if (v2 > v || (v2 == v && i2 < i)) { v = v2; i = i2; }
+// float -> int whose signed order equals the float order (-0 folded onto +0)
+__device__ __forceinline__ int32_t ordered_key(uint32_t bits) {
+    int32_t b = (int32_t)bits;
+    b = (b < 0) ? (b ^ 0x7fffffff) : b;
+    return (b == -1) ? 0 : b;            // -0.0f maps to -1 above; fold it onto +0.0f
+}
+__device__ __forceinline__ float key_to_float(int32_t k) {
+    return __int_as_float(k < 0 ? (k ^ 0x7fffffff) : k);
 }
 
-__global__ void __launch_bounds__(256)
-lmhead_tile_kernel(const uint16_t* __restrict__ hidden, const uint16_t* __restrict__ W,
-                   int M, int Hd, int V, int slabs, float* __restrict__ pmax, int32_t* __restrict__ pidx) {
-    __shared__ __align__(16) float As[kTK][kTM + 4];
-    __shared__ __align__(16) float Bs[kTK][kTN + 4];
-    const int tid = threadIdx.x;
-    const int r0 = blockIdx.x * kTM;
-    const int v0 = blockIdx.y * kTN;
-    const int ty = tid >> 4, tx = tid & 15;       // 16 x 16 threads: 4 rows x 8 vocab entries each
-    float acc[4][8];
-#pragma unroll
-    for (int i = 0; i < 4; ++i)
-#pragma unroll
-        for (int j = 0; j < 8; ++j) acc[i][j] = 0.f;
+template <int BK>
+__global__ void __launch_bounds__(kLmThreads, 1)
+lmhead_umma_kernel(const __grid_constant__ CUtensorMap tmW, const __grid_constant__ CUtensorMap tmH,
+                   const LmParams p, int32_t* status) {
+    constexpr int kSwz = BK * 2;                 // bytes per smem row = swizzle span
+    constexpr int kGroup = 8 * kSwz;             // 8-row swizzle group
+    extern __shared__ uint8_t smem_raw[];
+    uint8_t* smem = reinterpret_cast<uint8_t*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~(uintptr_t)1023);
+    const int a_bytes = kBM * kSwz;
+    const int stage_bytes = a_bytes + p.n_pad * kSwz;
 
-    for (int k0 = 0; k0 < Hd; k0 += kTK) {
-        {   // A tile: 64 rows x 32 k = 256 vectors of 8
-            const int r = tid >> 2, c = tid & 3;
-            uint4 u = make_uint4(0, 0, 0, 0);
-            if (r0 + r < M) u = *reinterpret_cast<const uint4*>(hidden + (size_t)(r0 + r) * Hd + k0 + c * 8);
-            const uint32_t w[4] = {u.x, u.y, u.z, u.w};
-#pragma unroll
-            for (int e = 0; e < 4; ++e) {
-                As[c * 8 + 2 * e][r] = bf16lo(w[e]);
-                As[c * 8 + 2 * e + 1][r] = bf16hi(w[e]);
-            }
-        }
-#pragma unroll
-        for (int it = 0; it < 2; ++it) {   // B tile: 128 vocab x 32 k = 512 vectors
-            const int idx = tid + it * 256;
-            const int r = idx >> 2, c = idx & 3;
-            uint4 u = make_uint4(0, 0, 0, 0);
-            if (v0 + r < V) u = *reinterpret_cast<const uint4*>(W + (size_t)(v0 + r) * Hd + k0 + c * 8);
-            const uint32_t w[4] = {u.x, u.y, u.z, u.w};
-#pragma unroll
-            for (int e = 0; e < 4; ++e) {
-                Bs[c * 8 + 2 * e][r] = bf16lo(w[e]);
-                Bs[c * 8 + 2 * e + 1][r] = bf16hi(w[e]);
-            }
-        }
-        __syncthreads();
-#pragma unroll
-        for (int k = 0; k < kTK; ++k) {
-            const float4 a = *reinterpret_cast<const float4*>(&As[k][ty * 4]);
-            const float4 b0 = *reinterpret_cast<const float4*>(&Bs[k][tx * 8]);
-            const float4 b1 = *reinterpret_cast<const float4*>(&Bs[k][tx * 8 + 4]);
-            const float av[4] = {a.x, a.y, a.z, a.w};
-            const float bv[8] = {b0.x, b0.y, b0.z, b0.w, b1.x, b1.y, b1.z, b1.w};
-#pragma unroll
-            for (int i = 0; i < 4; ++i)
-#pragma unroll
-                for (int j = 0; j < 8; ++j) acc[i][j] = fmaf(av[i], bv[j], acc[i][j]);
-        }
-        __syncthreads();
-    }
-#pragma unroll
-    for (int i = 0; i < 4; ++i) {
-        float bv = -INFINITY;
-        int bi = 0x7fffffff;
-#pragma unroll
-        for (int j = 0; j < 8; ++j) {
-            const int v = v0 + tx * 8 + j;
-            if (v < V) better(bv, bi, acc[i][j], v);
-        }
-#pragma unroll
-        for (int off = 8; off >= 1; off >>= 1) {
-            const float ov = __shfl_xor_sync(0xffffffffu, bv, off);
-            const int oi = __shfl_xor_sync(0xffffffffu, bi, off);
-            better(bv, bi, ov, oi);
-        }
-        const int r = r0 + ty * 4 + i;
-        if (tx == 0 && r < M) {
-            pmax[(size_t)r * slabs + blockIdx.y] = bv;
-            pidx[(size_t)r * slabs + blockIdx.y] = bi;
-        }
-    }
-}
+    __shared__ __align__(8) uint64_t full_bar[kMaxStages];
+    __shared__ __align__(8) uint64_t empty_bar[kMaxStages];
+    __shared__ __align__(8) uint64_t tmem_full[2];
+    __shared__ __align__(8) uint64_t tmem_empty[2];
+    __shared__ uint32_t tmem_base_slot;
+    __shared__ int abort_flag;
 
-// one warp per row
-__global__ void lmhead_reduce_kernel(const float* __restrict__ pmax, const int32_t* __restrict__ pidx,
-                                     int M, int slabs, int32_t* __restrict__ argmax, float* __restrict__ maxlogit) {
-    const int r = blockIdx.x * (blockDim.x >> 5) + (threadIdx.x >> 5);
+    const int warp = threadIdx.x >> 5;
     const int lane = threadIdx.x & 31;
-    if (r >= M) return;
-    float bv = -INFINITY;
-    int bi = 0x7fffffff;
-    for (int s = lane; s < slabs; s += 32) better(bv, bi, pmax[(size_t)r * slabs + s], pidx[(size_t)r * slabs + s]);
-#pragma unroll
-    for (int off = 16; off >= 1; off >>= 1) {
-        const float ov = __shfl_xor_sync(0xffffffffu, bv, off);
-        const int oi = __shfl_xor_sync(0xffffffffu, bi, off);
-        better(bv, bi, ov, oi);
+    const int kblocks = p.Hd / BK;
+    const int my_tiles = (p.n_tiles - (int)blockIdx.x + (int)gridDim.x - 1) / (int)gridDim.x;
+
+    if (threadIdx.x == 0) {
+        abort_flag = 0;
+        for (int s = 0; s < p.stages; ++s) { mbar_init(&full_bar[s], 1); mbar_init(&empty_bar[s], 1); }
+        for (int b = 0; b < 2; ++b) { mbar_init(&tmem_full[b], 1); mbar_init(&tmem_empty[b], 4); }
+        fence_barrier_init();
     }
-    if (lane == 0) {
-        argmax[r] = bi;
-        if (maxlogit) maxlogit[r] = bv;
+    if (warp == 5) {
+        tmem_alloc(&tmem_base_slot, (uint32_t)p.tmem_cols);
+        tmem_relinquish();
+    }
+    if (warp == 4 && lane == 0) { prefetch_tensormap(&tmW); prefetch_tensormap(&tmH); }
+    tc_fence_before_sync();
+    __syncthreads();
+    tc_fence_after_sync();
+    const uint32_t tmem_base = tmem_base_slot;
+
+    if (warp == 4) {
+        // ------------------------------------------------ TMA producer
+        if (lane == 0) {
+            const uint64_t pol_w = policy_evict_first();
+            const uint64_t pol_h = policy_evict_last();
+            int it = 0;
+            bool ok = true;
+            for (int t = 0; t < my_tiles && ok; ++t) {
+                const int v0 = ((int)blockIdx.x + t * (int)gridDim.x) * kBM;
+                for (int kb = 0; kb < kblocks; ++kb, ++it) {
+                    const int s = it % p.stages;
+                    const uint32_t ph = (uint32_t)(it / p.stages) & 1u;
+                    if (!mbar_wait(&empty_bar[s], ph ^ 1u, &abort_flag)) { ok = false; break; }
+                    uint8_t* a = smem + (size_t)s * stage_bytes;
+                    mbar_arrive_expect_tx(&full_bar[s], (uint32_t)stage_bytes);
+                    tma_load_2d(a, &tmW, kb * BK, v0, &full_bar[s], pol_w);
+                    for (int part = 0; part < p.n_parts; ++part)
+                        tma_load_2d(a + a_bytes + (size_t)part * p.part_n * kSwz, &tmH, kb * BK,
+                                    p.row0 + part * p.part_n, &full_bar[s], pol_h);
+                }
+            }
+            if (!ok) {
+                set_status(status, SD_ERR_TIMEOUT);
+                for (int i = 0; i < 1000; ++i) __nanosleep(1000);   // let copies in flight land
+            }
+        }
+    } else if (warp == 5) {
+        // ------------------------------------------------ MMA issuer
+        if (lane == 0) {
+            const uint32_t idesc = make_idesc_bf16(kBM, p.part_n, false, false);
+            int it = 0;
+            bool ok = true;
+            for (int t = 0; t < my_tiles && ok; ++t) {
+                const int buf = t % p.acc_bufs;
+                const uint32_t use = (uint32_t)(t / p.acc_bufs);
+                if (!mbar_wait(&tmem_empty[buf], (use & 1u) ^ 1u, &abort_flag)) { ok = false; break; }
+                tc_fence_after_sync();
+                const uint32_t d0 = tmem_base + (uint32_t)(buf * p.buf_stride);
+                for (int kb = 0; kb < kblocks; ++kb, ++it) {
+                    const int s = it % p.stages;
+                    const uint32_t ph = (uint32_t)(it / p.stages) & 1u;
+                    if (!mbar_wait(&full_bar[s], ph, &abort_flag)) { ok = false; break; }
+                    tc_fence_after_sync();
+                    const uint32_t a_addr = smem_u32(smem + (size_t)s * stage_bytes);
+                    const uint32_t b_addr = a_addr + (uint32_t)a_bytes;
+#pragma unroll
+                    for (int k = 0; k < BK / 16; ++k) {
+                        const uint64_t adesc = make_smem_desc(a_addr + k * 32, 16, kGroup, kSwz);
+                        for (int part = 0; part < p.n_parts; ++part) {
+                            const uint64_t bdesc =
+                                make_smem_desc(b_addr + (uint32_t)(part * p.part_n * kSwz) + k * 32, 16, kGroup, kSwz);
+                            mma_ss(d0 + (uint32_t)(part * p.part_n), adesc, bdesc, idesc, (kb | k) != 0 ? 1u : 0u);
+                        }
+                    }
+                    mma_commit(&empty_bar[s]);            // stage reusable once these MMAs have read it
+                }
+                if (ok) mma_commit(&tmem_full[buf]);       // accumulator complete
+            }
+            if (!ok) set_status(status, SD_ERR_TIMEOUT);
+        }
+    } else {
+        // ------------------------------------------------ epilogue warps 0..3 (TMEM lanes 32*warp ..)
+        int32_t best_key[kMaxCols / 32];
+        int32_t best_idx[kMaxCols / 32];
+#pragma unroll
+        for (int c = 0; c < kMaxCols / 32; ++c) { best_key[c] = INT32_MIN; best_idx[c] = 0x7fffffff; }
+        bool ok = true;
+        for (int t = 0; t < my_tiles && ok; ++t) {
+            const int buf = t % p.acc_bufs;
+            const uint32_t use = (uint32_t)(t / p.acc_bufs);
+            if (!mbar_wait(&tmem_full[buf], use & 1u, &abort_flag)) { ok = false; break; }
+            tc_fence_after_sync();
+            const int v_base = ((int)blockIdx.x + t * (int)gridDim.x) * kBM + warp * 32;
+            const bool v_ok = (v_base + lane) < p.V;
+            const uint32_t taddr = tmem_base + ((uint32_t)(warp * 32) << 16) + (uint32_t)(buf * p.buf_stride);
+#pragma unroll
+            for (int c = 0; c < kMaxCols / 32; ++c) {
+                if (c * 32 < p.n_pad) {
+                    uint32_t r[32];
+                    tmem_ld32(taddr + c * 32, r);
+                    tmem_ld_wait();
+                    int32_t ck = INT32_MIN, ci = 0x7fffffff;
+#pragma unroll
+                    for (int j = 0; j < 32; ++j) {
+                        const int32_t key = v_ok ? ordered_key(r[j]) : INT32_MIN;
+                        const int32_t mx = __reduce_max_sync(0xffffffffu, key);
+                        const uint32_t who = __ballot_sync(0xffffffffu, key == mx);
+                        if (lane == j) { ck = mx; ci = v_base + (__ffs(who) - 1); }
+                    }
+                    if (ck > best_key[c]) { best_key[c] = ck; best_idx[c] = ci; }
+                }
+            }
+            tc_fence_before_sync();
+            __syncwarp();
+            if (lane == 0) mbar_arrive(&tmem_empty[buf]);
+        }
+        // merge the four warps through shared memory (the pipeline stages are idle by now:
+        // the last accumulator was complete, so every copy has landed and every MMA has read it)
+        asm volatile("bar.sync 1, 128;" ::: "memory");
+        int32_t* red_key = reinterpret_cast<int32_t*>(smem);
+        int32_t* red_idx = red_key + 4 * kMaxCols;
+#pragma unroll
+        for (int c = 0; c < kMaxCols / 32; ++c) {
+            red_key[warp * kMaxCols + c * 32 + lane] = best_key[c];
+            red_idx[warp * kMaxCols + c * 32 + lane] = best_idx[c];
+        }
+        asm volatile("bar.sync 1, 128;" ::: "memory");
+        for (int col = threadIdx.x; col < kMaxCols; col += 128) {
+            int32_t k = red_key[col], i = red_idx[col];
+#pragma unroll
+            for (int w = 1; w < 4; ++w) {
+                const int32_t k2 = red_key[w * kMaxCols + col], i2 = red_idx[w * kMaxCols + col];
+                if (k2 > k || (k2 == k && i2 < i)) { k = k2; i = i2; }
+            }
+            p.part_key[(size_t)blockIdx.x * kMaxCols + col] = ok ? k : INT32_MIN;
+            p.part_idx[(size_t)blockIdx.x * kMaxCols + col] = i;
+        }
+    }
+    tc_fence_before_sync();
+    __syncthreads();
+    if (warp == 5) {
+        tc_fence_after_sync();
+        tmem_dealloc(tmem_base, (uint32_t)p.tmem_cols);
     }
 }
+
+// one thread per hidden row: merge the per-CTA candidates (lowest index on ties)
+__global__ void lmhead_merge_kernel(const int32_t* __restrict__ part_key, const int32_t* __restrict__ part_idx,
+                                    int n_ctas, int rows, int row0, int32_t* __restrict__ argmax,
+                                    float* __restrict__ maxlogit) {
+    const int col = blockIdx.x * blockDim.x + threadIdx.x;
+    if (col >= rows) return;
+    int32_t k = INT32_MIN, i = 0x7fffffff;
+    for (int c = 0; c < n_ctas; ++c) {
+        const int32_t k2 = part_key[(size_t)c * kMaxCols + col], i2 = part_idx[(size_t)c * kMaxCols + col];
+        if (k2 > k || (k2 == k && i2 < i)) { k = k2; i = i2; }
+    }
+    argmax[row0 + col] = i;
+    if (maxlogit) maxlogit[row0 + col] = key_to_float(k);
+}
+
+static int round_up(int x, int m) { return (x + m - 1) / m * m; }
 
 sd_status launch_lmhead(const void* hidden, const void* W, int M, int Hd, int V,
                         int32_t* argmax, float* maxlogit, void* ws, size_t ws_bytes,
                         int32_t* dev_status, cudaStream_t st) {
-    (void)dev_status;
     if (ws_bytes < lmhead_workspace_bytes(M, V)) return SD_ERR_WORKSPACE;
-    const int slabs = (V + kTN - 1) / kTN;
-    float* pmax = static_cast<float*>(ws);
-    int32_t* pidx = reinterpret_cast<int32_t*>(pmax + (size_t)M * slabs);
-    dim3 grid((M + kTM - 1) / kTM, slabs);
-    lmhead_tile_kernel<<<grid, 256, 0, st>>>(static_cast<const uint16_t*>(hidden), static_cast<const uint16_t*>(W),
-                                             M, Hd, V, slabs, pmax, pidx);
-    if (cudaGetLastError() != cudaSuccess) return SD_ERR_CUDA;
-    lmhead_reduce_kernel<<<(M + 3) / 4, 128, 0, st>>>(pmax, pidx, M, slabs, argmax, maxlogit);
-    return cuda_ok(cudaGetLastError());
+    int dev = 0, sms = 0;
+    if (cudaGetDevice(&dev) != cudaSuccess ||
+        cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev) != cudaSuccess)
+        return SD_ERR_CUDA;
+
+    const int n_blocks = (M + kMaxCols - 1) / kMaxCols;
+    const int rows_per_block = round_up((M + n_blocks - 1) / n_blocks, 16);
+    for (int rb = 0; rb < n_blocks; ++rb) {
+        LmParams p;
+        p.row0 = rb * rows_per_block;
+        p.rows = (M - p.row0 < rows_per_block) ? (M - p.row0) : rows_per_block;
+        p.Hd = Hd; p.V = V;
+        const int n16 = round_up(p.rows, 16);
+        p.n_parts = (n16 > 256) ? 2 : 1;
+        p.part_n = round_up((n16 + p.n_parts - 1) / p.n_parts, 16);
+        p.n_pad = p.n_parts * p.part_n;
+        p.buf_stride = round_up(p.n_pad, 32);
+        p.acc_bufs = (2 * p.buf_stride <= kMaxCols) ? 2 : 1;
+        int cols = 32;
+        while (cols < p.acc_bufs * p.buf_stride) cols *= 2;
+        p.tmem_cols = cols;
+        p.n_tiles = (V + kBM - 1) / kBM;
+        // contraction step: 64 (128-byte swizzle) while at least four stages fit, else 32
+        const int stage64 = (kBM + p.n_pad) * 128;
+        const int bk = (4 * stage64 <= kSmemBudget) ? 64 : 32;
+        const int stage_bytes = (kBM + p.n_pad) * bk * 2;
+        int stages = kSmemBudget / stage_bytes;
+        if (stages > kMaxStages) stages = kMaxStages;
+        if (stages < 2) return SD_ERR_UNSUPPORTED;
+        p.stages = stages;
+        p.part_key = static_cast<int32_t*>(ws);
+        p.part_idx = p.part_key + (size_t)kMaxCtas * kMaxCols;
+
+        CUtensorMap tmW, tmH;
+        if (!encode_tmap_bf16_2d(&tmW, W, (uint64_t)V, (uint64_t)Hd, (uint64_t)Hd * 2, (uint32_t)bk, kBM, bk * 2))
+            return SD_ERR_CUDA;
+        if (!encode_tmap_bf16_2d(&tmH, hidden, (uint64_t)M, (uint64_t)Hd, (uint64_t)Hd * 2, (uint32_t)bk,
+                                 (uint32_t)p.part_n, bk * 2))
+            return SD_ERR_CUDA;
+        int grid = sms < kMaxCtas ? sms : kMaxCtas;
+        if (grid > p.n_tiles) grid = p.n_tiles;
+        const size_t dyn = (size_t)stages * stage_bytes + 1024;
+        auto kern = (bk == 64) ? lmhead_umma_kernel<64> : lmhead_umma_kernel<32>;
+        if (cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)dyn) != cudaSuccess)
+            return SD_ERR_CUDA;
+        kern<<<grid, kLmThreads, dyn, st>>>(tmW, tmH, p, dev_status);
+        if (cudaGetLastError() != cudaSuccess) return SD_ERR_CUDA;
+        lmhead_merge_kernel<<<(p.rows + 127) / 128, 128, 0, st>>>(p.part_key, p.part_idx, grid, p.rows, p.row0,
+                                                                 argmax, maxlogit);
+        if (cudaGetLastError() != cudaSuccess) return SD_ERR_CUDA;
+    }
+    return SD_OK;
 }
 
 }  // namespace sdv
