@@ -1,199 +1,428 @@
-// Tree-masked GQA attention over a paged prefix cache plus the tree's own KV.
+// Tree-masked GQA attention over a paged prefix cache plus the tree's own KV,
+// on the 5th-generation tensor cores (tcgen05 + TMEM), split-KV.
 //
-// Split-KV flash-decode: the keys of one (sequence, KV head) are cut into
-// chunks; every chunk produces, for each of the T*G query rows that share this
-// KV head, a partial (running max, sum of exponentials, unnormalised output);
-// a merge kernel combines the partials in a fixed order.  The tree's own keys
-// form one extra chunk, masked by the per-node ancestor bitmask.
+// All T*G query rows that share one KV head (node-major: row = node*G + g) are
+// processed against every K/V byte exactly once per 128-row tile: with 60 nodes
+// and 7 grouped heads that is 420 rows per K/V row, which makes the step
+// compute-bound, so both S = Q.K^T and O += P.V run as tcgen05.mma with
+// accumulators in TMEM.
+//
+// One CTA = (sequence, KV head, 128-row tile, key chunk).  Its key tiles are the
+// 64-token cache blocks of the chunk (TMA, 128-byte swizzle, located through the
+// block table) and, for the last chunk, one extra tile holding the tree's own
+// keys, masked per row by the node's ancestor bitmask.  Softmax runs one thread
+// per row straight out of TMEM (no cross-thread reductions); the running maximum
+// is only raised when it grows by more than 2^8, so the accumulator in TMEM is
+// rescaled rarely.  With one chunk the CTA writes the output itself; otherwise it
+// writes (max, sum, unnormalised O) and a small kernel merges the chunks in a
+// fixed order.
 #include "common.cuh"
+#include "sm100.cuh"
 
 namespace sdv {
+using namespace sm100;
 
-constexpr int kRowsPerCta = 128;   // query rows (node, grouped head) per CTA
-constexpr int kKeyTile = 32;       // keys staged in shared memory at a time
-constexpr int kSub = 8;            // keys scored between two rescales
+constexpr int kRowTile = 128;                  // query rows per CTA (MMA M)
+constexpr int kKeyTile = 64;                   // keys per tile = one cache block
+constexpr int kAttThreads = 192;               // warps 0-3 softmax, warp 4 TMA, warp 5 MMA
+constexpr int kSubTile = kKeyTile * 128;       // bytes of a [64][64] bf16 swizzled sub-tile (8 KiB)
+constexpr int kQBytes = 2 * kRowTile * 128;    // Q tile: two D-halves of [128][64] bf16 (32 KiB)
+constexpr int kKVStage = 2 * kSubTile;         // one K (or V) tile: two D-halves (16 KiB)
+constexpr int kStages = 2;
+constexpr int kPBytes = kRowTile * 128;        // P tile [128][64] bf16 (16 KiB)
+constexpr int kAttSmem = kQBytes + 2 * kStages * kKVStage + kPBytes + 256;
+constexpr int kTmemCols = 256;                 // O: 0..127, S buffers: 128..191, 192..255
 constexpr float kLog2e = 1.4426950408889634f;
+constexpr float kRescaleThreshold = 8.0f;      // log2 units
 
 struct AttnPlan {
-    int chunk_keys;      // prefix keys per chunk (multiple of 64)
-    int n_chunks;        // prefix chunks + 1 tree chunk
-    int rows;            // T_max * G
-    int row_blocks;
+    int n_chunks;      // key chunks per sequence (the last one also takes the tree tile)
+    int rows;          // T_max * G
+    int row_tiles;
 };
 
-static AttnPlan make_plan(const sd_batch& bt) {
+static AttnPlan make_plan(const sd_batch& bt, int sms) {
     AttnPlan p;
     const int G = bt.Hq / bt.Hkv;
     p.rows = bt.T_max * G;
-    p.row_blocks = (p.rows + kRowsPerCta - 1) / kRowsPerCta;
-    const int max_keys = bt.max_blocks_per_seq * kBlock;
-    p.chunk_keys = 512;
-    p.n_chunks = (max_keys + p.chunk_keys - 1) / p.chunk_keys + 1;
+    p.row_tiles = (p.rows + kRowTile - 1) / kRowTile;
+    // Pick the chunk count that minimises (waves of CTAs) x (key tiles per CTA + fixed cost),
+    // two CTAs being resident per SM.  Few waves are counted whole; many waves balance out.
+    const int max_tiles = bt.max_blocks_per_seq;
+    const int base = bt.B * bt.Hkv * p.row_tiles;
+    const int slots = 2 * sms;
+    int n = 1;
+    double best = 1e30;
+    for (int c = 1; c <= 64 && c <= max_tiles; ++c) {
+        const double w = (double)base * c / slots;
+        const double waves = (w <= 2.0) ? (double)((base * c + slots - 1) / slots) : w;
+        const double cost = waves * ((max_tiles + c - 1) / c + 3);
+        if (cost < best - 1e-9) { best = cost; n = c; }
+    }
+    p.n_chunks = n;
     return p;
 }
 
-// workspace: per (b, kvh, chunk): m[rows4], l[rows4], acc[rows][D] (fp32), rows4 = rows rounded
-// up to a multiple of 4 so that every acc row stays 16-byte aligned
+// workspace per (b, kvh, chunk): m[rows4], l[rows4], acc[rows][D] (fp32); rows4 = rows rounded up
+// to a multiple of 4 so that every acc row stays 16-byte aligned
 __host__ __device__ static inline size_t rows4(const AttnPlan& p) { return (size_t)((p.rows + 3) & ~3); }
-__host__ __device__ static inline size_t partial_stride(const AttnPlan& p) { return 2 * rows4(p) + (size_t)p.rows * kD; }
+__host__ __device__ static inline size_t partial_stride(const AttnPlan& p) {
+    return 2 * rows4(p) + (size_t)p.rows * kD;
+}
+
+static int sm_count() {
+    static int sms = 0;
+    if (sms == 0) {
+        int dev = 0;
+        if (cudaGetDevice(&dev) != cudaSuccess ||
+            cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev) != cudaSuccess || sms <= 0)
+            sms = 148;
+    }
+    return sms;
+}
 
 size_t attention_workspace_bytes(const sd_batch& bt) {
-    AttnPlan p = make_plan(bt);
+    AttnPlan p = make_plan(bt, sm_count());
+    if (p.n_chunks == 1) return 256;
     return (size_t)bt.B * bt.Hkv * p.n_chunks * partial_stride(p) * sizeof(float);
 }
 
-// One thread per query row; K/V tiles are staged in shared memory as fp32 and
-// read by all threads at the same address (broadcast).
-__global__ void __launch_bounds__(kRowsPerCta)
-attn_partial_kernel(sd_batch bt, sd_kv_layer cache, const uint16_t* __restrict__ q,
-                    const uint16_t* __restrict__ kt, const uint16_t* __restrict__ vt,
-                    float scale_log2, float* __restrict__ ws, AttnPlan plan, int32_t* status) {
-    __shared__ __align__(16) float Ks[kKeyTile][kD];
-    __shared__ __align__(16) float Vs[kKeyTile][kD];
-    extern __shared__ __align__(16) float Qs[];          // [kD][kRowsPerCta]  (transposed)
+struct AttnMaps {
+    CUtensorMap k_cache, v_cache;   // 2-D [num_blocks*Hkv*64][128], box 64 x 64
+    CUtensorMap k_tree, v_tree;     // 3-D (128, Hkv, B*T_max), box 64 x 1 x 64
+};
 
+__global__ void __launch_bounds__(kAttThreads, 2)
+attn_umma_kernel(const __grid_constant__ AttnMaps maps, const sd_batch bt, const int num_blocks,
+                 const uint16_t* __restrict__ q, const float scale_log2, const AttnPlan plan,
+                 float* __restrict__ ws, __nv_bfloat16* __restrict__ out, float* __restrict__ lse,
+                 int32_t* status) {
+    extern __shared__ __align__(1024) uint8_t smem[];
+    uint8_t* q_smem = smem;
+    uint8_t* k_smem = smem + kQBytes;
+    uint8_t* v_smem = k_smem + kStages * kKVStage;
+    uint8_t* p_smem = v_smem + kStages * kKVStage;
+    uint64_t* bars = reinterpret_cast<uint64_t*>(p_smem + kPBytes);
+    uint64_t* k_full = bars;             // [2] TMA -> MMA
+    uint64_t* k_empty = bars + 2;        // [2] MMA -> TMA
+    uint64_t* v_full = bars + 4;         // [2]
+    uint64_t* v_empty = bars + 6;        // [2]
+    uint64_t* s_full = bars + 8;         // [2] MMA -> softmax
+    uint64_t* s_empty = bars + 10;       // [2] softmax -> MMA
+    uint64_t* p_full = bars + 12;        // softmax -> MMA   (P written, O rescaled)
+    uint64_t* pv_done = bars + 13;       // MMA -> softmax   (P consumed, O updated)
+    uint64_t* q_full = bars + 14;        // softmax -> MMA   (Q staged)
+    uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(bars + 16);
+    int* abort_flag = reinterpret_cast<int*>(bars + 17);
+
+    const int warp = threadIdx.x >> 5;
+    const int lane = threadIdx.x & 31;
     const int chunk = blockIdx.x;
-    const int rb = blockIdx.y;
+    const int rt = blockIdx.y;
     const int b = blockIdx.z / bt.Hkv;
     const int kvh = blockIdx.z % bt.Hkv;
-    const int tid = threadIdx.x;
     const int G = bt.Hq / bt.Hkv;
     const int T = bt.T_max;
-    const int n = min(bt.n_nodes[b], T);
-    const int len = bt.len[b];
-    const bool tree_chunk = (chunk == plan.n_chunks - 1);
+    const int n = min(max(bt.n_nodes[b], 0), T);
+    const int len = max(bt.len[b], 0);
 
-    int key0, key1;
-    if (tree_chunk) { key0 = 0; key1 = n; }
-    else {
-        key0 = chunk * plan.chunk_keys;
-        key1 = min(len, key0 + plan.chunk_keys);
-        if (key1 <= key0) return;                          // whole CTA: nothing to do
+    // key tiles of this CTA: cache blocks [t0, t1) and, for the last chunk, the tree tile
+    const int tiles_total = min((len + kKeyTile - 1) / kKeyTile, bt.max_blocks_per_seq);
+    const int tpc = (tiles_total + plan.n_chunks - 1) / plan.n_chunks;
+    const int t0 = min(chunk * tpc, tiles_total);
+    const int t1 = min(t0 + tpc, tiles_total);
+    const bool has_tree = (chunk == plan.n_chunks - 1);
+    const int nt = (t1 - t0) + (has_tree ? 1 : 0);
+    if (nt == 0) return;                                   // whole CTA, before any barrier or allocation
+    if ((smem_u32(smem) & 1023u) != 0) {                   // swizzled tiles need 1 KiB alignment
+        if (threadIdx.x == 0) set_status(status, SD_ERR_UNSUPPORTED);
+        return;
     }
-    const int row = rb * kRowsPerCta + tid;
-    const int node = row / G;
-    const int g = row - node * G;
-    const bool row_ok = (row < plan.rows) && (node < n);
-    const uint64_t amask = (row_ok && tree_chunk) ? bt.anc_mask[(size_t)b * T + node] : ~0ull;
 
-    // stage q transposed, pre-multiplied by scale * log2(e)
-    {
-        const uint16_t* qr = q + (((size_t)b * T + (row_ok ? node : 0)) * bt.Hq + kvh * G + (row_ok ? g : 0)) * kD;
-        for (int d = 0; d < kD; d += 8) {
-            uint4 u = *reinterpret_cast<const uint4*>(qr + d);
-            const uint32_t w[4] = {u.x, u.y, u.z, u.w};
-#pragma unroll
-            for (int e = 0; e < 4; ++e) {
-                Qs[(d + 2 * e) * kRowsPerCta + tid] = bf16lo(w[e]) * scale_log2;
-                Qs[(d + 2 * e + 1) * kRowsPerCta + tid] = bf16hi(w[e]) * scale_log2;
-            }
+    if (threadIdx.x == 0) {
+        *abort_flag = 0;
+        for (int i = 0; i < 2; ++i) {
+            mbar_init(&k_full[i], 1); mbar_init(&k_empty[i], 1);
+            mbar_init(&v_full[i], 1); mbar_init(&v_empty[i], 1);
+            mbar_init(&s_full[i], 1); mbar_init(&s_empty[i], 4);
         }
+        mbar_init(p_full, 4); mbar_init(pv_done, 1); mbar_init(q_full, 4);
+        fence_barrier_init();
     }
-    float acc[kD];
-#pragma unroll
-    for (int d = 0; d < kD; ++d) acc[d] = 0.f;
-    float m = -INFINITY, l = 0.f;
+    if (warp == 5) {
+        tmem_alloc(tmem_slot, kTmemCols);
+        tmem_relinquish();
+    }
+    if (warp == 4 && lane == 0) {
+        prefetch_tensormap(&maps.k_cache); prefetch_tensormap(&maps.v_cache);
+        prefetch_tensormap(&maps.k_tree); prefetch_tensormap(&maps.v_tree);
+    }
+    tc_fence_before_sync();
+    __syncthreads();
+    tc_fence_after_sync();
+    const uint32_t tmem_base = *tmem_slot;
+    const uint32_t tmem_o = tmem_base;
+    const uint32_t tmem_s = tmem_base + 128;
 
-    for (int t0 = key0; t0 < key1; t0 += kKeyTile) {
-        const int nk = min(kKeyTile, key1 - t0);
-        __syncthreads();
-        // cooperative load of nk keys: 16 vectors of 8 bf16 per row, K and V
-        for (int idx = tid; idx < kKeyTile * 16; idx += kRowsPerCta) {
-            const int kk = idx >> 4, c = idx & 15;
-            uint4 uk = make_uint4(0, 0, 0, 0), uv = uk;
-            if (kk < nk) {
-                const int t = t0 + kk;
-                const uint16_t *kp, *vp;
-                bool ok = true;
-                if (tree_chunk) {
-                    const size_t off = (((size_t)b * T + t) * bt.Hkv + kvh) * kD;
-                    kp = kt + off; vp = vt + off;
-                } else {
-                    const int blk = bt.block_table[(size_t)b * bt.max_blocks_per_seq + t / kBlock];
-                    if (blk < 0 || blk >= cache.num_blocks) { set_status(status, SD_ERR_BOUNDS); ok = false; }
-                    const size_t off = (((size_t)(ok ? blk : 0) * bt.Hkv + kvh) * kBlock + (t % kBlock)) * kD;
-                    kp = static_cast<const uint16_t*>(cache.k) + off;
-                    vp = static_cast<const uint16_t*>(cache.v) + off;
+    if (warp == 4) {
+        // ------------------------------------------------------------ TMA producer
+        const uint64_t pol = policy_evict_first();
+        bool ok = true;
+        int blk_cache = 0;
+        for (int j = 0; j < nt; ++j) {
+            const bool tree = (j >= t1 - t0);
+            if (!tree && (j & 31) == 0) {                  // fetch 32 block-table entries at a time
+                const int t = t0 + j + lane;
+                blk_cache = (t < t1) ? bt.block_table[(size_t)b * bt.max_blocks_per_seq + t] : 0;
+            }
+            int blk = __shfl_sync(0xffffffffu, blk_cache, j & 31);
+            if (!tree && (blk < 0 || blk >= num_blocks)) {
+                if (lane == 0) set_status(status, SD_ERR_BOUNDS);
+                blk = 0;
+            }
+            if (lane == 0 && ok) {
+                const int s = j & 1;
+                const uint32_t ph = (uint32_t)(j >> 1) & 1u;
+                if (!mbar_wait(&k_empty[s], ph ^ 1u, abort_flag)) ok = false;
+                if (ok) {
+                    mbar_arrive_expect_tx(&k_full[s], kKVStage);
+                    uint8_t* dst = k_smem + s * kKVStage;
+                    if (tree) {
+                        tma_load_3d(dst, &maps.k_tree, 0, kvh, b * T, &k_full[s], pol);
+                        tma_load_3d(dst + kSubTile, &maps.k_tree, 64, kvh, b * T, &k_full[s], pol);
+                    } else {
+                        const int y = (blk * bt.Hkv + kvh) * kKeyTile;
+                        tma_load_2d(dst, &maps.k_cache, 0, y, &k_full[s], pol);
+                        tma_load_2d(dst + kSubTile, &maps.k_cache, 64, y, &k_full[s], pol);
+                    }
+                    if (!mbar_wait(&v_empty[s], ph ^ 1u, abort_flag)) ok = false;
                 }
                 if (ok) {
-                    uk = *reinterpret_cast<const uint4*>(kp + c * 8);
-                    uv = *reinterpret_cast<const uint4*>(vp + c * 8);
+                    mbar_arrive_expect_tx(&v_full[s], kKVStage);
+                    uint8_t* dst = v_smem + s * kKVStage;
+                    if (tree) {
+                        tma_load_3d(dst, &maps.v_tree, 0, kvh, b * T, &v_full[s], pol);
+                        tma_load_3d(dst + kSubTile, &maps.v_tree, 64, kvh, b * T, &v_full[s], pol);
+                    } else {
+                        const int y = (blk * bt.Hkv + kvh) * kKeyTile;
+                        tma_load_2d(dst, &maps.v_cache, 0, y, &v_full[s], pol);
+                        tma_load_2d(dst + kSubTile, &maps.v_cache, 64, y, &v_full[s], pol);
+                    }
                 }
             }
-            const uint32_t wk[4] = {uk.x, uk.y, uk.z, uk.w};
-            const uint32_t wv[4] = {uv.x, uv.y, uv.z, uv.w};
-#pragma unroll
-            for (int e = 0; e < 4; ++e) {
-                Ks[kk][c * 8 + 2 * e] = bf16lo(wk[e]);
-                Ks[kk][c * 8 + 2 * e + 1] = bf16hi(wk[e]);
-                Vs[kk][c * 8 + 2 * e] = bf16lo(wv[e]);
-                Vs[kk][c * 8 + 2 * e + 1] = bf16hi(wv[e]);
-            }
+            __syncwarp();
         }
-        __syncthreads();
-        for (int s0 = 0; s0 < nk; s0 += kSub) {
-            float s[kSub];
+        if (lane == 0 && !ok) {
+            set_status(status, SD_ERR_TIMEOUT);
+            for (int i = 0; i < 1000; ++i) __nanosleep(1000);      // let copies in flight land
+        }
+    } else if (warp == 5) {
+        // ------------------------------------------------------------ MMA issuer
+        if (lane == 0) {
+            const uint32_t idesc_s = make_idesc_bf16(kRowTile, kKeyTile, false, false);   // S = Q . K^T
+            const uint32_t idesc_o = make_idesc_bf16(kRowTile, kD, false, true);          // O += P . V
+            const uint32_t q_addr = smem_u32(q_smem);
+            const uint32_t p_addr = smem_u32(p_smem);
+            bool ok = mbar_wait(q_full, 0, abort_flag);
+            auto issue_s = [&](int j) -> bool {
+                const int s = j & 1;
+                const uint32_t ph = (uint32_t)(j >> 1) & 1u;
+                if (!mbar_wait(&s_empty[s], ph ^ 1u, abort_flag)) return false;
+                if (!mbar_wait(&k_full[s], ph, abort_flag)) return false;
+                tc_fence_after_sync();
+                const uint32_t k_addr = smem_u32(k_smem + s * kKVStage);
 #pragma unroll
-            for (int j = 0; j < kSub; ++j) s[j] = 0.f;
-#pragma unroll 4
-            for (int d = 0; d < kD; d += 4) {
-                const float q0 = Qs[(d + 0) * kRowsPerCta + tid];
-                const float q1 = Qs[(d + 1) * kRowsPerCta + tid];
-                const float q2 = Qs[(d + 2) * kRowsPerCta + tid];
-                const float q3 = Qs[(d + 3) * kRowsPerCta + tid];
+                for (int k = 0; k < kD / 16; ++k) {
+                    const uint64_t ad = make_smem_desc(q_addr + (k >> 2) * (kRowTile * 128) + (k & 3) * 32, 16, 1024, 128);
+                    const uint64_t bd = make_smem_desc(k_addr + (k >> 2) * kSubTile + (k & 3) * 32, 16, 1024, 128);
+                    mma_ss(tmem_s + s * kKeyTile, ad, bd, idesc_s, k != 0 ? 1u : 0u);
+                }
+                mma_commit(&k_empty[s]);
+                mma_commit(&s_full[s]);
+                return true;
+            };
+            if (ok) ok = issue_s(0);
+            for (int j = 0; j < nt && ok; ++j) {
+                if (j + 1 < nt) ok = issue_s(j + 1);
+                if (!ok) break;
+                const int s = j & 1;
+                const uint32_t ph = (uint32_t)(j >> 1) & 1u;
+                if (!mbar_wait(p_full, (uint32_t)j & 1u, abort_flag)) { ok = false; break; }
+                if (!mbar_wait(&v_full[s], ph, abort_flag)) { ok = false; break; }
+                tc_fence_after_sync();
+                const uint32_t v_addr = smem_u32(v_smem + s * kKVStage);
 #pragma unroll
-                for (int j = 0; j < kSub; ++j) {
-                    const float4 k4 = *reinterpret_cast<const float4*>(&Ks[s0 + j][d]);
-                    s[j] = fmaf(q0, k4.x, s[j]);
-                    s[j] = fmaf(q1, k4.y, s[j]);
-                    s[j] = fmaf(q2, k4.z, s[j]);
-                    s[j] = fmaf(q3, k4.w, s[j]);
+                for (int k = 0; k < kKeyTile / 16; ++k) {
+                    const uint64_t ad = make_smem_desc(p_addr + k * 32, 16, 1024, 128);
+                    // V is stored [key][d]: N (= d) contiguous; D-halves kSubTile apart, 8-key groups 1 KiB apart
+                    const uint64_t bd = make_smem_desc(v_addr + k * 2048, kSubTile, 1024, 128);
+                    mma_ss(tmem_o, ad, bd, idesc_o, (j | k) != 0 ? 1u : 0u);
+                }
+                mma_commit(&v_empty[s]);
+                mma_commit(pv_done);
+            }
+            if (!ok) set_status(status, SD_ERR_TIMEOUT);
+        }
+    } else {
+        // ------------------------------------------------------------ softmax: one thread per row
+        const int row_in_tile = warp * 32 + lane;
+        const int row = rt * kRowTile + row_in_tile;
+        const int node = row / G;
+        const int g = row - node * G;
+        const bool row_ok = (row < plan.rows) && (node < n);
+        {   // stage this row of Q (zeros for padding rows) in the swizzled K-major layout
+            const uint4* src = reinterpret_cast<const uint4*>(
+                q + (((size_t)b * T + (row_ok ? node : 0)) * bt.Hq + kvh * G + (row_ok ? g : 0)) * kD);
+#pragma unroll
+            for (int c = 0; c < 16; ++c) {
+                uint4 u = row_ok ? __ldg(src + c) : make_uint4(0, 0, 0, 0);
+                uint8_t* dst = q_smem + (c >> 3) * (kRowTile * 128) + row_in_tile * 128 + (((c & 7) ^ (row_in_tile & 7)) << 4);
+                *reinterpret_cast<uint4*>(dst) = u;
+            }
+            fence_proxy_async_smem();
+            __syncwarp();
+            if (lane == 0) mbar_arrive(q_full);
+        }
+        const uint64_t amask = row_ok ? bt.anc_mask[(size_t)b * T + node] : ~0ull;
+        const uint32_t lane_field = (uint32_t)(warp * 32) << 16;
+        float m_used = -INFINITY, l = 0.f;
+        bool ok = true;
+        for (int j = 0; j < nt && ok; ++j) {
+            const int s = j & 1;
+            const uint32_t ph = (uint32_t)(j >> 1) & 1u;
+            if (!mbar_wait(&s_full[s], ph, abort_flag)) { ok = false; break; }
+            tc_fence_after_sync();
+            uint32_t r0[32], r1[32];
+            tmem_ld32(tmem_s + lane_field + s * kKeyTile, r0);
+            tmem_ld32(tmem_s + lane_field + s * kKeyTile + 32, r1);
+            tmem_ld_wait();
+            tc_fence_before_sync();
+            __syncwarp();
+            if (lane == 0) mbar_arrive(&s_empty[s]);
+
+            float sc[64];
+#pragma unroll
+            for (int c = 0; c < 32; ++c) { sc[c] = __uint_as_float(r0[c]) * scale_log2; sc[32 + c] = __uint_as_float(r1[c]) * scale_log2; }
+            const bool tree = (j >= t1 - t0);
+            if (tree) {
+#pragma unroll
+                for (int c = 0; c < 64; ++c) sc[c] = ((amask >> c) & 1ull) ? sc[c] : -INFINITY;
+            } else {
+                const int valid = len - (t0 + j) * kKeyTile;        // keys of this block inside the prefix
+                if (valid < kKeyTile) {
+#pragma unroll
+                    for (int c = 0; c < 64; ++c) sc[c] = (c < valid) ? sc[c] : -INFINITY;
                 }
             }
-            float mnew = m;
+            float mt = sc[0];
 #pragma unroll
-            for (int j = 0; j < kSub; ++j) {
-                const int t = t0 + s0 + j;
-                const bool vis = (s0 + j < nk) && (!tree_chunk || ((amask >> t) & 1ull));
-                s[j] = vis ? s[j] : -INFINITY;
-                mnew = fmaxf(mnew, s[j]);
+            for (int c = 1; c < 64; ++c) mt = fmaxf(mt, sc[c]);
+            // raise the reference maximum only when it would grow by more than the threshold
+            const bool raise = mt > m_used + kRescaleThreshold;      // true on the first tile (m_used = -inf)
+            bool waited_pv = false;
+            if (__any_sync(0xffffffffu, raise)) {
+                if (j > 0) {
+                    if (!mbar_wait(pv_done, (uint32_t)(j - 1) & 1u, abort_flag)) { ok = false; break; }
+                    waited_pv = true;
+                    tc_fence_after_sync();
+                    const float alpha = raise ? exp2f(m_used - mt) : 1.f;
+#pragma unroll
+                    for (int cc = 0; cc < 4; ++cc) {
+                        uint32_t o[32];
+                        tmem_ld32(tmem_o + lane_field + cc * 32, o);
+                        tmem_ld_wait();
+#pragma unroll
+                        for (int c = 0; c < 32; ++c) o[c] = __float_as_uint(__uint_as_float(o[c]) * alpha);
+                        tmem_st32(tmem_o + lane_field + cc * 32, o);
+                    }
+                    tmem_st_wait();
+                    l *= alpha;
+                }
+                if (raise) m_used = mt;
             }
-            if (mnew == -INFINITY) continue;              // nothing visible yet for this row
-            const float alpha = exp2f(m - mnew);          // m = -inf gives 0
-            float p[kSub];
+            uint32_t pk[32];
             float psum = 0.f;
 #pragma unroll
-            for (int j = 0; j < kSub; ++j) { p[j] = exp2f(s[j] - mnew); psum += p[j]; }
-            l = l * alpha + psum;
-            m = mnew;
-#pragma unroll
-            for (int d = 0; d < kD; d += 4) {
-                float4 o = make_float4(acc[d] * alpha, acc[d + 1] * alpha, acc[d + 2] * alpha, acc[d + 3] * alpha);
-#pragma unroll
-                for (int j = 0; j < kSub; ++j) {
-                    const float4 v4 = *reinterpret_cast<const float4*>(&Vs[s0 + j][d]);
-                    o.x = fmaf(p[j], v4.x, o.x);
-                    o.y = fmaf(p[j], v4.y, o.y);
-                    o.z = fmaf(p[j], v4.z, o.z);
-                    o.w = fmaf(p[j], v4.w, o.w);
-                }
-                acc[d] = o.x; acc[d + 1] = o.y; acc[d + 2] = o.z; acc[d + 3] = o.w;
+            for (int c = 0; c < 32; ++c) {
+                const float p0 = exp2f(sc[2 * c] - m_used);
+                const float p1 = exp2f(sc[2 * c + 1] - m_used);
+                psum += p0 + p1;
+                __nv_bfloat162 h = __floats2bfloat162_rn(p0, p1);
+                pk[c] = *reinterpret_cast<uint32_t*>(&h);
             }
+            l += psum;
+            if (j > 0 && !waited_pv) {
+                if (!mbar_wait(pv_done, (uint32_t)(j - 1) & 1u, abort_flag)) { ok = false; break; }
+            }
+#pragma unroll
+            for (int c = 0; c < 8; ++c) {
+                uint8_t* dst = p_smem + row_in_tile * 128 + ((c ^ (row_in_tile & 7)) << 4);
+                *reinterpret_cast<uint4*>(dst) = make_uint4(pk[4 * c], pk[4 * c + 1], pk[4 * c + 2], pk[4 * c + 3]);
+            }
+            fence_proxy_async_smem();
+            tc_fence_before_sync();
+            __syncwarp();
+            if (lane == 0) mbar_arrive(p_full);
+        }
+        // ------------------------------------------------------------ epilogue
+        if (ok) ok = mbar_wait(pv_done, (uint32_t)(nt - 1) & 1u, abort_flag);
+        if (ok) {
+            tc_fence_after_sync();
+            const bool direct = (plan.n_chunks == 1);
+            const int h = kvh * G + g;
+            const size_t orow = ((size_t)b * T + node) * bt.Hq + h;
+            float* part = nullptr;
+            if (!direct)
+                part = ws + ((size_t)(b * bt.Hkv + kvh) * plan.n_chunks + chunk) * partial_stride(plan);
+            const float inv = 1.f / l;
+#pragma unroll
+            for (int cc = 0; cc < 4; ++cc) {
+                uint32_t o[32];
+                tmem_ld32(tmem_o + lane_field + cc * 32, o);
+                tmem_ld_wait();
+                if (row < plan.rows) {
+                    if (direct) {
+                        uint32_t w[16];
+#pragma unroll
+                        for (int c = 0; c < 16; ++c) {
+                            const float a = row_ok ? __uint_as_float(o[2 * c]) * inv : 0.f;
+                            const float bb = row_ok ? __uint_as_float(o[2 * c + 1]) * inv : 0.f;
+                            __nv_bfloat162 hh = __floats2bfloat162_rn(a, bb);
+                            w[c] = *reinterpret_cast<uint32_t*>(&hh);
+                        }
+                        uint4* dst = reinterpret_cast<uint4*>(out + orow * kD + cc * 32);
+#pragma unroll
+                        for (int c = 0; c < 4; ++c) dst[c] = make_uint4(w[4 * c], w[4 * c + 1], w[4 * c + 2], w[4 * c + 3]);
+                    } else {
+                        uint4* dst = reinterpret_cast<uint4*>(part + 2 * rows4(plan) + (size_t)row * kD + cc * 32);
+#pragma unroll
+                        for (int c = 0; c < 8; ++c) dst[c] = make_uint4(o[4 * c], o[4 * c + 1], o[4 * c + 2], o[4 * c + 3]);
+                    }
+                }
+            }
+            if (row < plan.rows) {
+                if (direct) {
+                    if (lse) lse[orow] = row_ok ? (m_used + log2f(l)) * 0.6931471805599453f : 0.f;
+                } else {
+                    part[row] = m_used;
+                    part[rows4(plan) + row] = l;
+                }
+            }
+        } else if (lane == 0) {
+            set_status(status, SD_ERR_TIMEOUT);
         }
     }
-    if (row < plan.rows) {
-        float* base = ws + ((size_t)(b * bt.Hkv + kvh) * plan.n_chunks + chunk) * partial_stride(plan);
-        base[row] = m;
-        base[rows4(plan) + row] = l;
-        float4* o = reinterpret_cast<float4*>(base + 2 * rows4(plan) + (size_t)row * kD);
-#pragma unroll
-        for (int d = 0; d < kD; d += 4) o[d / 4] = make_float4(acc[d], acc[d + 1], acc[d + 2], acc[d + 3]);
+    tc_fence_before_sync();
+    __syncthreads();
+    if (warp == 5) {
+        tc_fence_after_sync();
+        tmem_dealloc(tmem_base, kTmemCols);
     }
 }
 
-// grid (T_max*G rows, Hkv, B), kD threads: thread d merges output column d.
+// grid (T_max*G rows, Hkv, B), kD threads: thread d merges output column d over the chunks.
 __global__ void __launch_bounds__(kD)
-attn_merge_kernel(sd_batch bt, const float* __restrict__ ws, AttnPlan plan,
+attn_merge_kernel(const sd_batch bt, const float* __restrict__ ws, const AttnPlan plan,
                   __nv_bfloat16* __restrict__ out, float* __restrict__ lse) {
     const int row = blockIdx.x, kvh = blockIdx.y, b = blockIdx.z;
     const int d = threadIdx.x;
@@ -202,22 +431,24 @@ attn_merge_kernel(sd_batch bt, const float* __restrict__ ws, AttnPlan plan,
     const int node = row / G, g = row - node * G;
     const int h = kvh * G + g;
     const size_t orow = ((size_t)b * T + node) * bt.Hq + h;
-    const int n = min(bt.n_nodes[b], T);
+    const int n = min(max(bt.n_nodes[b], 0), T);
     if (node >= n) {
         out[orow * kD + d] = __float2bfloat16(0.f);
         if (lse && d == 0) lse[orow] = 0.f;
         return;
     }
-    const int len = bt.len[b];
+    const int len = max(bt.len[b], 0);
+    const int tiles_total = min((len + kKeyTile - 1) / kKeyTile, bt.max_blocks_per_seq);
+    const int tpc = (tiles_total + plan.n_chunks - 1) / plan.n_chunks;
     const float* base = ws + (size_t)(b * bt.Hkv + kvh) * plan.n_chunks * partial_stride(plan);
     float M = -INFINITY;
     for (int c = 0; c < plan.n_chunks; ++c) {
-        const bool live = (c == plan.n_chunks - 1) || (c * plan.chunk_keys < len);
+        const bool live = (c == plan.n_chunks - 1) || (c * tpc < tiles_total);
         if (live) M = fmaxf(M, base[(size_t)c * partial_stride(plan) + row]);
     }
     float num = 0.f, den = 0.f;
     for (int c = 0; c < plan.n_chunks; ++c) {
-        const bool live = (c == plan.n_chunks - 1) || (c * plan.chunk_keys < len);
+        const bool live = (c == plan.n_chunks - 1) || (c * tpc < tiles_total);
         if (!live) continue;
         const float* pc = base + (size_t)c * partial_stride(plan);
         const float w = exp2f(pc[row] - M);
@@ -231,20 +462,33 @@ attn_merge_kernel(sd_batch bt, const float* __restrict__ ws, AttnPlan plan,
 sd_status launch_attention(const sd_batch& bt, const sd_kv_layer& cache, const void* q,
                            const void* kt, const void* vt, float scale, void* out, float* lse,
                            void* ws, size_t ws_bytes, int32_t* dev_status, cudaStream_t st) {
-    AttnPlan plan = make_plan(bt);
+    const AttnPlan plan = make_plan(bt, sm_count());
     if (ws_bytes < attention_workspace_bytes(bt)) return SD_ERR_WORKSPACE;
-    const size_t dyn = (size_t)kD * kRowsPerCta * sizeof(float);
-    if (cudaFuncSetAttribute(attn_partial_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)dyn) != cudaSuccess)
+    AttnMaps maps;
+    const uint64_t cache_rows = (uint64_t)cache.num_blocks * bt.Hkv * kKeyTile;
+    if (!encode_tmap_bf16_2d(&maps.k_cache, cache.k, cache_rows, kD, kD * 2, 64, kKeyTile, 128) ||
+        !encode_tmap_bf16_2d(&maps.v_cache, cache.v, cache_rows, kD, kD * 2, 64, kKeyTile, 128))
         return SD_ERR_CUDA;
-    dim3 grid(plan.n_chunks, plan.row_blocks, bt.B * bt.Hkv);
-    attn_partial_kernel<<<grid, kRowsPerCta, dyn, st>>>(
-        bt, cache, static_cast<const uint16_t*>(q), static_cast<const uint16_t*>(kt),
-        static_cast<const uint16_t*>(vt), scale * kLog2e, static_cast<float*>(ws), plan, dev_status);
+    const uint64_t dims[3] = {(uint64_t)kD, (uint64_t)bt.Hkv, (uint64_t)bt.B * bt.T_max};
+    const uint64_t strides[2] = {(uint64_t)kD * 2, (uint64_t)bt.Hkv * kD * 2};
+    const uint32_t box[3] = {64, 1, kKeyTile};
+    if (!encode_tmap_bf16_3d(&maps.k_tree, kt, dims, strides, box, 128) ||
+        !encode_tmap_bf16_3d(&maps.v_tree, vt, dims, strides, box, 128))
+        return SD_ERR_CUDA;
+    if (cudaFuncSetAttribute(attn_umma_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, kAttSmem) != cudaSuccess)
+        return SD_ERR_CUDA;
+    dim3 grid(plan.n_chunks, plan.row_tiles, bt.B * bt.Hkv);
+    attn_umma_kernel<<<grid, kAttThreads, kAttSmem, st>>>(
+        maps, bt, cache.num_blocks, static_cast<const uint16_t*>(q), scale * kLog2e, plan,
+        static_cast<float*>(ws), static_cast<__nv_bfloat16*>(out), lse, dev_status);
     if (cudaGetLastError() != cudaSuccess) return SD_ERR_CUDA;
-    dim3 mgrid(plan.rows, bt.Hkv, bt.B);
-    attn_merge_kernel<<<mgrid, kD, 0, st>>>(bt, static_cast<const float*>(ws), plan,
-                                            static_cast<__nv_bfloat16*>(out), lse);
-    return cuda_ok(cudaGetLastError());
+    if (plan.n_chunks > 1) {
+        dim3 mgrid(plan.rows, bt.Hkv, bt.B);
+        attn_merge_kernel<<<mgrid, kD, 0, st>>>(bt, static_cast<const float*>(ws), plan,
+                                                static_cast<__nv_bfloat16*>(out), lse);
+        if (cudaGetLastError() != cudaSuccess) return SD_ERR_CUDA;
+    }
+    return SD_OK;
 }
 
 }  // namespace sdv
