@@ -148,6 +148,39 @@ sd_status sd_lmhead_argmax(const void *hidden, const void *W,
                            int32_t *dev_status, void *stream);
 
 /*
+ * sd_lmhead_argmax without any scratch argument.  (The paper has no counterpart
+ * to this call; it exists for the way some programs have to use the library.)
+ *
+ * Who needs it: code that is not allowed to obtain device memory at the point
+ * where it verifies a draft - a decode loop whose memory was budgeted and
+ * carved up once at start-up, a plug-in running inside a server that hands it
+ * a fixed arena, a latency-critical path where cudaMalloc's implicit device
+ * synchronisation is unacceptable.  Such callers cannot size and allocate the
+ * workspace sd_lmhead_argmax asks for, so here the library brings its own: a
+ * fixed 1 MiB table compiled into the library image, resident on every GPU
+ * that loads the library until the process ends.  This call allocates and
+ * frees nothing, on the host or on the device.
+ *
+ * Same arithmetic, arguments and results as sd_lmhead_argmax, with these
+ * differences:
+ *   - M is limited to SD_LMHEAD_STATIC_MAX_ROWS (512) rows per call, the
+ *     number the built-in table holds; larger M returns SD_ERR_UNSUPPORTED and
+ *     launches nothing (call it once per slice of rows instead).
+ *   - The first call on each device looks up the table's device address.
+ *     Make that first call during start-up, before any stream capture begins.
+ *   - All calls on a device share the one table, and it keeps whatever the
+ *     previous call left in it.  No entry needs clearing between calls (each
+ *     call overwrites every entry it later reads), but two calls whose kernels
+ *     overlap on the GPU - different streams, no ordering between them - race
+ *     on it and give wrong answers.  Keep calls on one stream, or order them.
+ */
+#define SD_LMHEAD_STATIC_MAX_ROWS 512
+sd_status sd_lmhead_argmax_static(const void *hidden, const void *W,
+                                  int32_t M, int32_t Hd, int32_t V,
+                                  int32_t *argmax, float *maxlogit,
+                                  int32_t *dev_status, void *stream);
+
+/*
  * Greedy acceptance (Sec. 1 "validated"; Sec. 4.1 reports the average
  * acceptance length this step produces).  Node j >= 1 matches when
  * draft_tok[b][j] == target_argmax[b][parents[b][j]]; a node is valid when

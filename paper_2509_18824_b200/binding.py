@@ -29,7 +29,8 @@ KERNELS_PER_ATTENTION = 2      # split-KV partials + merge
 KERNELS_PER_LMHEAD = 2         # tiles + cross-slab reduce
 
 EXPORTS = ["sd_version", "sd_status_string", "sd_workspace_bytes", "sd_tree_prepare",
-           "sd_verify_attention", "sd_lmhead_argmax", "sd_accept_tree", "sd_compact_kv"]
+           "sd_verify_attention", "sd_lmhead_argmax", "sd_lmhead_argmax_static", "sd_accept_tree",
+           "sd_compact_kv"]
 
 
 class sd_kv_layer(C.Structure):
@@ -62,6 +63,9 @@ def _load() -> C.CDLL:
     lib.sd_lmhead_argmax.restype = C.c_int
     lib.sd_lmhead_argmax.argtypes = [C.c_void_p, C.c_void_p, C.c_int32, C.c_int32, C.c_int32,
                                      C.c_void_p, C.c_void_p, C.c_void_p, C.c_size_t, C.c_void_p, C.c_void_p]
+    lib.sd_lmhead_argmax_static.restype = C.c_int
+    lib.sd_lmhead_argmax_static.argtypes = [C.c_void_p, C.c_void_p, C.c_int32, C.c_int32, C.c_int32,
+                                            C.c_void_p, C.c_void_p, C.c_void_p, C.c_void_p]
     lib.sd_accept_tree.restype = C.c_int
     lib.sd_accept_tree.argtypes = [C.c_void_p] * 9
     lib.sd_compact_kv.restype = C.c_int
@@ -167,6 +171,16 @@ def sd_lmhead_argmax(hidden, W, argmax, maxlogit, workspace, status, stream=None
     _check(lib.sd_lmhead_argmax(_ptr(hidden), _ptr(W), int(M), int(Hd), int(V), _ptr(argmax),
                                 _ptr(maxlogit), _ptr(workspace),
                                 workspace.numel() * workspace.element_size(), _ptr(status), _stream(stream)))
+
+
+def sd_lmhead_argmax_static(hidden, W, argmax, maxlogit, status, stream=None) -> None:
+    """LM-head arg-max using the scratch table built into the library: for callers
+    that may not allocate device memory.  At most 512 rows per call."""
+    M, Hd = hidden.shape
+    V = W.shape[0]
+    assert W.shape[1] == Hd
+    _check(lib.sd_lmhead_argmax_static(_ptr(hidden), _ptr(W), int(M), int(Hd), int(V), _ptr(argmax),
+                                       _ptr(maxlogit), _ptr(status), _stream(stream)))
 
 
 def sd_accept_tree(batch: Batch, draft_tok, target_argmax, n_acc, path, out_tok, new_len,

@@ -291,4 +291,50 @@ sd_status launch_lmhead(const void* hidden, const void* W, int M, int Hd, int V,
     return SD_OK;
 }
 
+
+// ---------------------------------------------------------------------------
+// Variant that needs no caller-provided scratch: the per-CTA candidate table
+// lives in a fixed array inside the library image (1 MiB on every GPU that
+// loads the library, held until the process exits).
+// ---------------------------------------------------------------------------
+constexpr size_t kStaticScratchBytes = (size_t)kMaxCtas * kMaxCols * 2 * sizeof(int32_t);
+static __device__ __align__(256) unsigned char g_lmhead_scratch[kStaticScratchBytes];
+
+constexpr int kMaxDevices = 64;
+static void* g_scratch_addr[kMaxDevices];     // device address of the array, per device ordinal
+
+// The array's name is only a host-side handle here; the device address has to be
+// asked for, once per device, with that device current.
+static sd_status static_scratch(void** ptr) {
+    int dev = 0;
+    if (cudaGetDevice(&dev) != cudaSuccess) return SD_ERR_CUDA;
+    if (dev < 0 || dev >= kMaxDevices) return SD_ERR_UNSUPPORTED;
+    if (!g_scratch_addr[dev]) {
+        void* p = nullptr;
+        if (cudaGetSymbolAddress(&p, g_lmhead_scratch) != cudaSuccess || !p) return SD_ERR_CUDA;
+        g_scratch_addr[dev] = p;
+    }
+    *ptr = g_scratch_addr[dev];
+    return SD_OK;
+}
+
 }  // namespace sdv
+
+extern "C" sd_status sd_lmhead_argmax_static(const void* hidden, const void* W,
+                                             int32_t M, int32_t Hd, int32_t V,
+                                             int32_t* argmax, float* maxlogit,
+                                             int32_t* dev_status, void* stream) {
+    using namespace sdv;
+    if (!hidden || !W || !argmax || !dev_status) return SD_ERR_INVALID_ARG;
+    if (!aligned16(hidden) || !aligned16(W)) return SD_ERR_INVALID_ARG;
+    if (M < 1 || V < 1 || Hd < 1) return SD_ERR_INVALID_ARG;
+    if (Hd % 64 != 0) return SD_ERR_UNSUPPORTED;
+    if (M > SD_LMHEAD_STATIC_MAX_ROWS) return SD_ERR_UNSUPPORTED;   // the built-in table holds one pass of rows
+    void* scratch = nullptr;
+    sd_status s = static_scratch(&scratch);
+    if (s != SD_OK) return s;
+    // Nothing in the table has to start at zero: every entry the merge reads is
+    // written by this call's own CTAs first.
+    return launch_lmhead(hidden, W, M, Hd, V, argmax, maxlogit, scratch, kStaticScratchBytes, dev_status,
+                         static_cast<cudaStream_t>(stream));
+}
