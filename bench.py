@@ -184,6 +184,8 @@ def main():
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
     ap.add_argument("--config", default="c5")
     ap.add_argument("--no-cpu-baseline", action="store_true")
+    ap.add_argument("--layers", type=int, default=0,
+                    help="override the number of layers (small cases for profiler captures only)")
     args = ap.parse_args()
     if args.impl == "reference":
         return run_reference(args)
@@ -202,7 +204,8 @@ def main():
         dist.init_process_group("nccl", device_id=torch.device("cuda", local_rank))
 
     # synthetic batch (each replica its own seed)
-    w = wl.make(args.config, seed=wl.spec(args.config).seed + 1000 * rank)
+    over = {"L": args.layers} if args.layers > 0 else {}
+    w = wl.make(args.config, seed=wl.spec(args.config).seed + 1000 * rank, **over)
     vs = VerifyStep(w, keep_host_inputs=True)
     # planted draft tokens follow the target's arg-max, taken here from the library's own LM head
     vs.lmhead()

@@ -29,11 +29,17 @@ constexpr int kSubTile = kKeyTile * 128;       // bytes of a [64][64] bf16 swizz
 constexpr int kQBytes = 2 * kRowTile * 128;    // Q tile: two D-halves of [128][64] bf16 (32 KiB)
 constexpr int kKVStage = 2 * kSubTile;         // one K (or V) tile: two D-halves (16 KiB)
 constexpr int kStages = 2;
-constexpr int kPBytes = kRowTile * 128;        // P tile [128][64] bf16 (16 KiB)
-constexpr int kAttSmem = kQBytes + 2 * kStages * kKVStage + kPBytes + 256;
-constexpr int kTmemCols = 256;                 // O: 0..127, S buffers: 128..191, 192..255
+constexpr int kAttSmem = kQBytes + 2 * kStages * kKVStage + 256;
+constexpr int kTmemCols = 256;                 // O: 0..127, S/P buffers: 128..191, 192..255
+// P (bf16, two keys per 32-bit column) overwrites the first 32 columns of the S buffer it came from
 constexpr float kLog2e = 1.4426950408889634f;
 constexpr float kRescaleThreshold = 8.0f;      // log2 units
+
+__device__ __forceinline__ float ex2_approx(float x) {
+    float y;
+    asm("ex2.approx.ftz.f32 %0, %1;" : "=f"(y) : "f"(x));
+    return y;
+}
 
 struct AttnPlan {
     int n_chunks;      // key chunks per sequence (the last one also takes the tree tile)
@@ -55,7 +61,7 @@ static AttnPlan make_plan(const sd_batch& bt, int sms) {
     double best = 1e30;
     for (int c = 1; c <= 64 && c <= max_tiles; ++c) {
         const double w = (double)base * c / slots;
-        const double waves = (w <= 2.0) ? (double)((base * c + slots - 1) / slots) : w;
+        const double waves = (w <= 4.0) ? (double)((base * c + slots - 1) / slots) : w;
         const double cost = waves * ((max_tiles + c - 1) / c + 3);
         if (cost < best - 1e-9) { best = cost; n = c; }
     }
@@ -101,16 +107,17 @@ attn_umma_kernel(const __grid_constant__ AttnMaps maps, const sd_batch bt, const
     uint8_t* q_smem = smem;
     uint8_t* k_smem = smem + kQBytes;
     uint8_t* v_smem = k_smem + kStages * kKVStage;
-    uint8_t* p_smem = v_smem + kStages * kKVStage;
-    uint64_t* bars = reinterpret_cast<uint64_t*>(p_smem + kPBytes);
+    uint64_t* bars = reinterpret_cast<uint64_t*>(v_smem + kStages * kKVStage);
     uint64_t* k_full = bars;             // [2] TMA -> MMA
     uint64_t* k_empty = bars + 2;        // [2] MMA -> TMA
     uint64_t* v_full = bars + 4;         // [2]
     uint64_t* v_empty = bars + 6;        // [2]
     uint64_t* s_full = bars + 8;         // [2] MMA -> softmax
-    uint64_t* s_empty = bars + 10;       // [2] softmax -> MMA
-    uint64_t* p_full = bars + 12;        // softmax -> MMA   (P written, O rescaled)
-    uint64_t* pv_done = bars + 13;       // MMA -> softmax   (P consumed, O updated)
+    uint64_t* p_full = bars + 10;        // [2] softmax -> MMA (P written into S buffer j&1, O rescaled);
+                                         //     one barrier per buffer so that a warp running a tile ahead
+                                         //     cannot complete the previous tile's phase
+    uint64_t* pv_done = bars + 13;       // MMA -> softmax   (O updated by tile j; phase j)
+    uint64_t* o_full = bars + 12;        // MMA -> softmax   (single use: every MMA of the CTA has completed)
     uint64_t* q_full = bars + 14;        // softmax -> MMA   (Q staged)
     uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(bars + 16);
     int* abort_flag = reinterpret_cast<int*>(bars + 17);
@@ -144,9 +151,9 @@ attn_umma_kernel(const __grid_constant__ AttnMaps maps, const sd_batch bt, const
         for (int i = 0; i < 2; ++i) {
             mbar_init(&k_full[i], 1); mbar_init(&k_empty[i], 1);
             mbar_init(&v_full[i], 1); mbar_init(&v_empty[i], 1);
-            mbar_init(&s_full[i], 1); mbar_init(&s_empty[i], 4);
+            mbar_init(&s_full[i], 1); mbar_init(&p_full[i], 4);
         }
-        mbar_init(p_full, 4); mbar_init(pv_done, 1); mbar_init(q_full, 4);
+        mbar_init(pv_done, 1); mbar_init(q_full, 4); mbar_init(o_full, 1);
         fence_barrier_init();
     }
     if (warp == 5) {
@@ -222,12 +229,10 @@ attn_umma_kernel(const __grid_constant__ AttnMaps maps, const sd_batch bt, const
             const uint32_t idesc_s = make_idesc_bf16(kRowTile, kKeyTile, false, false);   // S = Q . K^T
             const uint32_t idesc_o = make_idesc_bf16(kRowTile, kD, false, true);          // O += P . V
             const uint32_t q_addr = smem_u32(q_smem);
-            const uint32_t p_addr = smem_u32(p_smem);
             bool ok = mbar_wait(q_full, 0, abort_flag);
             auto issue_s = [&](int j) -> bool {
                 const int s = j & 1;
                 const uint32_t ph = (uint32_t)(j >> 1) & 1u;
-                if (!mbar_wait(&s_empty[s], ph ^ 1u, abort_flag)) return false;
                 if (!mbar_wait(&k_full[s], ph, abort_flag)) return false;
                 tc_fence_after_sync();
                 const uint32_t k_addr = smem_u32(k_smem + s * kKVStage);
@@ -247,20 +252,21 @@ attn_umma_kernel(const __grid_constant__ AttnMaps maps, const sd_batch bt, const
                 if (!ok) break;
                 const int s = j & 1;
                 const uint32_t ph = (uint32_t)(j >> 1) & 1u;
-                if (!mbar_wait(p_full, (uint32_t)j & 1u, abort_flag)) { ok = false; break; }
+                if (!mbar_wait(&p_full[s], ph, abort_flag)) { ok = false; break; }
                 if (!mbar_wait(&v_full[s], ph, abort_flag)) { ok = false; break; }
                 tc_fence_after_sync();
                 const uint32_t v_addr = smem_u32(v_smem + s * kKVStage);
 #pragma unroll
                 for (int k = 0; k < kKeyTile / 16; ++k) {
-                    const uint64_t ad = make_smem_desc(p_addr + k * 32, 16, 1024, 128);
                     // V is stored [key][d]: N (= d) contiguous; D-halves kSubTile apart, 8-key groups 1 KiB apart
                     const uint64_t bd = make_smem_desc(v_addr + k * 2048, kSubTile, 1024, 128);
-                    mma_ss(tmem_o, ad, bd, idesc_o, (j | k) != 0 ? 1u : 0u);
+                    // P comes straight from TMEM: 16 keys = 8 packed columns per MMA
+                    mma_ts(tmem_o, tmem_s + s * kKeyTile + k * 8, bd, idesc_o, (j | k) != 0 ? 1u : 0u);
                 }
                 mma_commit(&v_empty[s]);
                 mma_commit(pv_done);
             }
+            if (ok) mma_commit(o_full);
             if (!ok) set_status(status, SD_ERR_TIMEOUT);
         }
     } else {
@@ -296,13 +302,11 @@ attn_umma_kernel(const __grid_constant__ AttnMaps maps, const sd_batch bt, const
             tmem_ld32(tmem_s + lane_field + s * kKeyTile, r0);
             tmem_ld32(tmem_s + lane_field + s * kKeyTile + 32, r1);
             tmem_ld_wait();
-            tc_fence_before_sync();
-            __syncwarp();
-            if (lane == 0) mbar_arrive(&s_empty[s]);
 
+            // raw scores stay unscaled; scale * log2(e) is folded into the exponent's FMA
             float sc[64];
 #pragma unroll
-            for (int c = 0; c < 32; ++c) { sc[c] = __uint_as_float(r0[c]) * scale_log2; sc[32 + c] = __uint_as_float(r1[c]) * scale_log2; }
+            for (int c = 0; c < 32; ++c) { sc[c] = __uint_as_float(r0[c]); sc[32 + c] = __uint_as_float(r1[c]); }
             const bool tree = (j >= t1 - t0);
             if (tree) {
 #pragma unroll
@@ -314,16 +318,18 @@ attn_umma_kernel(const __grid_constant__ AttnMaps maps, const sd_batch bt, const
                     for (int c = 0; c < 64; ++c) sc[c] = (c < valid) ? sc[c] : -INFINITY;
                 }
             }
-            float mt = sc[0];
+            float mx[4] = {sc[0], sc[1], sc[2], sc[3]};
 #pragma unroll
-            for (int c = 1; c < 64; ++c) mt = fmaxf(mt, sc[c]);
+            for (int c = 4; c < 64; c += 4) {
+                mx[0] = fmaxf(mx[0], sc[c]); mx[1] = fmaxf(mx[1], sc[c + 1]);
+                mx[2] = fmaxf(mx[2], sc[c + 2]); mx[3] = fmaxf(mx[3], sc[c + 3]);
+            }
+            const float mt = fmaxf(fmaxf(mx[0], mx[1]), fmaxf(mx[2], mx[3])) * scale_log2;   // scale > 0
             // raise the reference maximum only when it would grow by more than the threshold
             const bool raise = mt > m_used + kRescaleThreshold;      // true on the first tile (m_used = -inf)
-            bool waited_pv = false;
-            if (__any_sync(0xffffffffu, raise)) {
+                        if (__any_sync(0xffffffffu, raise)) {
                 if (j > 0) {
                     if (!mbar_wait(pv_done, (uint32_t)(j - 1) & 1u, abort_flag)) { ok = false; break; }
-                    waited_pv = true;
                     tc_fence_after_sync();
                     const float alpha = raise ? exp2f(m_used - mt) : 1.f;
 #pragma unroll
@@ -341,31 +347,28 @@ attn_umma_kernel(const __grid_constant__ AttnMaps maps, const sd_batch bt, const
                 if (raise) m_used = mt;
             }
             uint32_t pk[32];
-            float psum = 0.f;
+            float ps[4] = {0.f, 0.f, 0.f, 0.f};
+            const float neg_m = -m_used;
 #pragma unroll
             for (int c = 0; c < 32; ++c) {
-                const float p0 = exp2f(sc[2 * c] - m_used);
-                const float p1 = exp2f(sc[2 * c + 1] - m_used);
-                psum += p0 + p1;
+                const float p0 = ex2_approx(fmaf(sc[2 * c], scale_log2, neg_m));
+                const float p1 = ex2_approx(fmaf(sc[2 * c + 1], scale_log2, neg_m));
+                ps[c & 3] += p0 + p1;
                 __nv_bfloat162 h = __floats2bfloat162_rn(p0, p1);
                 pk[c] = *reinterpret_cast<uint32_t*>(&h);
             }
+            const float psum = (ps[0] + ps[1]) + (ps[2] + ps[3]);
             l += psum;
-            if (j > 0 && !waited_pv) {
-                if (!mbar_wait(pv_done, (uint32_t)(j - 1) & 1u, abort_flag)) { ok = false; break; }
-            }
-#pragma unroll
-            for (int c = 0; c < 8; ++c) {
-                uint8_t* dst = p_smem + row_in_tile * 128 + ((c ^ (row_in_tile & 7)) << 4);
-                *reinterpret_cast<uint4*>(dst) = make_uint4(pk[4 * c], pk[4 * c + 1], pk[4 * c + 2], pk[4 * c + 3]);
-            }
-            fence_proxy_async_smem();
+            // P replaces the S columns this thread has just consumed (its own TMEM lane)
+            tmem_st32(tmem_s + lane_field + s * kKeyTile, pk);
+            tmem_st_wait();
             tc_fence_before_sync();
             __syncwarp();
-            if (lane == 0) mbar_arrive(p_full);
+            if (lane == 0) mbar_arrive(&p_full[s]);
         }
         // ------------------------------------------------------------ epilogue
-        if (ok) ok = mbar_wait(pv_done, (uint32_t)(nt - 1) & 1u, abort_flag);
+        // (a parity wait on pv_done would be ambiguous here: the softmax may be two phases ahead of it)
+        if (ok) ok = mbar_wait(o_full, 0, abort_flag);
         if (ok) {
             tc_fence_after_sync();
             const bool direct = (plan.n_chunks == 1);
@@ -420,43 +423,61 @@ attn_umma_kernel(const __grid_constant__ AttnMaps maps, const sd_batch bt, const
     }
 }
 
-// grid (T_max*G rows, Hkv, B), kD threads: thread d merges output column d over the chunks.
-__global__ void __launch_bounds__(kD)
+// grid (ceil(rows / 8), Hkv, B), 128 threads: 16 threads per row, 8 output columns each.
+constexpr int kMergeRows = 8;
+__global__ void __launch_bounds__(128)
 attn_merge_kernel(const sd_batch bt, const float* __restrict__ ws, const AttnPlan plan,
                   __nv_bfloat16* __restrict__ out, float* __restrict__ lse) {
-    const int row = blockIdx.x, kvh = blockIdx.y, b = blockIdx.z;
-    const int d = threadIdx.x;
+    const int row = blockIdx.x * kMergeRows + (threadIdx.x >> 4);
+    const int c8 = threadIdx.x & 15;
+    const int kvh = blockIdx.y, b = blockIdx.z;
+    if (row >= plan.rows) return;
     const int G = bt.Hq / bt.Hkv;
     const int T = bt.T_max;
     const int node = row / G, g = row - node * G;
     const int h = kvh * G + g;
     const size_t orow = ((size_t)b * T + node) * bt.Hq + h;
+    uint4* dst = reinterpret_cast<uint4*>(out + orow * kD + c8 * 8);
     const int n = min(max(bt.n_nodes[b], 0), T);
     if (node >= n) {
-        out[orow * kD + d] = __float2bfloat16(0.f);
-        if (lse && d == 0) lse[orow] = 0.f;
+        *dst = make_uint4(0, 0, 0, 0);
+        if (lse && c8 == 0) lse[orow] = 0.f;
         return;
     }
     const int len = max(bt.len[b], 0);
     const int tiles_total = min((len + kKeyTile - 1) / kKeyTile, bt.max_blocks_per_seq);
     const int tpc = (tiles_total + plan.n_chunks - 1) / plan.n_chunks;
-    const float* base = ws + (size_t)(b * bt.Hkv + kvh) * plan.n_chunks * partial_stride(plan);
+    const size_t stride = partial_stride(plan);
+    const float* base = ws + (size_t)(b * bt.Hkv + kvh) * plan.n_chunks * stride;
     float M = -INFINITY;
     for (int c = 0; c < plan.n_chunks; ++c) {
         const bool live = (c == plan.n_chunks - 1) || (c * tpc < tiles_total);
-        if (live) M = fmaxf(M, base[(size_t)c * partial_stride(plan) + row]);
+        if (live) M = fmaxf(M, base[(size_t)c * stride + row]);
     }
-    float num = 0.f, den = 0.f;
+    float num[8] = {0.f, 0.f, 0.f, 0.f, 0.f, 0.f, 0.f, 0.f};
+    float den = 0.f;
     for (int c = 0; c < plan.n_chunks; ++c) {
         const bool live = (c == plan.n_chunks - 1) || (c * tpc < tiles_total);
         if (!live) continue;
-        const float* pc = base + (size_t)c * partial_stride(plan);
+        const float* pc = base + (size_t)c * stride;
         const float w = exp2f(pc[row] - M);
         den = fmaf(w, pc[rows4(plan) + row], den);
-        num = fmaf(w, pc[2 * rows4(plan) + (size_t)row * kD + d], num);
+        const float4* o = reinterpret_cast<const float4*>(pc + 2 * rows4(plan) + (size_t)row * kD + c8 * 8);
+        const float4 a0 = o[0], a1 = o[1];
+        num[0] = fmaf(w, a0.x, num[0]); num[1] = fmaf(w, a0.y, num[1]);
+        num[2] = fmaf(w, a0.z, num[2]); num[3] = fmaf(w, a0.w, num[3]);
+        num[4] = fmaf(w, a1.x, num[4]); num[5] = fmaf(w, a1.y, num[5]);
+        num[6] = fmaf(w, a1.z, num[6]); num[7] = fmaf(w, a1.w, num[7]);
     }
-    out[orow * kD + d] = __float2bfloat16(num / den);
-    if (lse && d == 0) lse[orow] = (M + log2f(den)) * 0.6931471805599453f;
+    const float inv = 1.f / den;
+    uint32_t wd[4];
+#pragma unroll
+    for (int i = 0; i < 4; ++i) {
+        __nv_bfloat162 hh = __floats2bfloat162_rn(num[2 * i] * inv, num[2 * i + 1] * inv);
+        wd[i] = *reinterpret_cast<uint32_t*>(&hh);
+    }
+    *dst = make_uint4(wd[0], wd[1], wd[2], wd[3]);
+    if (lse && c8 == 0) lse[orow] = (M + log2f(den)) * 0.6931471805599453f;
 }
 
 sd_status launch_attention(const sd_batch& bt, const sd_kv_layer& cache, const void* q,
@@ -483,8 +504,8 @@ sd_status launch_attention(const sd_batch& bt, const sd_kv_layer& cache, const v
         static_cast<float*>(ws), static_cast<__nv_bfloat16*>(out), lse, dev_status);
     if (cudaGetLastError() != cudaSuccess) return SD_ERR_CUDA;
     if (plan.n_chunks > 1) {
-        dim3 mgrid(plan.rows, bt.Hkv, bt.B);
-        attn_merge_kernel<<<mgrid, kD, 0, st>>>(bt, static_cast<const float*>(ws), plan,
+        dim3 mgrid((plan.rows + kMergeRows - 1) / kMergeRows, bt.Hkv, bt.B);
+        attn_merge_kernel<<<mgrid, 128, 0, st>>>(bt, static_cast<const float*>(ws), plan,
                                                 static_cast<__nv_bfloat16*>(out), lse);
         if (cudaGetLastError() != cudaSuccess) return SD_ERR_CUDA;
     }

@@ -150,6 +150,24 @@ def test_attention_configs_full_compare(cfg, gain):
     np.testing.assert_allclose(lse, rlse, rtol=2e-3, atol=2e-3)
 
 
+def test_attention_is_deterministic_run_to_run():
+    """Many short CTAs (17 key chunks of two tiles): repeated runs must give identical bits,
+    which a lost synchronisation between the MMA, softmax and epilogue roles would not."""
+    w = wl.make("c2", lmhead=False, q_gain=45.0)
+    ref, _ = oracle.attention(oracle.Geometry.of(w), w.k_cache[0], w.v_cache[0], w.q[0], w.k_tree[0],
+                              w.v_tree[0], w.scale)
+    first = None
+    for rep in range(6):
+        out, lse, status = gpu_attention(w, layer=0)
+        assert status == 0
+        check_attention(out, ref, f"run {rep}")
+        if first is None:
+            first = (out.copy(), lse.copy())
+        else:
+            np.testing.assert_array_equal(out, first[0])
+            np.testing.assert_array_equal(lse, first[1])
+
+
 def sample_rows(w, n, seed):
     g = np.random.default_rng(seed)
     rows = np.stack([g.integers(0, w.B, n), g.integers(0, w.T_max, n), g.integers(0, w.Hq, n)], 1).astype(np.int32)
