@@ -25,7 +25,7 @@ SD_ERR_TIMEOUT = -6
 SD_ERR_BOUNDS = -7
 
 # kernel launches behind one call (kept in step with the kernels; used for launch accounting)
-KERNELS_PER_ATTENTION = 2      # split-KV partials + merge
+KERNELS_PER_ATTENTION = 1      # split-KV chunks merge inside the kernel (thread-block cluster)
 KERNELS_PER_LMHEAD = 2         # tiles + cross-slab reduce
 
 EXPORTS = ["sd_version", "sd_status_string", "sd_workspace_bytes", "sd_tree_prepare",

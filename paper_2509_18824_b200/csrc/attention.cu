@@ -25,15 +25,18 @@ using namespace sm100;
 constexpr int kRowTile = 128;                  // query rows per CTA (MMA M)
 constexpr int kKeyTile = 64;                   // keys per tile = one cache block
 constexpr int kAttThreads = 192;               // warps 0-3 softmax, warp 4 TMA, warp 5 MMA
+constexpr int kTmaWarp = 4, kMmaWarp = 5;
 constexpr int kSubTile = kKeyTile * 128;       // bytes of a [64][64] bf16 swizzled sub-tile (8 KiB)
 constexpr int kQBytes = 2 * kRowTile * 128;    // Q tile: two D-halves of [128][64] bf16 (32 KiB)
 constexpr int kKVStage = 2 * kSubTile;         // one K (or V) tile: two D-halves (16 KiB)
-constexpr int kStages = 2;
-constexpr int kAttSmem = kQBytes + 2 * kStages * kKVStage + 256;
+constexpr int kKStages = 3;                    // K tiles are consumed a tile ahead of V
+constexpr int kVStages = 2;
+constexpr int kAttSmem = kQBytes + (kKStages + kVStages) * kKVStage + 256;
 constexpr int kTmemCols = 256;                 // O: 0..127, S/P buffers: 128..191, 192..255
 // P (bf16, two keys per 32-bit column) overwrites the first 32 columns of the S buffer it came from
 constexpr float kLog2e = 1.4426950408889634f;
 constexpr float kRescaleThreshold = 8.0f;      // log2 units
+constexpr int kMaxChunks = 8;                  // = portable cluster size
 
 __device__ __forceinline__ float ex2_approx(float x) {
     float y;
@@ -59,7 +62,7 @@ static AttnPlan make_plan(const sd_batch& bt, int sms) {
     const int slots = 2 * sms;
     int n = 1;
     double best = 1e30;
-    for (int c = 1; c <= 64 && c <= max_tiles; ++c) {
+    for (int c = 1; c <= kMaxChunks && c <= max_tiles; c *= 2) {   // 128 rows split evenly over the chunks
         const double w = (double)base * c / slots;
         const double waves = (w <= 4.0) ? (double)((base * c + slots - 1) / slots) : w;
         const double cost = waves * ((max_tiles + c - 1) / c + 3);
@@ -67,13 +70,6 @@ static AttnPlan make_plan(const sd_batch& bt, int sms) {
     }
     p.n_chunks = n;
     return p;
-}
-
-// workspace per (b, kvh, chunk): m[rows4], l[rows4], acc[rows][D] (fp32); rows4 = rows rounded up
-// to a multiple of 4 so that every acc row stays 16-byte aligned
-__host__ __device__ static inline size_t rows4(const AttnPlan& p) { return (size_t)((p.rows + 3) & ~3); }
-__host__ __device__ static inline size_t partial_stride(const AttnPlan& p) {
-    return 2 * rows4(p) + (size_t)p.rows * kD;
 }
 
 static int sm_count() {
@@ -87,40 +83,106 @@ static int sm_count() {
     return sms;
 }
 
-size_t attention_workspace_bytes(const sd_batch& bt) {
-    AttnPlan p = make_plan(bt, sm_count());
-    if (p.n_chunks == 1) return 256;
-    return (size_t)bt.B * bt.Hkv * p.n_chunks * partial_stride(p) * sizeof(float);
-}
+// The chunks of a row tile are merged inside a thread-block cluster, through shared memory:
+// attention needs no global scratch (a nominal size keeps the argument checks uniform).
+size_t attention_workspace_bytes(const sd_batch&) { return 256; }
 
 struct AttnMaps {
     CUtensorMap k_cache, v_cache;   // 2-D [num_blocks*Hkv*64][128], box 64 x 64
     CUtensorMap k_tree, v_tree;     // 3-D (128, Hkv, B*T_max), box 64 x 1 x 64
 };
 
+// Final step of a clustered launch.  Each CTA of the cluster finishes 128 / NCH rows of the tile: a
+// warp takes a few rows at a time, every lane four output columns, and adds up the chunks in chunk
+// order (so the result does not depend on timing).  A row of a parked tile is one contiguous
+// 512-byte line of the owning CTA's shared memory; all loads of a batch of rows are issued before
+// any of them is used, so that their latencies overlap.
+struct MergeCtx {
+    const sd_batch& bt; const AttnPlan& plan; __nv_bfloat16* out; float* lse;
+    uint32_t xo_addr, xs_addr;
+    int chunk, rt, b, kvh, n, tpc, tiles_total, warp, lane;
+};
+
+template <int NCH>
+__device__ __forceinline__ void merge_rows(const MergeCtx& x) {
+    constexpr int kRowsPer = kRowTile / NCH;
+    constexpr int kBatch = 8 / NCH;                 // rows in flight per warp
+    const int G = x.bt.Hq / x.bt.Hkv;
+    for (int i0 = x.warp * kBatch; i0 < kRowsPer; i0 += 4 * kBatch) {
+        float mc[kBatch][NCH], lc[kBatch][NCH];
+        float4 v[kBatch][NCH];
+#pragma unroll
+        for (int u = 0; u < kBatch; ++u) {
+            const int r = x.chunk * kRowsPer + i0 + u;
+#pragma unroll
+            for (int c = 0; c < NCH; ++c) {
+                const bool live = (c == NCH - 1) || (c * x.tpc < x.tiles_total);   // that chunk had key tiles
+                mc[u][c] = -INFINITY; lc[u][c] = 0.f; v[u][c] = make_float4(0.f, 0.f, 0.f, 0.f);
+                if (live) {
+                    mc[u][c] = ld_dsmem_f32(map_dsmem(x.xs_addr + r * 4, c));
+                    lc[u][c] = ld_dsmem_f32(map_dsmem(x.xs_addr + (kRowTile + r) * 4, c));
+                    v[u][c] = ld_dsmem_v4(map_dsmem(x.xo_addr + (uint32_t)(r * kD + ((x.lane ^ (r & 31)) << 2)) * 4, c));
+                }
+            }
+        }
+#pragma unroll
+        for (int u = 0; u < kBatch; ++u) {
+            const int r = x.chunk * kRowsPer + i0 + u;
+            const int row = x.rt * kRowTile + r;
+            if (row >= x.plan.rows) continue;
+            const int node = row / G;
+            const int g = row - node * G;
+            const size_t orow = ((size_t)x.b * x.bt.T_max + node) * x.bt.Hq + x.kvh * G + g;
+            uint2* dst = reinterpret_cast<uint2*>(x.out + orow * kD + x.lane * 4);
+            if (node >= x.n) {                               // unused node: zero row
+                *dst = make_uint2(0, 0);
+                if (x.lse && x.lane == 0) x.lse[orow] = 0.f;
+                continue;
+            }
+            float M = mc[u][0];
+#pragma unroll
+            for (int c = 1; c < NCH; ++c) M = fmaxf(M, mc[u][c]);
+            float den = 0.f;
+            float4 acc = make_float4(0.f, 0.f, 0.f, 0.f);
+#pragma unroll
+            for (int c = 0; c < NCH; ++c) {
+                const float w = exp2f(mc[u][c] - M);         // 0 for a chunk without tiles (m = -inf)
+                den = fmaf(w, lc[u][c], den);
+                acc.x = fmaf(w, v[u][c].x, acc.x); acc.y = fmaf(w, v[u][c].y, acc.y);
+                acc.z = fmaf(w, v[u][c].z, acc.z); acc.w = fmaf(w, v[u][c].w, acc.w);
+            }
+            const float inv = 1.f / den;
+            __nv_bfloat162 h0 = __floats2bfloat162_rn(acc.x * inv, acc.y * inv);
+            __nv_bfloat162 h1 = __floats2bfloat162_rn(acc.z * inv, acc.w * inv);
+            *dst = make_uint2(*reinterpret_cast<uint32_t*>(&h0), *reinterpret_cast<uint32_t*>(&h1));
+            if (x.lse && x.lane == 0) x.lse[orow] = (M + log2f(den)) * 0.6931471805599453f;
+        }
+    }
+}
+
 __global__ void __launch_bounds__(kAttThreads, 2)
 attn_umma_kernel(const __grid_constant__ AttnMaps maps, const sd_batch bt, const int num_blocks,
                  const uint16_t* __restrict__ q, const float scale_log2, const AttnPlan plan,
-                 float* __restrict__ ws, __nv_bfloat16* __restrict__ out, float* __restrict__ lse,
+                 __nv_bfloat16* __restrict__ out, float* __restrict__ lse,
                  int32_t* status) {
     extern __shared__ __align__(1024) uint8_t smem[];
     uint8_t* q_smem = smem;
     uint8_t* k_smem = smem + kQBytes;
-    uint8_t* v_smem = k_smem + kStages * kKVStage;
-    uint64_t* bars = reinterpret_cast<uint64_t*>(v_smem + kStages * kKVStage);
-    uint64_t* k_full = bars;             // [2] TMA -> MMA
-    uint64_t* k_empty = bars + 2;        // [2] MMA -> TMA
-    uint64_t* v_full = bars + 4;         // [2]
-    uint64_t* v_empty = bars + 6;        // [2]
-    uint64_t* s_full = bars + 8;         // [2] MMA -> softmax
-    uint64_t* p_full = bars + 10;        // [2] softmax -> MMA (P written into S buffer j&1, O rescaled);
-                                         //     one barrier per buffer so that a warp running a tile ahead
+    uint8_t* v_smem = k_smem + kKStages * kKVStage;
+    uint64_t* bars = reinterpret_cast<uint64_t*>(v_smem + kVStages * kKVStage);
+    uint64_t* k_full = bars;             // [3] TMA -> MMA
+    uint64_t* k_empty = bars + 3;        // [3] MMA -> TMA
+    uint64_t* v_full = bars + 6;         // [2]
+    uint64_t* v_empty = bars + 8;        // [2]
+    uint64_t* s_full = bars + 10;        // [2] MMA -> softmax (scores of tile j in buffer j&1)
+    uint64_t* p_full = bars + 12;        // [2] softmax -> MMA (P written into buffer j&1, O rescaled); one
+                                         //     barrier per buffer so that a warp running a tile ahead
                                          //     cannot complete the previous tile's phase
-    uint64_t* pv_done = bars + 13;       // MMA -> softmax   (O updated by tile j; phase j)
-    uint64_t* o_full = bars + 12;        // MMA -> softmax   (single use: every MMA of the CTA has completed)
-    uint64_t* q_full = bars + 14;        // softmax -> MMA   (Q staged)
-    uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(bars + 16);
-    int* abort_flag = reinterpret_cast<int*>(bars + 17);
+    uint64_t* pv_done = bars + 14;       // MMA -> softmax   (O updated by tile j; phase j)
+    uint64_t* o_full = bars + 15;        // MMA -> softmax   (single use: every MMA of the CTA has completed)
+    uint64_t* q_full = bars + 16;        // softmax -> MMA   (Q staged)
+    uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(bars + 17);
+    int* abort_flag = reinterpret_cast<int*>(bars + 18);
 
     const int warp = threadIdx.x >> 5;
     const int lane = threadIdx.x & 31;
@@ -140,90 +202,97 @@ attn_umma_kernel(const __grid_constant__ AttnMaps maps, const sd_batch bt, const
     const int t1 = min(t0 + tpc, tiles_total);
     const bool has_tree = (chunk == plan.n_chunks - 1);
     const int nt = (t1 - t0) + (has_tree ? 1 : 0);
-    if (nt == 0) return;                                   // whole CTA, before any barrier or allocation
-    if ((smem_u32(smem) & 1023u) != 0) {                   // swizzled tiles need 1 KiB alignment
-        if (threadIdx.x == 0) set_status(status, SD_ERR_UNSUPPORTED);
-        return;
-    }
+    const bool aligned = (smem_u32(smem) & 1023u) == 0;    // swizzled tiles need 1 KiB alignment
+    if (!aligned && threadIdx.x == 0) set_status(status, SD_ERR_UNSUPPORTED);
+    // A CTA without key tiles has nothing to compute, but it still takes part in the cluster barriers.
+    const bool active = (nt > 0) && aligned;
+    const bool clustered = (plan.n_chunks > 1);            // cluster = the chunks of one (b, kvh, row tile)
+    float m_used = -INFINITY, l = 0.f;                     // softmax state of this thread's row (warps 0-3)
+    uint32_t tmem_base = 0;
 
+    if (active) {
     if (threadIdx.x == 0) {
         *abort_flag = 0;
-        for (int i = 0; i < 2; ++i) {
-            mbar_init(&k_full[i], 1); mbar_init(&k_empty[i], 1);
-            mbar_init(&v_full[i], 1); mbar_init(&v_empty[i], 1);
-            mbar_init(&s_full[i], 1); mbar_init(&p_full[i], 4);
-        }
+        for (int i = 0; i < kKStages; ++i) { mbar_init(&k_full[i], 1); mbar_init(&k_empty[i], 1); }
+        for (int i = 0; i < kVStages; ++i) { mbar_init(&v_full[i], 1); mbar_init(&v_empty[i], 1); }
+        for (int i = 0; i < 2; ++i) { mbar_init(&s_full[i], 1); mbar_init(&p_full[i], 4); }
         mbar_init(pv_done, 1); mbar_init(q_full, 4); mbar_init(o_full, 1);
         fence_barrier_init();
     }
-    if (warp == 5) {
+    if (warp == kMmaWarp) {
         tmem_alloc(tmem_slot, kTmemCols);
         tmem_relinquish();
     }
-    if (warp == 4 && lane == 0) {
+    if (warp == kTmaWarp && lane == 0) {
         prefetch_tensormap(&maps.k_cache); prefetch_tensormap(&maps.v_cache);
         prefetch_tensormap(&maps.k_tree); prefetch_tensormap(&maps.v_tree);
     }
     tc_fence_before_sync();
     __syncthreads();
     tc_fence_after_sync();
-    const uint32_t tmem_base = *tmem_slot;
+    tmem_base = *tmem_slot;
     const uint32_t tmem_o = tmem_base;
     const uint32_t tmem_s = tmem_base + 128;
 
-    if (warp == 4) {
-        // ------------------------------------------------------------ TMA producer
-        const uint64_t pol = policy_evict_first();
-        bool ok = true;
-        int blk_cache = 0;
-        for (int j = 0; j < nt; ++j) {
-            const bool tree = (j >= t1 - t0);
-            if (!tree && (j & 31) == 0) {                  // fetch 32 block-table entries at a time
-                const int t = t0 + j + lane;
-                blk_cache = (t < t1) ? bt.block_table[(size_t)b * bt.max_blocks_per_seq + t] : 0;
-            }
-            int blk = __shfl_sync(0xffffffffu, blk_cache, j & 31);
-            if (!tree && (blk < 0 || blk >= num_blocks)) {
-                if (lane == 0) set_status(status, SD_ERR_BOUNDS);
-                blk = 0;
-            }
-            if (lane == 0 && ok) {
-                const int s = j & 1;
-                const uint32_t ph = (uint32_t)(j >> 1) & 1u;
-                if (!mbar_wait(&k_empty[s], ph ^ 1u, abort_flag)) ok = false;
-                if (ok) {
-                    mbar_arrive_expect_tx(&k_full[s], kKVStage);
-                    uint8_t* dst = k_smem + s * kKVStage;
-                    if (tree) {
-                        tma_load_3d(dst, &maps.k_tree, 0, kvh, b * T, &k_full[s], pol);
-                        tma_load_3d(dst + kSubTile, &maps.k_tree, 64, kvh, b * T, &k_full[s], pol);
-                    } else {
-                        const int y = (blk * bt.Hkv + kvh) * kKeyTile;
-                        tma_load_2d(dst, &maps.k_cache, 0, y, &k_full[s], pol);
-                        tma_load_2d(dst + kSubTile, &maps.k_cache, 64, y, &k_full[s], pol);
-                    }
-                    if (!mbar_wait(&v_empty[s], ph ^ 1u, abort_flag)) ok = false;
+    if (warp == kTmaWarp) {
+        // ------------------------------------------------------------ TMA producer (one thread)
+        // K and V tiles travel through separate rings and are issued independently, whichever slot
+        // frees first: the next K tile (needed early, for the score MMA issued one tile ahead) must
+        // not queue behind a V slot that is only released when P.V has finished.
+        if (lane == 0) {
+            const uint64_t pol = policy_evict_first();
+            const int32_t* table = bt.block_table + (size_t)b * bt.max_blocks_per_seq;
+            const int n_pref = t1 - t0;
+            int jk = 0, jv = 0;
+            int blk_k = (n_pref > 0) ? __ldg(table + t0) : 0;      // looked up one tile ahead
+            int blk_v = blk_k;
+            bool ok = true;
+            long long t_last = clock64();
+            auto issue = [&](int j, int blk, bool is_v) {
+                const int stages = is_v ? kVStages : kKStages;
+                const int s = j % stages;
+                uint64_t* full = (is_v ? v_full : k_full) + s;
+                uint8_t* dst = (is_v ? v_smem : k_smem) + s * kKVStage;
+                mbar_arrive_expect_tx(full, kKVStage);
+                if (j >= n_pref) {
+                    const CUtensorMap* m = is_v ? &maps.v_tree : &maps.k_tree;
+                    tma_load_3d(dst, m, 0, kvh, b * T, full, pol);
+                    tma_load_3d(dst + kSubTile, m, 64, kvh, b * T, full, pol);
+                } else {
+                    if (blk < 0 || blk >= num_blocks) { set_status(status, SD_ERR_BOUNDS); blk = 0; }
+                    const CUtensorMap* m = is_v ? &maps.v_cache : &maps.k_cache;
+                    const int y = (blk * bt.Hkv + kvh) * kKeyTile;
+                    tma_load_2d(dst, m, 0, y, full, pol);
+                    tma_load_2d(dst + kSubTile, m, 64, y, full, pol);
                 }
-                if (ok) {
-                    mbar_arrive_expect_tx(&v_full[s], kKVStage);
-                    uint8_t* dst = v_smem + s * kKVStage;
-                    if (tree) {
-                        tma_load_3d(dst, &maps.v_tree, 0, kvh, b * T, &v_full[s], pol);
-                        tma_load_3d(dst + kSubTile, &maps.v_tree, 64, kvh, b * T, &v_full[s], pol);
-                    } else {
-                        const int y = (blk * bt.Hkv + kvh) * kKeyTile;
-                        tma_load_2d(dst, &maps.v_cache, 0, y, &v_full[s], pol);
-                        tma_load_2d(dst + kSubTile, &maps.v_cache, 64, y, &v_full[s], pol);
-                    }
+            };
+            while ((jk < nt || jv < nt) && ok) {
+                bool progress = false;
+                if (jk < nt && mbar_try_wait(&k_empty[jk % kKStages], ((uint32_t)(jk / kKStages) & 1u) ^ 1u)) {
+                    issue(jk, blk_k, false);
+                    ++jk;
+                    if (jk < n_pref) blk_k = __ldg(table + t0 + jk);
+                    progress = true;
+                }
+                if (jv < nt && mbar_try_wait(&v_empty[jv % kVStages], ((uint32_t)(jv / kVStages) & 1u) ^ 1u)) {
+                    issue(jv, blk_v, true);
+                    ++jv;
+                    if (jv < n_pref) blk_v = __ldg(table + t0 + jv);
+                    progress = true;
+                }
+                if (progress) {
+                    t_last = clock64();
+                } else if (*reinterpret_cast<volatile int*>(abort_flag) || clock64() - t_last > kWaitCycles) {
+                    *reinterpret_cast<volatile int*>(abort_flag) = 1;
+                    ok = false;
                 }
             }
-            __syncwarp();
+            if (!ok) {
+                set_status(status, SD_ERR_TIMEOUT);
+                for (int i = 0; i < 1000; ++i) __nanosleep(1000);      // let copies in flight land
+            }
         }
-        if (lane == 0 && !ok) {
-            set_status(status, SD_ERR_TIMEOUT);
-            for (int i = 0; i < 1000; ++i) __nanosleep(1000);      // let copies in flight land
-        }
-    } else if (warp == 5) {
+    } else if (warp == kMmaWarp) {
         // ------------------------------------------------------------ MMA issuer
         if (lane == 0) {
             const uint32_t idesc_s = make_idesc_bf16(kRowTile, kKeyTile, false, false);   // S = Q . K^T
@@ -231,18 +300,18 @@ attn_umma_kernel(const __grid_constant__ AttnMaps maps, const sd_batch bt, const
             const uint32_t q_addr = smem_u32(q_smem);
             bool ok = mbar_wait(q_full, 0, abort_flag);
             auto issue_s = [&](int j) -> bool {
-                const int s = j & 1;
-                const uint32_t ph = (uint32_t)(j >> 1) & 1u;
-                if (!mbar_wait(&k_full[s], ph, abort_flag)) return false;
+                const int s = j & 1;                               // score buffer
+                const int ks = j % kKStages;                       // K ring slot
+                if (!mbar_wait(&k_full[ks], (uint32_t)(j / kKStages) & 1u, abort_flag)) return false;
                 tc_fence_after_sync();
-                const uint32_t k_addr = smem_u32(k_smem + s * kKVStage);
+                const uint32_t k_addr = smem_u32(k_smem + ks * kKVStage);
 #pragma unroll
                 for (int k = 0; k < kD / 16; ++k) {
                     const uint64_t ad = make_smem_desc(q_addr + (k >> 2) * (kRowTile * 128) + (k & 3) * 32, 16, 1024, 128);
                     const uint64_t bd = make_smem_desc(k_addr + (k >> 2) * kSubTile + (k & 3) * 32, 16, 1024, 128);
                     mma_ss(tmem_s + s * kKeyTile, ad, bd, idesc_s, k != 0 ? 1u : 0u);
                 }
-                mma_commit(&k_empty[s]);
+                mma_commit(&k_empty[ks]);
                 mma_commit(&s_full[s]);
                 return true;
             };
@@ -253,9 +322,10 @@ attn_umma_kernel(const __grid_constant__ AttnMaps maps, const sd_batch bt, const
                 const int s = j & 1;
                 const uint32_t ph = (uint32_t)(j >> 1) & 1u;
                 if (!mbar_wait(&p_full[s], ph, abort_flag)) { ok = false; break; }
-                if (!mbar_wait(&v_full[s], ph, abort_flag)) { ok = false; break; }
+                const int vs = j % kVStages;
+                if (!mbar_wait(&v_full[vs], (uint32_t)(j / kVStages) & 1u, abort_flag)) { ok = false; break; }
                 tc_fence_after_sync();
-                const uint32_t v_addr = smem_u32(v_smem + s * kKVStage);
+                const uint32_t v_addr = smem_u32(v_smem + vs * kKVStage);
 #pragma unroll
                 for (int k = 0; k < kKeyTile / 16; ++k) {
                     // V is stored [key][d]: N (= d) contiguous; D-halves kSubTile apart, 8-key groups 1 KiB apart
@@ -263,13 +333,13 @@ attn_umma_kernel(const __grid_constant__ AttnMaps maps, const sd_batch bt, const
                     // P comes straight from TMEM: 16 keys = 8 packed columns per MMA
                     mma_ts(tmem_o, tmem_s + s * kKeyTile + k * 8, bd, idesc_o, (j | k) != 0 ? 1u : 0u);
                 }
-                mma_commit(&v_empty[s]);
+                mma_commit(&v_empty[vs]);
                 mma_commit(pv_done);
             }
             if (ok) mma_commit(o_full);
             if (!ok) set_status(status, SD_ERR_TIMEOUT);
         }
-    } else {
+    } else if (warp < 4) {
         // ------------------------------------------------------------ softmax: one thread per row
         const int row_in_tile = warp * 32 + lane;
         const int row = rt * kRowTile + row_in_tile;
@@ -291,7 +361,6 @@ attn_umma_kernel(const __grid_constant__ AttnMaps maps, const sd_batch bt, const
         }
         const uint64_t amask = row_ok ? bt.anc_mask[(size_t)b * T + node] : ~0ull;
         const uint32_t lane_field = (uint32_t)(warp * 32) << 16;
-        float m_used = -INFINITY, l = 0.f;
         bool ok = true;
         for (int j = 0; j < nt && ok; ++j) {
             const int s = j & 1;
@@ -369,14 +438,11 @@ attn_umma_kernel(const __grid_constant__ AttnMaps maps, const sd_batch bt, const
         // ------------------------------------------------------------ epilogue
         // (a parity wait on pv_done would be ambiguous here: the softmax may be two phases ahead of it)
         if (ok) ok = mbar_wait(o_full, 0, abort_flag);
-        if (ok) {
+        if (ok && !clustered) {
+            // single chunk: normalise and write bf16 output
             tc_fence_after_sync();
-            const bool direct = (plan.n_chunks == 1);
             const int h = kvh * G + g;
             const size_t orow = ((size_t)b * T + node) * bt.Hq + h;
-            float* part = nullptr;
-            if (!direct)
-                part = ws + ((size_t)(b * bt.Hkv + kvh) * plan.n_chunks + chunk) * partial_stride(plan);
             const float inv = 1.f / l;
 #pragma unroll
             for (int cc = 0; cc < 4; ++cc) {
@@ -384,107 +450,78 @@ attn_umma_kernel(const __grid_constant__ AttnMaps maps, const sd_batch bt, const
                 tmem_ld32(tmem_o + lane_field + cc * 32, o);
                 tmem_ld_wait();
                 if (row < plan.rows) {
-                    if (direct) {
-                        uint32_t w[16];
+                    uint32_t w[16];
 #pragma unroll
-                        for (int c = 0; c < 16; ++c) {
-                            const float a = row_ok ? __uint_as_float(o[2 * c]) * inv : 0.f;
-                            const float bb = row_ok ? __uint_as_float(o[2 * c + 1]) * inv : 0.f;
-                            __nv_bfloat162 hh = __floats2bfloat162_rn(a, bb);
-                            w[c] = *reinterpret_cast<uint32_t*>(&hh);
-                        }
-                        uint4* dst = reinterpret_cast<uint4*>(out + orow * kD + cc * 32);
-#pragma unroll
-                        for (int c = 0; c < 4; ++c) dst[c] = make_uint4(w[4 * c], w[4 * c + 1], w[4 * c + 2], w[4 * c + 3]);
-                    } else {
-                        uint4* dst = reinterpret_cast<uint4*>(part + 2 * rows4(plan) + (size_t)row * kD + cc * 32);
-#pragma unroll
-                        for (int c = 0; c < 8; ++c) dst[c] = make_uint4(o[4 * c], o[4 * c + 1], o[4 * c + 2], o[4 * c + 3]);
+                    for (int c = 0; c < 16; ++c) {
+                        const float a = row_ok ? __uint_as_float(o[2 * c]) * inv : 0.f;
+                        const float bb = row_ok ? __uint_as_float(o[2 * c + 1]) * inv : 0.f;
+                        __nv_bfloat162 hh = __floats2bfloat162_rn(a, bb);
+                        w[c] = *reinterpret_cast<uint32_t*>(&hh);
                     }
+                    uint4* dst = reinterpret_cast<uint4*>(out + orow * kD + cc * 32);
+#pragma unroll
+                    for (int c = 0; c < 4; ++c) dst[c] = make_uint4(w[4 * c], w[4 * c + 1], w[4 * c + 2], w[4 * c + 3]);
                 }
             }
-            if (row < plan.rows) {
-                if (direct) {
-                    if (lse) lse[orow] = row_ok ? (m_used + log2f(l)) * 0.6931471805599453f : 0.f;
-                } else {
-                    part[row] = m_used;
-                    part[rows4(plan) + row] = l;
-                }
+            if (row < plan.rows && lse) lse[orow] = row_ok ? (m_used + log2f(l)) * 0.6931471805599453f : 0.f;
+        } else if (ok) {
+            // several chunks: park (m, l, unnormalised O) in this CTA's own shared memory, where the
+            // CTAs of the cluster read it.  The K/V rings are idle by now (every MMA has completed).
+            // 16-byte pieces of a row are XOR-swizzled by the row index so that the per-row accesses
+            // of a warp spread over the banks.
+            tc_fence_after_sync();
+            float* xo = reinterpret_cast<float*>(k_smem);
+            float* xs = xo + kRowTile * kD;
+#pragma unroll
+            for (int cc = 0; cc < 4; ++cc) {
+                uint32_t o[32];
+                tmem_ld32(tmem_o + lane_field + cc * 32, o);
+                tmem_ld_wait();
+#pragma unroll
+                for (int k = 0; k < 8; ++k)
+                    *reinterpret_cast<uint4*>(xo + row_in_tile * kD + (((cc * 8 + k) ^ (row_in_tile & 31)) << 2)) =
+                        make_uint4(o[4 * k], o[4 * k + 1], o[4 * k + 2], o[4 * k + 3]);
             }
-        } else if (lane == 0) {
+            xs[row_in_tile] = m_used;
+            xs[kRowTile + row_in_tile] = l;
+        } else if (!ok && lane == 0) {
             set_status(status, SD_ERR_TIMEOUT);
         }
     }
+    }   // active
+
+    if (clustered) {
+        // every thread of every CTA of the cluster: exchange areas are complete and visible
+        __syncwarp();
+        cluster_arrive_release();
+        cluster_wait_acquire();
+        if (warp < 4) {
+            const uint32_t xo_addr = smem_u32(k_smem);
+            const MergeCtx mc{bt, plan, out, lse, xo_addr, xo_addr + kRowTile * kD * 4,
+                              chunk, rt, b, kvh, n, tpc, tiles_total, warp, lane};
+            if (plan.n_chunks == 2) merge_rows<2>(mc);
+            else if (plan.n_chunks == 4) merge_rows<4>(mc);
+            else merge_rows<8>(mc);
+        }
+        // every CTA keeps its shared memory alive until all the others have read it
+        __syncwarp();
+        cluster_arrive_release();
+        cluster_wait_acquire();
+    }
+    if (!active) return;
     tc_fence_before_sync();
     __syncthreads();
-    if (warp == 5) {
+    if (warp == kMmaWarp) {
         tc_fence_after_sync();
         tmem_dealloc(tmem_base, kTmemCols);
     }
-}
-
-// grid (ceil(rows / 8), Hkv, B), 128 threads: 16 threads per row, 8 output columns each.
-constexpr int kMergeRows = 8;
-__global__ void __launch_bounds__(128)
-attn_merge_kernel(const sd_batch bt, const float* __restrict__ ws, const AttnPlan plan,
-                  __nv_bfloat16* __restrict__ out, float* __restrict__ lse) {
-    const int row = blockIdx.x * kMergeRows + (threadIdx.x >> 4);
-    const int c8 = threadIdx.x & 15;
-    const int kvh = blockIdx.y, b = blockIdx.z;
-    if (row >= plan.rows) return;
-    const int G = bt.Hq / bt.Hkv;
-    const int T = bt.T_max;
-    const int node = row / G, g = row - node * G;
-    const int h = kvh * G + g;
-    const size_t orow = ((size_t)b * T + node) * bt.Hq + h;
-    uint4* dst = reinterpret_cast<uint4*>(out + orow * kD + c8 * 8);
-    const int n = min(max(bt.n_nodes[b], 0), T);
-    if (node >= n) {
-        *dst = make_uint4(0, 0, 0, 0);
-        if (lse && c8 == 0) lse[orow] = 0.f;
-        return;
-    }
-    const int len = max(bt.len[b], 0);
-    const int tiles_total = min((len + kKeyTile - 1) / kKeyTile, bt.max_blocks_per_seq);
-    const int tpc = (tiles_total + plan.n_chunks - 1) / plan.n_chunks;
-    const size_t stride = partial_stride(plan);
-    const float* base = ws + (size_t)(b * bt.Hkv + kvh) * plan.n_chunks * stride;
-    float M = -INFINITY;
-    for (int c = 0; c < plan.n_chunks; ++c) {
-        const bool live = (c == plan.n_chunks - 1) || (c * tpc < tiles_total);
-        if (live) M = fmaxf(M, base[(size_t)c * stride + row]);
-    }
-    float num[8] = {0.f, 0.f, 0.f, 0.f, 0.f, 0.f, 0.f, 0.f};
-    float den = 0.f;
-    for (int c = 0; c < plan.n_chunks; ++c) {
-        const bool live = (c == plan.n_chunks - 1) || (c * tpc < tiles_total);
-        if (!live) continue;
-        const float* pc = base + (size_t)c * stride;
-        const float w = exp2f(pc[row] - M);
-        den = fmaf(w, pc[rows4(plan) + row], den);
-        const float4* o = reinterpret_cast<const float4*>(pc + 2 * rows4(plan) + (size_t)row * kD + c8 * 8);
-        const float4 a0 = o[0], a1 = o[1];
-        num[0] = fmaf(w, a0.x, num[0]); num[1] = fmaf(w, a0.y, num[1]);
-        num[2] = fmaf(w, a0.z, num[2]); num[3] = fmaf(w, a0.w, num[3]);
-        num[4] = fmaf(w, a1.x, num[4]); num[5] = fmaf(w, a1.y, num[5]);
-        num[6] = fmaf(w, a1.z, num[6]); num[7] = fmaf(w, a1.w, num[7]);
-    }
-    const float inv = 1.f / den;
-    uint32_t wd[4];
-#pragma unroll
-    for (int i = 0; i < 4; ++i) {
-        __nv_bfloat162 hh = __floats2bfloat162_rn(num[2 * i] * inv, num[2 * i + 1] * inv);
-        wd[i] = *reinterpret_cast<uint32_t*>(&hh);
-    }
-    *dst = make_uint4(wd[0], wd[1], wd[2], wd[3]);
-    if (lse && c8 == 0) lse[orow] = (M + log2f(den)) * 0.6931471805599453f;
 }
 
 sd_status launch_attention(const sd_batch& bt, const sd_kv_layer& cache, const void* q,
                            const void* kt, const void* vt, float scale, void* out, float* lse,
                            void* ws, size_t ws_bytes, int32_t* dev_status, cudaStream_t st) {
     const AttnPlan plan = make_plan(bt, sm_count());
-    if (ws_bytes < attention_workspace_bytes(bt)) return SD_ERR_WORKSPACE;
+    (void)ws_bytes;
     AttnMaps maps;
     const uint64_t cache_rows = (uint64_t)cache.num_blocks * bt.Hkv * kKeyTile;
     if (!encode_tmap_bf16_2d(&maps.k_cache, cache.k, cache_rows, kD, kD * 2, 64, kKeyTile, 128) ||
@@ -498,17 +535,22 @@ sd_status launch_attention(const sd_batch& bt, const sd_kv_layer& cache, const v
         return SD_ERR_CUDA;
     if (cudaFuncSetAttribute(attn_umma_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, kAttSmem) != cudaSuccess)
         return SD_ERR_CUDA;
-    dim3 grid(plan.n_chunks, plan.row_tiles, bt.B * bt.Hkv);
-    attn_umma_kernel<<<grid, kAttThreads, kAttSmem, st>>>(
-        maps, bt, cache.num_blocks, static_cast<const uint16_t*>(q), scale * kLog2e, plan,
-        static_cast<float*>(ws), static_cast<__nv_bfloat16*>(out), lse, dev_status);
-    if (cudaGetLastError() != cudaSuccess) return SD_ERR_CUDA;
-    if (plan.n_chunks > 1) {
-        dim3 mgrid((plan.rows + kMergeRows - 1) / kMergeRows, bt.Hkv, bt.B);
-        attn_merge_kernel<<<mgrid, 128, 0, st>>>(bt, static_cast<const float*>(ws), plan,
-                                                static_cast<__nv_bfloat16*>(out), lse);
-        if (cudaGetLastError() != cudaSuccess) return SD_ERR_CUDA;
-    }
+    cudaLaunchConfig_t cfg = {};
+    cfg.gridDim = dim3(plan.n_chunks, plan.row_tiles, bt.B * bt.Hkv);
+    cfg.blockDim = dim3(kAttThreads);
+    cfg.dynamicSmemBytes = kAttSmem;
+    cfg.stream = st;
+    cudaLaunchAttribute attr[1];
+    attr[0].id = cudaLaunchAttributeClusterDimension;      // the chunks of one row tile form a cluster
+    attr[0].val.clusterDim.x = plan.n_chunks;
+    attr[0].val.clusterDim.y = 1;
+    attr[0].val.clusterDim.z = 1;
+    cfg.attrs = attr;
+    cfg.numAttrs = 1;
+    if (cudaLaunchKernelEx(&cfg, attn_umma_kernel, maps, bt, cache.num_blocks, static_cast<const uint16_t*>(q),
+                           scale * kLog2e, plan, static_cast<__nv_bfloat16*>(out), lse, dev_status) != cudaSuccess)
+        return SD_ERR_CUDA;
+    (void)ws;
     return SD_OK;
 }
 
