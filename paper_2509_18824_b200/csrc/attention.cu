@@ -106,7 +106,7 @@ struct MergeCtx {
 template <int NCH>
 __device__ __forceinline__ void merge_rows(const MergeCtx& x) {
     constexpr int kRowsPer = kRowTile / NCH;
-    constexpr int kBatch = 8 / NCH;                 // rows in flight per warp
+    constexpr int kBatch = 16 / NCH;                // rows in flight per warp
     const int G = x.bt.Hq / x.bt.Hkv;
     for (int i0 = x.warp * kBatch; i0 < kRowsPer; i0 += 4 * kBatch) {
         float mc[kBatch][NCH], lc[kBatch][NCH];
@@ -118,7 +118,11 @@ __device__ __forceinline__ void merge_rows(const MergeCtx& x) {
             for (int c = 0; c < NCH; ++c) {
                 const bool live = (c == NCH - 1) || (c * x.tpc < x.tiles_total);   // that chunk had key tiles
                 mc[u][c] = -INFINITY; lc[u][c] = 0.f; v[u][c] = make_float4(0.f, 0.f, 0.f, 0.f);
-                if (live) {
+                if (live && c == x.chunk) {                  // this CTA's own chunk: plain shared-memory reads
+                    mc[u][c] = ld_smem_f32(x.xs_addr + r * 4);
+                    lc[u][c] = ld_smem_f32(x.xs_addr + (kRowTile + r) * 4);
+                    v[u][c] = ld_smem_v4(x.xo_addr + (uint32_t)(r * kD + ((x.lane ^ (r & 31)) << 2)) * 4);
+                } else if (live) {
                     mc[u][c] = ld_dsmem_f32(map_dsmem(x.xs_addr + r * 4, c));
                     lc[u][c] = ld_dsmem_f32(map_dsmem(x.xs_addr + (kRowTile + r) * 4, c));
                     v[u][c] = ld_dsmem_v4(map_dsmem(x.xo_addr + (uint32_t)(r * kD + ((x.lane ^ (r & 31)) << 2)) * 4, c));

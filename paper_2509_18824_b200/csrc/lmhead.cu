@@ -216,6 +216,185 @@ lmhead_umma_kernel(const __grid_constant__ CUtensorMap tmW, const __grid_constan
     }
 }
 
+// ---------------------------------------------------------------------------
+// Two-CTA version (cta_group::2): a cluster of two CTAs works on 256 vocabulary
+// rows at a time.  Each CTA streams its own 128 rows of W and HALF of the hidden
+// rows of every k-step; one tcgen05.mma issued by the leader CTA multiplies both
+// halves against both W slabs and fills the accumulators in both CTAs' TMEM.
+// The hidden matrix is therefore re-read from L2 half as often per W byte.
+// ---------------------------------------------------------------------------
+template <int BK>
+__global__ void __launch_bounds__(kLmThreads, 1)
+lmhead_umma_pair_kernel(const __grid_constant__ CUtensorMap tmW, const __grid_constant__ CUtensorMap tmH,
+                        const LmParams p, int32_t* status) {
+    constexpr int kSwz = BK * 2;
+    constexpr int kGroup = 8 * kSwz;
+    extern __shared__ uint8_t smem_raw[];
+    uint8_t* smem = reinterpret_cast<uint8_t*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~(uintptr_t)1023);
+    const int a_bytes = kBM * kSwz;
+    const int half_n = p.part_n / 2;                          // hidden rows of one MMA held by this CTA
+    const int stage_bytes = a_bytes + p.n_parts * half_n * kSwz;
+
+    __shared__ __align__(8) uint64_t full_bar[kMaxStages];   // used in the leader: both CTAs' loads
+    __shared__ __align__(8) uint64_t empty_bar[kMaxStages];  // in each CTA: stage consumed
+    __shared__ __align__(8) uint64_t tmem_full[2];           // in each CTA: accumulator complete
+    __shared__ __align__(8) uint64_t tmem_empty[2];          // used in the leader: 8 epilogue warps done
+    __shared__ uint32_t tmem_base_slot;
+    __shared__ int abort_flag;
+
+    const int warp = threadIdx.x >> 5;
+    const int lane = threadIdx.x & 31;
+    const uint32_t rank = cluster_ctarank();                  // 0 = leader
+    const int pair = blockIdx.x >> 1;
+    const int n_pairs = gridDim.x >> 1;
+    const int kblocks = p.Hd / BK;
+    const int my_tiles = (p.n_tiles - pair + n_pairs - 1) / n_pairs;   // tiles of 256 vocabulary rows
+
+    if (threadIdx.x == 0) {
+        abort_flag = 0;
+        for (int s = 0; s < p.stages; ++s) { mbar_init(&full_bar[s], 1); mbar_init(&empty_bar[s], 1); }
+        for (int b = 0; b < 2; ++b) { mbar_init(&tmem_full[b], 1); mbar_init(&tmem_empty[b], 8); }
+        fence_barrier_init();
+    }
+    if (warp == 5) {
+        tmem_alloc_pair(&tmem_base_slot, (uint32_t)p.tmem_cols);
+        tmem_relinquish_pair();
+    }
+    if (warp == 4 && lane == 0) { prefetch_tensormap(&tmW); prefetch_tensormap(&tmH); }
+    tc_fence_before_sync();
+    __syncthreads();
+    cluster_arrive_release();          // the partner's barriers exist before anything signals them
+    cluster_wait_acquire();
+    tc_fence_after_sync();
+    const uint32_t tmem_base = tmem_base_slot;
+
+    if (warp == 4) {
+        // ------------------------------------------------ TMA producer (one per CTA)
+        if (lane == 0) {
+            const uint64_t pol_w = policy_evict_first();
+            const uint64_t pol_h = policy_evict_last();
+            int it = 0;
+            bool ok = true;
+            for (int t = 0; t < my_tiles && ok; ++t) {
+                const int v0 = ((pair + t * n_pairs) * 2 + (int)rank) * kBM;
+                for (int kb = 0; kb < kblocks; ++kb, ++it) {
+                    const int s = it % p.stages;
+                    const uint32_t ph = (uint32_t)(it / p.stages) & 1u;
+                    if (!mbar_wait(&empty_bar[s], ph ^ 1u, &abort_flag)) { ok = false; break; }
+                    uint8_t* a = smem + (size_t)s * stage_bytes;
+                    if (rank == 0) mbar_arrive_expect_tx(&full_bar[s], 2u * (uint32_t)stage_bytes);
+                    const uint32_t bar = map_dsmem(smem_u32(&full_bar[s]), 0);     // the leader's barrier
+                    tma_load_2d_pair(a, &tmW, kb * BK, v0, bar, pol_w);
+                    for (int part = 0; part < p.n_parts; ++part)
+                        tma_load_2d_pair(a + a_bytes + (size_t)part * half_n * kSwz, &tmH, kb * BK,
+                                         p.row0 + part * p.part_n + (int)rank * half_n, bar, pol_h);
+                }
+            }
+            if (!ok) {
+                set_status(status, SD_ERR_TIMEOUT);
+                for (int i = 0; i < 1000; ++i) __nanosleep(1000);   // let copies in flight land
+            }
+        }
+    } else if (warp == 5) {
+        // ------------------------------------------------ MMA issuer (leader CTA only)
+        if (lane == 0 && rank == 0) {
+            const uint32_t idesc = make_idesc_bf16(2 * kBM, p.part_n, false, false);
+            int it = 0;
+            bool ok = true;
+            for (int t = 0; t < my_tiles && ok; ++t) {
+                const int buf = t % p.acc_bufs;
+                const uint32_t use = (uint32_t)(t / p.acc_bufs);
+                if (!mbar_wait(&tmem_empty[buf], (use & 1u) ^ 1u, &abort_flag)) { ok = false; break; }
+                tc_fence_after_sync();
+                const uint32_t d0 = tmem_base + (uint32_t)(buf * p.buf_stride);
+                for (int kb = 0; kb < kblocks; ++kb, ++it) {
+                    const int s = it % p.stages;
+                    const uint32_t ph = (uint32_t)(it / p.stages) & 1u;
+                    if (!mbar_wait(&full_bar[s], ph, &abort_flag)) { ok = false; break; }
+                    tc_fence_after_sync();
+                    const uint32_t a_addr = smem_u32(smem + (size_t)s * stage_bytes);
+                    const uint32_t b_addr = a_addr + (uint32_t)a_bytes;
+#pragma unroll
+                    for (int k = 0; k < BK / 16; ++k) {
+                        const uint64_t adesc = make_smem_desc(a_addr + k * 32, 16, kGroup, kSwz);
+                        for (int part = 0; part < p.n_parts; ++part) {
+                            const uint64_t bdesc =
+                                make_smem_desc(b_addr + (uint32_t)(part * half_n * kSwz) + k * 32, 16, kGroup, kSwz);
+                            mma_ss_pair(d0 + (uint32_t)(part * p.part_n), adesc, bdesc, idesc, (kb | k) != 0 ? 1u : 0u);
+                        }
+                    }
+                    mma_commit_pair(&empty_bar[s], 3);        // both CTAs may refill this stage
+                }
+                if (ok) mma_commit_pair(&tmem_full[buf], 3);  // accumulators complete in both CTAs
+            }
+            if (!ok) set_status(status, SD_ERR_TIMEOUT);
+        }
+    } else {
+        // ------------------------------------------------ epilogue warps 0..3 (TMEM lanes 32*warp ..)
+        int32_t best_key[kMaxCols / 32];
+        int32_t best_idx[kMaxCols / 32];
+#pragma unroll
+        for (int c = 0; c < kMaxCols / 32; ++c) { best_key[c] = INT32_MIN; best_idx[c] = 0x7fffffff; }
+        bool ok = true;
+        for (int t = 0; t < my_tiles && ok; ++t) {
+            const int buf = t % p.acc_bufs;
+            const uint32_t use = (uint32_t)(t / p.acc_bufs);
+            if (!mbar_wait(&tmem_full[buf], use & 1u, &abort_flag)) { ok = false; break; }
+            tc_fence_after_sync();
+            const int v_base = ((pair + t * n_pairs) * 2 + (int)rank) * kBM + warp * 32;
+            const bool v_ok = (v_base + lane) < p.V;
+            const uint32_t taddr = tmem_base + ((uint32_t)(warp * 32) << 16) + (uint32_t)(buf * p.buf_stride);
+#pragma unroll
+            for (int c = 0; c < kMaxCols / 32; ++c) {
+                if (c * 32 < p.n_pad) {
+                    uint32_t r[32];
+                    tmem_ld32(taddr + c * 32, r);
+                    tmem_ld_wait();
+                    int32_t ck = INT32_MIN, ci = 0x7fffffff;
+#pragma unroll
+                    for (int j = 0; j < 32; ++j) {
+                        const int32_t key = v_ok ? ordered_key(r[j]) : INT32_MIN;
+                        const int32_t mx = __reduce_max_sync(0xffffffffu, key);
+                        const uint32_t who = __ballot_sync(0xffffffffu, key == mx);
+                        if (lane == j) { ck = mx; ci = v_base + (__ffs(who) - 1); }
+                    }
+                    if (ck > best_key[c]) { best_key[c] = ck; best_idx[c] = ci; }
+                }
+            }
+            tc_fence_before_sync();
+            __syncwarp();
+            if (lane == 0) mbar_arrive_remote(map_dsmem(smem_u32(&tmem_empty[buf]), 0));
+        }
+        asm volatile("bar.sync 1, 128;" ::: "memory");
+        int32_t* red_key = reinterpret_cast<int32_t*>(smem);
+        int32_t* red_idx = red_key + 4 * kMaxCols;
+#pragma unroll
+        for (int c = 0; c < kMaxCols / 32; ++c) {
+            red_key[warp * kMaxCols + c * 32 + lane] = best_key[c];
+            red_idx[warp * kMaxCols + c * 32 + lane] = best_idx[c];
+        }
+        asm volatile("bar.sync 1, 128;" ::: "memory");
+        for (int col = threadIdx.x; col < kMaxCols; col += 128) {
+            int32_t k = red_key[col], i = red_idx[col];
+#pragma unroll
+            for (int w = 1; w < 4; ++w) {
+                const int32_t k2 = red_key[w * kMaxCols + col], i2 = red_idx[w * kMaxCols + col];
+                if (k2 > k || (k2 == k && i2 < i)) { k = k2; i = i2; }
+            }
+            p.part_key[(size_t)blockIdx.x * kMaxCols + col] = ok ? k : INT32_MIN;
+            p.part_idx[(size_t)blockIdx.x * kMaxCols + col] = i;
+        }
+    }
+    tc_fence_before_sync();
+    __syncthreads();
+    cluster_arrive_release();          // neither CTA leaves while the other may still signal it
+    cluster_wait_acquire();
+    if (warp == 5) {
+        tc_fence_after_sync();
+        tmem_dealloc_pair(tmem_base, (uint32_t)p.tmem_cols);
+    }
+}
+
 // one thread per hidden row: merge the per-CTA candidates (lowest index on ties)
 __global__ void lmhead_merge_kernel(const int32_t* __restrict__ part_key, const int32_t* __restrict__ part_idx,
                                     int n_ctas, int rows, int row0, int32_t* __restrict__ argmax,
@@ -259,10 +438,18 @@ sd_status launch_lmhead(const void* hidden, const void* W, int M, int Hd, int V,
         while (cols < p.acc_bufs * p.buf_stride) cols *= 2;
         p.tmem_cols = cols;
         p.n_tiles = (V + kBM - 1) / kBM;
+        // Two-CTA tiles whenever a pair has work (the common case); rows per MMA part must then
+        // split evenly over the two CTAs in whole 8-row swizzle groups.
+        const bool pair = (sms >= 2) && (V > kBM);
+        if (pair) {
+            p.part_n = round_up(p.part_n, 16);
+            p.n_tiles = (V + 2 * kBM - 1) / (2 * kBM);
+        }
+        const int b_rows = pair ? p.n_pad / 2 : p.n_pad;      // hidden rows staged per CTA and k-step
         // contraction step: 64 (128-byte swizzle) while at least four stages fit, else 32
-        const int stage64 = (kBM + p.n_pad) * 128;
+        const int stage64 = (kBM + b_rows) * 128;
         const int bk = (4 * stage64 <= kSmemBudget) ? 64 : 32;
-        const int stage_bytes = (kBM + p.n_pad) * bk * 2;
+        const int stage_bytes = (kBM + b_rows) * bk * 2;
         int stages = kSmemBudget / stage_bytes;
         if (stages > kMaxStages) stages = kMaxStages;
         if (stages < 2) return SD_ERR_UNSUPPORTED;
@@ -274,16 +461,37 @@ sd_status launch_lmhead(const void* hidden, const void* W, int M, int Hd, int V,
         if (!encode_tmap_bf16_2d(&tmW, W, (uint64_t)V, (uint64_t)Hd, (uint64_t)Hd * 2, (uint32_t)bk, kBM, bk * 2))
             return SD_ERR_CUDA;
         if (!encode_tmap_bf16_2d(&tmH, hidden, (uint64_t)M, (uint64_t)Hd, (uint64_t)Hd * 2, (uint32_t)bk,
-                                 (uint32_t)p.part_n, bk * 2))
+                                 (uint32_t)(pair ? p.part_n / 2 : p.part_n), bk * 2))
             return SD_ERR_CUDA;
         int grid = sms < kMaxCtas ? sms : kMaxCtas;
-        if (grid > p.n_tiles) grid = p.n_tiles;
         const size_t dyn = (size_t)stages * stage_bytes + 1024;
-        auto kern = (bk == 64) ? lmhead_umma_kernel<64> : lmhead_umma_kernel<32>;
-        if (cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)dyn) != cudaSuccess)
-            return SD_ERR_CUDA;
-        kern<<<grid, kLmThreads, dyn, st>>>(tmW, tmH, p, dev_status);
-        if (cudaGetLastError() != cudaSuccess) return SD_ERR_CUDA;
+        if (pair) {
+            grid &= ~1;
+            if (grid > 2 * p.n_tiles) grid = 2 * p.n_tiles;
+            auto kern = (bk == 64) ? lmhead_umma_pair_kernel<64> : lmhead_umma_pair_kernel<32>;
+            if (cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)dyn) != cudaSuccess)
+                return SD_ERR_CUDA;
+            cudaLaunchConfig_t cfg = {};
+            cfg.gridDim = dim3(grid);
+            cfg.blockDim = dim3(kLmThreads);
+            cfg.dynamicSmemBytes = dyn;
+            cfg.stream = st;
+            cudaLaunchAttribute attr[1];
+            attr[0].id = cudaLaunchAttributeClusterDimension;
+            attr[0].val.clusterDim.x = 2;
+            attr[0].val.clusterDim.y = 1;
+            attr[0].val.clusterDim.z = 1;
+            cfg.attrs = attr;
+            cfg.numAttrs = 1;
+            if (cudaLaunchKernelEx(&cfg, kern, tmW, tmH, p, dev_status) != cudaSuccess) return SD_ERR_CUDA;
+        } else {
+            if (grid > p.n_tiles) grid = p.n_tiles;
+            auto kern = (bk == 64) ? lmhead_umma_kernel<64> : lmhead_umma_kernel<32>;
+            if (cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)dyn) != cudaSuccess)
+                return SD_ERR_CUDA;
+            kern<<<grid, kLmThreads, dyn, st>>>(tmW, tmH, p, dev_status);
+            if (cudaGetLastError() != cudaSuccess) return SD_ERR_CUDA;
+        }
         lmhead_merge_kernel<<<(p.rows + 127) / 128, 128, 0, st>>>(p.part_key, p.part_idx, grid, p.rows, p.row0,
                                                                  argmax, maxlogit);
         if (cudaGetLastError() != cudaSuccess) return SD_ERR_CUDA;
