@@ -1,0 +1,131 @@
+"""Per-call measurements beyond the headline step: every workload's attention,
+the LM head at several row counts, and the bandwidth-regime cases (chain
+decoding, a compaction stress shape).  One JSON line per measurement.
+
+    python -m paper_2509_18824_b200.supplements [attention] [lmhead] [compact]
+
+Timing: CUDA events on the launching stream, >= 3 warm-up calls, inputs rotated
+over several layers so that the working set exceeds L2.
+"""
+from __future__ import annotations
+
+import json
+import os
+import sys
+
+import numpy as np
+import torch
+
+from . import binding as sd
+from . import workloads as wl
+from .step import to_device
+
+
+def _peaks():
+    fn = os.path.join(os.path.dirname(os.path.dirname(os.path.abspath(__file__))), "MEASURED_PEAKS.json")
+    if os.path.exists(fn):
+        p = json.load(open(fn))
+        return float(p["hbm_gbs"]), float(p["bf16_tflops"]), "measured"
+    return 6650.0, 1590.0, "fallback"
+
+
+def _time(fn, reps):
+    for _ in range(3):
+        fn()
+    torch.cuda.synchronize()
+    e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    e0.record()
+    for _ in range(reps):
+        fn()
+    e1.record()
+    torch.cuda.synchronize()
+    return e0.elapsed_time(e1) / reps
+
+
+def attention(configs=("c2", "c3", "c4", "c5", "chain11")):
+    hbm, tens, src = _peaks()
+    for cfg in configs:
+        sp = wl.spec(cfg)
+        sp.L = 4                                   # 4 distinct layers: > L2 for every config but c2
+        w = wl.make_geometry(sp)
+        wl.fill_attention(w)
+        bt = sd.Batch.of(w)
+        st = sd.new_status()
+        sd.sd_tree_prepare(bt, st)
+        kc = [to_device(x) for x in w.k_cache]; vc = [to_device(x) for x in w.v_cache]
+        q = [to_device(x) for x in w.q]; kt = [to_device(x) for x in w.k_tree]; vt = [to_device(x) for x in w.v_tree]
+        out = torch.zeros((w.B, w.T_max, w.Hq, w.D), dtype=torch.bfloat16, device="cuda")
+        ws = torch.empty(sd.sd_workspace_bytes(bt), dtype=torch.uint8, device="cuda")
+        caches = [sd.kv_layer(k, v) for k, v in zip(kc, vc)]
+
+        def run():
+            for l in range(w.L):
+                sd.sd_verify_attention(bt, caches[l], q[l], kt[l], vt[l], w.scale, out, None, ws, st)
+        ms = _time(run, 10) / w.L
+        vis = sum(int((int(w.len[b]) + wl.node_depths(w.parents[b]) + 1).sum()) for b in range(w.B))
+        flops = 4.0 * w.D * w.Hq * vis
+        nbytes = (sum(int(w.len[b]) + w.T_max for b in range(w.B)) * w.Hkv * w.D * 4
+                  + 2 * w.B * w.T_max * w.Hq * w.D * 2)
+        print(json.dumps({"call": "sd_verify_attention", "workload": cfg, "us": ms * 1e3,
+                          "tflops": flops / ms / 1e9, "frac_tensor_burst": flops / ms / 1e9 / tens,
+                          "gbs": nbytes / ms / 1e6, "frac_hbm": nbytes / ms / 1e6 / hbm,
+                          "frac_hbm_nominal_8TBs": nbytes / ms / 1e6 / 8000.0,
+                          "flop_per_byte": flops / nbytes, "peaks": src, "status": int(st.item())}))
+        del kc, vc, q, kt, vt
+        torch.cuda.empty_cache()
+
+
+def lmhead(rows=(60, 240, 480, 960), V=152064, Hd=3584):
+    hbm, tens, src = _peaks()
+    W = to_device(wl.normal_bf16(7, "W", (V, Hd), 1.0 / np.sqrt(Hd)))
+    for M in rows:
+        h = to_device(wl.normal_bf16(7, f"h{M}", (M, Hd), 1.0 / np.sqrt(Hd)))
+        am = torch.zeros(M, dtype=torch.int32, device="cuda")
+        mx = torch.zeros(M, dtype=torch.float32, device="cuda")
+        ws = torch.empty(sd.sd_workspace_bytes(None, M, V), dtype=torch.uint8, device="cuda")
+        st = sd.new_status()
+        ms = _time(lambda: sd.sd_lmhead_argmax(h, W, am, mx, ws, st), 10)
+        flops = 2.0 * M * V * Hd
+        nbytes = (V + M) * Hd * 2
+        print(json.dumps({"call": "sd_lmhead_argmax", "rows": M, "us": ms * 1e3, "tflops": flops / ms / 1e9,
+                          "frac_tensor_burst": flops / ms / 1e9 / tens, "gbs": nbytes / ms / 1e6,
+                          "frac_hbm": nbytes / ms / 1e6 / hbm, "peaks": src, "status": int(st.item())}))
+
+
+def compact(B=1024, L=8, T=64, Hkv=4, D=128):
+    """Stress shape for compaction: every node of every tree accepted (a 64-node chain), 1024
+    sequences, 8 layers: 2 x 1.07 GB moved per call."""
+    hbm, _, src = _peaks()
+    g = np.random.default_rng(0)
+    lens = g.integers(0, 64, size=B).astype(np.int32)
+    table = np.arange(2 * B, dtype=np.int32).reshape(B, 2)
+    parents = np.stack([wl.chain_tree(T)] * B)
+    geo = type("G", (), dict(B=B, T_max=T, Hq=Hkv, Hkv=Hkv, D=D, block_table=table, len=lens,
+                             n_nodes=np.full(B, T, np.int32), parents=parents))
+    bt = sd.Batch.of(geo)
+    st = sd.new_status()
+    kc = [torch.zeros((2 * B, Hkv, 64, D), dtype=torch.int16, device="cuda") for _ in range(L)]
+    vc = [torch.zeros((2 * B, Hkv, 64, D), dtype=torch.int16, device="cuda") for _ in range(L)]
+    kt = [torch.randint(-30000, 30000, (B, T, Hkv, D), dtype=torch.int16, device="cuda") for _ in range(L)]
+    vt = [torch.randint(-30000, 30000, (B, T, Hkv, D), dtype=torch.int16, device="cuda") for _ in range(L)]
+    n_acc = torch.full((B,), T, dtype=torch.int32, device="cuda")
+    path = torch.arange(T, dtype=torch.int32, device="cuda").repeat(B, 1).contiguous()
+    ls = sd.LayerSet(kc, vc, kt, vt)
+    ms = _time(lambda: sd.sd_compact_kv(bt, ls, n_acc, path, st), 10)
+    moved = 2.0 * B * T * Hkv * D * 2 * 2 * L          # read + write, K and V
+    ok = all(torch.equal(kc[l][2 * b + (int(lens[b]) + 5) // 64, :, (int(lens[b]) + 5) % 64], kt[l][b, 5])
+             for l in (0, L - 1) for b in (0, B - 1))
+    print(json.dumps({"call": "sd_compact_kv", "workload": f"stress B={B} L={L} all {T} nodes accepted",
+                      "us": ms * 1e3, "gbs": moved / ms / 1e6, "frac_hbm": moved / ms / 1e6 / hbm,
+                      "frac_hbm_nominal_8TBs": moved / ms / 1e6 / 8000.0, "bytes": moved, "peaks": src,
+                      "spot_check": bool(ok), "status": int(st.item())}))
+
+
+if __name__ == "__main__":
+    what = sys.argv[1:] or ["attention", "lmhead", "compact"]
+    if "attention" in what:
+        attention()
+    if "lmhead" in what:
+        lmhead()
+    if "compact" in what:
+        compact()
