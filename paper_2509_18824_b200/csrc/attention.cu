@@ -301,20 +301,27 @@ attn_umma_kernel(const __grid_constant__ AttnMaps maps, const sd_batch bt, const
         if (lane == 0) {
             const uint32_t idesc_s = make_idesc_bf16(kRowTile, kKeyTile, false, false);   // S = Q . K^T
             const uint32_t idesc_o = make_idesc_bf16(kRowTile, kD, false, true);          // O += P . V
-            const uint32_t q_addr = smem_u32(q_smem);
+            // Descriptors are prepared outside the issue sequences: every instruction between two
+            // tcgen05.mma of one thread delays the second one.  k-steps only move the (16-byte
+            // granular) start-address field in the low bits.
+            uint64_t qdesc[kD / 16];
+#pragma unroll
+            for (int k = 0; k < kD / 16; ++k)
+                qdesc[k] = make_smem_desc(smem_u32(q_smem) + (k >> 2) * (kRowTile * 128) + (k & 3) * 32, 16, 1024, 128);
+            const uint64_t kdesc_base = make_smem_desc(smem_u32(k_smem), 16, 1024, 128);
+            // V is stored [key][d]: N (= d) contiguous; D-halves kSubTile apart, 8-key groups 1 KiB apart
+            const uint64_t vdesc_base = make_smem_desc(smem_u32(v_smem), kSubTile, 1024, 128);
             bool ok = mbar_wait(q_full, 0, abort_flag);
             auto issue_s = [&](int j) -> bool {
                 const int s = j & 1;                               // score buffer
                 const int ks = j % kKStages;                       // K ring slot
                 if (!mbar_wait(&k_full[ks], (uint32_t)(j / kKStages) & 1u, abort_flag)) return false;
                 tc_fence_after_sync();
-                const uint32_t k_addr = smem_u32(k_smem + ks * kKVStage);
+                const uint64_t kd = kdesc_base + (uint64_t)(ks * (kKVStage >> 4));
+                const uint32_t d = tmem_s + s * kKeyTile;
 #pragma unroll
-                for (int k = 0; k < kD / 16; ++k) {
-                    const uint64_t ad = make_smem_desc(q_addr + (k >> 2) * (kRowTile * 128) + (k & 3) * 32, 16, 1024, 128);
-                    const uint64_t bd = make_smem_desc(k_addr + (k >> 2) * kSubTile + (k & 3) * 32, 16, 1024, 128);
-                    mma_ss(tmem_s + s * kKeyTile, ad, bd, idesc_s, k != 0 ? 1u : 0u);
-                }
+                for (int k = 0; k < kD / 16; ++k)
+                    mma_ss(d, qdesc[k], kd + (uint64_t)((k >> 2) * (kSubTile >> 4) + (k & 3) * 2), idesc_s, k != 0 ? 1u : 0u);
                 mma_commit(&k_empty[ks]);
                 mma_commit(&s_full[s]);
                 return true;
@@ -329,14 +336,12 @@ attn_umma_kernel(const __grid_constant__ AttnMaps maps, const sd_batch bt, const
                 const int vs = j % kVStages;
                 if (!mbar_wait(&v_full[vs], (uint32_t)(j / kVStages) & 1u, abort_flag)) { ok = false; break; }
                 tc_fence_after_sync();
-                const uint32_t v_addr = smem_u32(v_smem + vs * kKVStage);
+                const uint64_t vd = vdesc_base + (uint64_t)(vs * (kKVStage >> 4));
+                const uint32_t pa = tmem_s + s * kKeyTile;        // P comes straight from TMEM: 16 keys = 8 columns
+                const uint32_t first = (j != 0) ? 1u : 0u;
 #pragma unroll
-                for (int k = 0; k < kKeyTile / 16; ++k) {
-                    // V is stored [key][d]: N (= d) contiguous; D-halves kSubTile apart, 8-key groups 1 KiB apart
-                    const uint64_t bd = make_smem_desc(v_addr + k * 2048, kSubTile, 1024, 128);
-                    // P comes straight from TMEM: 16 keys = 8 packed columns per MMA
-                    mma_ts(tmem_o, tmem_s + s * kKeyTile + k * 8, bd, idesc_o, (j | k) != 0 ? 1u : 0u);
-                }
+                for (int k = 0; k < kKeyTile / 16; ++k)
+                    mma_ts(tmem_o, pa + k * 8, vd + (uint64_t)(k * (2048 >> 4)), idesc_o, k != 0 ? 1u : first);
                 mma_commit(&v_empty[vs]);
                 mma_commit(pv_done);
             }

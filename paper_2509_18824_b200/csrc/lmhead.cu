@@ -223,7 +223,7 @@ lmhead_umma_kernel(const __grid_constant__ CUtensorMap tmW, const __grid_constan
 // halves against both W slabs and fills the accumulators in both CTAs' TMEM.
 // The hidden matrix is therefore re-read from L2 half as often per W byte.
 // ---------------------------------------------------------------------------
-template <int BK>
+template <int BK, int NPARTS>
 __global__ void __launch_bounds__(kLmThreads, 1)
 lmhead_umma_pair_kernel(const __grid_constant__ CUtensorMap tmW, const __grid_constant__ CUtensorMap tmH,
                         const LmParams p, int32_t* status) {
@@ -299,6 +299,7 @@ lmhead_umma_pair_kernel(const __grid_constant__ CUtensorMap tmW, const __grid_co
         // ------------------------------------------------ MMA issuer (leader CTA only)
         if (lane == 0 && rank == 0) {
             const uint32_t idesc = make_idesc_bf16(2 * kBM, p.part_n, false, false);
+            const uint32_t part_step = (uint32_t)(half_n * kSwz) >> 4;   // next part's B rows, in descriptor units
             int it = 0;
             bool ok = true;
             for (int t = 0; t < my_tiles && ok; ++t) {
@@ -312,15 +313,17 @@ lmhead_umma_pair_kernel(const __grid_constant__ CUtensorMap tmW, const __grid_co
                     const uint32_t ph = (uint32_t)(it / p.stages) & 1u;
                     if (!mbar_wait(&full_bar[s], ph, &abort_flag)) { ok = false; break; }
                     tc_fence_after_sync();
+                    // descriptors of the stage; k-steps and parts only move the 16-byte-granular start address
                     const uint32_t a_addr = smem_u32(smem + (size_t)s * stage_bytes);
-                    const uint32_t b_addr = a_addr + (uint32_t)a_bytes;
+                    const uint64_t adesc0 = make_smem_desc(a_addr, 16, kGroup, kSwz);
+                    const uint64_t bdesc0 = make_smem_desc(a_addr + (uint32_t)a_bytes, 16, kGroup, kSwz);
+                    const uint32_t first = (kb != 0) ? 1u : 0u;
 #pragma unroll
                     for (int k = 0; k < BK / 16; ++k) {
-                        const uint64_t adesc = make_smem_desc(a_addr + k * 32, 16, kGroup, kSwz);
-                        for (int part = 0; part < p.n_parts; ++part) {
-                            const uint64_t bdesc =
-                                make_smem_desc(b_addr + (uint32_t)(part * half_n * kSwz) + k * 32, 16, kGroup, kSwz);
-                            mma_ss_pair(d0 + (uint32_t)(part * p.part_n), adesc, bdesc, idesc, (kb | k) != 0 ? 1u : 0u);
+#pragma unroll
+                        for (int part = 0; part < NPARTS; ++part) {
+                            mma_ss_pair(d0 + (uint32_t)(part * p.part_n), adesc0 + (uint64_t)(k * 2),
+                                        bdesc0 + (uint64_t)(part * part_step + k * 2), idesc, k != 0 ? 1u : first);
                         }
                     }
                     mma_commit_pair(&empty_bar[s], 3);        // both CTAs may refill this stage
@@ -468,7 +471,8 @@ sd_status launch_lmhead(const void* hidden, const void* W, int M, int Hd, int V,
         if (pair) {
             grid &= ~1;
             if (grid > 2 * p.n_tiles) grid = 2 * p.n_tiles;
-            auto kern = (bk == 64) ? lmhead_umma_pair_kernel<64> : lmhead_umma_pair_kernel<32>;
+            auto kern = (bk == 64) ? (p.n_parts == 2 ? lmhead_umma_pair_kernel<64, 2> : lmhead_umma_pair_kernel<64, 1>)
+                                   : (p.n_parts == 2 ? lmhead_umma_pair_kernel<32, 2> : lmhead_umma_pair_kernel<32, 1>);
             if (cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)dyn) != cudaSuccess)
                 return SD_ERR_CUDA;
             cudaLaunchConfig_t cfg = {};
