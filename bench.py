@@ -29,6 +29,11 @@ import numpy as np
 ROOT = os.path.dirname(os.path.abspath(__file__))
 sys.path.insert(0, ROOT)
 
+# dram__bytes_read.sum + dram__bytes_write.sum of one attn_umma_kernel launch, from the ncu capture
+# summarised in profiles/attn_umma_kernel_c5_layer_ncu.md (same grid and tile shape as the bench's
+# launches).  Set an entry to None whenever the kernel changes until the counters are retaken.
+ATTENTION_DRAM_BYTES_PER_LAUNCH = {"c5": 75.5e6}
+
 METRIC = "tree_verify_steps_per_s"
 UNIT = "steps/s"
 
@@ -289,7 +294,10 @@ def main():
         # grouped heads per KV head its arithmetic intensity (~420 flop/B) puts it on the tensor roof
         roofline = {"kernel": "sd_verify_attention", "bound": "tensor", "achieved": att_tflops,
                     "peak": peaks["tensor_sustained"], "unit": "TFLOP/s",
-                    "frac": att_tflops / peaks["tensor_sustained"], "traffic": None,
+                    "frac": att_tflops / peaks["tensor_sustained"],
+                    "traffic": ATTENTION_DRAM_BYTES_PER_LAUNCH.get(args.config),
+                    "traffic_unit": "bytes per launch (dram read + write, one ncu capture)",
+                    "algorithmic_bytes_per_launch": work["att_bytes"],
                     "peak_source": peaks["source"] + " (sustained bf16)",
                     "hbm_gbs": att_gbs, "hbm_frac_of_measured": att_gbs / peaks["hbm"],
                     "hbm_frac_of_nominal_8TBs": att_gbs / 8000.0,

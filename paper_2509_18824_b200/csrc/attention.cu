@@ -13,9 +13,10 @@
 // keys, masked per row by the node's ancestor bitmask.  Softmax runs one thread
 // per row straight out of TMEM (no cross-thread reductions); the running maximum
 // is only raised when it grows by more than 2^8, so the accumulator in TMEM is
-// rescaled rarely.  With one chunk the CTA writes the output itself; otherwise it
-// writes (max, sum, unnormalised O) and a small kernel merges the chunks in a
-// fixed order.
+// rescaled rarely.  P goes back into TMEM and feeds the second MMA from there.
+// With one chunk the CTA writes the output itself; otherwise the chunks of a row
+// tile form a thread-block cluster and merge their (max, sum, unnormalised O)
+// through distributed shared memory in a fixed order.
 #include "common.cuh"
 #include "sm100.cuh"
 
