@@ -147,6 +147,22 @@ def cpu_step_estimate(w, att_rows=6720, lm_rows=96):
     return total, sample, oracle.num_threads()
 
 
+def max_over_ranks(values, device):
+    """Slowest rank decides: element-wise maximum of `values` over all ranks (identity on one rank)."""
+    import torch
+    import torch.distributed as dist
+    t = torch.tensor(list(values), dtype=torch.float64, device=device)
+    if dist.is_available() and dist.is_initialized() and dist.get_world_size() > 1:
+        dist.all_reduce(t, op=dist.ReduceOp.MAX)
+    return [float(x) for x in t]
+
+
+def job_throughput(world, steps, ms_total):
+    """Whole-job steps/s of `world` independent replicas that each ran `steps` steps; `ms_total` is
+    the slowest rank's time."""
+    return world * steps / (ms_total * 1e-3)
+
+
 def run_reference(args):
     """The fp64 CPU checker timed as the reference arm (rank 0 only)."""
     if int(os.environ.get("RANK", "0")) != 0:
@@ -273,16 +289,13 @@ def main():
     n_acc = vs.host_out["n_acc"].numpy().copy()
     assert (n_acc == w.planted_len + 1).all(), "planted paths were not recovered"
 
-    t = torch.tensor([ms_total, ms_e2e], dtype=torch.float64, device="cuda")
-    if world > 1:
-        dist.all_reduce(t, op=dist.ReduceOp.MAX)
-    ms_total, ms_e2e = float(t[0]), float(t[1])
+    ms_total, ms_e2e = max_over_ranks([ms_total, ms_e2e], "cuda")
 
     if rank == 0:
         peaks = read_peaks()
         work = algorithmic_work(w)
         ms_step = ms_total / args.steps
-        value = world * args.steps / (ms_total * 1e-3)
+        value = job_throughput(world, args.steps, ms_total)
         tokens_per_step = int(n_acc.sum())
         att_s = per_call_ms["attention"] * 1e-3
         lm_s = per_call_ms["lmhead"] * 1e-3
