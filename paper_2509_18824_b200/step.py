@@ -68,6 +68,7 @@ class VerifyStep:
         self.scale = float(w.scale)
         sd.sd_tree_prepare(self.batch, self.status)
         # pinned host copies for the end-to-end path
+        self._copy_stream = None
         self.host = None
         if keep_host_inputs:
             self.host = dict(
@@ -119,18 +120,38 @@ class VerifyStep:
 
     def run_from_host(self):
         """End-to-end step: this step's inputs come from pinned host memory, the
-        accepted tokens go back to the host; caches and weights stay resident."""
+        accepted tokens go back to the host; caches and weights stay resident.
+        The host-to-device copies run on a second stream, one layer ahead of the
+        layer that is being computed; every call that reads a buffer first waits
+        for the event recorded behind that buffer's copy."""
         h = self.host
-        for l in range(self.L):
-            self.q[l].copy_(h["q"][l], non_blocking=True)
-            self.k_tree[l].copy_(h["k_tree"][l], non_blocking=True)
-            self.v_tree[l].copy_(h["v_tree"][l], non_blocking=True)
-        self.hidden.copy_(h["hidden"], non_blocking=True)
-        self.draft_tok.copy_(h["draft_tok"], non_blocking=True)
-        self.batch.parents.copy_(h["parents"], non_blocking=True)
-        self.batch.n_nodes.copy_(h["n_nodes"], non_blocking=True)
+        main = torch.cuda.current_stream()
+        if self._copy_stream is None:
+            self._copy_stream = torch.cuda.Stream(device=self.device)
+            self._ev_small = torch.cuda.Event()
+            self._ev_layer = [torch.cuda.Event() for _ in range(self.L)]
+        cs = self._copy_stream
+        cs.wait_stream(main)            # the previous step no longer reads the input buffers
+        with torch.cuda.stream(cs):
+            self.batch.parents.copy_(h["parents"], non_blocking=True)
+            self.batch.n_nodes.copy_(h["n_nodes"], non_blocking=True)
+            self._ev_small.record(cs)
+            for l in range(self.L):
+                self.q[l].copy_(h["q"][l], non_blocking=True)
+                self.k_tree[l].copy_(h["k_tree"][l], non_blocking=True)
+                self.v_tree[l].copy_(h["v_tree"][l], non_blocking=True)
+                self._ev_layer[l].record(cs)
+            self.hidden.copy_(h["hidden"], non_blocking=True)
+            self.draft_tok.copy_(h["draft_tok"], non_blocking=True)
+        main.wait_event(self._ev_small)
         sd.sd_tree_prepare(self.batch, self.status)
-        self.run()
+        for l in range(self.L):
+            main.wait_event(self._ev_layer[l])
+            self.attention(l)
+        main.wait_stream(cs)            # hidden states and draft tokens have arrived
+        self.lmhead()
+        self.accept()
+        self.compact()
         self.host_out["n_acc"].copy_(self.n_acc, non_blocking=True)
         self.host_out["path"].copy_(self.path, non_blocking=True)
         self.host_out["out_tok"].copy_(self.out_tok, non_blocking=True)
