@@ -118,6 +118,20 @@ def test_attention_gqa7_wide_trees_and_unused_nodes():
     np.testing.assert_allclose(lse[ok], rlse[ok], rtol=2e-3, atol=2e-3)
 
 
+@pytest.mark.parametrize("Hq,Hkv,T", [(8, 1, 64), (3, 3, 5), (16, 2, 33), (4, 4, 1)])
+def test_attention_group_sizes_and_tree_sizes(Hq, Hkv, T):
+    """Largest supported shape (64 nodes x 8 grouped heads = 512 rows per KV head), no grouping at
+    all, a single-node tree (plain decoding), odd sizes."""
+    g = np.random.default_rng(Hq * 100 + T)
+    par = np.stack([np.array([-1] + [int(g.integers(0, i)) for i in range(1, T)]) for _ in range(2)])
+    p = tiny128(40 + T, B=2, T=T, Hq=Hq, Hkv=Hkv, lens=(257, 64), parents=par, gain=3.0)
+    out, lse, status = gpu_attention(p)
+    assert status == 0
+    ref, rlse = oracle.attention(oracle.Geometry.of(p), p.k_cache, p.v_cache, p.q, p.k_tree, p.v_tree, p.scale)
+    check_attention(out, ref, f"Hq={Hq} Hkv={Hkv} T={T}")
+    np.testing.assert_allclose(lse, rlse, rtol=2e-3, atol=2e-3)
+
+
 def test_attention_planted_key_large_v_and_bad_block_table():
     p = tiny128(6, B=1, T=8, Hq=4, Hkv=1, lens=(900,), gain=1.0)
     # one key with score ~ +30, V rows scaled by 64
@@ -194,6 +208,17 @@ def test_attention_full_size_sampled_rows(cfg, gain):
 @pytest.mark.parametrize("M,Hd,V", [(1, 64, 1), (5, 128, 1000), (8, 256, 1024), (61, 192, 129), (130, 64, 4099)])
 def test_lmhead_small_shapes_crisp(M, Hd, V):
     g = np.random.default_rng(M + V)
+    h = wl.f32_to_bf16_bits(g.standard_normal((M, Hd)).astype(np.float32))
+    W = wl.f32_to_bf16_bits((g.standard_normal((V, Hd)) / np.sqrt(Hd)).astype(np.float32))
+    am, mx = gpu_lmhead(h, W)
+    ram, t1, t2 = oracle.lmhead(h, W)
+    check_argmax(am, mx, ram, t1, t2)
+
+
+def test_lmhead_more_rows_than_one_pass():
+    """More than 512 rows are processed in several passes over the vocabulary."""
+    g = np.random.default_rng(11)
+    M, Hd, V = 1100, 128, 2500
     h = wl.f32_to_bf16_bits(g.standard_normal((M, Hd)).astype(np.float32))
     W = wl.f32_to_bf16_bits((g.standard_normal((V, Hd)) / np.sqrt(Hd)).astype(np.float32))
     am, mx = gpu_lmhead(h, W)
