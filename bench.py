@@ -29,10 +29,10 @@ import numpy as np
 ROOT = os.path.dirname(os.path.abspath(__file__))
 sys.path.insert(0, ROOT)
 
-# dram__bytes_read.sum + dram__bytes_write.sum of one attn_umma_kernel launch, from the ncu capture
-# summarised in profiles/attn_umma_kernel_c5_layer_ncu.md (same grid and tile shape as the bench's
-# launches).  Set an entry to None whenever the kernel changes until the counters are retaken.
-ATTENTION_DRAM_BYTES_PER_LAUNCH = {"c5": 75.5e6}
+# dram__bytes_read.sum + dram__bytes_write.sum of attn_umma_kernel per layer, from the ncu capture
+# summarised under profiles/.  Set an entry to None whenever the kernel changes until the counters
+# are retaken.
+ATTENTION_DRAM_BYTES_PER_LAYER = {"c5": None}
 
 METRIC = "tree_verify_steps_per_s"
 UNIT = "steps/s"
@@ -258,18 +258,20 @@ def main():
     ms_total = e0.elapsed_time(e1)
 
     # per-call durations, same steps, events around every call (same stream)
-    names = ["attention", "lmhead", "accept", "compact"]
+    names = ["attention", "attention_single_layer_call", "lmhead", "accept", "compact"]
     ev = {n: [] for n in names}
     def timed(name, fn):
         a, b = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
         a.record(); fn(); b.record()
         ev[name].append((a, b))
     for _ in range(args.steps):
-        for l in range(vs.L):
-            timed("attention", lambda: vs.attention(l))
+        timed("attention", vs.attention_layers)           # all layers, one library call
         timed("lmhead", vs.lmhead)
         timed("accept", vs.accept)
         timed("compact", vs.compact)
+    for _ in range(max(1, args.steps // 10)):             # for comparison: one call per layer
+        for l in range(vs.L):
+            timed("attention_single_layer_call", lambda: vs.attention(l))
     torch.cuda.synchronize()
     clocks = sampler.stop() if rank == 0 else None
     per_call_ms = {n: sum(a.elapsed_time(b) for a, b in ev[n]) / len(ev[n]) for n in names}
@@ -297,24 +299,30 @@ def main():
         ms_step = ms_total / args.steps
         value = job_throughput(world, args.steps, ms_total)
         tokens_per_step = int(n_acc.sum())
-        att_s = per_call_ms["attention"] * 1e-3
+        n_att_launches = (vs.L + sd.ATTENTION_LAYERS_PER_LAUNCH - 1) // sd.ATTENTION_LAYERS_PER_LAUNCH
+        layers_per_launch = vs.L / n_att_launches
+        att_s = per_call_ms["attention"] * 1e-3 / n_att_launches          # one launch = layers_per_launch layers
         lm_s = per_call_ms["lmhead"] * 1e-3
-        att_tflops = work["att_flops"] / att_s / 1e12
-        att_gbs = work["att_bytes"] / att_s / 1e9
+        att_tflops = work["att_flops"] * layers_per_launch / att_s / 1e12
+        att_gbs = work["att_bytes"] * layers_per_launch / att_s / 1e9
         lm_tflops = work["lm_flops"] / lm_s / 1e12
         lm_gbs = work["lm_bytes"] / lm_s / 1e9
-        # dominant kernel: per-layer tree attention (28 launches per step); at 60 nodes x 7
+        # dominant kernel: tree attention, all layers of the step in one launch; at 60 nodes x 7
         # grouped heads per KV head its arithmetic intensity (~420 flop/B) puts it on the tensor roof
-        roofline = {"kernel": "sd_verify_attention", "bound": "tensor", "achieved": att_tflops,
+        traffic = ATTENTION_DRAM_BYTES_PER_LAYER.get(args.config)
+        roofline = {"kernel": "sd_verify_attention_layers (attn_umma_kernel)", "bound": "tensor", "achieved": att_tflops,
                     "peak": peaks["tensor_sustained"], "unit": "TFLOP/s",
                     "frac": att_tflops / peaks["tensor_sustained"],
-                    "traffic": ATTENTION_DRAM_BYTES_PER_LAUNCH.get(args.config),
-                    "traffic_unit": "bytes per launch (dram read + write, one ncu capture)",
-                    "algorithmic_bytes_per_launch": work["att_bytes"],
+                    "traffic": traffic * layers_per_launch if traffic else None,
+                    "traffic_unit": "bytes per launch (dram read + write; ncu capture of a 4-layer launch, "
+                                    "scaled by layers per launch)",
+                    "layers_per_launch": layers_per_launch,
+                    "algorithmic_bytes_per_launch": work["att_bytes"] * layers_per_launch,
+                    "algorithmic_flops_per_launch": work["att_flops"] * layers_per_launch,
                     "peak_source": peaks["source"] + " (sustained bf16)",
                     "hbm_gbs": att_gbs, "hbm_frac_of_measured": att_gbs / peaks["hbm"],
                     "hbm_frac_of_nominal_8TBs": att_gbs / 8000.0,
-                    "avg_launch_ms": per_call_ms["attention"]}
+                    "avg_launch_ms": att_s * 1e3}
         line = {"metric": METRIC, "value": value, "unit": UNIT, "n_gpus": world, "steps": args.steps,
                 "warmup": max(args.warmup, 3), "ms_per_step": ms_step, "higher_is_better": True,
                 "scaling": "weak", "vs_baseline": None, "dtype": "bf16", "data": "synthetic",
@@ -326,7 +334,9 @@ def main():
                         "h2d_bytes_per_step": vs.h2d_bytes(), "d2h_bytes_per_step": vs.d2h_bytes()},
                 "gpu_launches": vs.launches_per_step * args.steps,
                 "roofline": roofline,
-                "calls": {"attention_ms_per_layer": per_call_ms["attention"],
+                "calls": {"attention_ms_all_layers": per_call_ms["attention"],
+                          "attention_ms_per_layer": per_call_ms["attention"] / vs.L,
+                          "attention_ms_single_layer_call": per_call_ms["attention_single_layer_call"],
                           "lmhead_ms": per_call_ms["lmhead"], "accept_ms": per_call_ms["accept"],
                           "compact_ms": per_call_ms["compact"],
                           "lmhead_tflops": lm_tflops, "lmhead_frac_of_tensor_peak": lm_tflops / peaks["tensor_sustained"],

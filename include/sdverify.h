@@ -131,6 +131,33 @@ sd_status sd_verify_attention(const sd_batch *batch, const sd_kv_layer *cache,
                               int32_t *dev_status, void *stream);
 
 /*
+ * The same attention for L layers in one call (Sec. 1: one parallel validation
+ * pass of the target model; every layer attends over its own cache and its own
+ * tree K/V with the same trees and masks).  Layer l computes exactly what
+ * sd_verify_attention computes from caches[l], q_layers[l], k_tree_layers[l],
+ * v_tree_layers[l] into out_layers[l] (and lse_layers[l]), to within fp32
+ * rounding (the keys of a sequence may be split into a different number of
+ * chunks than in a single-layer call).  The layers are independent, so they
+ * share kernel launches: the grid runs over (layer, sequence, KV head, row
+ * tile), which fills the GPU without splitting the keys of a sequence and
+ * hides every per-launch cost but one.  Usable when all layers' q and tree K/V
+ * exist before the call (as in this library's verify step, where they are
+ * inputs); a decoder that produces them layer by layer calls
+ * sd_verify_attention per layer instead.
+ *   caches                     : host array [L] of cache descriptors
+ *   q_layers, k_tree_layers,
+ *   v_tree_layers, out_layers  : host arrays [L] of dev pointers, layouts above
+ *   lse_layers                 : NULL, or host array [L] of dev pointers (entries may be NULL)
+ * The host arrays are read before the call returns.  Errors as sd_verify_attention.
+ */
+sd_status sd_verify_attention_layers(const sd_batch *batch, const sd_kv_layer *caches, int32_t L,
+                                     const void *const *q_layers, const void *const *k_tree_layers,
+                                     const void *const *v_tree_layers, float scale,
+                                     void *const *out_layers, float *const *lse_layers,
+                                     void *workspace, size_t workspace_bytes,
+                                     int32_t *dev_status, void *stream);
+
+/*
  * LM-head projection with fused arg-max (Sec. 1 / Sec. 4.1: the target's own
  * greedy prediction at every speculative position).
  *   logits[r][v] = sum_k hidden[r][k] * W[v][k]     (never written to memory)

@@ -26,10 +26,11 @@ SD_ERR_BOUNDS = -7
 
 # kernel launches behind one call (kept in step with the kernels; used for launch accounting)
 KERNELS_PER_ATTENTION = 1      # split-KV chunks merge inside the kernel (thread-block cluster)
+ATTENTION_LAYERS_PER_LAUNCH = 32   # sd_verify_attention_layers: layers sharing one launch
 KERNELS_PER_LMHEAD = 2         # tiles + cross-slab reduce
 
 EXPORTS = ["sd_version", "sd_status_string", "sd_workspace_bytes", "sd_tree_prepare",
-           "sd_verify_attention", "sd_lmhead_argmax", "sd_lmhead_argmax_static", "sd_accept_tree",
+           "sd_verify_attention", "sd_verify_attention_layers", "sd_lmhead_argmax", "sd_lmhead_argmax_static", "sd_accept_tree",
            "sd_compact_kv"]
 
 
@@ -60,6 +61,10 @@ def _load() -> C.CDLL:
     lib.sd_verify_attention.argtypes = [C.c_void_p, C.c_void_p, C.c_void_p, C.c_void_p, C.c_void_p,
                                         C.c_float, C.c_void_p, C.c_void_p, C.c_void_p, C.c_size_t,
                                         C.c_void_p, C.c_void_p]
+    lib.sd_verify_attention_layers.restype = C.c_int
+    lib.sd_verify_attention_layers.argtypes = [C.c_void_p, C.c_void_p, C.c_int32, C.c_void_p, C.c_void_p,
+                                               C.c_void_p, C.c_float, C.c_void_p, C.c_void_p, C.c_void_p,
+                                               C.c_size_t, C.c_void_p, C.c_void_p]
     lib.sd_lmhead_argmax.restype = C.c_int
     lib.sd_lmhead_argmax.argtypes = [C.c_void_p, C.c_void_p, C.c_int32, C.c_int32, C.c_int32,
                                      C.c_void_p, C.c_void_p, C.c_void_p, C.c_size_t, C.c_void_p, C.c_void_p]
@@ -162,6 +167,30 @@ def sd_verify_attention(batch: Batch, cache: sd_kv_layer, q, k_tree, v_tree, sca
                                    C.c_float(scale), _ptr(out), _ptr(lse), _ptr(workspace),
                                    workspace.numel() * workspace.element_size(), _ptr(status),
                                    _stream(stream)))
+
+
+class AttentionLayerSet:
+    """Host arrays of per-layer pointers for ``sd_verify_attention_layers`` (built once, reused)."""
+
+    def __init__(self, k_caches, v_caches, qs, k_trees, v_trees, outs, lses=None):
+        L = len(k_caches)
+        self.L = L
+        self.caches = (sd_kv_layer * L)(*[kv_layer(k, v) for k, v in zip(k_caches, v_caches)])
+        self.q = (C.c_void_p * L)(*[_ptr(t) for t in qs])
+        self.kt = (C.c_void_p * L)(*[_ptr(t) for t in k_trees])
+        self.vt = (C.c_void_p * L)(*[_ptr(t) for t in v_trees])
+        self.out = (C.c_void_p * L)(*[_ptr(t) for t in outs])
+        self.lse = (C.c_void_p * L)(*[_ptr(t) for t in lses]) if lses is not None else None
+        self._keep = (list(k_caches), list(v_caches), list(qs), list(k_trees), list(v_trees), list(outs),
+                      list(lses) if lses is not None else None)
+
+
+def sd_verify_attention_layers(batch: Batch, layers: AttentionLayerSet, scale: float, workspace, status,
+                               stream=None) -> None:
+    _check(lib.sd_verify_attention_layers(batch.ref(), layers.caches, layers.L, layers.q, layers.kt, layers.vt,
+                                          C.c_float(scale), layers.out, layers.lse, _ptr(workspace),
+                                          workspace.numel() * workspace.element_size(), _ptr(status),
+                                          _stream(stream)))
 
 
 def sd_lmhead_argmax(hidden, W, argmax, maxlogit, workspace, status, stream=None) -> None:

@@ -74,6 +74,28 @@ sd_status sd_verify_attention(const sd_batch* batch, const sd_kv_layer* cache,
                             workspace_bytes, dev_status, static_cast<cudaStream_t>(stream));
 }
 
+sd_status sd_verify_attention_layers(const sd_batch* batch, const sd_kv_layer* caches, int32_t L,
+                                     const void* const* q_layers, const void* const* k_tree_layers,
+                                     const void* const* v_tree_layers, float scale,
+                                     void* const* out_layers, float* const* lse_layers,
+                                     void* workspace, size_t workspace_bytes,
+                                     int32_t* dev_status, void* stream) {
+    sd_status s = check_geometry(batch, true);
+    if (s != SD_OK) return s;
+    if (!caches || L < 1 || !q_layers || !k_tree_layers || !v_tree_layers || !out_layers) return SD_ERR_INVALID_ARG;
+    if (!ok_ptr(batch->anc_mask) || !ok_ptr(workspace) || !dev_status) return SD_ERR_INVALID_ARG;
+    if (!(scale > 0.f)) return SD_ERR_INVALID_ARG;
+    for (int l = 0; l < L; ++l) {
+        if (!ok_ptr(caches[l].k) || !ok_ptr(caches[l].v) || caches[l].num_blocks < 1) return SD_ERR_INVALID_ARG;
+        if (!ok_ptr(q_layers[l]) || !ok_ptr(k_tree_layers[l]) || !ok_ptr(v_tree_layers[l]) || !ok_ptr(out_layers[l]))
+            return SD_ERR_INVALID_ARG;
+        if (lse_layers && lse_layers[l] && (reinterpret_cast<uintptr_t>(lse_layers[l]) & 3u)) return SD_ERR_INVALID_ARG;
+    }
+    (void)workspace_bytes;
+    return launch_attention_layers(*batch, caches, L, q_layers, k_tree_layers, v_tree_layers, scale, out_layers,
+                                   lse_layers, dev_status, static_cast<cudaStream_t>(stream));
+}
+
 sd_status sd_lmhead_argmax(const void* hidden, const void* W, int32_t M, int32_t Hd, int32_t V,
                            int32_t* argmax, float* maxlogit, void* workspace, size_t workspace_bytes,
                            int32_t* dev_status, void* stream) {

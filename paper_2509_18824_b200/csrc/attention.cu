@@ -51,7 +51,7 @@ struct AttnPlan {
     int row_tiles;
 };
 
-static AttnPlan make_plan(const sd_batch& bt, int sms) {
+static AttnPlan make_plan(const sd_batch& bt, int n_layers, int sms) {
     AttnPlan p;
     const int G = bt.Hq / bt.Hkv;
     p.rows = bt.T_max * G;
@@ -59,7 +59,7 @@ static AttnPlan make_plan(const sd_batch& bt, int sms) {
     // Pick the chunk count that minimises (waves of CTAs) x (key tiles per CTA + fixed cost),
     // two CTAs being resident per SM.  Few waves are counted whole; many waves balance out.
     const int max_tiles = bt.max_blocks_per_seq;
-    const int base = bt.B * bt.Hkv * p.row_tiles;
+    const int base = n_layers * bt.B * bt.Hkv * p.row_tiles;
     const int slots = 2 * sms;
     int n = 1;
     double best = 1e30;
@@ -88,10 +88,19 @@ static int sm_count() {
 // attention needs no global scratch (a nominal size keeps the argument checks uniform).
 size_t attention_workspace_bytes(const sd_batch&) { return 256; }
 
-struct AttnMaps {
+// Everything the CTAs of one layer need.  A launch covers up to kMaxLayersPerLaunch layers (the
+// descriptors travel as kernel parameters); blockIdx.z enumerates (layer, sequence, KV head).
+struct AttnLayer {
     CUtensorMap k_cache, v_cache;   // 2-D [num_blocks*Hkv*64][128], box 64 x 64
     CUtensorMap k_tree, v_tree;     // 3-D (128, Hkv, B*T_max), box 64 x 1 x 64
+    const uint16_t* q;              // bf16 [B][T_max][Hq][D]
+    __nv_bfloat16* out;             // bf16 [B][T_max][Hq][D]
+    float* lse;                     // f32  [B][T_max][Hq] or null
+    int32_t num_blocks;
 };
+constexpr int kMaxLayersPerLaunch = 32;
+template <int NL>
+struct AttnLayers { AttnLayer l[NL]; };
 
 // Final step of a clustered launch.  Each CTA of the cluster finishes 128 / NCH rows of the tile: a
 // warp takes a few rows at a time, every lane four output columns, and adds up the chunks in chunk
@@ -165,11 +174,10 @@ __device__ __forceinline__ void merge_rows(const MergeCtx& x) {
     }
 }
 
+template <int NL>
 __global__ void __launch_bounds__(kAttThreads, 2)
-attn_umma_kernel(const __grid_constant__ AttnMaps maps, const sd_batch bt, const int num_blocks,
-                 const uint16_t* __restrict__ q, const float scale_log2, const AttnPlan plan,
-                 __nv_bfloat16* __restrict__ out, float* __restrict__ lse,
-                 int32_t* status) {
+attn_umma_kernel(const __grid_constant__ AttnLayers<NL> layers, const sd_batch bt,
+                 const float scale_log2, const AttnPlan plan, int32_t* status) {
     extern __shared__ __align__(1024) uint8_t smem[];
     uint8_t* q_smem = smem;
     uint8_t* k_smem = smem + kQBytes;
@@ -193,8 +201,18 @@ attn_umma_kernel(const __grid_constant__ AttnMaps maps, const sd_batch bt, const
     const int lane = threadIdx.x & 31;
     const int chunk = blockIdx.x;
     const int rt = blockIdx.y;
-    const int b = blockIdx.z / bt.Hkv;
     const int kvh = blockIdx.z % bt.Hkv;
+    const int lb = blockIdx.z / bt.Hkv;
+    const int b = lb % bt.B;
+    const AttnLayer& ly = layers.l[lb / bt.B];
+    const CUtensorMap* const map_kc = &ly.k_cache;
+    const CUtensorMap* const map_vc = &ly.v_cache;
+    const CUtensorMap* const map_kt = &ly.k_tree;
+    const CUtensorMap* const map_vt = &ly.v_tree;
+    const uint16_t* __restrict__ q = ly.q;
+    __nv_bfloat16* __restrict__ out = ly.out;
+    float* __restrict__ lse = ly.lse;
+    const int num_blocks = ly.num_blocks;
     const int G = bt.Hq / bt.Hkv;
     const int T = bt.T_max;
     const int n = min(max(bt.n_nodes[b], 0), T);
@@ -229,8 +247,8 @@ attn_umma_kernel(const __grid_constant__ AttnMaps maps, const sd_batch bt, const
         tmem_relinquish();
     }
     if (warp == kTmaWarp && lane == 0) {
-        prefetch_tensormap(&maps.k_cache); prefetch_tensormap(&maps.v_cache);
-        prefetch_tensormap(&maps.k_tree); prefetch_tensormap(&maps.v_tree);
+        prefetch_tensormap(map_kc); prefetch_tensormap(map_vc);
+        prefetch_tensormap(map_kt); prefetch_tensormap(map_vt);
     }
     tc_fence_before_sync();
     __syncthreads();
@@ -260,12 +278,12 @@ attn_umma_kernel(const __grid_constant__ AttnMaps maps, const sd_batch bt, const
                 uint8_t* dst = (is_v ? v_smem : k_smem) + s * kKVStage;
                 mbar_arrive_expect_tx(full, kKVStage);
                 if (j >= n_pref) {
-                    const CUtensorMap* m = is_v ? &maps.v_tree : &maps.k_tree;
+                    const CUtensorMap* m = is_v ? map_vt : map_kt;
                     tma_load_3d(dst, m, 0, kvh, b * T, full, pol);
                     tma_load_3d(dst + kSubTile, m, 64, kvh, b * T, full, pol);
                 } else {
                     if (blk < 0 || blk >= num_blocks) { set_status(status, SD_ERR_BOUNDS); blk = 0; }
-                    const CUtensorMap* m = is_v ? &maps.v_cache : &maps.k_cache;
+                    const CUtensorMap* m = is_v ? map_vc : map_kc;
                     const int y = (blk * bt.Hkv + kvh) * kKeyTile;
                     tma_load_2d(dst, m, 0, y, full, pol);
                     tma_load_2d(dst + kSubTile, m, 64, y, full, pol);
@@ -527,26 +545,34 @@ attn_umma_kernel(const __grid_constant__ AttnMaps maps, const sd_batch bt, const
     }
 }
 
-sd_status launch_attention(const sd_batch& bt, const sd_kv_layer& cache, const void* q,
-                           const void* kt, const void* vt, float scale, void* out, float* lse,
-                           void* ws, size_t ws_bytes, int32_t* dev_status, cudaStream_t st) {
-    const AttnPlan plan = make_plan(bt, sm_count());
-    (void)ws_bytes;
-    AttnMaps maps;
+static bool fill_layer(AttnLayer* ly, const sd_batch& bt, const sd_kv_layer& cache, const void* q,
+                       const void* kt, const void* vt, void* out, float* lse) {
     const uint64_t cache_rows = (uint64_t)cache.num_blocks * bt.Hkv * kKeyTile;
-    if (!encode_tmap_bf16_2d(&maps.k_cache, cache.k, cache_rows, kD, kD * 2, 64, kKeyTile, 128) ||
-        !encode_tmap_bf16_2d(&maps.v_cache, cache.v, cache_rows, kD, kD * 2, 64, kKeyTile, 128))
-        return SD_ERR_CUDA;
+    if (!encode_tmap_bf16_2d(&ly->k_cache, cache.k, cache_rows, kD, kD * 2, 64, kKeyTile, 128) ||
+        !encode_tmap_bf16_2d(&ly->v_cache, cache.v, cache_rows, kD, kD * 2, 64, kKeyTile, 128))
+        return false;
     const uint64_t dims[3] = {(uint64_t)kD, (uint64_t)bt.Hkv, (uint64_t)bt.B * bt.T_max};
     const uint64_t strides[2] = {(uint64_t)kD * 2, (uint64_t)bt.Hkv * kD * 2};
     const uint32_t box[3] = {64, 1, kKeyTile};
-    if (!encode_tmap_bf16_3d(&maps.k_tree, kt, dims, strides, box, 128) ||
-        !encode_tmap_bf16_3d(&maps.v_tree, vt, dims, strides, box, 128))
-        return SD_ERR_CUDA;
-    if (cudaFuncSetAttribute(attn_umma_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, kAttSmem) != cudaSuccess)
+    if (!encode_tmap_bf16_3d(&ly->k_tree, kt, dims, strides, box, 128) ||
+        !encode_tmap_bf16_3d(&ly->v_tree, vt, dims, strides, box, 128))
+        return false;
+    ly->q = static_cast<const uint16_t*>(q);
+    ly->out = static_cast<__nv_bfloat16*>(out);
+    ly->lse = lse;
+    ly->num_blocks = cache.num_blocks;
+    return true;
+}
+
+template <int NL>
+static sd_status launch_group(const AttnLayers<NL>& layers, int n_layers, const sd_batch& bt, float scale,
+                              int32_t* dev_status, cudaStream_t st) {
+    const AttnPlan plan = make_plan(bt, n_layers, sm_count());
+    auto kern = attn_umma_kernel<NL>;
+    if (cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, kAttSmem) != cudaSuccess)
         return SD_ERR_CUDA;
     cudaLaunchConfig_t cfg = {};
-    cfg.gridDim = dim3(plan.n_chunks, plan.row_tiles, bt.B * bt.Hkv);
+    cfg.gridDim = dim3(plan.n_chunks, plan.row_tiles, n_layers * bt.B * bt.Hkv);
     cfg.blockDim = dim3(kAttThreads);
     cfg.dynamicSmemBytes = kAttSmem;
     cfg.stream = st;
@@ -557,11 +583,48 @@ sd_status launch_attention(const sd_batch& bt, const sd_kv_layer& cache, const v
     attr[0].val.clusterDim.z = 1;
     cfg.attrs = attr;
     cfg.numAttrs = 1;
-    if (cudaLaunchKernelEx(&cfg, attn_umma_kernel, maps, bt, cache.num_blocks, static_cast<const uint16_t*>(q),
-                           scale * kLog2e, plan, static_cast<__nv_bfloat16*>(out), lse, dev_status) != cudaSuccess)
+    if (cudaLaunchKernelEx(&cfg, kern, layers, bt, scale * kLog2e, plan, dev_status) != cudaSuccess)
         return SD_ERR_CUDA;
-    (void)ws;
     return SD_OK;
+}
+
+// One launch per group of layers: at most kMaxLayersPerLaunch descriptors fit the kernel's
+// parameter space and gridDim.z is limited to 65535.
+sd_status launch_attention_layers(const sd_batch& bt, const sd_kv_layer* caches, int L,
+                                  const void* const* q, const void* const* kt, const void* const* vt,
+                                  float scale, void* const* out, float* const* lse,
+                                  int32_t* dev_status, cudaStream_t st) {
+    const int per_layer_z = bt.B * bt.Hkv;
+    if (per_layer_z > 65535) return SD_ERR_UNSUPPORTED;
+    int group = 65535 / per_layer_z;
+    if (group > kMaxLayersPerLaunch) group = kMaxLayersPerLaunch;
+    for (int l0 = 0; l0 < L; l0 += group) {
+        const int nl = (L - l0 < group) ? (L - l0) : group;
+        if (nl == 1) {
+            AttnLayers<1> one;
+            if (!fill_layer(&one.l[0], bt, caches[l0], q[l0], kt[l0], vt[l0], out[l0], lse ? lse[l0] : nullptr))
+                return SD_ERR_CUDA;
+            sd_status s = launch_group<1>(one, 1, bt, scale, dev_status, st);
+            if (s != SD_OK) return s;
+        } else {
+            AttnLayers<kMaxLayersPerLaunch> many;
+            for (int i = 0; i < nl; ++i)
+                if (!fill_layer(&many.l[i], bt, caches[l0 + i], q[l0 + i], kt[l0 + i], vt[l0 + i], out[l0 + i],
+                                lse ? lse[l0 + i] : nullptr))
+                    return SD_ERR_CUDA;
+            for (int i = nl; i < kMaxLayersPerLaunch; ++i) many.l[i] = many.l[0];
+            sd_status s = launch_group<kMaxLayersPerLaunch>(many, nl, bt, scale, dev_status, st);
+            if (s != SD_OK) return s;
+        }
+    }
+    return SD_OK;
+}
+
+sd_status launch_attention(const sd_batch& bt, const sd_kv_layer& cache, const void* q,
+                           const void* kt, const void* vt, float scale, void* out, float* lse,
+                           void* ws, size_t ws_bytes, int32_t* dev_status, cudaStream_t st) {
+    (void)ws; (void)ws_bytes;
+    return launch_attention_layers(bt, &cache, 1, &q, &kt, &vt, scale, &out, &lse, dev_status, st);
 }
 
 }  // namespace sdv

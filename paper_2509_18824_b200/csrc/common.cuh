@@ -38,6 +38,10 @@ size_t attention_workspace_bytes(const sd_batch& bt);
 sd_status launch_attention(const sd_batch& bt, const sd_kv_layer& cache, const void* q,
                            const void* kt, const void* vt, float scale, void* out, float* lse,
                            void* ws, size_t ws_bytes, int32_t* dev_status, cudaStream_t st);
+sd_status launch_attention_layers(const sd_batch& bt, const sd_kv_layer* caches, int L,
+                                  const void* const* q, const void* const* kt, const void* const* vt,
+                                  float scale, void* const* out, float* const* lse,
+                                  int32_t* dev_status, cudaStream_t st);
 size_t lmhead_workspace_bytes(int M, int V);
 sd_status launch_lmhead(const void* hidden, const void* W, int M, int Hd, int V,
                         int32_t* argmax, float* maxlogit, void* ws, size_t ws_bytes,

@@ -65,6 +65,8 @@ class VerifyStep:
         self.workspace = torch.empty(max(nbytes, 256), dtype=torch.uint8, device=d)
         self.caches = [sd.kv_layer(k, v) for k, v in zip(self.k_cache, self.v_cache)]
         self.layerset = sd.LayerSet(self.k_cache, self.v_cache, self.k_tree, self.v_tree)
+        self.att_all = self._attention_set(0, self.L)
+        self._att_groups = {}
         self.scale = float(w.scale)
         sd.sd_tree_prepare(self.batch, self.status)
         # pinned host copies for the end-to-end path
@@ -86,6 +88,22 @@ class VerifyStep:
         sd.sd_verify_attention(self.batch, self.caches[l], self.q[l], self.k_tree[l], self.v_tree[l],
                                self.scale, self.out[l], self.lse[l], self.workspace, self.status, stream)
 
+    def _attention_set(self, l0: int, l1: int):
+        s = slice(l0, l1)
+        return sd.AttentionLayerSet(self.k_cache[s], self.v_cache[s], self.q[s], self.k_tree[s], self.v_tree[s],
+                                    self.out[s], self.lse[s])
+
+    def attention_layers(self, l0: int = 0, l1: Optional[int] = None, stream=None):
+        """Layers l0..l1-1 in one library call (all layers by default)."""
+        l1 = self.L if l1 is None else l1
+        if (l0, l1) == (0, self.L):
+            ls = self.att_all
+        else:
+            ls = self._att_groups.get((l0, l1))
+            if ls is None:
+                ls = self._att_groups[(l0, l1)] = self._attention_set(l0, l1)
+        sd.sd_verify_attention_layers(self.batch, ls, self.scale, self.workspace, self.status, stream)
+
     def lmhead(self, stream=None):
         sd.sd_lmhead_argmax(self.hidden, self.W, self.argmax, self.maxlogit, self.workspace, self.status, stream)
 
@@ -97,18 +115,24 @@ class VerifyStep:
         sd.sd_compact_kv(self.batch, self.layerset, self.n_acc, self.path, self.status, stream)
 
     # -- the whole step -------------------------------------------------
-    def run(self, stream=None):
-        for l in range(self.L):
-            self.attention(l, stream)
+    def run(self, stream=None, per_layer=False):
+        """All layers' attention in one call (the step's q and tree K/V are all present up front);
+        per_layer=True issues one call per layer, as a decoder that interleaves its own layers would."""
+        if per_layer:
+            for l in range(self.L):
+                self.attention(l, stream)
+        else:
+            self.attention_layers(stream=stream)
         self.lmhead(stream)
         self.accept(None, stream)
         self.compact(stream)
 
     @property
     def launches_per_step(self) -> int:
-        """Kernel launches of one run(): per layer the partial and the merge kernel;
-        the LM-head kernels; acceptance; compaction."""
-        return self.L * sd.KERNELS_PER_ATTENTION + sd.KERNELS_PER_LMHEAD + 1 + (self.L + 63) // 64
+        """Kernel launches of one run(): attention (one launch per group of up to 32 layers), the
+        LM-head kernels, acceptance, compaction."""
+        return ((self.L + sd.ATTENTION_LAYERS_PER_LAUNCH - 1) // sd.ATTENTION_LAYERS_PER_LAUNCH
+                + sd.KERNELS_PER_LMHEAD + 1 + (self.L + 63) // 64)
 
     def h2d_bytes(self) -> int:
         h = self.host
@@ -118,12 +142,12 @@ class VerifyStep:
     def d2h_bytes(self) -> int:
         return sum(t.numel() * t.element_size() for t in self.host_out.values())
 
-    def run_from_host(self):
+    def run_from_host(self, group: int = 7):
         """End-to-end step: this step's inputs come from pinned host memory, the
         accepted tokens go back to the host; caches and weights stay resident.
-        The host-to-device copies run on a second stream, one layer ahead of the
-        layer that is being computed; every call that reads a buffer first waits
-        for the event recorded behind that buffer's copy."""
+        The host-to-device copies run on a second stream, ahead of the compute:
+        attention is issued in groups of `group` layers, each group as soon as
+        its layers' copies have landed (an event recorded behind them)."""
         h = self.host
         main = torch.cuda.current_stream()
         if self._copy_stream is None:
@@ -145,9 +169,10 @@ class VerifyStep:
             self.draft_tok.copy_(h["draft_tok"], non_blocking=True)
         main.wait_event(self._ev_small)
         sd.sd_tree_prepare(self.batch, self.status)
-        for l in range(self.L):
-            main.wait_event(self._ev_layer[l])
-            self.attention(l)
+        for l0 in range(0, self.L, group):
+            l1 = min(l0 + group, self.L)
+            main.wait_event(self._ev_layer[l1 - 1])
+            self.attention_layers(l0, l1)
         main.wait_stream(cs)            # hidden states and draft tokens have arrived
         self.lmhead()
         self.accept()

@@ -204,6 +204,74 @@ def test_attention_full_size_sampled_rows(cfg, gain):
     assert np.isfinite(out).all()
 
 
+def gpu_attention_layers(w, layers):
+    """sd_verify_attention_layers over the listed layers of a workload; returns per-layer (out, lse)."""
+    bt = sd.Batch.of(w)
+    st = sd.new_status()
+    sd.sd_tree_prepare(bt, st)
+    dev = lambda xs: [to_device(xs[l]) for l in layers]
+    kc, vc, q, kt, vt = dev(w.k_cache), dev(w.v_cache), dev(w.q), dev(w.k_tree), dev(w.v_tree)
+    out = [torch.full((w.B, w.T_max, w.Hq, w.D), 7.0, dtype=torch.bfloat16, device="cuda") for _ in layers]
+    lse = [torch.full((w.B, w.T_max, w.Hq), 7.0, dtype=torch.float32, device="cuda") for _ in layers]
+    ws = torch.empty(sd.sd_workspace_bytes(bt), dtype=torch.uint8, device="cuda")
+    ls = sd.AttentionLayerSet(kc, vc, q, kt, vt, out, lse)
+    sd.sd_verify_attention_layers(bt, ls, float(w.scale), ws, st)
+    torch.cuda.synchronize()
+    assert int(st.item()) == 0
+    return [(o.float().cpu().numpy(), l.cpu().numpy()) for o, l in zip(out, lse)]
+
+
+@pytest.mark.parametrize("cfg,L,gain", [("c1", 3, 45.0), ("c2", 2, 45.0), ("c2", 5, 1.0)])
+def test_attention_layers_call_full_compare(cfg, L, gain):
+    """Several layers in one call (few enough that the keys are still split into chunks): every
+    layer against the checker, element by element."""
+    w = wl.make(cfg, lmhead=False, q_gain=gain, L=L)
+    got = gpu_attention_layers(w, list(range(L)))
+    G = oracle.Geometry.of(w)
+    for l in range(L):
+        ref, rlse = oracle.attention(G, w.k_cache[l], w.v_cache[l], w.q[l], w.k_tree[l], w.v_tree[l], w.scale)
+        check_attention(got[l][0], ref, f"{cfg} layer {l}")
+        np.testing.assert_allclose(got[l][1], rlse, rtol=2e-3, atol=2e-3)
+
+
+def test_attention_layers_call_many_layers_ragged():
+    """More layers than one launch holds (33 > 32), ragged lengths, unused nodes, shuffled blocks:
+    every layer must land in its own output and agree with the checker."""
+    L = 33
+    g = np.random.default_rng(21)
+    T = 24
+    par = np.stack([np.array([-1] + [int(g.integers(max(0, i - 5), i)) for i in range(1, T)]) for _ in range(2)])
+    w = tiny128(100, B=2, T=T, Hq=14, Hkv=2, lens=(130, 61), parents=par, gain=3.0)
+    w.n_nodes = np.array([24, 9], dtype=np.int32)
+
+    class Layer:
+        pass
+    ps = []
+    for l in range(L):                                 # same geometry for all layers, own tensors each
+        p = Layer()
+        gl = np.random.default_rng(500 + l)
+        for name, k in (("q", 3.0), ("k_tree", 1.0), ("v_tree", 0.3), ("k_cache", 1.0), ("v_cache", 0.3)):
+            shape = getattr(w, name).shape
+            setattr(p, name, wl.f32_to_bf16_bits((gl.standard_normal(shape) * k).astype(np.float32)))
+        ps.append(p)
+
+    class Stack:
+        pass
+    sw = Stack()
+    for name in ("B", "T_max", "Hq", "Hkv", "D", "block_table", "len", "n_nodes", "parents", "scale"):
+        setattr(sw, name, getattr(w, name))
+    for name in ("k_cache", "v_cache", "q", "k_tree", "v_tree"):
+        setattr(sw, name, [getattr(p, name) for p in ps])
+    got = gpu_attention_layers(sw, list(range(L)))
+    G = oracle.Geometry.of(w)
+    for l in range(L):
+        ref, rlse = oracle.attention(G, ps[l].k_cache, ps[l].v_cache, ps[l].q, ps[l].k_tree, ps[l].v_tree, w.scale)
+        check_attention(got[l][0], ref, f"layer {l}")
+        ok = np.isfinite(rlse)
+        np.testing.assert_allclose(got[l][1][ok], rlse[ok], rtol=2e-3, atol=2e-3)
+        assert (got[l][0][1, 9:] == 0).all()
+
+
 # ------------------------------------------------------------------ LM head
 @pytest.mark.parametrize("M,Hd,V", [(1, 64, 1), (5, 128, 1000), (8, 256, 1024), (61, 192, 129), (130, 64, 4099)])
 def test_lmhead_small_shapes_crisp(M, Hd, V):
@@ -309,11 +377,19 @@ def test_full_step_c5_shapes():
     np.testing.assert_array_equal(ref_acc[0], w.planted_len + 1)
 
     vs = VerifyStep(w)
-    for l in range(vs.L):
+    for l in range(vs.L):                              # one call per layer ...
         vs.attention(l)
+    torch.cuda.synchronize()
+    single = [o.clone() for o in vs.out]
+    for o in vs.out:
+        o.fill_(7.0)
+    vs.attention_layers()                              # ... and all layers in one call, as run() does
     vs.lmhead()
     torch.cuda.synchronize()
     vs.check_status()
+    for l in range(vs.L):                              # the two ways differ only by fp32 merge rounding
+        d = (vs.out[l].float() - single[l].float()).abs().max().item()
+        assert d <= 2e-3, f"layer {l}: all-layers call differs from the single-layer call by {d}"
     am = vs.argmax.cpu().numpy()
     in_band, mis_in, mis_out = check_argmax(am, vs.maxlogit.cpu().numpy(), ram, t1, t2)
     print(f"c5 LM head: rows {len(am)}, in band {in_band}, mismatches in band {mis_in}, outside {mis_out}")
