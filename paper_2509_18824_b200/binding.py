@@ -45,11 +45,11 @@ class sd_batch(C.Structure):
                 ("parents", C.c_void_p), ("anc_mask", C.c_void_p)]
 
 
-def _load() -> C.CDLL:
-    if not os.path.exists(LIB_PATH):
+def _load(path: str = LIB_PATH) -> C.CDLL:
+    if path == LIB_PATH and not os.path.exists(LIB_PATH):
         from . import build as _build          # needs nvcc; raises if it fails
         _build.build()
-    lib = C.CDLL(LIB_PATH)
+    lib = C.CDLL(path)
     lib.sd_version.restype = C.c_int
     lib.sd_status_string.restype = C.c_char_p
     lib.sd_status_string.argtypes = [C.c_int]

@@ -25,7 +25,7 @@ using namespace sm100;
 
 constexpr int kRowTile = 128;                  // query rows per CTA (MMA M)
 constexpr int kKeyTile = 64;                   // keys per tile = one cache block
-constexpr int kAttThreads = 192;               // warps 0-3 softmax, warp 4 TMA, warp 5 MMA
+constexpr int kAttThreads = 161;               // warps 0-3 softmax, warp 4 TMA, warp 5 = ONE thread: MMA issuer
 constexpr int kTmaWarp = 4, kMmaWarp = 5;
 constexpr int kSubTile = kKeyTile * 128;       // bytes of a [64][64] bf16 swizzled sub-tile (8 KiB)
 constexpr int kQBytes = 2 * kRowTile * 128;    // Q tile: two D-halves of [128][64] bf16 (32 KiB)
@@ -39,6 +39,11 @@ constexpr float kLog2e = 1.4426950408889634f;
 constexpr float kRescaleThreshold = 8.0f;      // log2 units
 constexpr int kMaxChunks = 8;                  // = portable cluster size
 
+__device__ __forceinline__ float max3(float a, float b, float c) {
+    float d;
+    asm("max.f32 %0, %1, %2, %3;" : "=f"(d) : "f"(a), "f"(b), "f"(c));
+    return d;
+}
 __device__ __forceinline__ float ex2_approx(float x) {
     float y;
     asm("ex2.approx.ftz.f32 %0, %1;" : "=f"(y) : "f"(x));
@@ -197,7 +202,9 @@ attn_umma_kernel(const __grid_constant__ AttnLayers<NL> layers, const sd_batch b
     uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(bars + 17);
     int* abort_flag = reinterpret_cast<int*>(bars + 18);
 
-    const int warp = threadIdx.x >> 5;
+    // warp index as a value the compiler knows to be warp-uniform, so that role dispatch is uniform
+    // control flow (a warp's non-existent lanes do not take part in the shuffle)
+    const int warp = __shfl_sync(0xffffffffu, (int)(threadIdx.x >> 5), 0);
     const int lane = threadIdx.x & 31;
     const int chunk = blockIdx.x;
     const int rt = blockIdx.y;
@@ -242,7 +249,7 @@ attn_umma_kernel(const __grid_constant__ AttnLayers<NL> layers, const sd_batch b
         mbar_init(pv_done, 1); mbar_init(q_full, 4); mbar_init(o_full, 1);
         fence_barrier_init();
     }
-    if (warp == kMmaWarp) {
+    if (warp == kTmaWarp) {                                // a full warp (the MMA warp is a single thread)
         tmem_alloc(tmem_slot, kTmemCols);
         tmem_relinquish();
     }
@@ -317,16 +324,15 @@ attn_umma_kernel(const __grid_constant__ AttnLayers<NL> layers, const sd_batch b
         }
     } else if (warp == kMmaWarp) {
         // ------------------------------------------------------------ MMA issuer
-        if (lane == 0) {
+        // This warp consists of one thread (the block has 5 * 32 + 1 threads), so everything in
+        // here is uniform control flow on warp-uniform values: tcgen05.mma takes its descriptors
+        // from uniform registers, and inside a divergent "lane 0 only" region of a full warp every
+        // descriptor would first have to be moved there, instruction by instruction.
+        {
             const uint32_t idesc_s = make_idesc_bf16(kRowTile, kKeyTile, false, false);   // S = Q . K^T
             const uint32_t idesc_o = make_idesc_bf16(kRowTile, kD, false, true);          // O += P . V
-            // Descriptors are prepared outside the issue sequences: every instruction between two
-            // tcgen05.mma of one thread delays the second one.  k-steps only move the (16-byte
-            // granular) start-address field in the low bits.
-            uint64_t qdesc[kD / 16];
-#pragma unroll
-            for (int k = 0; k < kD / 16; ++k)
-                qdesc[k] = make_smem_desc(smem_u32(q_smem) + (k >> 2) * (kRowTile * 128) + (k & 3) * 32, 16, 1024, 128);
+            // k-steps only move the (16-byte granular) start-address field in the low bits
+            const uint64_t qdesc_base = make_smem_desc(smem_u32(q_smem), 16, 1024, 128);
             const uint64_t kdesc_base = make_smem_desc(smem_u32(k_smem), 16, 1024, 128);
             // V is stored [key][d]: N (= d) contiguous; D-halves kSubTile apart, 8-key groups 1 KiB apart
             const uint64_t vdesc_base = make_smem_desc(smem_u32(v_smem), kSubTile, 1024, 128);
@@ -340,7 +346,8 @@ attn_umma_kernel(const __grid_constant__ AttnLayers<NL> layers, const sd_batch b
                 const uint32_t d = tmem_s + s * kKeyTile;
 #pragma unroll
                 for (int k = 0; k < kD / 16; ++k)
-                    mma_ss(d, qdesc[k], kd + (uint64_t)((k >> 2) * (kSubTile >> 4) + (k & 3) * 2), idesc_s, k != 0 ? 1u : 0u);
+                    mma_ss(d, qdesc_base + (uint64_t)((k >> 2) * ((kRowTile * 128) >> 4) + (k & 3) * 2),
+                           kd + (uint64_t)((k >> 2) * (kSubTile >> 4) + (k & 3) * 2), idesc_s, k != 0 ? 1u : 0u);
                 mma_commit(&k_empty[ks]);
                 mma_commit(&s_full[s]);
                 return true;
@@ -395,36 +402,61 @@ attn_umma_kernel(const __grid_constant__ AttnLayers<NL> layers, const sd_batch b
             const uint32_t ph = (uint32_t)(j >> 1) & 1u;
             if (!mbar_wait(&s_full[s], ph, abort_flag)) { ok = false; break; }
             tc_fence_after_sync();
+            // The scores arrive in two halves; the second half is in flight while the first is
+            // processed.  Raw scores stay unscaled: scale * log2(e) is folded into the exponent's FMA.
             uint32_t r0[32], r1[32];
             tmem_ld32(tmem_s + lane_field + s * kKeyTile, r0);
-            tmem_ld32(tmem_s + lane_field + s * kKeyTile + 32, r1);
             tmem_ld_wait();
-
-            // raw scores stay unscaled; scale * log2(e) is folded into the exponent's FMA
-            float sc[64];
-#pragma unroll
-            for (int c = 0; c < 32; ++c) { sc[c] = __uint_as_float(r0[c]); sc[32 + c] = __uint_as_float(r1[c]); }
+            tmem_ld32(tmem_s + lane_field + s * kKeyTile + 32, r1);
             const bool tree = (j >= t1 - t0);
-            if (tree) {
+            const int valid = tree ? kKeyTile : len - (t0 + j) * kKeyTile;   // keys of this block inside the prefix
+            const uint32_t mask_lo = tree ? (uint32_t)amask : (valid >= 32 ? ~0u : ((1u << max(valid, 0)) - 1u));
+            const uint32_t mask_hi = tree ? (uint32_t)(amask >> 32)
+                                          : (valid >= 64 ? ~0u : (valid <= 32 ? 0u : ((1u << (valid - 32)) - 1u)));
+            const bool masked = tree || valid < kKeyTile;
+            if (masked) {
 #pragma unroll
-                for (int c = 0; c < 64; ++c) sc[c] = ((amask >> c) & 1ull) ? sc[c] : -INFINITY;
-            } else {
-                const int valid = len - (t0 + j) * kKeyTile;        // keys of this block inside the prefix
-                if (valid < kKeyTile) {
-#pragma unroll
-                    for (int c = 0; c < 64; ++c) sc[c] = (c < valid) ? sc[c] : -INFINITY;
-                }
+                for (int c = 0; c < 32; ++c)
+                    r0[c] = ((mask_lo >> c) & 1u) ? r0[c] : 0xff800000u;      // -inf
             }
-            float mx[4] = {sc[0], sc[1], sc[2], sc[3]};
+            // The exponentials are taken against the current reference maximum right away, while the
+            // tile's own maximum is found alongside (independent instruction streams); only when that
+            // maximum turns out to exceed the reference by more than the threshold (rare after the
+            // first tiles) is the reference raised and the tile's exponentials redone.
+            uint32_t pk[32];
+            float ps[4] = {0.f, 0.f, 0.f, 0.f};
+            float mx[4] = {-INFINITY, -INFINITY, -INFINITY, -INFINITY};
+            const float neg_m = -m_used;
 #pragma unroll
-            for (int c = 4; c < 64; c += 4) {
-                mx[0] = fmaxf(mx[0], sc[c]); mx[1] = fmaxf(mx[1], sc[c + 1]);
-                mx[2] = fmaxf(mx[2], sc[c + 2]); mx[3] = fmaxf(mx[3], sc[c + 3]);
+            for (int c = 0; c < 16; ++c) {
+                const float a = __uint_as_float(r0[2 * c]), bq = __uint_as_float(r0[2 * c + 1]);
+                mx[c & 3] = max3(mx[c & 3], a, bq);
+                const float p0 = ex2_approx(fmaf(a, scale_log2, neg_m));
+                const float p1 = ex2_approx(fmaf(bq, scale_log2, neg_m));
+                ps[c & 3] += p0 + p1;
+                __nv_bfloat162 h = __floats2bfloat162_rn(p0, p1);
+                pk[c] = *reinterpret_cast<uint32_t*>(&h);
+            }
+            tmem_ld_wait();
+            if (masked) {
+#pragma unroll
+                for (int c = 0; c < 32; ++c)
+                    r1[c] = ((mask_hi >> c) & 1u) ? r1[c] : 0xff800000u;
+            }
+#pragma unroll
+            for (int c = 0; c < 16; ++c) {
+                const float a = __uint_as_float(r1[2 * c]), bq = __uint_as_float(r1[2 * c + 1]);
+                mx[c & 3] = max3(mx[c & 3], a, bq);
+                const float p0 = ex2_approx(fmaf(a, scale_log2, neg_m));
+                const float p1 = ex2_approx(fmaf(bq, scale_log2, neg_m));
+                ps[c & 3] += p0 + p1;
+                __nv_bfloat162 h = __floats2bfloat162_rn(p0, p1);
+                pk[16 + c] = *reinterpret_cast<uint32_t*>(&h);
             }
             const float mt = fmaxf(fmaxf(mx[0], mx[1]), fmaxf(mx[2], mx[3])) * scale_log2;   // scale > 0
             // raise the reference maximum only when it would grow by more than the threshold
             const bool raise = mt > m_used + kRescaleThreshold;      // true on the first tile (m_used = -inf)
-                        if (__any_sync(0xffffffffu, raise)) {
+            if (__any_sync(0xffffffffu, raise)) {
                 if (j > 0) {
                     if (!mbar_wait(pv_done, (uint32_t)(j - 1) & 1u, abort_flag)) { ok = false; break; }
                     tc_fence_after_sync();
@@ -442,17 +474,21 @@ attn_umma_kernel(const __grid_constant__ AttnLayers<NL> layers, const sd_batch b
                     l *= alpha;
                 }
                 if (raise) m_used = mt;
-            }
-            uint32_t pk[32];
-            float ps[4] = {0.f, 0.f, 0.f, 0.f};
-            const float neg_m = -m_used;
+                // redo the tile against the new reference (same values for rows that did not raise)
+                const float neg_m2 = -m_used;
+                ps[0] = ps[1] = ps[2] = ps[3] = 0.f;
 #pragma unroll
-            for (int c = 0; c < 32; ++c) {
-                const float p0 = ex2_approx(fmaf(sc[2 * c], scale_log2, neg_m));
-                const float p1 = ex2_approx(fmaf(sc[2 * c + 1], scale_log2, neg_m));
-                ps[c & 3] += p0 + p1;
-                __nv_bfloat162 h = __floats2bfloat162_rn(p0, p1);
-                pk[c] = *reinterpret_cast<uint32_t*>(&h);
+                for (int c = 0; c < 16; ++c) {
+                    const float p0 = ex2_approx(fmaf(__uint_as_float(r0[2 * c]), scale_log2, neg_m2));
+                    const float p1 = ex2_approx(fmaf(__uint_as_float(r0[2 * c + 1]), scale_log2, neg_m2));
+                    const float p2 = ex2_approx(fmaf(__uint_as_float(r1[2 * c]), scale_log2, neg_m2));
+                    const float p3 = ex2_approx(fmaf(__uint_as_float(r1[2 * c + 1]), scale_log2, neg_m2));
+                    ps[c & 3] += (p0 + p1) + (p2 + p3);
+                    __nv_bfloat162 h0 = __floats2bfloat162_rn(p0, p1);
+                    __nv_bfloat162 h1 = __floats2bfloat162_rn(p2, p3);
+                    pk[c] = *reinterpret_cast<uint32_t*>(&h0);
+                    pk[16 + c] = *reinterpret_cast<uint32_t*>(&h1);
+                }
             }
             const float psum = (ps[0] + ps[1]) + (ps[2] + ps[3]);
             l += psum;
@@ -539,7 +575,7 @@ attn_umma_kernel(const __grid_constant__ AttnLayers<NL> layers, const sd_batch b
     if (!active) return;
     tc_fence_before_sync();
     __syncthreads();
-    if (warp == kMmaWarp) {
+    if (warp == kTmaWarp) {
         tc_fence_after_sync();
         tmem_dealloc(tmem_base, kTmemCols);
     }
