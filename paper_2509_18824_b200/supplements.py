@@ -2,7 +2,7 @@
 the LM head at several row counts, and the bandwidth-regime cases (chain
 decoding, a compaction stress shape).  One JSON line per measurement.
 
-    python -m paper_2509_18824_b200.supplements [attention] [lmhead] [compact]
+    python -m paper_2509_18824_b200.supplements [attention] [attention_layers] [lmhead] [compact]
 
 Timing: CUDA events on the launching stream, >= 3 warm-up calls, inputs rotated
 over several layers so that the working set exceeds L2.
@@ -75,6 +75,38 @@ def attention(configs=("c2", "c3", "c4", "c5", "chain11")):
         torch.cuda.empty_cache()
 
 
+def attention_layers(configs=("c5", "chain11", "c4"), L=28):
+    """All L layers through sd_verify_attention_layers (one launch): the regime of a whole verify
+    step, where per-launch costs are paid once.  chain11 is the bandwidth-bound case."""
+    hbm, tens, src = _peaks()
+    for cfg in configs:
+        sp = wl.spec(cfg)
+        sp.L = L if cfg != "c4" else 8             # c4's caches are 4x larger per layer
+        w = wl.make_geometry(sp)
+        wl.fill_attention(w)
+        bt = sd.Batch.of(w)
+        st = sd.new_status()
+        sd.sd_tree_prepare(bt, st)
+        kc = [to_device(x) for x in w.k_cache]; vc = [to_device(x) for x in w.v_cache]
+        q = [to_device(x) for x in w.q]; kt = [to_device(x) for x in w.k_tree]; vt = [to_device(x) for x in w.v_tree]
+        out = [torch.zeros((w.B, w.T_max, w.Hq, w.D), dtype=torch.bfloat16, device="cuda") for _ in range(w.L)]
+        ws = torch.empty(sd.sd_workspace_bytes(bt), dtype=torch.uint8, device="cuda")
+        ls = sd.AttentionLayerSet(kc, vc, q, kt, vt, out)
+        ms = _time(lambda: sd.sd_verify_attention_layers(bt, ls, w.scale, ws, st), 20)
+        vis = sum(int((int(w.len[b]) + wl.node_depths(w.parents[b]) + 1).sum()) for b in range(w.B))
+        flops = 4.0 * w.D * w.Hq * vis * w.L
+        nbytes = (sum(int(w.len[b]) + w.T_max for b in range(w.B)) * w.Hkv * w.D * 4
+                  + 2 * w.B * w.T_max * w.Hq * w.D * 2) * w.L
+        print(json.dumps({"call": "sd_verify_attention_layers", "workload": cfg, "layers": w.L, "us": ms * 1e3,
+                          "us_per_layer": ms * 1e3 / w.L,
+                          "tflops": flops / ms / 1e9, "frac_tensor_burst": flops / ms / 1e9 / tens,
+                          "gbs": nbytes / ms / 1e6, "frac_hbm": nbytes / ms / 1e6 / hbm,
+                          "frac_hbm_nominal_8TBs": nbytes / ms / 1e6 / 8000.0,
+                          "flop_per_byte": flops / nbytes, "peaks": src, "status": int(st.item())}))
+        del kc, vc, q, kt, vt, out, ls
+        torch.cuda.empty_cache()
+
+
 def lmhead(rows=(60, 240, 480, 960), V=152064, Hd=3584):
     hbm, tens, src = _peaks()
     W = to_device(wl.normal_bf16(7, "W", (V, Hd), 1.0 / np.sqrt(Hd)))
@@ -122,9 +154,11 @@ def compact(B=1024, L=8, T=64, Hkv=4, D=128):
 
 
 if __name__ == "__main__":
-    what = sys.argv[1:] or ["attention", "lmhead", "compact"]
+    what = sys.argv[1:] or ["attention", "attention_layers", "lmhead", "compact"]
     if "attention" in what:
         attention()
+    if "attention_layers" in what:
+        attention_layers()
     if "lmhead" in what:
         lmhead()
     if "compact" in what:
