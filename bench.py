@@ -32,7 +32,7 @@ sys.path.insert(0, ROOT)
 # dram__bytes_read.sum + dram__bytes_write.sum of attn_umma_kernel per layer, from the ncu capture
 # summarised under profiles/.  Set an entry to None whenever the kernel changes until the counters
 # are retaken.
-ATTENTION_DRAM_BYTES_PER_LAYER = {"c5": None}
+ATTENTION_DRAM_BYTES_PER_LAYER = {"c5": 72.37e6}
 
 METRIC = "tree_verify_steps_per_s"
 UNIT = "steps/s"
@@ -258,7 +258,7 @@ def main():
     ms_total = e0.elapsed_time(e1)
 
     # per-call durations, same steps, events around every call (same stream)
-    names = ["attention", "attention_single_layer_call", "lmhead", "accept", "compact"]
+    names = ["attention", "attention_single_layer_call", "tail", "lmhead", "accept", "compact"]
     ev = {n: [] for n in names}
     def timed(name, fn):
         a, b = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
@@ -266,7 +266,8 @@ def main():
         ev[name].append((a, b))
     for _ in range(args.steps):
         timed("attention", vs.attention_layers)           # all layers, one library call
-        timed("lmhead", vs.lmhead)
+        timed("tail", vs.tail)                            # LM head + acceptance + compaction, one call
+        timed("lmhead", vs.lmhead)                        # the same three as separate calls
         timed("accept", vs.accept)
         timed("compact", vs.compact)
     for _ in range(max(1, args.steps // 10)):             # for comparison: one call per layer
@@ -337,6 +338,7 @@ def main():
                 "calls": {"attention_ms_all_layers": per_call_ms["attention"],
                           "attention_ms_per_layer": per_call_ms["attention"] / vs.L,
                           "attention_ms_single_layer_call": per_call_ms["attention_single_layer_call"],
+                          "lmhead_accept_compact_ms": per_call_ms["tail"],
                           "lmhead_ms": per_call_ms["lmhead"], "accept_ms": per_call_ms["accept"],
                           "compact_ms": per_call_ms["compact"],
                           "lmhead_tflops": lm_tflops, "lmhead_frac_of_tensor_peak": lm_tflops / peaks["tensor_sustained"],

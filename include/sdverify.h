@@ -96,8 +96,8 @@ const char *sd_status_string(sd_status s);
 
 /*
  * Scratch bytes that sd_verify_attention (for this geometry; only the host
- * scalars of *geom are read) and sd_lmhead_argmax (for M rows, vocabulary V)
- * need; the larger of the two.  Pass M = 0 or V = 0 to size for attention
+ * scalars of *geom are read) and sd_lmhead_argmax / sd_lmhead_accept_compact
+ * (for M rows, vocabulary V) need; the larger of the two.  Pass M = 0 or V = 0 to size for attention
  * only, geom = NULL for the LM head only.
  */
 size_t sd_workspace_bytes(const sd_batch *geom, int32_t M, int32_t V);
@@ -243,6 +243,28 @@ sd_status sd_compact_kv(const sd_batch *batch, const sd_kv_layer *layers, int32_
                         const void *const *k_tree_layers, const void *const *v_tree_layers,
                         const int32_t *n_acc, const int32_t *path,
                         int32_t *dev_status, void *stream);
+
+/*
+ * LM head, acceptance and compaction in one call (Sec. 1: validation ends with the
+ * target's tokens deciding which drafts survive; Sec. 4.1: the survivors' KV joins
+ * the context).  Equivalent, output for output and byte for byte, to
+ *     sd_lmhead_argmax(hidden, W, M = B * T_max, ...)      row b * T_max + i = node i of sequence b
+ *     sd_accept_tree(batch, draft_tok, argmax, ...)
+ *     sd_compact_kv(batch, layers, L, ..., n_acc, path)
+ * but after the LM-head tiles a single kernel (one CTA per sequence) merges the
+ * arg-max candidates, picks the accepted path and copies the accepted K/V rows,
+ * instead of three launches of a few microseconds each.  Arguments as in the three
+ * calls; argmax [B * T_max] and maxlogit (nullable) are outputs as well.
+ * B * T_max > 512 or L > 64 falls back to the three separate steps internally.
+ */
+sd_status sd_lmhead_accept_compact(const sd_batch *batch, const void *hidden, const void *W,
+                                   int32_t Hd, int32_t V, const int32_t *draft_tok,
+                                   const sd_kv_layer *layers, int32_t L,
+                                   const void *const *k_tree_layers, const void *const *v_tree_layers,
+                                   int32_t *argmax, float *maxlogit,
+                                   int32_t *n_acc, int32_t *path, int32_t *out_tok, int32_t *new_len,
+                                   void *workspace, size_t workspace_bytes,
+                                   int32_t *dev_status, void *stream);
 
 #ifdef __cplusplus
 }

@@ -27,11 +27,12 @@ SD_ERR_BOUNDS = -7
 # kernel launches behind one call (kept in step with the kernels; used for launch accounting)
 KERNELS_PER_ATTENTION = 1      # split-KV chunks merge inside the kernel (thread-block cluster)
 ATTENTION_LAYERS_PER_LAUNCH = 32   # sd_verify_attention_layers: layers sharing one launch
+KERNELS_PER_TAIL = 2               # sd_lmhead_accept_compact: LM-head tiles + fused tail kernel
 KERNELS_PER_LMHEAD = 2         # tiles + cross-slab reduce
 
 EXPORTS = ["sd_version", "sd_status_string", "sd_workspace_bytes", "sd_tree_prepare",
            "sd_verify_attention", "sd_verify_attention_layers", "sd_lmhead_argmax", "sd_lmhead_argmax_static", "sd_accept_tree",
-           "sd_compact_kv"]
+           "sd_compact_kv", "sd_lmhead_accept_compact"]
 
 
 class sd_kv_layer(C.Structure):
@@ -76,6 +77,11 @@ def _load(path: str = LIB_PATH) -> C.CDLL:
     lib.sd_compact_kv.restype = C.c_int
     lib.sd_compact_kv.argtypes = [C.c_void_p, C.c_void_p, C.c_int32, C.c_void_p, C.c_void_p,
                                   C.c_void_p, C.c_void_p, C.c_void_p, C.c_void_p]
+    lib.sd_lmhead_accept_compact.restype = C.c_int
+    lib.sd_lmhead_accept_compact.argtypes = [C.c_void_p, C.c_void_p, C.c_void_p, C.c_int32, C.c_int32, C.c_void_p,
+                                             C.c_void_p, C.c_int32, C.c_void_p, C.c_void_p,
+                                             C.c_void_p, C.c_void_p, C.c_void_p, C.c_void_p, C.c_void_p, C.c_void_p,
+                                             C.c_void_p, C.c_size_t, C.c_void_p, C.c_void_p]
     return lib
 
 
@@ -234,3 +240,16 @@ class LayerSet:
 def sd_compact_kv(batch: Batch, layers: LayerSet, n_acc, path, status, stream=None) -> None:
     _check(lib.sd_compact_kv(batch.ref(), layers.layers, layers.L, layers.kt, layers.vt,
                              _ptr(n_acc), _ptr(path), _ptr(status), _stream(stream)))
+
+
+def sd_lmhead_accept_compact(batch: Batch, hidden, W, draft_tok, layers: LayerSet, argmax, maxlogit,
+                             n_acc, path, out_tok, new_len, workspace, status, stream=None) -> None:
+    """LM-head arg-max over the B * T_max rows of `hidden`, greedy acceptance and KV compaction in all
+    layers; the three steps share one tail kernel."""
+    M, Hd = hidden.shape
+    V = W.shape[0]
+    assert W.shape[1] == Hd and M == batch.B * batch.T_max
+    _check(lib.sd_lmhead_accept_compact(batch.ref(), _ptr(hidden), _ptr(W), int(Hd), int(V), _ptr(draft_tok),
+                                        layers.layers, layers.L, layers.kt, layers.vt, _ptr(argmax), _ptr(maxlogit),
+                                        _ptr(n_acc), _ptr(path), _ptr(out_tok), _ptr(new_len), _ptr(workspace),
+                                        workspace.numel() * workspace.element_size(), _ptr(status), _stream(stream)))

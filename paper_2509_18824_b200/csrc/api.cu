@@ -45,7 +45,7 @@ const char* sd_status_string(sd_status s) {
 size_t sd_workspace_bytes(const sd_batch* geom, int32_t M, int32_t V) {
     size_t a = 0, l = 0;
     if (geom && check_geometry(geom, false) == SD_OK) a = attention_workspace_bytes(*geom);
-    if (M > 0 && V > 0) l = lmhead_workspace_bytes(M, V);
+    if (M > 0 && V > 0) l = tail_workspace_bytes(M, V);     // covers sd_lmhead_argmax and the fused tail
     size_t n = a > l ? a : l;
     return (n + 255) & ~(size_t)255;
 }
@@ -130,6 +130,28 @@ sd_status sd_compact_kv(const sd_batch* batch, const sd_kv_layer* layers, int32_
     }
     return launch_compact(*batch, layers, L, k_tree_layers, v_tree_layers, n_acc, path, dev_status,
                           static_cast<cudaStream_t>(stream));
+}
+
+sd_status sd_lmhead_accept_compact(const sd_batch* batch, const void* hidden, const void* W, int32_t Hd, int32_t V,
+                                   const int32_t* draft_tok, const sd_kv_layer* layers, int32_t L,
+                                   const void* const* k_tree_layers, const void* const* v_tree_layers,
+                                   int32_t* argmax, float* maxlogit,
+                                   int32_t* n_acc, int32_t* path, int32_t* out_tok, int32_t* new_len,
+                                   void* workspace, size_t workspace_bytes, int32_t* dev_status, void* stream) {
+    sd_status s = check_geometry(batch, true);
+    if (s != SD_OK) return s;
+    if (!ok_ptr(hidden) || !ok_ptr(W) || !argmax || !ok_ptr(workspace) || !dev_status) return SD_ERR_INVALID_ARG;
+    if (V < 1 || Hd < 1) return SD_ERR_INVALID_ARG;
+    if (Hd % 64 != 0) return SD_ERR_UNSUPPORTED;
+    if (!draft_tok || !n_acc || !path || !out_tok || !new_len) return SD_ERR_INVALID_ARG;
+    if (!layers || L < 1 || !k_tree_layers || !v_tree_layers) return SD_ERR_INVALID_ARG;
+    for (int l = 0; l < L; ++l) {
+        if (!ok_ptr(layers[l].k) || !ok_ptr(layers[l].v) || layers[l].num_blocks < 1) return SD_ERR_INVALID_ARG;
+        if (!ok_ptr(k_tree_layers[l]) || !ok_ptr(v_tree_layers[l])) return SD_ERR_INVALID_ARG;
+    }
+    return launch_lmhead_accept_compact(*batch, hidden, W, Hd, V, draft_tok, layers, L, k_tree_layers, v_tree_layers,
+                                        argmax, maxlogit, n_acc, path, out_tok, new_len, workspace, workspace_bytes,
+                                        dev_status, static_cast<cudaStream_t>(stream));
 }
 
 }  // extern "C"

@@ -43,8 +43,16 @@ sd_status launch_attention_layers(const sd_batch& bt, const sd_kv_layer* caches,
                                   float scale, void* const* out, float* const* lse,
                                   int32_t* dev_status, cudaStream_t st);
 size_t lmhead_workspace_bytes(int M, int V);
+size_t tail_workspace_bytes(int M, int V);
 sd_status launch_lmhead(const void* hidden, const void* W, int M, int Hd, int V,
                         int32_t* argmax, float* maxlogit, void* ws, size_t ws_bytes,
                         int32_t* dev_status, cudaStream_t st);
+
+sd_status launch_lmhead_accept_compact(const sd_batch& bt, const void* hidden, const void* W, int Hd, int V,
+                                       const int32_t* draft, const sd_kv_layer* layers, int L,
+                                       const void* const* kt, const void* const* vt,
+                                       int32_t* argmax, float* maxlogit, int32_t* n_acc, int32_t* path,
+                                       int32_t* out_tok, int32_t* new_len, void* ws, size_t ws_bytes,
+                                       int32_t* dev_status, cudaStream_t st);
 
 }  // namespace sdv

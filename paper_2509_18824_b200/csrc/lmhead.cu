@@ -7,7 +7,7 @@
 // leaves TMEM: the epilogue warps reduce each column over the 128 vocabulary
 // lanes (max + lowest index) and keep a running best per hidden row; only
 // (max, index) pairs per CTA reach memory, and a tiny kernel merges them.
-#include "common.cuh"
+#include "tree_device.cuh"
 #include "sm100.cuh"
 
 namespace sdv {
@@ -15,7 +15,7 @@ using namespace sm100;
 
 constexpr int kBM = 128;            // vocabulary rows per tile (MMA M)
 constexpr int kLmThreads = 192;     // warps 0-3 epilogue, warp 4 TMA producer, warp 5 MMA issuer
-constexpr int kMaxCols = 512;       // hidden rows per launch (TMEM columns)
+constexpr int kMaxCols = kLmMaxCols; // hidden rows per launch (TMEM columns)
 constexpr int kMaxCtas = 256;
 constexpr int kMaxStages = 8;
 constexpr int kSmemBudget = 227 * 1024 - 2048;
@@ -40,15 +40,17 @@ size_t lmhead_workspace_bytes(int M, int V) {
     (void)M; (void)V;
     return (size_t)kMaxCtas * kMaxCols * 2 * sizeof(int32_t);
 }
+// the fused tail also parks the acceptance outputs of its non-writing CTAs: per layer
+// 2 * B + 2 * B * T_max <= 4 * 512 words, for up to 64 layers
+size_t tail_workspace_bytes(int M, int V) {
+    return lmhead_workspace_bytes(M, V) + (size_t)kLayersPerLaunch * 4 * kMaxCols * sizeof(int32_t);
+}
 
 // float -> int whose signed order equals the float order (-0 folded onto +0)
 __device__ __forceinline__ int32_t ordered_key(uint32_t bits) {
     int32_t b = (int32_t)bits;
     b = (b < 0) ? (b ^ 0x7fffffff) : b;
     return (b == -1) ? 0 : b;            // -0.0f maps to -1 above; fold it onto +0.0f
-}
-__device__ __forceinline__ float key_to_float(int32_t k) {
-    return __int_as_float(k < 0 ? (k ^ 0x7fffffff) : k);
 }
 
 template <int BK>
@@ -415,10 +417,13 @@ __global__ void lmhead_merge_kernel(const int32_t* __restrict__ part_key, const 
 
 static int round_up(int x, int m) { return (x + m - 1) / m * m; }
 
-sd_status launch_lmhead(const void* hidden, const void* W, int M, int Hd, int V,
-                        int32_t* argmax, float* maxlogit, void* ws, size_t ws_bytes,
-                        int32_t* dev_status, cudaStream_t st) {
+// tiles_only_ctas != nullptr (M <= 512 required): launch only the tile kernel and report how many
+// CTAs filled the candidate tables; the caller merges them itself (the fused tail kernel).
+static sd_status launch_lmhead_impl(const void* hidden, const void* W, int M, int Hd, int V,
+                                    int32_t* argmax, float* maxlogit, void* ws, size_t ws_bytes,
+                                    int32_t* dev_status, cudaStream_t st, int* tiles_only_ctas) {
     if (ws_bytes < lmhead_workspace_bytes(M, V)) return SD_ERR_WORKSPACE;
+    if (tiles_only_ctas && M > kMaxCols) return SD_ERR_UNSUPPORTED;
     int dev = 0, sms = 0;
     if (cudaGetDevice(&dev) != cudaSuccess ||
         cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev) != cudaSuccess)
@@ -496,11 +501,117 @@ sd_status launch_lmhead(const void* hidden, const void* W, int M, int Hd, int V,
             kern<<<grid, kLmThreads, dyn, st>>>(tmW, tmH, p, dev_status);
             if (cudaGetLastError() != cudaSuccess) return SD_ERR_CUDA;
         }
+        if (tiles_only_ctas) {
+            *tiles_only_ctas = grid;
+            return SD_OK;
+        }
         lmhead_merge_kernel<<<(p.rows + 127) / 128, 128, 0, st>>>(p.part_key, p.part_idx, grid, p.rows, p.row0,
                                                                  argmax, maxlogit);
         if (cudaGetLastError() != cudaSuccess) return SD_ERR_CUDA;
     }
     return SD_OK;
+}
+
+sd_status launch_lmhead(const void* hidden, const void* W, int M, int Hd, int V,
+                        int32_t* argmax, float* maxlogit, void* ws, size_t ws_bytes,
+                        int32_t* dev_status, cudaStream_t st) {
+    return launch_lmhead_impl(hidden, W, M, Hd, V, argmax, maxlogit, ws, ws_bytes, dev_status, st, nullptr);
+}
+
+// ---------------------------------------------------------------------------
+// Fused tail of a verify step.  CTA (b, l) merges the LM-head candidates of sequence b's rows
+// (row = b * T_max + node), runs greedy acceptance on the resulting arg-max, and copies the
+// accepted nodes' K/V into the cache of layer l.  The merge and the acceptance are a few
+// microseconds of latency-bound work, so every layer's CTA repeats them rather than waiting for
+// another CTA's result; only the CTAs of layer 0 write the arg-max and acceptance outputs.
+// Replaces three launches (candidate merge, acceptance, compaction).
+// ---------------------------------------------------------------------------
+__global__ void __launch_bounds__(256)
+tail_kernel(sd_batch bt, const __grid_constant__ CompactLayers ly,
+            const int32_t* __restrict__ part_key, const int32_t* __restrict__ part_idx, int n_ctas,
+            const int32_t* __restrict__ draft, int32_t* __restrict__ argmax, float* __restrict__ maxlogit,
+            int32_t* n_acc, int32_t* path, int32_t* out_tok, int32_t* new_len, int32_t* status,
+            int32_t* scratch /* [B][4 * T_max + 2]: outputs of the CTAs that must not write the real ones */) {
+    __shared__ int32_t s_target[kMaxT];
+    __shared__ int32_t s_path[kMaxT];
+    __shared__ int s_na;
+    const int b = blockIdx.x;
+    const int layer = blockIdx.y;
+    const int T = bt.T_max;
+    const bool writer = (layer == 0);
+    // 1. arg-max of this sequence's rows: eight threads per row, each an eighth of the CTAs' candidates
+    for (int row0 = 0; row0 < T; row0 += 32) {
+        const int row = row0 + (threadIdx.x >> 3), sub = threadIdx.x & 7;
+        int32_t k = INT32_MIN, i = 0x7fffffff;
+        if (row < T) {
+            const int col = b * T + row;
+#pragma unroll 4
+            for (int c = sub; c < n_ctas; c += 8)
+                take_better(k, i, __ldg(part_key + (size_t)c * kMaxCols + col), __ldg(part_idx + (size_t)c * kMaxCols + col));
+        }
+#pragma unroll
+        for (int d = 1; d <= 4; d <<= 1) {
+            const int32_t k2 = __shfl_xor_sync(0xffffffffu, k, d), i2 = __shfl_xor_sync(0xffffffffu, i, d);
+            take_better(k, i, k2, i2);
+        }
+        if (row < T && sub == 0) {
+            if (writer) {
+                argmax[b * T + row] = i;
+                if (maxlogit) maxlogit[b * T + row] = key_to_float(k);
+            }
+            s_target[row] = i;
+        }
+    }
+    if (threadIdx.x == 0) s_na = 0;
+    __syncthreads();
+    // 2. greedy acceptance (one warp); CTAs of other layers keep their copy of the outputs to themselves
+    if (threadIdx.x < 32) {
+        int32_t* priv = scratch + ((size_t)blockIdx.y * gridDim.x) * (2 * T + 2);   // this layer's private area
+        int32_t* o_nacc = writer ? n_acc : priv;                        // [B]
+        int32_t* o_newlen = writer ? new_len : priv + gridDim.x;        // [B]
+        int32_t* o_path = writer ? path : priv + 2 * gridDim.x;         // [B][T]
+        int32_t* o_tok = writer ? out_tok : priv + 2 * gridDim.x + (size_t)gridDim.x * T;
+        const int na = accept_sequence(bt, b, threadIdx.x, bt.parents + (size_t)b * T, draft + (size_t)b * T,
+                                       s_target, o_nacc, o_path, o_tok, o_newlen, s_path, status);
+        if (threadIdx.x == 0) s_na = na;
+    }
+    __syncthreads();
+    // 3. accepted rows into this layer's cache
+    compact_sequence(bt, ly, layer, 1, b, s_na, s_path, threadIdx.x, blockDim.x, status);
+}
+
+void fill_compact_layers(CompactLayers* ly, const sd_kv_layer* layers, const void* const* kt, const void* const* vt,
+                         int l0, int nl);
+
+sd_status launch_lmhead_accept_compact(const sd_batch& bt, const void* hidden, const void* W, int Hd, int V,
+                                       const int32_t* draft, const sd_kv_layer* layers, int L,
+                                       const void* const* kt, const void* const* vt,
+                                       int32_t* argmax, float* maxlogit, int32_t* n_acc, int32_t* path,
+                                       int32_t* out_tok, int32_t* new_len, void* ws, size_t ws_bytes,
+                                       int32_t* dev_status, cudaStream_t st) {
+    const int M = bt.B * bt.T_max;
+    if (M > kMaxCols || L > kLayersPerLaunch) {
+        // shapes beyond one pass of the candidate tables or one set of layer descriptors: the same
+        // three steps as separate launches
+        sd_status s = launch_lmhead(hidden, W, M, Hd, V, argmax, maxlogit, ws, ws_bytes, dev_status, st);
+        if (s != SD_OK) return s;
+        s = launch_accept(bt, draft, argmax, n_acc, path, out_tok, new_len, dev_status, st);
+        if (s != SD_OK) return s;
+        return launch_compact(bt, layers, L, kt, vt, n_acc, path, dev_status, st);
+    }
+    if (ws_bytes < tail_workspace_bytes(M, V)) return SD_ERR_WORKSPACE;
+    int n_ctas = 0;
+    sd_status s = launch_lmhead_impl(hidden, W, M, Hd, V, argmax, maxlogit, ws, ws_bytes, dev_status, st, &n_ctas);
+    if (s != SD_OK) return s;
+    CompactLayers ly;
+    fill_compact_layers(&ly, layers, kt, vt, 0, L);
+    const int32_t* part_key = static_cast<const int32_t*>(ws);
+    const int32_t* part_idx = part_key + (size_t)kMaxCtas * kMaxCols;
+    // scratch for the non-writing CTAs' acceptance outputs: behind the candidate tables
+    int32_t* scratch = static_cast<int32_t*>(ws) + (size_t)kMaxCtas * kMaxCols * 2;
+    tail_kernel<<<dim3(bt.B, L), 256, 0, st>>>(bt, ly, part_key, part_idx, n_ctas, draft, argmax, maxlogit,
+                                               n_acc, path, out_tok, new_len, dev_status, scratch);
+    return cuda_ok(cudaGetLastError());
 }
 
 

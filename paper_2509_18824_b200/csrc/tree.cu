@@ -1,6 +1,6 @@
 // Tree bookkeeping kernels: ancestor masks and greedy acceptance.
 // Integer work only; one warp per sequence.
-#include "common.cuh"
+#include "tree_device.cuh"
 
 namespace sdv {
 
@@ -46,53 +46,9 @@ __global__ void accept_kernel(sd_batch bt, const int32_t* __restrict__ draft,
                               int32_t* n_acc, int32_t* path, int32_t* out_tok, int32_t* new_len,
                               int32_t* status) {
     const int b = blockIdx.x;
-    const int lane = threadIdx.x;
     const int T = bt.T_max;
-    const int n = bt.n_nodes[b];
-    const int32_t* par = bt.parents + (size_t)b * T;
-    const int32_t* dt = draft + (size_t)b * T;
-    const int32_t* tg = target + (size_t)b * T;
-    bool bad = (n < 1 || n > T);
-    if (!bad)
-        for (int i = lane; i < n; i += 32) {
-            int p = par[i];
-            if (i == 0 ? (p != -1) : (p < 0 || p >= i)) bad = true;
-        }
-    if (__any_sync(0xffffffffu, bad)) {
-        if (lane == 0) set_status(status, SD_ERR_INVALID_TREE);
-        return;
-    }
-    // key = depth * 64 + (63 - index) for valid nodes: max key = deepest, lowest index
-    int best_key = -1;
-    for (int i = lane; i < n; i += 32) {
-        bool ok = true;
-        int depth = 0;
-        int j = i;
-        for (int step = 0; step < kMaxT && j > 0; ++step) {
-            int p = par[j];
-            ok = ok && (dt[j] == tg[p]);
-            ++depth;
-            j = p;
-        }
-        if (ok) best_key = max(best_key, depth * 64 + (63 - i));
-    }
-    best_key = __reduce_max_sync(0xffffffffu, best_key);   // node 0 is always valid
-    const int best = 63 - (best_key & 63);
-    const int na = (best_key >> 6) + 1;
-    int32_t* pa = path + (size_t)b * T;
-    int32_t* ot = out_tok + (size_t)b * T;
-    for (int k = na + lane; k < T; k += 32) { pa[k] = -1; ot[k] = -1; }
-    if (lane == 0) {
-        n_acc[b] = na;
-        new_len[b] = bt.len[b] + na;
-        int j = best;
-        for (int k = na - 1; k >= 0; --k) {
-            pa[k] = j;
-            if (k >= 1) ot[k - 1] = dt[j];
-            j = par[j];
-        }
-        ot[na - 1] = tg[best];
-    }
+    accept_sequence(bt, b, threadIdx.x, bt.parents + (size_t)b * T, draft + (size_t)b * T, target + (size_t)b * T,
+                    n_acc, path, out_tok, new_len, nullptr, status);
 }
 
 sd_status launch_tree_prepare(const sd_batch& bt, int32_t* dev_status, cudaStream_t st) {

@@ -114,25 +114,36 @@ class VerifyStep:
     def compact(self, stream=None):
         sd.sd_compact_kv(self.batch, self.layerset, self.n_acc, self.path, self.status, stream)
 
+    def tail(self, stream=None):
+        """LM head, acceptance and compaction through the one fused call."""
+        sd.sd_lmhead_accept_compact(self.batch, self.hidden, self.W, self.draft_tok, self.layerset, self.argmax,
+                                    self.maxlogit, self.n_acc, self.path, self.out_tok, self.new_len,
+                                    self.workspace, self.status, stream)
+
     # -- the whole step -------------------------------------------------
-    def run(self, stream=None, per_layer=False):
-        """All layers' attention in one call (the step's q and tree K/V are all present up front);
-        per_layer=True issues one call per layer, as a decoder that interleaves its own layers would."""
+    def run(self, stream=None, per_layer=False, fused_tail=True):
+        """All layers' attention in one call (the step's q and tree K/V are all present up front), then
+        LM head + acceptance + compaction in one call.  per_layer=True issues one attention call per
+        layer, as a decoder that interleaves its own layers would; fused_tail=False issues the three
+        tail calls separately."""
         if per_layer:
             for l in range(self.L):
                 self.attention(l, stream)
         else:
             self.attention_layers(stream=stream)
-        self.lmhead(stream)
-        self.accept(None, stream)
-        self.compact(stream)
+        if fused_tail:
+            self.tail(stream)
+        else:
+            self.lmhead(stream)
+            self.accept(None, stream)
+            self.compact(stream)
 
     @property
     def launches_per_step(self) -> int:
         """Kernel launches of one run(): attention (one launch per group of up to 32 layers), the
-        LM-head kernels, acceptance, compaction."""
+        LM-head tiles and the fused merge/acceptance/compaction kernel."""
         return ((self.L + sd.ATTENTION_LAYERS_PER_LAUNCH - 1) // sd.ATTENTION_LAYERS_PER_LAUNCH
-                + sd.KERNELS_PER_LMHEAD + 1 + (self.L + 63) // 64)
+                + sd.KERNELS_PER_TAIL)
 
     def h2d_bytes(self) -> int:
         h = self.host
@@ -174,9 +185,7 @@ class VerifyStep:
             main.wait_event(self._ev_layer[l1 - 1])
             self.attention_layers(l0, l1)
         main.wait_stream(cs)            # hidden states and draft tokens have arrived
-        self.lmhead()
-        self.accept()
-        self.compact()
+        self.tail()
         self.host_out["n_acc"].copy_(self.n_acc, non_blocking=True)
         self.host_out["path"].copy_(self.path, non_blocking=True)
         self.host_out["out_tok"].copy_(self.out_tok, non_blocking=True)

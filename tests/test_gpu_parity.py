@@ -366,6 +366,59 @@ def test_chained_step_tiny():
     np.testing.assert_array_equal(vs.v_cache[0].cpu().numpy().view(np.uint16), rv)
 
 
+@pytest.mark.parametrize("cfg,over", [("c1", dict(L=1)), ("c2", dict(L=3)),
+                                      ("c5", dict(L=2, V=8192, Hd=512, prefix=200)),
+                                      ("c4", dict(L=2, V=4096, Hd=256, prefix_range=(40, 300)))])
+def test_fused_tail_equals_separate_calls(cfg, over):
+    """sd_lmhead_accept_compact against sd_lmhead_argmax + sd_accept_tree + sd_compact_kv on the same
+    inputs: every output and every cache byte identical; acceptance also against the checker."""
+    w = wl.make(cfg, hidden_gain=16.0, **over)        # c4: 960 rows, more than one LM-head pass
+    L = w.L
+    ram, t1, t2 = oracle.lmhead(w.hidden, w.W)
+    g = np.random.default_rng(3)
+    wl.plant(w, ram.reshape(w.B, w.T_max), g.integers(0, 4, size=w.B))
+    res = []
+    for fused in (False, True):
+        vs = VerifyStep(w)
+        if fused:
+            vs.tail()
+        else:
+            vs.lmhead(); vs.accept(); vs.compact()
+        torch.cuda.synchronize()
+        vs.check_status()
+        res.append(dict(argmax=vs.argmax.cpu().numpy(), maxlogit=vs.maxlogit.cpu().numpy(),
+                        n_acc=vs.n_acc.cpu().numpy(), path=vs.path.cpu().numpy(), out_tok=vs.out_tok.cpu().numpy(),
+                        new_len=vs.new_len.cpu().numpy(),
+                        k=[x.cpu().numpy() for x in vs.k_cache], v=[x.cpu().numpy() for x in vs.v_cache]))
+    for key in ("argmax", "maxlogit", "n_acc", "path", "out_tok", "new_len"):
+        np.testing.assert_array_equal(res[0][key], res[1][key], err_msg=key)
+    for l in range(L):
+        np.testing.assert_array_equal(res[0]["k"][l], res[1]["k"][l])
+        np.testing.assert_array_equal(res[0]["v"][l], res[1]["v"][l])
+    np.testing.assert_array_equal(res[1]["argmax"], ram)             # crisp logits: every row must match
+    G = oracle.Geometry.of(w)
+    ref_acc = oracle.accept(G, w.draft_tok, ram.reshape(w.B, w.T_max))
+    for got, ref in zip((res[1]["n_acc"], res[1]["path"], res[1]["out_tok"], res[1]["new_len"]), ref_acc):
+        np.testing.assert_array_equal(got, ref)
+    for l in range(L):
+        rk, rv = w.k_cache[l].copy(), w.v_cache[l].copy()
+        oracle.compact(G, rk, rv, w.k_tree[l], w.v_tree[l], ref_acc[0], ref_acc[1])
+        np.testing.assert_array_equal(res[1]["k"][l].view(np.uint16), rk)
+        np.testing.assert_array_equal(res[1]["v"][l].view(np.uint16), rv)
+
+
+def test_fused_tail_bad_tree_touches_no_cache():
+    w = wl.make("c1", hidden_gain=16.0)
+    w.parents = w.parents.copy(); w.parents[0, 3] = 5
+    vs = VerifyStep(w)
+    before_k = vs.k_cache[0].clone()
+    vs.status.zero_()
+    vs.tail()
+    torch.cuda.synchronize()
+    assert int(vs.status.item()) == sd.SD_ERR_INVALID_TREE
+    assert torch.equal(before_k, vs.k_cache[0])
+
+
 def test_full_step_c5_shapes():
     """28 layers, batch 8, prefix 4096: planted paths are recovered bit-exactly,
     attention agrees on sampled rows in every layer, caches match after compaction."""
