@@ -315,7 +315,7 @@ def main():
                     "peak": peaks["tensor_sustained"], "unit": "TFLOP/s",
                     "frac": att_tflops / peaks["tensor_sustained"],
                     "traffic": traffic * layers_per_launch if traffic else None,
-                    "traffic_unit": "bytes per launch (dram read + write; ncu capture of a 4-layer launch, "
+                    "traffic_unit": "bytes per launch (dram read + write; ncu capture of an 8-layer launch, "
                                     "scaled by layers per launch)",
                     "layers_per_launch": layers_per_launch,
                     "algorithmic_bytes_per_launch": work["att_bytes"] * layers_per_launch,

@@ -44,14 +44,19 @@ class VerifyStep:
         self.k_cache = [to_device(x, d) for x in w.k_cache]
         self.v_cache = [to_device(x, d) for x in w.v_cache]
         self.W = to_device(w.W, d) if w.W is not None else None
-        # per-step inputs
-        self.q = [to_device(x, d) for x in w.q]
-        self.k_tree = [to_device(x, d) for x in w.k_tree]
-        self.v_tree = [to_device(x, d) for x in w.v_tree]
+        # per-step inputs: q, tree K and tree V of all layers live in ONE device buffer (layer-major),
+        # so that the end-to-end path can bring a whole group of layers over in a single copy
+        B, T = w.B, w.T_max
+        self._nq, self._nkv = B * T * w.Hq * w.D, B * T * w.Hkv * w.D       # bf16 elements per layer
+        self._per_layer = self._nq + 2 * self._nkv
+        self._in_dev = torch.empty(self.L * self._per_layer, dtype=torch.int16, device=d)
+        self.q, self.k_tree, self.v_tree = self._layer_views(self._in_dev, w)
+        for l in range(self.L):
+            self.q[l].copy_(to_device(w.q[l], d)); self.k_tree[l].copy_(to_device(w.k_tree[l], d))
+            self.v_tree[l].copy_(to_device(w.v_tree[l], d))
         self.hidden = to_device(w.hidden, d) if w.hidden is not None else None
         self.draft_tok = to_device(w.draft_tok, d) if w.draft_tok is not None else None
         # outputs
-        B, T = w.B, w.T_max
         self.out = [torch.zeros((B, T, w.Hq, w.D), dtype=torch.bfloat16, device=d) for _ in range(self.L)]
         self.lse = [torch.zeros((B, T, w.Hq), dtype=torch.float32, device=d) for _ in range(self.L)]
         M = B * T
@@ -73,15 +78,31 @@ class VerifyStep:
         self._copy_stream = None
         self.host = None
         if keep_host_inputs:
+            self._in_host = torch.empty(self.L * self._per_layer, dtype=torch.int16).pin_memory()
+            hq, hk, hv = self._layer_views(self._in_host, w)
+            for l in range(self.L):
+                hq[l].copy_(torch.from_numpy(w.q[l].view(np.int16)))
+                hk[l].copy_(torch.from_numpy(w.k_tree[l].view(np.int16)))
+                hv[l].copy_(torch.from_numpy(w.v_tree[l].view(np.int16)))
             self.host = dict(
-                q=[pinned(x) for x in w.q], k_tree=[pinned(x) for x in w.k_tree],
-                v_tree=[pinned(x) for x in w.v_tree], hidden=pinned(w.hidden),
+                q=hq, k_tree=hk, v_tree=hv, hidden=pinned(w.hidden),
                 draft_tok=pinned(w.draft_tok), parents=pinned(w.parents), n_nodes=pinned(w.n_nodes))
             self.host_out = dict(
                 n_acc=torch.zeros(B, dtype=torch.int32).pin_memory(),
                 path=torch.zeros((B, T), dtype=torch.int32).pin_memory(),
                 out_tok=torch.zeros((B, T), dtype=torch.int32).pin_memory(),
                 new_len=torch.zeros(B, dtype=torch.int32).pin_memory())
+
+    def _layer_views(self, flat: torch.Tensor, w):
+        """Per-layer q / tree K / tree V views of a flat layer-major buffer."""
+        B, T = w.B, w.T_max
+        q, kt, vt = [], [], []
+        for l in range(self.L):
+            o = l * self._per_layer
+            q.append(flat[o:o + self._nq].view(B, T, w.Hq, w.D))
+            kt.append(flat[o + self._nq:o + self._nq + self._nkv].view(B, T, w.Hkv, w.D))
+            vt.append(flat[o + self._nq + self._nkv:o + self._per_layer].view(B, T, w.Hkv, w.D))
+        return q, kt, vt
 
     # -- pieces ---------------------------------------------------------
     def attention(self, l: int, stream=None):
@@ -171,11 +192,11 @@ class VerifyStep:
             self.batch.parents.copy_(h["parents"], non_blocking=True)
             self.batch.n_nodes.copy_(h["n_nodes"], non_blocking=True)
             self._ev_small.record(cs)
-            for l in range(self.L):
-                self.q[l].copy_(h["q"][l], non_blocking=True)
-                self.k_tree[l].copy_(h["k_tree"][l], non_blocking=True)
-                self.v_tree[l].copy_(h["v_tree"][l], non_blocking=True)
-                self._ev_layer[l].record(cs)
+            for l0 in range(0, self.L, group):          # one copy per group of layers
+                l1 = min(l0 + group, self.L)
+                sl = slice(l0 * self._per_layer, l1 * self._per_layer)
+                self._in_dev[sl].copy_(self._in_host[sl], non_blocking=True)
+                self._ev_layer[l1 - 1].record(cs)
             self.hidden.copy_(h["hidden"], non_blocking=True)
             self.draft_tok.copy_(h["draft_tok"], non_blocking=True)
         main.wait_event(self._ev_small)
