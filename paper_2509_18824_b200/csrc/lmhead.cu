@@ -53,6 +53,47 @@ __device__ __forceinline__ int32_t ordered_key(uint32_t bits) {
     return (b == -1) ? 0 : b;            // -0.0f maps to -1 above; fold it onto +0.0f
 }
 
+__device__ __forceinline__ float redux_max_f32(float v) {
+    float d;
+    asm volatile("redux.sync.max.f32 %0, %1, 0xffffffff;" : "=f"(d) : "f"(v));
+    return d;
+}
+
+// element `lane` of a 32-entry register array, by a binary tree of selects on the lane's bits
+// (register arrays cannot be indexed by a run-time value)
+template <typename T>
+__device__ __forceinline__ T pick_lane(const T (&x)[32], int lane) {
+    T a[16], b[8], c[4], d[2];
+#pragma unroll
+    for (int i = 0; i < 16; ++i) a[i] = (lane & 16) ? x[i + 16] : x[i];
+#pragma unroll
+    for (int i = 0; i < 8; ++i) b[i] = (lane & 8) ? a[i + 8] : a[i];
+#pragma unroll
+    for (int i = 0; i < 4; ++i) c[i] = (lane & 4) ? b[i + 4] : b[i];
+#pragma unroll
+    for (int i = 0; i < 2; ++i) d[i] = (lane & 2) ? c[i + 2] : c[i];
+    return (lane & 1) ? d[1] : d[0];
+}
+
+// Arg-max over the 32 lanes (vocabulary rows) of each of 32 accumulator columns (hidden rows):
+// lane j ends up with column j's maximum and the lowest vocabulary row attaining it.  The passes
+// are kept apart on purpose: 32 independent warp reductions are in flight together, then 32
+// independent votes; interleaved per column, every reduction's latency (and then every vote's)
+// would be paid one after the other.
+__device__ __forceinline__ void column_argmax32(const uint32_t (&r)[32], bool v_ok, int v_base, int lane,
+                                                float& cv, int32_t& ci) {
+    float v[32], mx[32];
+#pragma unroll
+    for (int j = 0; j < 32; ++j) v[j] = v_ok ? __uint_as_float(r[j]) : -INFINITY;
+#pragma unroll
+    for (int j = 0; j < 32; ++j) mx[j] = redux_max_f32(v[j]);
+    uint32_t who[32];
+#pragma unroll
+    for (int j = 0; j < 32; ++j) who[j] = __ballot_sync(0xffffffffu, v[j] == mx[j]);
+    cv = pick_lane(mx, lane);
+    ci = v_base + (__ffs(pick_lane(who, lane)) - 1);
+}
+
 template <int BK>
 __global__ void __launch_bounds__(kLmThreads, 1)
 lmhead_umma_kernel(const __grid_constant__ CUtensorMap tmW, const __grid_constant__ CUtensorMap tmH,
@@ -154,10 +195,10 @@ lmhead_umma_kernel(const __grid_constant__ CUtensorMap tmW, const __grid_constan
         }
     } else {
         // ------------------------------------------------ epilogue warps 0..3 (TMEM lanes 32*warp ..)
-        int32_t best_key[kMaxCols / 32];
+        float best_val[kMaxCols / 32];
         int32_t best_idx[kMaxCols / 32];
 #pragma unroll
-        for (int c = 0; c < kMaxCols / 32; ++c) { best_key[c] = INT32_MIN; best_idx[c] = 0x7fffffff; }
+        for (int c = 0; c < kMaxCols / 32; ++c) { best_val[c] = -INFINITY; best_idx[c] = 0x7fffffff; }
         bool ok = true;
         for (int t = 0; t < my_tiles && ok; ++t) {
             const int buf = t % p.acc_bufs;
@@ -173,15 +214,10 @@ lmhead_umma_kernel(const __grid_constant__ CUtensorMap tmW, const __grid_constan
                     uint32_t r[32];
                     tmem_ld32(taddr + c * 32, r);
                     tmem_ld_wait();
-                    int32_t ck = INT32_MIN, ci = 0x7fffffff;
-#pragma unroll
-                    for (int j = 0; j < 32; ++j) {
-                        const int32_t key = v_ok ? ordered_key(r[j]) : INT32_MIN;
-                        const int32_t mx = __reduce_max_sync(0xffffffffu, key);
-                        const uint32_t who = __ballot_sync(0xffffffffu, key == mx);
-                        if (lane == j) { ck = mx; ci = v_base + (__ffs(who) - 1); }
-                    }
-                    if (ck > best_key[c]) { best_key[c] = ck; best_idx[c] = ci; }
+                    float cv;
+                    int32_t ci;
+                    column_argmax32(r, v_ok, v_base, lane, cv, ci);
+                    if (cv > best_val[c]) { best_val[c] = cv; best_idx[c] = ci; }
                 }
             }
             tc_fence_before_sync();
@@ -195,7 +231,7 @@ lmhead_umma_kernel(const __grid_constant__ CUtensorMap tmW, const __grid_constan
         int32_t* red_idx = red_key + 4 * kMaxCols;
 #pragma unroll
         for (int c = 0; c < kMaxCols / 32; ++c) {
-            red_key[warp * kMaxCols + c * 32 + lane] = best_key[c];
+            red_key[warp * kMaxCols + c * 32 + lane] = ordered_key(__float_as_uint(best_val[c]));
             red_idx[warp * kMaxCols + c * 32 + lane] = best_idx[c];
         }
         asm volatile("bar.sync 1, 128;" ::: "memory");
@@ -336,10 +372,10 @@ lmhead_umma_pair_kernel(const __grid_constant__ CUtensorMap tmW, const __grid_co
         }
     } else {
         // ------------------------------------------------ epilogue warps 0..3 (TMEM lanes 32*warp ..)
-        int32_t best_key[kMaxCols / 32];
+        float best_val[kMaxCols / 32];
         int32_t best_idx[kMaxCols / 32];
 #pragma unroll
-        for (int c = 0; c < kMaxCols / 32; ++c) { best_key[c] = INT32_MIN; best_idx[c] = 0x7fffffff; }
+        for (int c = 0; c < kMaxCols / 32; ++c) { best_val[c] = -INFINITY; best_idx[c] = 0x7fffffff; }
         bool ok = true;
         for (int t = 0; t < my_tiles && ok; ++t) {
             const int buf = t % p.acc_bufs;
@@ -355,15 +391,10 @@ lmhead_umma_pair_kernel(const __grid_constant__ CUtensorMap tmW, const __grid_co
                     uint32_t r[32];
                     tmem_ld32(taddr + c * 32, r);
                     tmem_ld_wait();
-                    int32_t ck = INT32_MIN, ci = 0x7fffffff;
-#pragma unroll
-                    for (int j = 0; j < 32; ++j) {
-                        const int32_t key = v_ok ? ordered_key(r[j]) : INT32_MIN;
-                        const int32_t mx = __reduce_max_sync(0xffffffffu, key);
-                        const uint32_t who = __ballot_sync(0xffffffffu, key == mx);
-                        if (lane == j) { ck = mx; ci = v_base + (__ffs(who) - 1); }
-                    }
-                    if (ck > best_key[c]) { best_key[c] = ck; best_idx[c] = ci; }
+                    float cv;
+                    int32_t ci;
+                    column_argmax32(r, v_ok, v_base, lane, cv, ci);
+                    if (cv > best_val[c]) { best_val[c] = cv; best_idx[c] = ci; }
                 }
             }
             tc_fence_before_sync();
@@ -375,7 +406,7 @@ lmhead_umma_pair_kernel(const __grid_constant__ CUtensorMap tmW, const __grid_co
         int32_t* red_idx = red_key + 4 * kMaxCols;
 #pragma unroll
         for (int c = 0; c < kMaxCols / 32; ++c) {
-            red_key[warp * kMaxCols + c * 32 + lane] = best_key[c];
+            red_key[warp * kMaxCols + c * 32 + lane] = ordered_key(__float_as_uint(best_val[c]));
             red_idx[warp * kMaxCols + c * 32 + lane] = best_idx[c];
         }
         asm volatile("bar.sync 1, 128;" ::: "memory");
