@@ -14,7 +14,9 @@ namespace sdv {
 using namespace sm100;
 
 constexpr int kBM = 128;            // vocabulary rows per tile (MMA M)
-constexpr int kLmThreads = 192;     // warps 0-3 epilogue, warp 4 TMA producer, warp 5 MMA issuer
+constexpr int kLmThreads = 161;     // warps 0-3 epilogue, warp 4 TMA producer, warp 5 = ONE thread: MMA issuer
+                                    // (a one-thread warp keeps the issue loop in uniform control flow, so
+                                    //  the MMA descriptors stay in uniform registers)
 constexpr int kMaxCols = kLmMaxCols; // hidden rows per launch (TMEM columns)
 constexpr int kMaxCtas = 256;
 constexpr int kMaxStages = 8;
@@ -112,7 +114,7 @@ lmhead_umma_kernel(const __grid_constant__ CUtensorMap tmW, const __grid_constan
     __shared__ uint32_t tmem_base_slot;
     __shared__ int abort_flag;
 
-    const int warp = threadIdx.x >> 5;
+    const int warp = __shfl_sync(0xffffffffu, (int)(threadIdx.x >> 5), 0);   // warp-uniform for the compiler
     const int lane = threadIdx.x & 31;
     const int kblocks = p.Hd / BK;
     const int my_tiles = (p.n_tiles - (int)blockIdx.x + (int)gridDim.x - 1) / (int)gridDim.x;
@@ -123,7 +125,7 @@ lmhead_umma_kernel(const __grid_constant__ CUtensorMap tmW, const __grid_constan
         for (int b = 0; b < 2; ++b) { mbar_init(&tmem_full[b], 1); mbar_init(&tmem_empty[b], 4); }
         fence_barrier_init();
     }
-    if (warp == 5) {
+    if (warp == 4) {                   // a full warp
         tmem_alloc(&tmem_base_slot, (uint32_t)p.tmem_cols);
         tmem_relinquish();
     }
@@ -160,8 +162,8 @@ lmhead_umma_kernel(const __grid_constant__ CUtensorMap tmW, const __grid_constan
             }
         }
     } else if (warp == 5) {
-        // ------------------------------------------------ MMA issuer
-        if (lane == 0) {
+        // ------------------------------------------------ MMA issuer (this warp is one thread)
+        {
             const uint32_t idesc = make_idesc_bf16(kBM, p.part_n, false, false);
             int it = 0;
             bool ok = true;
@@ -248,7 +250,7 @@ lmhead_umma_kernel(const __grid_constant__ CUtensorMap tmW, const __grid_constan
     }
     tc_fence_before_sync();
     __syncthreads();
-    if (warp == 5) {
+    if (warp == 4) {
         tc_fence_after_sync();
         tmem_dealloc(tmem_base, (uint32_t)p.tmem_cols);
     }
@@ -280,7 +282,7 @@ lmhead_umma_pair_kernel(const __grid_constant__ CUtensorMap tmW, const __grid_co
     __shared__ uint32_t tmem_base_slot;
     __shared__ int abort_flag;
 
-    const int warp = threadIdx.x >> 5;
+    const int warp = __shfl_sync(0xffffffffu, (int)(threadIdx.x >> 5), 0);   // warp-uniform for the compiler
     const int lane = threadIdx.x & 31;
     const uint32_t rank = cluster_ctarank();                  // 0 = leader
     const int pair = blockIdx.x >> 1;
@@ -294,7 +296,7 @@ lmhead_umma_pair_kernel(const __grid_constant__ CUtensorMap tmW, const __grid_co
         for (int b = 0; b < 2; ++b) { mbar_init(&tmem_full[b], 1); mbar_init(&tmem_empty[b], 8); }
         fence_barrier_init();
     }
-    if (warp == 5) {
+    if (warp == 4) {                   // a full warp
         tmem_alloc_pair(&tmem_base_slot, (uint32_t)p.tmem_cols);
         tmem_relinquish_pair();
     }
@@ -334,8 +336,8 @@ lmhead_umma_pair_kernel(const __grid_constant__ CUtensorMap tmW, const __grid_co
             }
         }
     } else if (warp == 5) {
-        // ------------------------------------------------ MMA issuer (leader CTA only)
-        if (lane == 0 && rank == 0) {
+        // ------------------------------------------------ MMA issuer (leader CTA only; this warp is one thread)
+        if (rank == 0) {
             const uint32_t idesc = make_idesc_bf16(2 * kBM, p.part_n, false, false);
             const uint32_t part_step = (uint32_t)(half_n * kSwz) >> 4;   // next part's B rows, in descriptor units
             int it = 0;
@@ -425,7 +427,7 @@ lmhead_umma_pair_kernel(const __grid_constant__ CUtensorMap tmW, const __grid_co
     __syncthreads();
     cluster_arrive_release();          // neither CTA leaves while the other may still signal it
     cluster_wait_acquire();
-    if (warp == 5) {
+    if (warp == 4) {
         tc_fence_after_sync();
         tmem_dealloc_pair(tmem_base, (uint32_t)p.tmem_cols);
     }
