@@ -264,13 +264,13 @@ def main():
         a, b = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
         a.record(); fn(); b.record()
         ev[name].append((a, b))
-    for _ in range(args.steps):
+    for _ in range(args.steps):                           # the same two calls as the timed step
         timed("attention", vs.attention_layers)           # all layers, one library call
         timed("tail", vs.tail)                            # LM head + acceptance + compaction, one call
-        timed("lmhead", vs.lmhead)                        # the same three as separate calls
+    for _ in range(max(1, args.steps // 10)):             # for comparison: the tail as three calls,
+        timed("lmhead", vs.lmhead)                        # attention as one call per layer
         timed("accept", vs.accept)
         timed("compact", vs.compact)
-    for _ in range(max(1, args.steps // 10)):             # for comparison: one call per layer
         for l in range(vs.L):
             timed("attention_single_layer_call", lambda: vs.attention(l))
     torch.cuda.synchronize()
@@ -303,7 +303,7 @@ def main():
         n_att_launches = (vs.L + sd.ATTENTION_LAYERS_PER_LAUNCH - 1) // sd.ATTENTION_LAYERS_PER_LAUNCH
         layers_per_launch = vs.L / n_att_launches
         att_s = per_call_ms["attention"] * 1e-3 / n_att_launches          # one launch = layers_per_launch layers
-        lm_s = per_call_ms["lmhead"] * 1e-3
+        lm_s = per_call_ms["tail"] * 1e-3                  # LM-head tiles + the 18 us tail kernel
         att_tflops = work["att_flops"] * layers_per_launch / att_s / 1e12
         att_gbs = work["att_bytes"] * layers_per_launch / att_s / 1e9
         lm_tflops = work["lm_flops"] / lm_s / 1e12

@@ -14,7 +14,9 @@ namespace sdv {
 using namespace sm100;
 
 constexpr int kBM = 128;            // vocabulary rows per tile (MMA M)
-constexpr int kLmThreads = 161;     // warps 0-3 epilogue, warp 4 TMA producer, warp 5 = ONE thread: MMA issuer
+constexpr int kEpiWarps = 8;        // two epilogue warps per TMEM lane quadrant: even and odd 32-column chunks
+constexpr int kTmaWarpLm = kEpiWarps, kMmaWarpLm = kEpiWarps + 1;
+constexpr int kLmThreads = kEpiWarps * 32 + 32 + 1;   // epilogue warps, TMA producer warp, ONE thread: MMA issuer
                                     // (a one-thread warp keeps the issue loop in uniform control flow, so
                                     //  the MMA descriptors stay in uniform registers)
 constexpr int kMaxCols = kLmMaxCols; // hidden rows per launch (TMEM columns)
@@ -122,20 +124,20 @@ lmhead_umma_kernel(const __grid_constant__ CUtensorMap tmW, const __grid_constan
     if (threadIdx.x == 0) {
         abort_flag = 0;
         for (int s = 0; s < p.stages; ++s) { mbar_init(&full_bar[s], 1); mbar_init(&empty_bar[s], 1); }
-        for (int b = 0; b < 2; ++b) { mbar_init(&tmem_full[b], 1); mbar_init(&tmem_empty[b], 4); }
+        for (int b = 0; b < 2; ++b) { mbar_init(&tmem_full[b], 1); mbar_init(&tmem_empty[b], kEpiWarps); }
         fence_barrier_init();
     }
-    if (warp == 4) {                   // a full warp
+    if (warp == kTmaWarpLm) {          // a full warp
         tmem_alloc(&tmem_base_slot, (uint32_t)p.tmem_cols);
         tmem_relinquish();
     }
-    if (warp == 4 && lane == 0) { prefetch_tensormap(&tmW); prefetch_tensormap(&tmH); }
+    if (warp == kTmaWarpLm && lane == 0) { prefetch_tensormap(&tmW); prefetch_tensormap(&tmH); }
     tc_fence_before_sync();
     __syncthreads();
     tc_fence_after_sync();
     const uint32_t tmem_base = tmem_base_slot;
 
-    if (warp == 4) {
+    if (warp == kTmaWarpLm) {
         // ------------------------------------------------ TMA producer
         if (lane == 0) {
             const uint64_t pol_w = policy_evict_first();
@@ -161,7 +163,7 @@ lmhead_umma_kernel(const __grid_constant__ CUtensorMap tmW, const __grid_constan
                 for (int i = 0; i < 1000; ++i) __nanosleep(1000);   // let copies in flight land
             }
         }
-    } else if (warp == 5) {
+    } else if (warp == kMmaWarpLm) {
         // ------------------------------------------------ MMA issuer (this warp is one thread)
         {
             const uint32_t idesc = make_idesc_bf16(kBM, p.part_n, false, false);
@@ -196,22 +198,26 @@ lmhead_umma_kernel(const __grid_constant__ CUtensorMap tmW, const __grid_constan
             if (!ok) set_status(status, SD_ERR_TIMEOUT);
         }
     } else {
-        // ------------------------------------------------ epilogue warps 0..3 (TMEM lanes 32*warp ..)
-        float best_val[kMaxCols / 32];
-        int32_t best_idx[kMaxCols / 32];
+        // ------------------------------------------------ epilogue warps 0..7
+        // warp w works on TMEM lanes 32 * (w & 3) .. +31 (the only ones it may read) and on the
+        // 32-column chunks of parity w >> 2
+        const int quad = warp & 3, par = warp >> 2;
+        float best_val[kMaxCols / 64];
+        int32_t best_idx[kMaxCols / 64];
 #pragma unroll
-        for (int c = 0; c < kMaxCols / 32; ++c) { best_val[c] = -INFINITY; best_idx[c] = 0x7fffffff; }
+        for (int c = 0; c < kMaxCols / 64; ++c) { best_val[c] = -INFINITY; best_idx[c] = 0x7fffffff; }
         bool ok = true;
         for (int t = 0; t < my_tiles && ok; ++t) {
             const int buf = t % p.acc_bufs;
             const uint32_t use = (uint32_t)(t / p.acc_bufs);
             if (!mbar_wait(&tmem_full[buf], use & 1u, &abort_flag)) { ok = false; break; }
             tc_fence_after_sync();
-            const int v_base = ((int)blockIdx.x + t * (int)gridDim.x) * kBM + warp * 32;
+            const int v_base = ((int)blockIdx.x + t * (int)gridDim.x) * kBM + quad * 32;
             const bool v_ok = (v_base + lane) < p.V;
-            const uint32_t taddr = tmem_base + ((uint32_t)(warp * 32) << 16) + (uint32_t)(buf * p.buf_stride);
+            const uint32_t taddr = tmem_base + ((uint32_t)(quad * 32) << 16) + (uint32_t)(buf * p.buf_stride);
 #pragma unroll
-            for (int c = 0; c < kMaxCols / 32; ++c) {
+            for (int h = 0; h < kMaxCols / 64; ++h) {
+                const int c = 2 * h + par;                 // this warp's chunk of the pair (2h, 2h + 1)
                 if (c * 32 < p.n_pad) {
                     uint32_t r[32];
                     tmem_ld32(taddr + c * 32, r);
@@ -219,7 +225,7 @@ lmhead_umma_kernel(const __grid_constant__ CUtensorMap tmW, const __grid_constan
                     float cv;
                     int32_t ci;
                     column_argmax32(r, v_ok, v_base, lane, cv, ci);
-                    if (cv > best_val[c]) { best_val[c] = cv; best_idx[c] = ci; }
+                    if (cv > best_val[h]) { best_val[h] = cv; best_idx[h] = ci; }
                 }
             }
             tc_fence_before_sync();
@@ -228,16 +234,16 @@ lmhead_umma_kernel(const __grid_constant__ CUtensorMap tmW, const __grid_constan
         }
         // merge the four warps through shared memory (the pipeline stages are idle by now:
         // the last accumulator was complete, so every copy has landed and every MMA has read it)
-        asm volatile("bar.sync 1, 128;" ::: "memory");
+        asm volatile("bar.sync 1, %0;" ::"n"(kEpiWarps * 32) : "memory");
         int32_t* red_key = reinterpret_cast<int32_t*>(smem);
         int32_t* red_idx = red_key + 4 * kMaxCols;
 #pragma unroll
-        for (int c = 0; c < kMaxCols / 32; ++c) {
-            red_key[warp * kMaxCols + c * 32 + lane] = ordered_key(__float_as_uint(best_val[c]));
-            red_idx[warp * kMaxCols + c * 32 + lane] = best_idx[c];
+        for (int h = 0; h < kMaxCols / 64; ++h) {
+            red_key[quad * kMaxCols + (2 * h + par) * 32 + lane] = ordered_key(__float_as_uint(best_val[h]));
+            red_idx[quad * kMaxCols + (2 * h + par) * 32 + lane] = best_idx[h];
         }
-        asm volatile("bar.sync 1, 128;" ::: "memory");
-        for (int col = threadIdx.x; col < kMaxCols; col += 128) {
+        asm volatile("bar.sync 1, %0;" ::"n"(kEpiWarps * 32) : "memory");
+        for (int col = threadIdx.x; col < kMaxCols; col += kEpiWarps * 32) {
             int32_t k = red_key[col], i = red_idx[col];
 #pragma unroll
             for (int w = 1; w < 4; ++w) {
@@ -250,7 +256,7 @@ lmhead_umma_kernel(const __grid_constant__ CUtensorMap tmW, const __grid_constan
     }
     tc_fence_before_sync();
     __syncthreads();
-    if (warp == 4) {
+    if (warp == kTmaWarpLm) {
         tc_fence_after_sync();
         tmem_dealloc(tmem_base, (uint32_t)p.tmem_cols);
     }
@@ -293,14 +299,14 @@ lmhead_umma_pair_kernel(const __grid_constant__ CUtensorMap tmW, const __grid_co
     if (threadIdx.x == 0) {
         abort_flag = 0;
         for (int s = 0; s < p.stages; ++s) { mbar_init(&full_bar[s], 1); mbar_init(&empty_bar[s], 1); }
-        for (int b = 0; b < 2; ++b) { mbar_init(&tmem_full[b], 1); mbar_init(&tmem_empty[b], 8); }
+        for (int b = 0; b < 2; ++b) { mbar_init(&tmem_full[b], 1); mbar_init(&tmem_empty[b], 2 * kEpiWarps); }
         fence_barrier_init();
     }
-    if (warp == 4) {                   // a full warp
+    if (warp == kTmaWarpLm) {          // a full warp
         tmem_alloc_pair(&tmem_base_slot, (uint32_t)p.tmem_cols);
         tmem_relinquish_pair();
     }
-    if (warp == 4 && lane == 0) { prefetch_tensormap(&tmW); prefetch_tensormap(&tmH); }
+    if (warp == kTmaWarpLm && lane == 0) { prefetch_tensormap(&tmW); prefetch_tensormap(&tmH); }
     tc_fence_before_sync();
     __syncthreads();
     cluster_arrive_release();          // the partner's barriers exist before anything signals them
@@ -308,7 +314,7 @@ lmhead_umma_pair_kernel(const __grid_constant__ CUtensorMap tmW, const __grid_co
     tc_fence_after_sync();
     const uint32_t tmem_base = tmem_base_slot;
 
-    if (warp == 4) {
+    if (warp == kTmaWarpLm) {
         // ------------------------------------------------ TMA producer (one per CTA)
         if (lane == 0) {
             const uint64_t pol_w = policy_evict_first();
@@ -335,7 +341,7 @@ lmhead_umma_pair_kernel(const __grid_constant__ CUtensorMap tmW, const __grid_co
                 for (int i = 0; i < 1000; ++i) __nanosleep(1000);   // let copies in flight land
             }
         }
-    } else if (warp == 5) {
+    } else if (warp == kMmaWarpLm) {
         // ------------------------------------------------ MMA issuer (leader CTA only; this warp is one thread)
         if (rank == 0) {
             const uint32_t idesc = make_idesc_bf16(2 * kBM, p.part_n, false, false);
@@ -373,22 +379,26 @@ lmhead_umma_pair_kernel(const __grid_constant__ CUtensorMap tmW, const __grid_co
             if (!ok) set_status(status, SD_ERR_TIMEOUT);
         }
     } else {
-        // ------------------------------------------------ epilogue warps 0..3 (TMEM lanes 32*warp ..)
-        float best_val[kMaxCols / 32];
-        int32_t best_idx[kMaxCols / 32];
+        // ------------------------------------------------ epilogue warps 0..7
+        // warp w works on TMEM lanes 32 * (w & 3) .. +31 (the only ones it may read) and on the
+        // 32-column chunks of parity w >> 2
+        const int quad = warp & 3, par = warp >> 2;
+        float best_val[kMaxCols / 64];
+        int32_t best_idx[kMaxCols / 64];
 #pragma unroll
-        for (int c = 0; c < kMaxCols / 32; ++c) { best_val[c] = -INFINITY; best_idx[c] = 0x7fffffff; }
+        for (int c = 0; c < kMaxCols / 64; ++c) { best_val[c] = -INFINITY; best_idx[c] = 0x7fffffff; }
         bool ok = true;
         for (int t = 0; t < my_tiles && ok; ++t) {
             const int buf = t % p.acc_bufs;
             const uint32_t use = (uint32_t)(t / p.acc_bufs);
             if (!mbar_wait(&tmem_full[buf], use & 1u, &abort_flag)) { ok = false; break; }
             tc_fence_after_sync();
-            const int v_base = ((pair + t * n_pairs) * 2 + (int)rank) * kBM + warp * 32;
+            const int v_base = ((pair + t * n_pairs) * 2 + (int)rank) * kBM + quad * 32;
             const bool v_ok = (v_base + lane) < p.V;
-            const uint32_t taddr = tmem_base + ((uint32_t)(warp * 32) << 16) + (uint32_t)(buf * p.buf_stride);
+            const uint32_t taddr = tmem_base + ((uint32_t)(quad * 32) << 16) + (uint32_t)(buf * p.buf_stride);
 #pragma unroll
-            for (int c = 0; c < kMaxCols / 32; ++c) {
+            for (int h = 0; h < kMaxCols / 64; ++h) {
+                const int c = 2 * h + par;                 // this warp's chunk of the pair (2h, 2h + 1)
                 if (c * 32 < p.n_pad) {
                     uint32_t r[32];
                     tmem_ld32(taddr + c * 32, r);
@@ -396,23 +406,23 @@ lmhead_umma_pair_kernel(const __grid_constant__ CUtensorMap tmW, const __grid_co
                     float cv;
                     int32_t ci;
                     column_argmax32(r, v_ok, v_base, lane, cv, ci);
-                    if (cv > best_val[c]) { best_val[c] = cv; best_idx[c] = ci; }
+                    if (cv > best_val[h]) { best_val[h] = cv; best_idx[h] = ci; }
                 }
             }
             tc_fence_before_sync();
             __syncwarp();
             if (lane == 0) mbar_arrive_remote(map_dsmem(smem_u32(&tmem_empty[buf]), 0));
         }
-        asm volatile("bar.sync 1, 128;" ::: "memory");
+        asm volatile("bar.sync 1, %0;" ::"n"(kEpiWarps * 32) : "memory");
         int32_t* red_key = reinterpret_cast<int32_t*>(smem);
         int32_t* red_idx = red_key + 4 * kMaxCols;
 #pragma unroll
-        for (int c = 0; c < kMaxCols / 32; ++c) {
-            red_key[warp * kMaxCols + c * 32 + lane] = ordered_key(__float_as_uint(best_val[c]));
-            red_idx[warp * kMaxCols + c * 32 + lane] = best_idx[c];
+        for (int h = 0; h < kMaxCols / 64; ++h) {
+            red_key[quad * kMaxCols + (2 * h + par) * 32 + lane] = ordered_key(__float_as_uint(best_val[h]));
+            red_idx[quad * kMaxCols + (2 * h + par) * 32 + lane] = best_idx[h];
         }
-        asm volatile("bar.sync 1, 128;" ::: "memory");
-        for (int col = threadIdx.x; col < kMaxCols; col += 128) {
+        asm volatile("bar.sync 1, %0;" ::"n"(kEpiWarps * 32) : "memory");
+        for (int col = threadIdx.x; col < kMaxCols; col += kEpiWarps * 32) {
             int32_t k = red_key[col], i = red_idx[col];
 #pragma unroll
             for (int w = 1; w < 4; ++w) {
@@ -427,7 +437,7 @@ lmhead_umma_pair_kernel(const __grid_constant__ CUtensorMap tmW, const __grid_co
     __syncthreads();
     cluster_arrive_release();          // neither CTA leaves while the other may still signal it
     cluster_wait_acquire();
-    if (warp == 4) {
+    if (warp == kTmaWarpLm) {
         tc_fence_after_sync();
         tmem_dealloc_pair(tmem_base, (uint32_t)p.tmem_cols);
     }

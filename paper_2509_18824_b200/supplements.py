@@ -2,7 +2,7 @@
 the LM head at several row counts, and the bandwidth-regime cases (chain
 decoding, a compaction stress shape).  One JSON line per measurement.
 
-    python -m paper_2509_18824_b200.supplements [attention] [attention_layers] [lmhead] [compact]
+    python -m paper_2509_18824_b200.supplements [attention] [attention_layers] [lmhead] [lmhead480] [compact]
 
 Timing: CUDA events on the launching stream, >= 3 warm-up calls, inputs rotated
 over several layers so that the working set exceeds L2.
@@ -161,5 +161,7 @@ if __name__ == "__main__":
         attention_layers()
     if "lmhead" in what:
         lmhead()
+    if "lmhead480" in what:                # the bench's LM-head launch alone (profiler captures)
+        lmhead(rows=(480,))
     if "compact" in what:
         compact()
