@@ -1,0 +1,114 @@
+"""Reference for verification at a sampling temperature (TEST INFRASTRUCTURE ONLY).
+
+The paper validates the draft's tokens with the target model and keeps the
+target's output distribution unchanged (Sec. 1: "batch-validated by the target
+model", lossless; the speculative-sampling lineage it cites in Sec. 1 gives the
+rule for sampling: accept a drafted token x with probability min(1, p(x)/q(x)),
+otherwise resample from the normalised positive part of p - q).  The drafts of
+an EAGLE-style tree are chosen deterministically (top-k), i.e. q is a point
+mass on each child's token, and the rule becomes sequential rejection without
+replacement:
+
+    at node i with target distribution p_i = softmax(logits_i / tau), residual mass R = 1:
+      for every child c of i, in node order:
+          accept c  iff  u[c] * R < p_i(token[c]);     then continue at c with R = 1
+          otherwise R -= p_i(token[c])
+      if no child was accepted (or i is a leaf): emit one token from p_i restricted to the
+      tokens that are not children of i, by inverse CDF in vocabulary order with the
+      uniform w:  the first token t whose cumulative remaining mass reaches w * R.
+
+Every random number is an input (u per node, w per sequence).  Plain numpy,
+fp64 unless a dtype is passed; no code shared with the GPU library.  Siblings
+must carry distinct tokens.
+
+Parity with the paper's own acceptance statistics is unpinned (they need the
+trained models).  The functions are pinned in tests/test_oracle_sampling.py by
+Monte-Carlo frequencies against p, by the zero-temperature limit (the greedy
+rule), by the single-child case (the textbook accept test) and by numpy's
+cumsum/searchsorted for the inverse CDF.
+"""
+from __future__ import annotations
+
+import numpy as np
+
+
+def softmax_rows(logits: np.ndarray, inv_temp: float):
+    """p = softmax(logits * inv_temp) per row and lse = log sum exp(logits * inv_temp), fp64."""
+    z = np.asarray(logits, dtype=np.float64) * float(inv_temp)
+    m = z.max(axis=-1, keepdims=True)
+    e = np.exp(z - m)
+    s = e.sum(axis=-1, keepdims=True)
+    return e / s, (m + np.log(s))[..., 0]
+
+
+def children_of(parents: np.ndarray, n: int, i: int):
+    return [j for j in range(i + 1, n) if parents[j] == i]
+
+
+def accept_walk(parents, n_nodes, draft_tok, p_child, u, dtype=np.float64):
+    """The acceptance walk of ONE sequence.
+
+    p_child[j] = probability of draft_tok[j] under the target distribution at parent(j) (j >= 1),
+    u[j] = the uniform drawn for node j.  The comparison u * R < p and the update R -= p are done in
+    `dtype` (fp64 for the definition; float32 reproduces the kernel's arithmetic bit for bit).
+    Returns (path, R): the accepted root path and the residual mass left at its last node.
+    """
+    parents = np.asarray(parents)
+    p_child = np.asarray(p_child, dtype=dtype)
+    u = np.asarray(u, dtype=dtype)
+    n = int(n_nodes)
+    cur, path = 0, [0]
+    one = dtype(1.0)
+    R = one
+    while True:
+        nxt = -1
+        R = one
+        kids = children_of(parents, n, cur)
+        toks = [int(draft_tok[c]) for c in kids]
+        assert len(set(toks)) == len(toks), "siblings must carry distinct tokens"
+        for c in kids:
+            if dtype(u[c] * R) < p_child[c]:
+                nxt = c
+                break
+            R = dtype(R - p_child[c])
+        if nxt < 0:
+            return path, R
+        cur = nxt
+        path.append(cur)
+
+
+def residual_sample(p_row, excluded, R, w):
+    """First token t (vocabulary order, tokens in `excluded` carry no mass) whose cumulative mass
+    reaches w * R; the last token with mass if rounding leaves the sum short.  Returns (t, margin):
+    margin = distance of the target from the nearer end of t's CDF interval (how close the decision
+    was)."""
+    p = np.array(p_row, dtype=np.float64)
+    if len(excluded):
+        p[np.asarray(excluded, dtype=np.int64)] = 0.0
+    target = float(w) * float(R)
+    acc = 0.0
+    last = -1
+    for t in range(len(p)):
+        if p[t] <= 0.0:
+            continue
+        last = t
+        if acc + p[t] >= target:
+            return t, min(target - acc, acc + p[t] - target)
+        acc += p[t]
+    return last, 0.0
+
+
+def verify_sequence(parents, n_nodes, draft_tok, logits, inv_temp, u, w):
+    """Whole rule for one sequence from the target's logits [T, V] (fp64 definition).
+    Returns (path, out_tok): accepted nodes and the emitted tokens (accepted drafts, then the
+    residual sample at the last accepted node)."""
+    p, _ = softmax_rows(logits, inv_temp)
+    n = int(n_nodes)
+    p_child = np.zeros(len(parents))
+    for j in range(1, n):
+        p_child[j] = p[parents[j], draft_tok[j]]
+    path, R = accept_walk(parents, n, draft_tok, p_child, u)
+    last = path[-1]
+    excl = [int(draft_tok[c]) for c in children_of(parents, n, last)]
+    t, _ = residual_sample(p[last], excl, R, w)
+    return path, [int(draft_tok[j]) for j in path[1:]] + [t]
