@@ -266,6 +266,54 @@ sd_status sd_lmhead_accept_compact(const sd_batch *batch, const void *hidden, co
                                    void *workspace, size_t workspace_bytes,
                                    int32_t *dev_status, void *stream);
 
+/*
+ * LM head with soft-max statistics, for verification at a sampling temperature
+ * (Sec. 1: the drafts are validated by the target model without changing its
+ * output distribution; the speculative-sampling rule the paper builds on
+ * compares a draft's probability under the target with a uniform number).
+ * As sd_lmhead_argmax, plus
+ *   lse[r] = log sum_v exp(logits[r][v] * inv_temp)        (natural log, fp32)
+ * accumulated in the same epilogue (running reference and sum per row; logits
+ * still never reach memory).  argmax and maxlogit may be NULL.
+ *   inv_temp  : 1 / temperature, > 0
+ *   workspace : at least sd_workspace_bytes(NULL, M, V)
+ */
+sd_status sd_lmhead_stats(const void *hidden, const void *W, int32_t M, int32_t Hd, int32_t V,
+                          float inv_temp, int32_t *argmax, float *maxlogit, float *lse,
+                          void *workspace, size_t workspace_bytes,
+                          int32_t *dev_status, void *stream);
+
+/*
+ * Acceptance at a sampling temperature for a deterministically drafted tree
+ * (Sec. 1, lossless validation; rule of the cited speculative-sampling work with
+ * a point-mass draft distribution).  With p_i = softmax(logits_i * inv_temp) the
+ * target distribution at node i:
+ *   at node i, residual mass R = 1; for every child c of i in node order:
+ *       accept c  iff  u[b][c] * R < p_i(draft_tok[c]);  continue at c with R = 1
+ *       otherwise R -= p_i(draft_tok[c])
+ *   where no child is accepted the walk stops and one more token is drawn from
+ *   p_i restricted to the tokens that are not drafted children of i: the first
+ *   token, in vocabulary order, at which the cumulative remaining mass reaches
+ *   w[b] times the total remaining mass.
+ * Outputs as sd_accept_tree (out_tok = accepted drafts, then the drawn token).
+ * All random numbers are inputs: u dev f32 [B][T_max] in [0,1), w dev f32 [B].
+ *   hidden, W, Hd, V : the LM head's operands (row b * T_max + i = node i of sequence b)
+ *   lse              : dev f32 [B * T_max] from sd_lmhead_stats with the same inv_temp
+ *   workspace        : at least sd_workspace_bytes(batch, B * T_max, V); it receives,
+ *                      among other things, the stop nodes' probabilities over the
+ *                      vocabulary (B x V floats) - the only logits-sized data that
+ *                      reach memory, for one row per sequence
+ * Siblings must carry distinct tokens.  Arithmetic: fp32; a comparison whose two
+ * sides differ by less than rounding may fall either way.  A draft token outside
+ * [0, V) stores SD_ERR_BOUNDS, a bad tree SD_ERR_INVALID_TREE.
+ */
+sd_status sd_accept_tree_sampled(const sd_batch *batch, const void *hidden, const void *W,
+                                 int32_t Hd, int32_t V, float inv_temp, const float *lse,
+                                 const int32_t *draft_tok, const float *u, const float *w,
+                                 int32_t *n_acc, int32_t *path, int32_t *out_tok, int32_t *new_len,
+                                 void *workspace, size_t workspace_bytes,
+                                 int32_t *dev_status, void *stream);
+
 #ifdef __cplusplus
 }
 #endif

@@ -32,7 +32,7 @@ KERNELS_PER_LMHEAD = 2         # tiles + cross-slab reduce
 
 EXPORTS = ["sd_version", "sd_status_string", "sd_workspace_bytes", "sd_tree_prepare",
            "sd_verify_attention", "sd_verify_attention_layers", "sd_lmhead_argmax", "sd_lmhead_argmax_static", "sd_accept_tree",
-           "sd_compact_kv", "sd_lmhead_accept_compact"]
+           "sd_compact_kv", "sd_lmhead_accept_compact", "sd_lmhead_stats", "sd_accept_tree_sampled"]
 
 
 class sd_kv_layer(C.Structure):
@@ -82,6 +82,14 @@ def _load(path: str = LIB_PATH) -> C.CDLL:
                                              C.c_void_p, C.c_int32, C.c_void_p, C.c_void_p,
                                              C.c_void_p, C.c_void_p, C.c_void_p, C.c_void_p, C.c_void_p, C.c_void_p,
                                              C.c_void_p, C.c_size_t, C.c_void_p, C.c_void_p]
+    lib.sd_lmhead_stats.restype = C.c_int
+    lib.sd_lmhead_stats.argtypes = [C.c_void_p, C.c_void_p, C.c_int32, C.c_int32, C.c_int32, C.c_float,
+                                    C.c_void_p, C.c_void_p, C.c_void_p, C.c_void_p, C.c_size_t, C.c_void_p, C.c_void_p]
+    lib.sd_accept_tree_sampled.restype = C.c_int
+    lib.sd_accept_tree_sampled.argtypes = [C.c_void_p, C.c_void_p, C.c_void_p, C.c_int32, C.c_int32, C.c_float,
+                                           C.c_void_p, C.c_void_p, C.c_void_p, C.c_void_p,
+                                           C.c_void_p, C.c_void_p, C.c_void_p, C.c_void_p,
+                                           C.c_void_p, C.c_size_t, C.c_void_p, C.c_void_p]
     return lib
 
 
@@ -253,3 +261,25 @@ def sd_lmhead_accept_compact(batch: Batch, hidden, W, draft_tok, layers: LayerSe
                                         layers.layers, layers.L, layers.kt, layers.vt, _ptr(argmax), _ptr(maxlogit),
                                         _ptr(n_acc), _ptr(path), _ptr(out_tok), _ptr(new_len), _ptr(workspace),
                                         workspace.numel() * workspace.element_size(), _ptr(status), _stream(stream)))
+
+
+def sd_lmhead_stats(hidden, W, inv_temp: float, argmax, maxlogit, lse, workspace, status, stream=None) -> None:
+    """LM-head arg-max plus lse[r] = log sum_v exp(logit[r][v] * inv_temp)."""
+    M, Hd = hidden.shape
+    V = W.shape[0]
+    assert W.shape[1] == Hd
+    _check(lib.sd_lmhead_stats(_ptr(hidden), _ptr(W), int(M), int(Hd), int(V), C.c_float(inv_temp), _ptr(argmax),
+                               _ptr(maxlogit), _ptr(lse), _ptr(workspace),
+                               workspace.numel() * workspace.element_size(), _ptr(status), _stream(stream)))
+
+
+def sd_accept_tree_sampled(batch: Batch, hidden, W, inv_temp: float, lse, draft_tok, u, w,
+                           n_acc, path, out_tok, new_len, workspace, status, stream=None) -> None:
+    """Acceptance at a sampling temperature (uniforms u [B,T] and w [B] are inputs)."""
+    M, Hd = hidden.shape
+    V = W.shape[0]
+    assert W.shape[1] == Hd and M == batch.B * batch.T_max
+    _check(lib.sd_accept_tree_sampled(batch.ref(), _ptr(hidden), _ptr(W), int(Hd), int(V), C.c_float(inv_temp),
+                                      _ptr(lse), _ptr(draft_tok), _ptr(u), _ptr(w), _ptr(n_acc), _ptr(path),
+                                      _ptr(out_tok), _ptr(new_len), _ptr(workspace),
+                                      workspace.numel() * workspace.element_size(), _ptr(status), _stream(stream)))

@@ -45,7 +45,11 @@ const char* sd_status_string(sd_status s) {
 size_t sd_workspace_bytes(const sd_batch* geom, int32_t M, int32_t V) {
     size_t a = 0, l = 0;
     if (geom && check_geometry(geom, false) == SD_OK) a = attention_workspace_bytes(*geom);
-    if (M > 0 && V > 0) l = tail_workspace_bytes(M, V);     // covers sd_lmhead_argmax and the fused tail
+    if (M > 0 && V > 0) l = stats_workspace_bytes(M, V);    // covers sd_lmhead_argmax, the fused tail and sd_lmhead_stats
+    if (geom && V > 0 && check_geometry(geom, false) == SD_OK) {
+        const size_t sw = sampled_workspace_bytes(geom->B, geom->T_max, V);   // sd_accept_tree_sampled
+        if (sw > l) l = sw;
+    }
     size_t n = a > l ? a : l;
     return (n + 255) & ~(size_t)255;
 }
@@ -152,6 +156,31 @@ sd_status sd_lmhead_accept_compact(const sd_batch* batch, const void* hidden, co
     return launch_lmhead_accept_compact(*batch, hidden, W, Hd, V, draft_tok, layers, L, k_tree_layers, v_tree_layers,
                                         argmax, maxlogit, n_acc, path, out_tok, new_len, workspace, workspace_bytes,
                                         dev_status, static_cast<cudaStream_t>(stream));
+}
+
+sd_status sd_lmhead_stats(const void* hidden, const void* W, int32_t M, int32_t Hd, int32_t V, float inv_temp,
+                          int32_t* argmax, float* maxlogit, float* lse, void* workspace, size_t workspace_bytes,
+                          int32_t* dev_status, void* stream) {
+    if (!ok_ptr(hidden) || !ok_ptr(W) || !lse || !ok_ptr(workspace) || !dev_status) return SD_ERR_INVALID_ARG;
+    if (M < 1 || V < 1 || Hd < 1 || !(inv_temp > 0.f)) return SD_ERR_INVALID_ARG;
+    if (Hd % 64 != 0) return SD_ERR_UNSUPPORTED;
+    return launch_lmhead_stats(hidden, W, M, Hd, V, inv_temp, argmax, maxlogit, lse, workspace, workspace_bytes,
+                               dev_status, static_cast<cudaStream_t>(stream));
+}
+
+sd_status sd_accept_tree_sampled(const sd_batch* batch, const void* hidden, const void* W, int32_t Hd, int32_t V,
+                                 float inv_temp, const float* lse, const int32_t* draft_tok,
+                                 const float* u, const float* w,
+                                 int32_t* n_acc, int32_t* path, int32_t* out_tok, int32_t* new_len,
+                                 void* workspace, size_t workspace_bytes, int32_t* dev_status, void* stream) {
+    sd_status s = check_geometry(batch, true);
+    if (s != SD_OK) return s;
+    if (!ok_ptr(hidden) || !ok_ptr(W) || !lse || !draft_tok || !u || !w) return SD_ERR_INVALID_ARG;
+    if (!n_acc || !path || !out_tok || !new_len || !ok_ptr(workspace) || !dev_status) return SD_ERR_INVALID_ARG;
+    if (V < 1 || Hd < 1 || !(inv_temp > 0.f)) return SD_ERR_INVALID_ARG;
+    if (Hd % 64 != 0) return SD_ERR_UNSUPPORTED;
+    return launch_accept_sampled(*batch, hidden, W, Hd, V, inv_temp, lse, draft_tok, u, w, n_acc, path, out_tok,
+                                 new_len, workspace, workspace_bytes, dev_status, static_cast<cudaStream_t>(stream));
 }
 
 }  // extern "C"

@@ -38,6 +38,10 @@ struct LmParams {
     int stages;
     int32_t* part_key; // [gridDim.x][kMaxCols] order-preserving integer image of the max logit
     int32_t* part_idx; // [gridDim.x][kMaxCols]
+    // soft-max statistics (sampling at a temperature): c2 = log2(e) / temperature, 0 = not wanted
+    float c2;
+    float* part_ref;   // [gridDim.x][kMaxCols] reference logit of the partial sum
+    float* part_sum;   // [gridDim.x][kMaxCols] sum over the CTA's vocabulary rows of 2^((logit - ref) * c2)
 };
 
 size_t lmhead_workspace_bytes(int M, int V) {
@@ -48,6 +52,10 @@ size_t lmhead_workspace_bytes(int M, int V) {
 // 2 * B + 2 * B * T_max <= 4 * 512 words, for up to 64 layers
 size_t tail_workspace_bytes(int M, int V) {
     return lmhead_workspace_bytes(M, V) + (size_t)kLayersPerLaunch * 4 * kMaxCols * sizeof(int32_t);
+}
+// soft-max statistics: two more per-CTA tables (reference, partial sum), behind the tail's area
+size_t stats_workspace_bytes(int M, int V) {
+    return tail_workspace_bytes(M, V) + (size_t)kMaxCtas * kMaxCols * 2 * sizeof(float);
 }
 
 // float -> int whose signed order equals the float order (-0 folded onto +0)
@@ -96,6 +104,68 @@ __device__ __forceinline__ void column_argmax32(const uint32_t (&r)[32], bool v_
     for (int j = 0; j < 32; ++j) who[j] = __ballot_sync(0xffffffffu, v[j] == mx[j]);
     cv = pick_lane(mx, lane);
     ci = v_base + (__ffs(pick_lane(who, lane)) - 1);
+}
+
+__device__ __forceinline__ float ex2_lm(float x) {
+    float y;
+    asm("ex2.approx.ftz.f32 %0, %1;" : "=f"(y) : "f"(x));
+    return y;
+}
+
+// Sum over the 32 lanes of each of 32 per-lane values: lane j receives sum_lanes x[j].  Five
+// exchange steps; in each a lane keeps the half of its values whose column index has the step's
+// bit equal to its own lane bit and hands the other half to its partner (fixed order of additions).
+__device__ __forceinline__ float transpose_sum32(const float (&x)[32], int lane) {
+    float a[16], b[8], c[4], d[2];
+#pragma unroll
+    for (int i = 0; i < 16; ++i) {
+        const float keep = (lane & 16) ? x[i + 16] : x[i], send = (lane & 16) ? x[i] : x[i + 16];
+        a[i] = keep + __shfl_xor_sync(0xffffffffu, send, 16);
+    }
+#pragma unroll
+    for (int i = 0; i < 8; ++i) {
+        const float keep = (lane & 8) ? a[i + 8] : a[i], send = (lane & 8) ? a[i] : a[i + 8];
+        b[i] = keep + __shfl_xor_sync(0xffffffffu, send, 8);
+    }
+#pragma unroll
+    for (int i = 0; i < 4; ++i) {
+        const float keep = (lane & 4) ? b[i + 4] : b[i], send = (lane & 4) ? b[i] : b[i + 4];
+        c[i] = keep + __shfl_xor_sync(0xffffffffu, send, 4);
+    }
+#pragma unroll
+    for (int i = 0; i < 2; ++i) {
+        const float keep = (lane & 2) ? c[i + 2] : c[i], send = (lane & 2) ? c[i] : c[i + 2];
+        d[i] = keep + __shfl_xor_sync(0xffffffffu, send, 2);
+    }
+    const float keep = (lane & 1) ? d[1] : d[0], send = (lane & 1) ? d[0] : d[1];
+    return keep + __shfl_xor_sync(0xffffffffu, send, 1);
+}
+
+// The same arg-max plus, per column, sum over the 32 vocabulary rows of 2^((logit - column max) * c2):
+// lane j receives column j's sum in cs.
+__device__ __forceinline__ void column_argmax_stats32(const uint32_t (&r)[32], bool v_ok, int v_base, int lane,
+                                                      float c2, float& cv, int32_t& ci, float& cs) {
+    float v[32], mx[32];
+#pragma unroll
+    for (int j = 0; j < 32; ++j) v[j] = v_ok ? __uint_as_float(r[j]) : -INFINITY;
+#pragma unroll
+    for (int j = 0; j < 32; ++j) mx[j] = redux_max_f32(v[j]);
+    uint32_t who[32];
+#pragma unroll
+    for (int j = 0; j < 32; ++j) who[j] = __ballot_sync(0xffffffffu, v[j] == mx[j]);
+    cv = pick_lane(mx, lane);
+    ci = v_base + (__ffs(pick_lane(who, lane)) - 1);
+    float e[32];
+#pragma unroll
+    for (int j = 0; j < 32; ++j) e[j] = (v[j] == -INFINITY) ? 0.f : ex2_lm((v[j] - mx[j]) * c2);
+    cs = transpose_sum32(e, lane);
+}
+
+// running (reference, sum) of a column takes in a new partial (ref2, sum2)
+__device__ __forceinline__ void merge_sumexp(float& ref, float& sum, float ref2, float sum2, float c2) {
+    if (!(sum2 > 0.f)) return;
+    if (ref2 > ref) { sum = sum * ex2_lm((ref - ref2) * c2) + sum2; ref = ref2; }
+    else            { sum += sum2 * ex2_lm((ref2 - ref) * c2); }
 }
 
 template <int BK>
@@ -204,8 +274,12 @@ lmhead_umma_kernel(const __grid_constant__ CUtensorMap tmW, const __grid_constan
         const int quad = warp & 3, par = warp >> 2;
         float best_val[kMaxCols / 64];
         int32_t best_idx[kMaxCols / 64];
+        float run_ref[kMaxCols / 64], run_sum[kMaxCols / 64];
 #pragma unroll
-        for (int c = 0; c < kMaxCols / 64; ++c) { best_val[c] = -INFINITY; best_idx[c] = 0x7fffffff; }
+        for (int c = 0; c < kMaxCols / 64; ++c) {
+            best_val[c] = -INFINITY; best_idx[c] = 0x7fffffff; run_ref[c] = -INFINITY; run_sum[c] = 0.f;
+        }
+        const bool stats = p.c2 > 0.f;
         bool ok = true;
         for (int t = 0; t < my_tiles && ok; ++t) {
             const int buf = t % p.acc_bufs;
@@ -224,7 +298,13 @@ lmhead_umma_kernel(const __grid_constant__ CUtensorMap tmW, const __grid_constan
                     tmem_ld_wait();
                     float cv;
                     int32_t ci;
-                    column_argmax32(r, v_ok, v_base, lane, cv, ci);
+                    if (stats) {
+                        float cs;
+                        column_argmax_stats32(r, v_ok, v_base, lane, p.c2, cv, ci, cs);
+                        merge_sumexp(run_ref[h], run_sum[h], cv, cs, p.c2);
+                    } else {
+                        column_argmax32(r, v_ok, v_base, lane, cv, ci);
+                    }
                     if (cv > best_val[h]) { best_val[h] = cv; best_idx[h] = ci; }
                 }
             }
@@ -237,10 +317,16 @@ lmhead_umma_kernel(const __grid_constant__ CUtensorMap tmW, const __grid_constan
         asm volatile("bar.sync 1, %0;" ::"n"(kEpiWarps * 32) : "memory");
         int32_t* red_key = reinterpret_cast<int32_t*>(smem);
         int32_t* red_idx = red_key + 4 * kMaxCols;
+        float* red_ref = reinterpret_cast<float*>(red_idx + 4 * kMaxCols);
+        float* red_sum = red_ref + 4 * kMaxCols;
 #pragma unroll
         for (int h = 0; h < kMaxCols / 64; ++h) {
             red_key[quad * kMaxCols + (2 * h + par) * 32 + lane] = ordered_key(__float_as_uint(best_val[h]));
             red_idx[quad * kMaxCols + (2 * h + par) * 32 + lane] = best_idx[h];
+            if (stats) {
+                red_ref[quad * kMaxCols + (2 * h + par) * 32 + lane] = run_ref[h];
+                red_sum[quad * kMaxCols + (2 * h + par) * 32 + lane] = run_sum[h];
+            }
         }
         asm volatile("bar.sync 1, %0;" ::"n"(kEpiWarps * 32) : "memory");
         for (int col = threadIdx.x; col < kMaxCols; col += kEpiWarps * 32) {
@@ -252,6 +338,13 @@ lmhead_umma_kernel(const __grid_constant__ CUtensorMap tmW, const __grid_constan
             }
             p.part_key[(size_t)blockIdx.x * kMaxCols + col] = ok ? k : INT32_MIN;
             p.part_idx[(size_t)blockIdx.x * kMaxCols + col] = i;
+            if (stats) {
+                float rf = red_ref[col], sm = red_sum[col];
+#pragma unroll
+                for (int w = 1; w < 4; ++w) merge_sumexp(rf, sm, red_ref[w * kMaxCols + col], red_sum[w * kMaxCols + col], p.c2);
+                p.part_ref[(size_t)blockIdx.x * kMaxCols + col] = rf;
+                p.part_sum[(size_t)blockIdx.x * kMaxCols + col] = sm;
+            }
         }
     }
     tc_fence_before_sync();
@@ -385,8 +478,12 @@ lmhead_umma_pair_kernel(const __grid_constant__ CUtensorMap tmW, const __grid_co
         const int quad = warp & 3, par = warp >> 2;
         float best_val[kMaxCols / 64];
         int32_t best_idx[kMaxCols / 64];
+        float run_ref[kMaxCols / 64], run_sum[kMaxCols / 64];
 #pragma unroll
-        for (int c = 0; c < kMaxCols / 64; ++c) { best_val[c] = -INFINITY; best_idx[c] = 0x7fffffff; }
+        for (int c = 0; c < kMaxCols / 64; ++c) {
+            best_val[c] = -INFINITY; best_idx[c] = 0x7fffffff; run_ref[c] = -INFINITY; run_sum[c] = 0.f;
+        }
+        const bool stats = p.c2 > 0.f;
         bool ok = true;
         for (int t = 0; t < my_tiles && ok; ++t) {
             const int buf = t % p.acc_bufs;
@@ -405,7 +502,13 @@ lmhead_umma_pair_kernel(const __grid_constant__ CUtensorMap tmW, const __grid_co
                     tmem_ld_wait();
                     float cv;
                     int32_t ci;
-                    column_argmax32(r, v_ok, v_base, lane, cv, ci);
+                    if (stats) {
+                        float cs;
+                        column_argmax_stats32(r, v_ok, v_base, lane, p.c2, cv, ci, cs);
+                        merge_sumexp(run_ref[h], run_sum[h], cv, cs, p.c2);
+                    } else {
+                        column_argmax32(r, v_ok, v_base, lane, cv, ci);
+                    }
                     if (cv > best_val[h]) { best_val[h] = cv; best_idx[h] = ci; }
                 }
             }
@@ -416,10 +519,16 @@ lmhead_umma_pair_kernel(const __grid_constant__ CUtensorMap tmW, const __grid_co
         asm volatile("bar.sync 1, %0;" ::"n"(kEpiWarps * 32) : "memory");
         int32_t* red_key = reinterpret_cast<int32_t*>(smem);
         int32_t* red_idx = red_key + 4 * kMaxCols;
+        float* red_ref = reinterpret_cast<float*>(red_idx + 4 * kMaxCols);
+        float* red_sum = red_ref + 4 * kMaxCols;
 #pragma unroll
         for (int h = 0; h < kMaxCols / 64; ++h) {
             red_key[quad * kMaxCols + (2 * h + par) * 32 + lane] = ordered_key(__float_as_uint(best_val[h]));
             red_idx[quad * kMaxCols + (2 * h + par) * 32 + lane] = best_idx[h];
+            if (stats) {
+                red_ref[quad * kMaxCols + (2 * h + par) * 32 + lane] = run_ref[h];
+                red_sum[quad * kMaxCols + (2 * h + par) * 32 + lane] = run_sum[h];
+            }
         }
         asm volatile("bar.sync 1, %0;" ::"n"(kEpiWarps * 32) : "memory");
         for (int col = threadIdx.x; col < kMaxCols; col += kEpiWarps * 32) {
@@ -431,6 +540,13 @@ lmhead_umma_pair_kernel(const __grid_constant__ CUtensorMap tmW, const __grid_co
             }
             p.part_key[(size_t)blockIdx.x * kMaxCols + col] = ok ? k : INT32_MIN;
             p.part_idx[(size_t)blockIdx.x * kMaxCols + col] = i;
+            if (stats) {
+                float rf = red_ref[col], sm = red_sum[col];
+#pragma unroll
+                for (int w = 1; w < 4; ++w) merge_sumexp(rf, sm, red_ref[w * kMaxCols + col], red_sum[w * kMaxCols + col], p.c2);
+                p.part_ref[(size_t)blockIdx.x * kMaxCols + col] = rf;
+                p.part_sum[(size_t)blockIdx.x * kMaxCols + col] = sm;
+            }
         }
     }
     tc_fence_before_sync();
@@ -458,14 +574,33 @@ __global__ void lmhead_merge_kernel(const int32_t* __restrict__ part_key, const 
     if (maxlogit) maxlogit[row0 + col] = key_to_float(k);
 }
 
+// the same merge plus log sum exp(logit / temperature) of every hidden row (natural log)
+__global__ void lmhead_merge_stats_kernel(const int32_t* __restrict__ part_key, const int32_t* __restrict__ part_idx,
+                                          const float* __restrict__ part_ref, const float* __restrict__ part_sum,
+                                          int n_ctas, int rows, int row0, float c2, int32_t* __restrict__ argmax,
+                                          float* __restrict__ maxlogit, float* __restrict__ lse) {
+    const int col = blockIdx.x * blockDim.x + threadIdx.x;
+    if (col >= rows) return;
+    int32_t k = INT32_MIN, i = 0x7fffffff;
+    float rf = -INFINITY, sm = 0.f;
+    for (int c = 0; c < n_ctas; ++c) {
+        take_better(k, i, part_key[(size_t)c * kMaxCols + col], part_idx[(size_t)c * kMaxCols + col]);
+        merge_sumexp(rf, sm, part_ref[(size_t)c * kMaxCols + col], part_sum[(size_t)c * kMaxCols + col], c2);
+    }
+    if (argmax) argmax[row0 + col] = i;
+    if (maxlogit) maxlogit[row0 + col] = key_to_float(k);
+    lse[row0 + col] = (rf * c2 + log2f(sm)) * 0.6931471805599453f;
+}
+
 static int round_up(int x, int m) { return (x + m - 1) / m * m; }
 
 // tiles_only_ctas != nullptr (M <= 512 required): launch only the tile kernel and report how many
 // CTAs filled the candidate tables; the caller merges them itself (the fused tail kernel).
 static sd_status launch_lmhead_impl(const void* hidden, const void* W, int M, int Hd, int V,
                                     int32_t* argmax, float* maxlogit, void* ws, size_t ws_bytes,
-                                    int32_t* dev_status, cudaStream_t st, int* tiles_only_ctas) {
-    if (ws_bytes < lmhead_workspace_bytes(M, V)) return SD_ERR_WORKSPACE;
+                                    int32_t* dev_status, cudaStream_t st, int* tiles_only_ctas,
+                                    float inv_temp = 0.f, float* lse = nullptr) {
+    if (ws_bytes < (lse ? stats_workspace_bytes(M, V) : lmhead_workspace_bytes(M, V))) return SD_ERR_WORKSPACE;
     if (tiles_only_ctas && M > kMaxCols) return SD_ERR_UNSUPPORTED;
     int dev = 0, sms = 0;
     if (cudaGetDevice(&dev) != cudaSuccess ||
@@ -507,6 +642,9 @@ static sd_status launch_lmhead_impl(const void* hidden, const void* W, int M, in
         p.stages = stages;
         p.part_key = static_cast<int32_t*>(ws);
         p.part_idx = p.part_key + (size_t)kMaxCtas * kMaxCols;
+        p.c2 = lse ? inv_temp * 1.4426950408889634f : 0.f;
+        p.part_ref = reinterpret_cast<float*>(static_cast<char*>(ws) + tail_workspace_bytes(M, V));
+        p.part_sum = p.part_ref + (size_t)kMaxCtas * kMaxCols;
 
         CUtensorMap tmW, tmH;
         if (!encode_tmap_bf16_2d(&tmW, W, (uint64_t)V, (uint64_t)Hd, (uint64_t)Hd * 2, (uint32_t)bk, kBM, bk * 2))
@@ -548,11 +686,21 @@ static sd_status launch_lmhead_impl(const void* hidden, const void* W, int M, in
             *tiles_only_ctas = grid;
             return SD_OK;
         }
-        lmhead_merge_kernel<<<(p.rows + 127) / 128, 128, 0, st>>>(p.part_key, p.part_idx, grid, p.rows, p.row0,
-                                                                 argmax, maxlogit);
+        if (lse)
+            lmhead_merge_stats_kernel<<<(p.rows + 127) / 128, 128, 0, st>>>(p.part_key, p.part_idx, p.part_ref, p.part_sum,
+                                                                           grid, p.rows, p.row0, p.c2, argmax, maxlogit, lse);
+        else
+            lmhead_merge_kernel<<<(p.rows + 127) / 128, 128, 0, st>>>(p.part_key, p.part_idx, grid, p.rows, p.row0,
+                                                                     argmax, maxlogit);
         if (cudaGetLastError() != cudaSuccess) return SD_ERR_CUDA;
     }
     return SD_OK;
+}
+
+sd_status launch_lmhead_stats(const void* hidden, const void* W, int M, int Hd, int V, float inv_temp,
+                              int32_t* argmax, float* maxlogit, float* lse, void* ws, size_t ws_bytes,
+                              int32_t* dev_status, cudaStream_t st) {
+    return launch_lmhead_impl(hidden, W, M, Hd, V, argmax, maxlogit, ws, ws_bytes, dev_status, st, nullptr, inv_temp, lse);
 }
 
 sd_status launch_lmhead(const void* hidden, const void* W, int M, int Hd, int V,

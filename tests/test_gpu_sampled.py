@@ -1,0 +1,171 @@
+"""GPU parity of verification at a sampling temperature: sd_lmhead_stats and sd_accept_tree_sampled
+against oracle/sampling.py on the same seeded inputs (uniform numbers are inputs on both sides)."""
+import numpy as np
+import pytest
+import torch
+
+import oracle
+from oracle import sampling as smp
+from paper_2509_18824_b200 import binding as sd
+from paper_2509_18824_b200 import workloads as wl
+from paper_2509_18824_b200.step import to_device
+
+pytestmark = pytest.mark.gpu
+
+CLOSE = 2e-5          # a comparison u * R < p (or a CDF crossing) nearer than this may fall either way in fp32
+
+
+def run_stats(hidden, W, inv_temp):
+    h, Wd = to_device(hidden), to_device(W)
+    M, V = hidden.shape[0], W.shape[0]
+    am = torch.full((M,), -5, dtype=torch.int32, device="cuda")
+    mx = torch.zeros(M, dtype=torch.float32, device="cuda")
+    lse = torch.zeros(M, dtype=torch.float32, device="cuda")
+    ws = torch.empty(sd.sd_workspace_bytes(None, M, V), dtype=torch.uint8, device="cuda")
+    st = sd.new_status()
+    sd.sd_lmhead_stats(h, Wd, inv_temp, am, mx, lse, ws, st)
+    torch.cuda.synchronize()
+    assert int(st.item()) == 0
+    return am.cpu().numpy(), mx.cpu().numpy(), lse.cpu().numpy()
+
+
+@pytest.mark.parametrize("M,Hd,V,inv_temp", [(5, 128, 1000, 1.0), (61, 192, 129, 0.5), (130, 64, 4099, 2.0),
+                                             (600, 128, 2500, 1.0)])
+def test_lmhead_stats_small_shapes(M, Hd, V, inv_temp):
+    g = np.random.default_rng(M + V)
+    h = wl.f32_to_bf16_bits((g.standard_normal((M, Hd)) * 2).astype(np.float32))
+    W = wl.f32_to_bf16_bits((g.standard_normal((V, Hd)) / np.sqrt(Hd)).astype(np.float32))
+    am, mx, lse = run_stats(h, W, inv_temp)
+    lg = oracle.logits(h, W)
+    _, rlse = smp.softmax_rows(lg, inv_temp)
+    np.testing.assert_allclose(lse, rlse, rtol=0, atol=3e-4)
+    ram, t1, t2 = oracle.lmhead(h, W)
+    ok = (t1 - t2) > 1e-3
+    np.testing.assert_array_equal(am[ok], ram[ok])
+
+
+def test_lmhead_stats_full_vocabulary():
+    for gain, inv_temp in ((1.0, 1.0), (30.0, 1.0), (30.0, 0.25)):
+        w = wl.make("c2", attention=False, hidden_gain=gain)
+        am, mx, lse = run_stats(w.hidden, w.W, inv_temp)
+        lg = oracle.logits(w.hidden, w.W)
+        _, rlse = smp.softmax_rows(lg, inv_temp)
+        np.testing.assert_allclose(lse, rlse, rtol=0, atol=5e-4)
+
+
+def good_drafts(w, lg, seed):
+    """Children of every node get the target's most likely tokens at that node (a good drafter),
+    in shuffled order, so that some are accepted; siblings are distinct by construction."""
+    g = np.random.default_rng(seed)
+    tok = np.zeros((w.B, w.T_max), dtype=np.int32)
+    for b in range(w.B):
+        n = int(w.n_nodes[b])
+        for i in range(n):
+            kids = smp.children_of(w.parents[b], n, i)
+            if kids:
+                top = np.argsort(-lg[b * w.T_max + i])[:len(kids)]
+                tok[b, kids] = g.permutation(top)
+    return tok
+
+
+def run_sampled(w, tok, inv_temp, u, wv):
+    bt = sd.Batch.of(w)
+    st = sd.new_status()
+    h, Wd = to_device(w.hidden), to_device(w.W)
+    M, V = w.hidden.shape[0], w.W.shape[0]
+    B, T = w.B, w.T_max
+    ws = torch.zeros(sd.sd_workspace_bytes(bt, M, V), dtype=torch.uint8, device="cuda")
+    lse = torch.zeros(M, dtype=torch.float32, device="cuda")
+    sd.sd_lmhead_stats(h, Wd, inv_temp, None, None, lse, ws, st)
+    n_acc = torch.full((B,), -9, dtype=torch.int32, device="cuda")
+    path = torch.full((B, T), -9, dtype=torch.int32, device="cuda")
+    out_tok = torch.full((B, T), -9, dtype=torch.int32, device="cuda")
+    new_len = torch.full((B,), -9, dtype=torch.int32, device="cuda")
+    sd.sd_accept_tree_sampled(bt, h, Wd, inv_temp, lse, to_device(tok), to_device(u), to_device(wv),
+                              n_acc, path, out_tok, new_len, ws, st)
+    torch.cuda.synchronize()
+    p_child = ws[:B * T * 4].view(torch.float32).cpu().numpy().reshape(B, T)      # first area of the workspace
+    return (n_acc.cpu().numpy(), path.cpu().numpy(), out_tok.cpu().numpy(), new_len.cpu().numpy(),
+            p_child, int(st.item()))
+
+
+@pytest.mark.parametrize("cfg,over,inv_temp", [
+    ("c1", dict(), 1.0), ("c1", dict(), 3.0),
+    ("c5", dict(L=1, V=8192, Hd=512, prefix=100), 5.0),
+    ("c4", dict(L=1, V=4096, Hd=256, prefix_range=(40, 300)), 3.0),          # 16 sequences: two residual passes
+    ("chain11", dict(L=1, V=3000, Hd=128, prefix=70), 2.5),
+])
+def test_sampled_acceptance_against_the_reference(cfg, over, inv_temp):
+    w = wl.make(cfg, attention=False, hidden_gain=24.0, **over)
+    B, T, V = w.B, w.T_max, w.W.shape[0]
+    lg = oracle.logits(w.hidden, w.W)
+    tok = good_drafts(w, lg, 1)
+    g = np.random.default_rng(7)
+    p64, _ = smp.softmax_rows(lg, inv_temp)
+    accepted_total = 0
+    for rep in range(3 if B > 1 else 25):
+        u = g.random((B, T)).astype(np.float32)
+        wv = g.random(B).astype(np.float32)
+        n_acc, path, out_tok, new_len, p_child, status = run_sampled(w, tok, inv_temp, u, wv)
+        assert status == 0
+        close_calls = 0
+        for b in range(B):
+            n = int(w.n_nodes[b])
+            par = w.parents[b]
+            # (1) the probabilities the kernel compared against
+            for j in range(1, n):
+                ref = p64[b * T + par[j], tok[b, j]]
+                assert abs(p_child[b, j] - ref) <= 1e-4 * ref + 1e-7, (b, j, p_child[b, j], ref)
+            # (2) the walk, bit for bit, in the kernel's arithmetic on the kernel's probabilities
+            pth32, R32 = smp.accept_walk(par, n, tok[b], p_child[b], u[b], dtype=np.float32)
+            assert list(path[b, :n_acc[b]]) == pth32 and (path[b, n_acc[b]:] == -1).all()
+            assert new_len[b] == w.len[b] + n_acc[b]
+            assert list(out_tok[b, :n_acc[b] - 1]) == [int(tok[b, j]) for j in pth32[1:]]
+            # (3) against the fp64 definition: same path unless some comparison was a close call
+            pc64 = np.zeros(T)
+            for j in range(1, n):
+                pc64[j] = p64[b * T + par[j], tok[b, j]]
+            pth64, R64 = smp.accept_walk(par, n, tok[b], pc64, u[b].astype(np.float64))
+            if pth64 != pth32:
+                close_calls += 1
+                continue
+            # (4) the drawn token: inverse CDF over the stop row without its drafted children
+            last = pth64[-1]
+            excl = [int(tok[b, c]) for c in smp.children_of(par, n, last)]
+            t_ref, margin = smp.residual_sample(p64[b * T + last], excl, R64, float(wv[b]))
+            got = int(out_tok[b, n_acc[b] - 1])
+            assert got not in excl and 0 <= got < V
+            if got != t_ref:
+                assert margin <= CLOSE * max(R64, 1e-3), (b, got, t_ref, margin)
+                close_calls += 1
+            accepted_total += n_acc[b] - 1
+        assert close_calls <= max(1, B // 8), close_calls
+    assert accepted_total > 0          # the drafts were good enough for the walk to move at all
+
+
+def test_sampled_zero_temperature_equals_greedy_acceptance():
+    """Large inverse temperature: the sampled rule must reproduce sd_accept_tree's outputs exactly
+    (path, accepted drafts, and the bonus token = arg-max at the last accepted node)."""
+    w = wl.make("c5", attention=False, hidden_gain=40.0, L=1, V=8192, Hd=512, prefix=100)
+    ram, t1, t2 = oracle.lmhead(w.hidden, w.W)
+    assert (t1 - t2).min() > 2e-3
+    wl.plant(w, ram.reshape(w.B, w.T_max))
+    ref = oracle.accept(oracle.Geometry.of(w), w.draft_tok, ram.reshape(w.B, w.T_max))
+    g = np.random.default_rng(3)
+    u = (g.random((w.B, w.T_max)) * 0.98 + 0.01).astype(np.float32)
+    wv = (g.random(w.B) * 0.98 + 0.01).astype(np.float32)
+    n_acc, path, out_tok, new_len, _, status = run_sampled(w, w.draft_tok, 4000.0, u, wv)
+    assert status == 0
+    for got, want in zip((n_acc, path, out_tok, new_len), ref):
+        np.testing.assert_array_equal(got, want)
+
+
+def test_sampled_bad_inputs_are_reported():
+    w = wl.make("c1", attention=False, hidden_gain=16.0)
+    tok = np.zeros((1, 8), dtype=np.int32); tok[0, 3] = 5000                 # outside the vocabulary
+    u = np.full((1, 8), 0.5, np.float32); wv = np.full(1, 0.5, np.float32)
+    *_, status = run_sampled(w, tok, 1.0, u, wv)
+    assert status == sd.SD_ERR_BOUNDS
+    w.parents = w.parents.copy(); w.parents[0, 3] = 6
+    *_, status = run_sampled(w, np.arange(8, dtype=np.int32)[None], 1.0, u, wv)
+    assert status == sd.SD_ERR_INVALID_TREE
