@@ -47,7 +47,7 @@ size_t sd_workspace_bytes(const sd_batch* geom, int32_t M, int32_t V) {
     if (geom && check_geometry(geom, false) == SD_OK) a = attention_workspace_bytes(*geom);
     if (M > 0 && V > 0) l = stats_workspace_bytes(M, V);    // covers sd_lmhead_argmax, the fused tail and sd_lmhead_stats
     if (geom && V > 0 && check_geometry(geom, false) == SD_OK) {
-        const size_t sw = sampled_workspace_bytes(geom->B, geom->T_max, V);   // sd_accept_tree_sampled
+        const size_t sw = sampled_workspace_bytes(geom->B, geom->T_max, V, 16384);   // sd_accept_tree_sampled (Hd <= 16384)
         if (sw > l) l = sw;
     }
     size_t n = a > l ? a : l;

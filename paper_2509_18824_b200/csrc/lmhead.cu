@@ -42,6 +42,11 @@ struct LmParams {
     float c2;
     float* part_ref;   // [gridDim.x][kMaxCols] reference logit of the partial sum
     float* part_sum;   // [gridDim.x][kMaxCols] sum over the CTA's vocabulary rows of 2^((logit - ref) * c2)
+    // probability output (residual draw of the sampled acceptance): when mass_out is set, the epilogue
+    // stores exp(logit * inv_temp - col_lse[row]) for every (row, vocabulary entry) instead of reducing
+    float* mass_out;        // [rows of the call][V]
+    const float* col_lse;   // [rows of the call]
+    float inv_temp;
 };
 
 size_t lmhead_workspace_bytes(int M, int V) {
@@ -298,6 +303,18 @@ lmhead_umma_kernel(const __grid_constant__ CUtensorMap tmW, const __grid_constan
                     tmem_ld_wait();
                     float cv;
                     int32_t ci;
+                    if (p.mass_out) {
+                        if (v_ok) {
+#pragma unroll
+                            for (int j = 0; j < 32; ++j) {
+                                const int row = c * 32 + j;
+                                if (row < p.rows)
+                                    p.mass_out[(size_t)(p.row0 + row) * p.V + v_base + lane] =
+                                        __expf(__uint_as_float(r[j]) * p.inv_temp - __ldg(p.col_lse + p.row0 + row));
+                            }
+                        }
+                        continue;
+                    }
                     if (stats) {
                         float cs;
                         column_argmax_stats32(r, v_ok, v_base, lane, p.c2, cv, ci, cs);
@@ -502,6 +519,18 @@ lmhead_umma_pair_kernel(const __grid_constant__ CUtensorMap tmW, const __grid_co
                     tmem_ld_wait();
                     float cv;
                     int32_t ci;
+                    if (p.mass_out) {
+                        if (v_ok) {
+#pragma unroll
+                            for (int j = 0; j < 32; ++j) {
+                                const int row = c * 32 + j;
+                                if (row < p.rows)
+                                    p.mass_out[(size_t)(p.row0 + row) * p.V + v_base + lane] =
+                                        __expf(__uint_as_float(r[j]) * p.inv_temp - __ldg(p.col_lse + p.row0 + row));
+                            }
+                        }
+                        continue;
+                    }
                     if (stats) {
                         float cs;
                         column_argmax_stats32(r, v_ok, v_base, lane, p.c2, cv, ci, cs);
@@ -574,22 +603,38 @@ __global__ void lmhead_merge_kernel(const int32_t* __restrict__ part_key, const 
     if (maxlogit) maxlogit[row0 + col] = key_to_float(k);
 }
 
-// the same merge plus log sum exp(logit / temperature) of every hidden row (natural log)
-__global__ void lmhead_merge_stats_kernel(const int32_t* __restrict__ part_key, const int32_t* __restrict__ part_idx,
-                                          const float* __restrict__ part_ref, const float* __restrict__ part_sum,
-                                          int n_ctas, int rows, int row0, float c2, int32_t* __restrict__ argmax,
-                                          float* __restrict__ maxlogit, float* __restrict__ lse) {
-    const int col = blockIdx.x * blockDim.x + threadIdx.x;
-    if (col >= rows) return;
+// the same merge plus log sum exp(logit / temperature) of every hidden row (natural log);
+// eight threads per row share the CTAs' partials and combine through shuffles (fixed order)
+__global__ void __launch_bounds__(256)
+lmhead_merge_stats_kernel(const int32_t* __restrict__ part_key, const int32_t* __restrict__ part_idx,
+                          const float* __restrict__ part_ref, const float* __restrict__ part_sum,
+                          int n_ctas, int rows, int row0, float c2, int32_t* __restrict__ argmax,
+                          float* __restrict__ maxlogit, float* __restrict__ lse) {
+    const int col = blockIdx.x * 32 + (threadIdx.x >> 3), sub = threadIdx.x & 7;
     int32_t k = INT32_MIN, i = 0x7fffffff;
     float rf = -INFINITY, sm = 0.f;
-    for (int c = 0; c < n_ctas; ++c) {
-        take_better(k, i, part_key[(size_t)c * kMaxCols + col], part_idx[(size_t)c * kMaxCols + col]);
-        merge_sumexp(rf, sm, part_ref[(size_t)c * kMaxCols + col], part_sum[(size_t)c * kMaxCols + col], c2);
+    if (col < rows) {
+        for (int c = sub; c < n_ctas; c += 8) {
+            take_better(k, i, __ldg(part_key + (size_t)c * kMaxCols + col), __ldg(part_idx + (size_t)c * kMaxCols + col));
+            merge_sumexp(rf, sm, __ldg(part_ref + (size_t)c * kMaxCols + col), __ldg(part_sum + (size_t)c * kMaxCols + col), c2);
+        }
     }
-    if (argmax) argmax[row0 + col] = i;
-    if (maxlogit) maxlogit[row0 + col] = key_to_float(k);
-    lse[row0 + col] = (rf * c2 + log2f(sm)) * 0.6931471805599453f;
+#pragma unroll
+    for (int d = 1; d <= 4; d <<= 1) {
+        const int32_t k2 = __shfl_xor_sync(0xffffffffu, k, d), i2 = __shfl_xor_sync(0xffffffffu, i, d);
+        const float rf2 = __shfl_xor_sync(0xffffffffu, rf, d), sm2 = __shfl_xor_sync(0xffffffffu, sm, d);
+        take_better(k, i, k2, i2);
+        // both partners must end with the same bits: combine in the order (lower lane, higher lane)
+        float ra = (threadIdx.x & d) ? rf2 : rf, sa = (threadIdx.x & d) ? sm2 : sm;
+        const float rb = (threadIdx.x & d) ? rf : rf2, sb = (threadIdx.x & d) ? sm : sm2;
+        merge_sumexp(ra, sa, rb, sb, c2);
+        rf = ra; sm = sa;
+    }
+    if (col < rows && sub == 0) {
+        if (argmax) argmax[row0 + col] = i;
+        if (maxlogit) maxlogit[row0 + col] = key_to_float(k);
+        lse[row0 + col] = (rf * c2 + log2f(sm)) * 0.6931471805599453f;
+    }
 }
 
 static int round_up(int x, int m) { return (x + m - 1) / m * m; }
@@ -599,7 +644,8 @@ static int round_up(int x, int m) { return (x + m - 1) / m * m; }
 static sd_status launch_lmhead_impl(const void* hidden, const void* W, int M, int Hd, int V,
                                     int32_t* argmax, float* maxlogit, void* ws, size_t ws_bytes,
                                     int32_t* dev_status, cudaStream_t st, int* tiles_only_ctas,
-                                    float inv_temp = 0.f, float* lse = nullptr) {
+                                    float inv_temp = 0.f, float* lse = nullptr,
+                                    float* mass_out = nullptr, const float* col_lse = nullptr) {
     if (ws_bytes < (lse ? stats_workspace_bytes(M, V) : lmhead_workspace_bytes(M, V))) return SD_ERR_WORKSPACE;
     if (tiles_only_ctas && M > kMaxCols) return SD_ERR_UNSUPPORTED;
     int dev = 0, sms = 0;
@@ -645,6 +691,7 @@ static sd_status launch_lmhead_impl(const void* hidden, const void* W, int M, in
         p.c2 = lse ? inv_temp * 1.4426950408889634f : 0.f;
         p.part_ref = reinterpret_cast<float*>(static_cast<char*>(ws) + tail_workspace_bytes(M, V));
         p.part_sum = p.part_ref + (size_t)kMaxCtas * kMaxCols;
+        p.mass_out = mass_out; p.col_lse = col_lse; p.inv_temp = inv_temp;
 
         CUtensorMap tmW, tmH;
         if (!encode_tmap_bf16_2d(&tmW, W, (uint64_t)V, (uint64_t)Hd, (uint64_t)Hd * 2, (uint32_t)bk, kBM, bk * 2))
@@ -686,8 +733,9 @@ static sd_status launch_lmhead_impl(const void* hidden, const void* W, int M, in
             *tiles_only_ctas = grid;
             return SD_OK;
         }
+        if (mass_out) continue;                      // nothing to merge: the epilogue stored the probabilities
         if (lse)
-            lmhead_merge_stats_kernel<<<(p.rows + 127) / 128, 128, 0, st>>>(p.part_key, p.part_idx, p.part_ref, p.part_sum,
+            lmhead_merge_stats_kernel<<<(p.rows + 31) / 32, 256, 0, st>>>(p.part_key, p.part_idx, p.part_ref, p.part_sum,
                                                                            grid, p.rows, p.row0, p.c2, argmax, maxlogit, lse);
         else
             lmhead_merge_kernel<<<(p.rows + 127) / 128, 128, 0, st>>>(p.part_key, p.part_idx, grid, p.rows, p.row0,
@@ -695,6 +743,14 @@ static sd_status launch_lmhead_impl(const void* hidden, const void* W, int M, in
         if (cudaGetLastError() != cudaSuccess) return SD_ERR_CUDA;
     }
     return SD_OK;
+}
+
+// probabilities of M rows over the whole vocabulary: mass[r][v] = exp(logit[r][v] * inv_temp - row_lse[r])
+sd_status launch_lmhead_mass(const void* hidden, const void* W, int M, int Hd, int V, float inv_temp,
+                             const float* row_lse, float* mass, void* ws, size_t ws_bytes,
+                             int32_t* dev_status, cudaStream_t st) {
+    return launch_lmhead_impl(hidden, W, M, Hd, V, nullptr, nullptr, ws, ws_bytes, dev_status, st, nullptr, inv_temp,
+                              nullptr, mass, row_lse);
 }
 
 sd_status launch_lmhead_stats(const void* hidden, const void* W, int M, int Hd, int V, float inv_temp,

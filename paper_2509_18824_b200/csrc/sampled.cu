@@ -4,15 +4,15 @@
 //
 //   child_prob_kernel      p[b][j] = exp(logit(parent(j), token(j)) / temperature - lse(parent(j)))
 //   sampled_walk_kernel    the walk: accepted path, residual mass, the stop node's drafted tokens
-//   residual_mass_kernel   exp(logit / temperature - lse) of the stop node's row over the whole
-//                          vocabulary (drafted tokens zeroed), per 256-token block sums
+//   gather_stop_rows_kernel + the LM-head tcgen05 kernel in its store mode
+//                          exp(logit / temperature - lse) of the stop node's row over the whole vocabulary
+//   residual_blocksum_kernel  drafted tokens of the stop node zeroed, sums per 256-token block
 //   residual_pick_kernel   inverse CDF in vocabulary order; writes the final token
 #include "tree_device.cuh"
 
 namespace sdv {
 
 constexpr int kResBlock = 256;         // vocabulary tokens per CTA of residual_mass_kernel
-constexpr int kResMaxB = 8;            // sequences handled per launch (their hidden rows live in shared memory)
 
 struct SampledWs {                     // carved out of the caller's workspace
     float* p_child;                    // [B][T]
@@ -22,17 +22,22 @@ struct SampledWs {                     // carved out of the caller's workspace
     int32_t* excl;                     // [B][64] drafted tokens of the stop node's children
     float* block_sum;                  // [B][n_blocks]
     float* mass;                       // [B][V]
+    uint16_t* stop_hidden;             // [B rounded up to 16][Hd] hidden rows of the stop nodes
+    float* stop_lse;                   // [B]
+    void* lm_ws;                       // candidate tables of the LM-head launch
 };
 
 static size_t align256(size_t x) { return (x + 255) & ~(size_t)255; }
 
-size_t sampled_workspace_bytes(int B, int T, int V) {
+size_t sampled_workspace_bytes(int B, int T, int V, int Hd) {
     const size_t nb = (size_t)(V + kResBlock - 1) / kResBlock;
+    const size_t b16 = (size_t)(B + 15) / 16 * 16;
     return align256((size_t)B * T * 4) + align256((size_t)B * 4) * 3 + align256((size_t)B * 64 * 4) +
-           align256((size_t)B * nb * 4) + align256((size_t)B * V * 4);
+           align256((size_t)B * nb * 4) + align256((size_t)B * V * 4) + align256(b16 * Hd * 2) + align256((size_t)B * 4) +
+           align256(stats_workspace_bytes(B, V));
 }
 
-static SampledWs carve(void* ws, int B, int T, int V) {
+static SampledWs carve(void* ws, int B, int T, int V, int Hd) {
     const size_t nb = (size_t)(V + kResBlock - 1) / kResBlock;
     char* p = static_cast<char*>(ws);
     SampledWs w;
@@ -42,7 +47,10 @@ static SampledWs carve(void* ws, int B, int T, int V) {
     w.n_excl = reinterpret_cast<int32_t*>(p);  p += align256((size_t)B * 4);
     w.excl = reinterpret_cast<int32_t*>(p);    p += align256((size_t)B * 64 * 4);
     w.block_sum = reinterpret_cast<float*>(p); p += align256((size_t)B * nb * 4);
-    w.mass = reinterpret_cast<float*>(p);
+    w.mass = reinterpret_cast<float*>(p);      p += align256((size_t)B * V * 4);
+    w.stop_hidden = reinterpret_cast<uint16_t*>(p); p += align256((size_t)(B + 15) / 16 * 16 * Hd * 2);
+    w.stop_lse = reinterpret_cast<float*>(p);  p += align256((size_t)B * 4);
+    w.lm_ws = p;
     return w;
 }
 
@@ -149,113 +157,100 @@ __global__ void sampled_walk_kernel(sd_batch bt, const int32_t* __restrict__ dra
     }
 }
 
-// CTA = 256 consecutive vocabulary tokens, 8 warps x 32 tokens.  The stop rows of up to 8 sequences
-// sit in shared memory as fp32, so every W row is read (and widened) once for all of them.  Shared
-// layout of a row: the first four floats of every 8-element piece, then the second four, so that
-// the lanes of a warp read consecutive 16-byte words.
-__global__ void __launch_bounds__(256)
-residual_mass_kernel(const uint16_t* __restrict__ hidden, const uint16_t* __restrict__ W, int Hd, int V, int b0, int nb,
-                     float inv_temp, const float* __restrict__ lse, const int32_t* __restrict__ stop_row,
-                     const int32_t* __restrict__ n_excl, const int32_t* __restrict__ excl,
-                     float* __restrict__ mass, float* __restrict__ block_sum, int n_blocks) {
-    extern __shared__ __align__(16) uint8_t rsm[];
-    const int n_vec = Hd / 8;
-    float4* rows = reinterpret_cast<float4*>(rsm);                          // [nb][2][n_vec]
-    float* vals = reinterpret_cast<float*>(rsm + (size_t)nb * Hd * 4);      // [nb][256]
-    const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
-    for (int i = threadIdx.x; i < nb * n_vec; i += blockDim.x) {
-        const int b = i / n_vec, k = i - b * n_vec;
-        const uint4 x = __ldg(reinterpret_cast<const uint4*>(hidden + (size_t)stop_row[b0 + b] * Hd) + k);
-        rows[(size_t)(b * 2) * n_vec + k] = make_float4(bf16lo(x.x), bf16hi(x.x), bf16lo(x.y), bf16hi(x.y));
-        rows[(size_t)(b * 2 + 1) * n_vec + k] = make_float4(bf16lo(x.z), bf16hi(x.z), bf16lo(x.w), bf16hi(x.w));
-    }
-    __syncthreads();
-    for (int k = 0; k < 32; ++k) {
-        const int t_in = warp * 32 + k;
-        const int t = blockIdx.x * kResBlock + t_in;
-        float acc[kResMaxB];
-#pragma unroll
-        for (int b = 0; b < kResMaxB; ++b) acc[b] = 0.f;
-        if (t < V) {
-            const uint4* wrow = reinterpret_cast<const uint4*>(W + (size_t)t * Hd);
-            for (int i = lane; i < n_vec; i += 32) {
-                const uint4 x = __ldg(wrow + i);
-                const float w0 = bf16lo(x.x), w1 = bf16hi(x.x), w2 = bf16lo(x.y), w3 = bf16hi(x.y);
-                const float w4 = bf16lo(x.z), w5 = bf16hi(x.z), w6 = bf16lo(x.w), w7 = bf16hi(x.w);
-#pragma unroll
-                for (int b = 0; b < kResMaxB; ++b) {
-                    if (b < nb) {
-                        const float4 y0 = rows[(size_t)(b * 2) * n_vec + i], y1 = rows[(size_t)(b * 2 + 1) * n_vec + i];
-                        float a = acc[b];
-                        a = fmaf(w0, y0.x, a); a = fmaf(w1, y0.y, a); a = fmaf(w2, y0.z, a); a = fmaf(w3, y0.w, a);
-                        a = fmaf(w4, y1.x, a); a = fmaf(w5, y1.y, a); a = fmaf(w6, y1.z, a); a = fmaf(w7, y1.w, a);
-                        acc[b] = a;
-                    }
-                }
-            }
-        }
-#pragma unroll
-        for (int b = 0; b < kResMaxB; ++b) {
-            if (b < nb) {
-                float l = acc[b];
-#pragma unroll
-                for (int d = 16; d >= 1; d >>= 1) l += __shfl_xor_sync(0xffffffffu, l, d);
-                float m = 0.f;
-                if (t < V) {
-                    const int ne = n_excl[b0 + b];                     // drafted tokens of the stop node carry no mass
-                    bool hit = false;
-                    for (int e = lane; e < ne; e += 32) hit |= (excl[(size_t)(b0 + b) * 64 + e] == t);
-                    m = __any_sync(0xffffffffu, hit) ? 0.f : __expf(l * inv_temp - lse[stop_row[b0 + b]]);
-                }
-                if (lane == 0) {
-                    vals[b * kResBlock + t_in] = m;
-                    if (t < V) mass[(size_t)(b0 + b) * V + t] = m;
-                }
-            }
-        }
-    }
-    __syncthreads();
-    if (threadIdx.x < nb) {                                            // block sums in vocabulary order
-        float s = 0.f;
-        for (int i = 0; i < kResBlock; ++i) s += vals[threadIdx.x * kResBlock + i];
-        block_sum[(size_t)(b0 + threadIdx.x) * n_blocks + blockIdx.x] = s;
-    }
+// hidden rows (and their lse) of the stop nodes, gathered into a dense [B][Hd] matrix for the LM-head kernel
+__global__ void gather_stop_rows_kernel(const uint16_t* __restrict__ hidden, int Hd, const float* __restrict__ lse,
+                                        const int32_t* __restrict__ stop_row, uint16_t* __restrict__ stop_hidden,
+                                        float* __restrict__ stop_lse) {
+    const int b = blockIdx.x;
+    const int row = stop_row[b];
+    const uint4* src = reinterpret_cast<const uint4*>(hidden + (size_t)row * Hd);
+    uint4* dst = reinterpret_cast<uint4*>(stop_hidden + (size_t)b * Hd);
+    for (int i = threadIdx.x; i < Hd / 8; i += blockDim.x) dst[i] = __ldg(src + i);
+    if (threadIdx.x == 0) stop_lse[b] = lse[row];
 }
 
-// one thread per sequence walks the block sums, then the block's tokens, in vocabulary order
-__global__ void residual_pick_kernel(sd_batch bt, int V, const float* __restrict__ w, const float* __restrict__ mass,
-                                     const float* __restrict__ block_sum, int n_blocks, const int32_t* __restrict__ n_acc,
-                                     int32_t* out_tok, int32_t* status) {
-    const int b = blockIdx.x * blockDim.x + threadIdx.x;
-    if (b >= bt.B) return;
+// grid (blocks of 256 tokens, sequences): drafted tokens of the stop node lose their mass, then the
+// block's masses are summed in a fixed order (pairwise tree over the 256 positions)
+__global__ void __launch_bounds__(kResBlock)
+residual_blocksum_kernel(int V, const int32_t* __restrict__ n_excl, const int32_t* __restrict__ excl,
+                         float* __restrict__ mass, float* __restrict__ block_sum, int n_blocks) {
+    __shared__ float s_v[kResBlock];
+    const int b = blockIdx.y;
+    const int t = blockIdx.x * kResBlock + threadIdx.x;
+    float m = 0.f;
+    if (t < V) {
+        m = mass[(size_t)b * V + t];
+        const int ne = n_excl[b];
+        bool hit = false;
+        for (int e = 0; e < ne; ++e) hit |= (__ldg(excl + (size_t)b * 64 + e) == t);
+        if (hit) { m = 0.f; mass[(size_t)b * V + t] = 0.f; }
+    }
+    s_v[threadIdx.x] = m;
+    __syncthreads();
+    for (int d = kResBlock / 2; d >= 1; d >>= 1) {
+        if (threadIdx.x < d) s_v[threadIdx.x] += s_v[threadIdx.x + d];
+        __syncthreads();
+    }
+    if (threadIdx.x == 0) block_sum[(size_t)b * n_blocks + blockIdx.x] = s_v[0];
+}
+
+// One CTA per sequence.  The block sums, then the chosen block's masses, are brought into shared
+// memory by all threads; one thread walks them in vocabulary order (a fixed order of additions).
+constexpr int kPickMaxBlocks = 4096;   // vocabularies up to 1 Mi tokens
+__global__ void __launch_bounds__(kResBlock)
+residual_pick_kernel(sd_batch bt, int V, const float* __restrict__ w, const float* __restrict__ mass,
+                     const float* __restrict__ block_sum, int n_blocks, const int32_t* __restrict__ n_acc,
+                     int32_t* out_tok, int32_t* status) {
+    __shared__ float s_bs[kPickMaxBlocks];
+    __shared__ float s_m[kResBlock];
+    __shared__ float s_acc, s_target;
+    __shared__ int s_k, s_pick;
+    const int b = blockIdx.x;
     const int na = n_acc[b];
     if (na < 1 || na > bt.T_max) return;                               // bad tree: already reported
     const float* bs = block_sum + (size_t)b * n_blocks;
-    float total = 0.f;
-    for (int k = 0; k < n_blocks; ++k) total += bs[k];
-    const float target = w[b] * total;
-    float acc = 0.f;
-    int k = 0;
-    for (; k < n_blocks - 1; ++k) {
-        if (acc + bs[k] >= target) break;
-        acc += bs[k];
-    }
-    const float* m = mass + (size_t)b * V;
-    int pick = -1, last = -1;
-    // (if rounding leaves the sums short, fall through the following blocks to the last token with mass)
-    for (; k < n_blocks && pick < 0; ++k) {
-        const int t1 = min(V, (k + 1) * kResBlock);
-        for (int t = k * kResBlock; t < t1; ++t) {
-            const float mt = m[t];
-            if (mt <= 0.f) continue;
-            last = t;
-            if (acc + mt >= target) { pick = t; break; }
-            acc += mt;
+    for (int k = threadIdx.x; k < n_blocks; k += blockDim.x) s_bs[k] = bs[k];
+    __syncthreads();
+    if (threadIdx.x == 0) {
+        float total = 0.f;
+        for (int k = 0; k < n_blocks; ++k) total += s_bs[k];
+        const float target = w[b] * total;
+        float acc = 0.f;
+        int k = 0;
+        for (; k < n_blocks - 1; ++k) {
+            if (acc + s_bs[k] >= target) break;
+            acc += s_bs[k];
         }
+        s_acc = acc; s_target = target; s_k = k; s_pick = -1;
     }
-    if (pick < 0) pick = last;
-    if (pick < 0) { set_status(status, SD_ERR_BOUNDS); pick = 0; }      // no mass at all: inputs were not finite
-    out_tok[(size_t)b * bt.T_max + na - 1] = pick;
+    __syncthreads();
+    const float* m = mass + (size_t)b * V;
+    // (if rounding leaves the sums short, fall through the following blocks to the last token with mass)
+    int last = -1;
+    for (int k = s_k; k < n_blocks; ++k) {
+        const int t = k * kResBlock + threadIdx.x;
+        s_m[threadIdx.x] = t < V ? m[t] : 0.f;
+        __syncthreads();
+        if (threadIdx.x == 0) {
+            float acc = s_acc;
+            const float target = s_target;
+            for (int i = 0; i < kResBlock; ++i) {
+                const float mt = s_m[i];
+                if (mt <= 0.f) continue;
+                last = k * kResBlock + i;
+                if (acc + mt >= target) { s_pick = last; break; }
+                acc += mt;
+            }
+            s_acc = acc;
+        }
+        __syncthreads();
+        if (s_pick >= 0) break;
+    }
+    if (threadIdx.x == 0) {
+        int pick = s_pick >= 0 ? s_pick : last;
+        if (pick < 0) { set_status(status, SD_ERR_BOUNDS); pick = 0; }  // no mass at all: inputs were not finite
+        out_tok[(size_t)b * bt.T_max + na - 1] = pick;
+    }
 }
 
 sd_status launch_accept_sampled(const sd_batch& bt, const void* hidden, const void* W, int Hd, int V, float inv_temp,
@@ -263,24 +258,24 @@ sd_status launch_accept_sampled(const sd_batch& bt, const void* hidden, const vo
                                 int32_t* n_acc, int32_t* path, int32_t* out_tok, int32_t* new_len,
                                 void* ws, size_t ws_bytes, int32_t* dev_status, cudaStream_t st) {
     const int B = bt.B, T = bt.T_max;
-    if (ws_bytes < sampled_workspace_bytes(B, T, V)) return SD_ERR_WORKSPACE;
-    const SampledWs s = carve(ws, B, T, V);
+    if (Hd > 16384) return SD_ERR_UNSUPPORTED;
+    if (ws_bytes < sampled_workspace_bytes(B, T, V, 16384)) return SD_ERR_WORKSPACE;
+    const SampledWs s = carve(ws, B, T, V, 16384);
     const uint16_t* h = static_cast<const uint16_t*>(hidden);
     const uint16_t* Wp = static_cast<const uint16_t*>(W);
     const int n_blocks = (V + kResBlock - 1) / kResBlock;
     child_prob_kernel<<<(B * T * 32 + 127) / 128, 128, 0, st>>>(bt, h, Wp, Hd, V, inv_temp, lse, draft, s.p_child, dev_status);
     sampled_walk_kernel<<<B, 32, 0, st>>>(bt, draft, s.p_child, u, n_acc, path, out_tok, new_len, s.resid, s.stop_row,
                                          s.n_excl, s.excl, dev_status);
-    for (int b0 = 0; b0 < B; b0 += kResMaxB) {
-        const int nb = (B - b0 < kResMaxB) ? (B - b0) : kResMaxB;
-        const size_t smem = (size_t)nb * Hd * 4 + (size_t)nb * kResBlock * 4;
-        if (smem > 200 * 1024) return SD_ERR_UNSUPPORTED;
-        if (cudaFuncSetAttribute(residual_mass_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem) != cudaSuccess)
-            return SD_ERR_CUDA;
-        residual_mass_kernel<<<n_blocks, 256, smem, st>>>(h, Wp, Hd, V, b0, nb, inv_temp, lse, s.stop_row, s.n_excl, s.excl,
-                                                         s.mass, s.block_sum, n_blocks);
-    }
-    residual_pick_kernel<<<(B + 31) / 32, 32, 0, st>>>(bt, V, w, s.mass, s.block_sum, n_blocks, n_acc, out_tok, dev_status);
+    gather_stop_rows_kernel<<<B, 128, 0, st>>>(h, Hd, lse, s.stop_row, s.stop_hidden, s.stop_lse);
+    // probabilities of the stop rows over the vocabulary: one more pass of the tensor-core LM-head kernel,
+    // its epilogue storing instead of reducing (W is streamed once for all sequences)
+    sd_status ls = launch_lmhead_mass(s.stop_hidden, W, B, Hd, V, inv_temp, s.stop_lse, s.mass, s.lm_ws,
+                                      stats_workspace_bytes(B, V), dev_status, st);
+    if (ls != SD_OK) return ls;
+    residual_blocksum_kernel<<<dim3(n_blocks, B), kResBlock, 0, st>>>(V, s.n_excl, s.excl, s.mass, s.block_sum, n_blocks);
+    if (n_blocks > kPickMaxBlocks) return SD_ERR_UNSUPPORTED;
+    residual_pick_kernel<<<B, kResBlock, 0, st>>>(bt, V, w, s.mass, s.block_sum, n_blocks, n_acc, out_tok, dev_status);
     return cuda_ok(cudaGetLastError());
 }
 

@@ -2,7 +2,7 @@
 the LM head at several row counts, and the bandwidth-regime cases (chain
 decoding, a compaction stress shape).  One JSON line per measurement.
 
-    python -m paper_2509_18824_b200.supplements [attention] [attention_layers] [lmhead] [lmhead480] [compact]
+    python -m paper_2509_18824_b200.supplements [attention] [attention_layers] [lmhead] [lmhead480] [sampled] [compact]
 
 Timing: CUDA events on the launching stream, >= 3 warm-up calls, inputs rotated
 over several layers so that the working set exceeds L2.
@@ -124,6 +124,36 @@ def lmhead(rows=(60, 240, 480, 960), V=152064, Hd=3584):
                           "frac_hbm": nbytes / ms / 1e6 / hbm, "peaks": src, "status": int(st.item())}))
 
 
+def sampled(cfg="c5", inv_temp=1.0):
+    """The tail of a step at a sampling temperature (LM head with log-sum-exp, rejection walk, residual
+    draw) next to the greedy tail, on the bench's shapes."""
+    hbm, tens, src = _peaks()
+    from .step import VerifyStep
+    w = wl.make(cfg, attention=False, L=1)
+    wl.fill_attention(w, [0])
+    vs = VerifyStep(w)
+    B, T, M = w.B, w.T_max, w.B * w.T_max
+    g = torch.Generator(device="cuda"); g.manual_seed(0)
+    u = torch.rand((B, T), device="cuda", generator=g)
+    wv = torch.rand((B,), device="cuda", generator=g)
+    lse = torch.zeros(M, dtype=torch.float32, device="cuda")
+    ws = torch.empty(sd.sd_workspace_bytes(vs.batch, M, w.V), dtype=torch.uint8, device="cuda")
+    st = vs.status
+    flops = 2.0 * M * w.V * w.Hd
+    ms_greedy = _time(lambda: sd.sd_lmhead_argmax(vs.hidden, vs.W, vs.argmax, vs.maxlogit, ws, st), 10)
+    ms_stats = _time(lambda: sd.sd_lmhead_stats(vs.hidden, vs.W, inv_temp, vs.argmax, vs.maxlogit, lse, ws, st), 10)
+    ms_acc = _time(lambda: sd.sd_accept_tree_sampled(vs.batch, vs.hidden, vs.W, inv_temp, lse, vs.draft_tok, u, wv,
+                                                     vs.n_acc, vs.path, vs.out_tok, vs.new_len, ws, st), 10)
+    wbytes = w.V * w.Hd * 2
+    print(json.dumps({"call": "sampled tail", "workload": cfg, "rows": M,
+                      "sd_lmhead_argmax_us": ms_greedy * 1e3, "sd_lmhead_stats_us": ms_stats * 1e3,
+                      "stats_tflops": flops / ms_stats / 1e9, "stats_frac_tensor_burst": flops / ms_stats / 1e9 / tens,
+                      "sd_accept_tree_sampled_us": ms_acc * 1e3,
+                      "accept_weight_stream_gbs": wbytes * ((B + 7) // 8) / ms_acc / 1e6,
+                      "accept_frac_hbm": wbytes * ((B + 7) // 8) / ms_acc / 1e6 / hbm,
+                      "peaks": src, "status": int(st.item())}))
+
+
 def compact(B=1024, L=8, T=64, Hkv=4, D=128):
     """Stress shape for compaction: every node of every tree accepted (a 64-node chain), 1024
     sequences, 8 layers: 2 x 1.07 GB moved per call."""
@@ -154,7 +184,7 @@ def compact(B=1024, L=8, T=64, Hkv=4, D=128):
 
 
 if __name__ == "__main__":
-    what = sys.argv[1:] or ["attention", "attention_layers", "lmhead", "compact"]
+    what = sys.argv[1:] or ["attention", "attention_layers", "lmhead", "sampled", "compact"]
     if "attention" in what:
         attention()
     if "attention_layers" in what:
@@ -163,5 +193,7 @@ if __name__ == "__main__":
         lmhead()
     if "lmhead480" in what:                # the bench's LM-head launch alone (profiler captures)
         lmhead(rows=(480,))
+    if "sampled" in what:
+        sampled()
     if "compact" in what:
         compact()

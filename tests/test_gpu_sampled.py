@@ -169,3 +169,46 @@ def test_sampled_bad_inputs_are_reported():
     w.parents = w.parents.copy(); w.parents[0, 3] = 6
     *_, status = run_sampled(w, np.arange(8, dtype=np.int32)[None], 1.0, u, wv)
     assert status == sd.SD_ERR_INVALID_TREE
+
+
+def test_sampled_full_size_c5():
+    """Vocabulary 152064, 8 x 60-node trees: the walk bit for bit on the kernel's own probabilities,
+    those probabilities and the drawn tokens against fp64 logits of the rows the walks visited."""
+    w = wl.make("c5", attention=False, hidden_gain=40.0)
+    B, T, V = w.B, w.T_max, w.V
+    ram, t1, t2 = oracle.lmhead(w.hidden, w.W)                   # good drafts: children get the arg-max first
+    g = np.random.default_rng(11)
+    tok = g.integers(0, V, size=(B, T)).astype(np.int32)
+    for b in range(B):
+        for i in range(int(w.n_nodes[b])):
+            kids = smp.children_of(w.parents[b], int(w.n_nodes[b]), i)
+            if kids:
+                tok[b, kids[0]] = ram[b * T + i]
+                for k, c in enumerate(kids[1:]):
+                    tok[b, c] = (ram[b * T + i] + 1 + k) % V
+    inv_temp = 6.0
+    u = g.random((B, T)).astype(np.float32)
+    wv = g.random(B).astype(np.float32)
+    n_acc, path, out_tok, new_len, p_child, status = run_sampled(w, tok, inv_temp, u, wv)
+    assert status == 0
+    visited = sorted({b * T + int(path[b, k]) for b in range(B) for k in range(n_acc[b])})
+    lg = oracle.logits(w.hidden[visited], w.W)
+    p64, _ = smp.softmax_rows(lg, inv_temp)
+    row_of = {r: i for i, r in enumerate(visited)}
+    moved = 0
+    for b in range(B):
+        n, par = int(w.n_nodes[b]), w.parents[b]
+        pth32, R32 = smp.accept_walk(par, n, tok[b], p_child[b], u[b], dtype=np.float32)
+        assert list(path[b, :n_acc[b]]) == pth32
+        for i in pth32:                                           # children of visited nodes
+            for c in smp.children_of(par, n, i):
+                ref = p64[row_of[b * T + i], tok[b, c]]
+                assert abs(p_child[b, c] - ref) <= 2e-4 * ref + 1e-7
+        last = pth32[-1]
+        excl = [int(tok[b, c]) for c in smp.children_of(par, n, last)]
+        t_ref, margin = smp.residual_sample(p64[row_of[b * T + last]], excl, float(R32), float(wv[b]))
+        got = int(out_tok[b, n_acc[b] - 1])
+        assert got not in excl
+        assert got == t_ref or margin <= CLOSE, (b, got, t_ref, margin)
+        moved += n_acc[b] - 1
+    assert moved > 0
