@@ -314,6 +314,23 @@ sd_status sd_accept_tree_sampled(const sd_batch *batch, const void *hidden, cons
                                  void *workspace, size_t workspace_bytes,
                                  int32_t *dev_status, void *stream);
 
+/*
+ * Draft-side feature aggregation (Sec. 3.1.1, f_c^i = Flatten(CrossAttention(f_q, f_i, f_i))):
+ * Q meta queries, shared by all tokens, attend over the L target-layer features
+ * of every token.  This is the attention core for H heads of size 128
+ * (D = H * 128); the module's projections are ordinary GEMMs outside it:
+ *   for token i, head h:  p = softmax_l(scale * <qp[q, h], k[i, l, h]>),
+ *                         out[i, q, h] = sum_l p[q, l] * v[i, l, h]
+ *   qp  : dev bf16 [Q][D]      projected meta queries (the same for every token)
+ *   k,v : dev bf16 [S][L][D]   the tokens' (projected) layer features; may be the same buffer
+ *   out : dev bf16 [S][Q][D]   = [S][Q * D] flattened, as the paper uses it
+ * L <= 32, Q <= 8.  fp32 accumulation, bf16 output (round to nearest even).
+ * Every K and V row is read once; the call is bound by HBM bandwidth.
+ */
+sd_status sd_draft_feature_attention(const void *qp, const void *k, const void *v,
+                                     int32_t S, int32_t L, int32_t Q, int32_t H, int32_t D,
+                                     float scale, void *out, void *stream);
+
 #ifdef __cplusplus
 }
 #endif

@@ -32,7 +32,7 @@ KERNELS_PER_LMHEAD = 2         # tiles + cross-slab reduce
 
 EXPORTS = ["sd_version", "sd_status_string", "sd_workspace_bytes", "sd_tree_prepare",
            "sd_verify_attention", "sd_verify_attention_layers", "sd_lmhead_argmax", "sd_lmhead_argmax_static", "sd_accept_tree",
-           "sd_compact_kv", "sd_lmhead_accept_compact", "sd_lmhead_stats", "sd_accept_tree_sampled"]
+           "sd_compact_kv", "sd_lmhead_accept_compact", "sd_lmhead_stats", "sd_accept_tree_sampled", "sd_draft_feature_attention"]
 
 
 class sd_kv_layer(C.Structure):
@@ -90,6 +90,9 @@ def _load(path: str = LIB_PATH) -> C.CDLL:
                                            C.c_void_p, C.c_void_p, C.c_void_p, C.c_void_p,
                                            C.c_void_p, C.c_void_p, C.c_void_p, C.c_void_p,
                                            C.c_void_p, C.c_size_t, C.c_void_p, C.c_void_p]
+    lib.sd_draft_feature_attention.restype = C.c_int
+    lib.sd_draft_feature_attention.argtypes = [C.c_void_p, C.c_void_p, C.c_void_p, C.c_int32, C.c_int32, C.c_int32,
+                                               C.c_int32, C.c_int32, C.c_float, C.c_void_p, C.c_void_p]
     return lib
 
 
@@ -283,3 +286,11 @@ def sd_accept_tree_sampled(batch: Batch, hidden, W, inv_temp: float, lse, draft_
                                       _ptr(lse), _ptr(draft_tok), _ptr(u), _ptr(w), _ptr(n_acc), _ptr(path),
                                       _ptr(out_tok), _ptr(new_len), _ptr(workspace),
                                       workspace.numel() * workspace.element_size(), _ptr(status), _stream(stream)))
+
+
+def sd_draft_feature_attention(qp, k, v, H: int, scale: float, out, stream=None) -> None:
+    """Meta-query cross-attention core: qp [Q,D], k and v [S,L,D], out [S,Q,D]; D = H * 128."""
+    Q, D = qp.shape
+    S, L, _ = k.shape
+    _check(lib.sd_draft_feature_attention(_ptr(qp), _ptr(k), _ptr(v), int(S), int(L), int(Q), int(H), int(D),
+                                          C.c_float(scale), _ptr(out), _stream(stream)))

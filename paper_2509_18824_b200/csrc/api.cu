@@ -183,4 +183,12 @@ sd_status sd_accept_tree_sampled(const sd_batch* batch, const void* hidden, cons
                                  new_len, workspace, workspace_bytes, dev_status, static_cast<cudaStream_t>(stream));
 }
 
+sd_status sd_draft_feature_attention(const void* qp, const void* k, const void* v, int32_t S, int32_t L, int32_t Q,
+                                     int32_t H, int32_t D, float scale, void* out, void* stream) {
+    if (!ok_ptr(qp) || !ok_ptr(k) || !ok_ptr(v) || !ok_ptr(out)) return SD_ERR_INVALID_ARG;
+    if (S < 1 || L < 1 || Q < 1 || H < 1 || !(scale > 0.f)) return SD_ERR_INVALID_ARG;
+    if (D != H * 128 || L > 32 || Q > 8) return SD_ERR_UNSUPPORTED;
+    return launch_draft_feature_attention(qp, k, v, S, L, Q, H, scale, out, static_cast<cudaStream_t>(stream));
+}
+
 }  // extern "C"

@@ -55,6 +55,8 @@ sd_status launch_lmhead_accept_compact(const sd_batch& bt, const void* hidden, c
                                        int32_t* out_tok, int32_t* new_len, void* ws, size_t ws_bytes,
                                        int32_t* dev_status, cudaStream_t st);
 
+sd_status launch_draft_feature_attention(const void* qp, const void* k, const void* v, int S, int L, int Q, int H,
+                                         float scale, void* out, cudaStream_t st);
 size_t stats_workspace_bytes(int M, int V);
 sd_status launch_lmhead_stats(const void* hidden, const void* W, int M, int Hd, int V, float inv_temp,
                               int32_t* argmax, float* maxlogit, float* lse, void* ws, size_t ws_bytes,

@@ -2,7 +2,7 @@
 the LM head at several row counts, and the bandwidth-regime cases (chain
 decoding, a compaction stress shape).  One JSON line per measurement.
 
-    python -m paper_2509_18824_b200.supplements [attention] [attention_layers] [lmhead] [lmhead480] [sampled] [compact]
+    python -m paper_2509_18824_b200.supplements [attention] [attention_layers] [lmhead] [lmhead480] [sampled] [draft] [compact]
 
 Timing: CUDA events on the launching stream, >= 3 warm-up calls, inputs rotated
 over several layers so that the working set exceeds L2.
@@ -154,6 +154,23 @@ def sampled(cfg="c5", inv_temp=1.0):
                       "peaks": src, "status": int(st.item())}))
 
 
+def draft(S=4096, L=28, Q=4, H=28):
+    """Draft-side feature aggregation on a 7B-shaped prefill: S tokens x 28 layer features of width 3584."""
+    hbm, _, src = _peaks()
+    D = H * 128
+    g = torch.Generator(device="cuda"); g.manual_seed(0)
+    qp = torch.randn((Q, D), device="cuda", generator=g).to(torch.bfloat16)
+    k = torch.randn((S, L, D), device="cuda", generator=g).to(torch.bfloat16)
+    v = torch.randn((S, L, D), device="cuda", generator=g).to(torch.bfloat16)
+    out = torch.zeros((S, Q, D), dtype=torch.bfloat16, device="cuda")
+    for name, vv in (("separate K and V", v), ("K = V (un-projected features)", k)):
+        ms = _time(lambda: sd.sd_draft_feature_attention(qp, k, vv, H, 1.0 / np.sqrt(128.0), out), 10)
+        nbytes = S * L * D * 2 * (2 if vv is v else 1) + S * Q * D * 2
+        print(json.dumps({"call": "sd_draft_feature_attention", "workload": f"S={S} L={L} Q={Q} H={H}, {name}",
+                          "us": ms * 1e3, "gbs": nbytes / ms / 1e6, "frac_hbm": nbytes / ms / 1e6 / hbm,
+                          "frac_hbm_nominal_8TBs": nbytes / ms / 1e6 / 8000.0, "bytes": nbytes, "peaks": src}))
+
+
 def compact(B=1024, L=8, T=64, Hkv=4, D=128):
     """Stress shape for compaction: every node of every tree accepted (a 64-node chain), 1024
     sequences, 8 layers: 2 x 1.07 GB moved per call."""
@@ -184,7 +201,7 @@ def compact(B=1024, L=8, T=64, Hkv=4, D=128):
 
 
 if __name__ == "__main__":
-    what = sys.argv[1:] or ["attention", "attention_layers", "lmhead", "sampled", "compact"]
+    what = sys.argv[1:] or ["attention", "attention_layers", "lmhead", "sampled", "draft", "compact"]
     if "attention" in what:
         attention()
     if "attention_layers" in what:
@@ -195,5 +212,7 @@ if __name__ == "__main__":
         lmhead(rows=(480,))
     if "sampled" in what:
         sampled()
+    if "draft" in what:
+        draft()
     if "compact" in what:
         compact()
