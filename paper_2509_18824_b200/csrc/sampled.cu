@@ -194,8 +194,53 @@ residual_blocksum_kernel(int V, const int32_t* __restrict__ n_excl, const int32_
     if (threadIdx.x == 0) block_sum[(size_t)b * n_blocks + blockIdx.x] = s_v[0];
 }
 
-// One CTA per sequence.  The block sums, then the chosen block's masses, are brought into shared
-// memory by all threads; one thread walks them in vocabulary order (a fixed order of additions).
+// First index i in [0, n) at which base + v[0] + ... + v[i] reaches target, found by one warp: every
+// lane sums a contiguous chunk, an inclusive scan over the lanes gives each chunk's starting value,
+// and the first lane whose chunk contains the crossing walks it element by element (fixed order of
+// additions).  positive_only: elements <= 0 cannot be the answer (tokens without mass).  Returns -1
+// when the sum stays short; *acc_io then holds base + the whole sum; *last_pos the last index with v > 0.
+__device__ __forceinline__ int warp_find_crossing(const float* v, int n, float target, bool positive_only,
+                                                  float* acc_io, int* last_pos, int lane) {
+    const int chunk = (n + 31) / 32;
+    const int i0 = min(n, lane * chunk), i1 = min(n, i0 + chunk);
+    float sum = 0.f;
+    int lastp = -1;
+    for (int i = i0; i < i1; ++i) { sum += v[i]; if (v[i] > 0.f) lastp = i; }
+    float incl = sum;
+#pragma unroll
+    for (int d = 1; d < 32; d <<= 1) {
+        const float y = __shfl_up_sync(0xffffffffu, incl, d);
+        if (lane >= d) incl += y;
+    }
+    const float before = *acc_io + (incl - sum);
+    int found = -1;
+    float acc_at = 0.f;
+    // lanes in order: the first chunk in which the walk actually reaches the target
+    uint32_t cand = __ballot_sync(0xffffffffu, i0 < i1 && before + sum >= target);
+    while (cand && found < 0) {
+        const int L0 = __ffs(cand) - 1;
+        cand &= cand - 1;
+        int idx = -1;
+        float acc = before;
+        if (lane == L0) {
+            for (int i = i0; i < i1; ++i) {
+                if (positive_only && !(v[i] > 0.f)) continue;
+                if (acc + v[i] >= target) { idx = i; break; }
+                acc += v[i];
+            }
+        }
+        found = __shfl_sync(0xffffffffu, idx, L0);
+        acc_at = __shfl_sync(0xffffffffu, acc, L0);
+    }
+    const float total = __shfl_sync(0xffffffffu, incl, 31);
+    const int lp = __reduce_max_sync(0xffffffffu, lastp);
+    if (last_pos && lp >= 0) *last_pos = lp;
+    *acc_io = found >= 0 ? acc_at : *acc_io + total;
+    return found;
+}
+
+// One CTA per sequence.  The block sums, then the masses of one block at a time, are brought into
+// shared memory by all threads; warp 0 finds where the cumulative mass reaches w * (total mass).
 constexpr int kPickMaxBlocks = 4096;   // vocabularies up to 1 Mi tokens
 __global__ void __launch_bounds__(kResBlock)
 residual_pick_kernel(sd_batch bt, int V, const float* __restrict__ w, const float* __restrict__ mass,
@@ -204,50 +249,48 @@ residual_pick_kernel(sd_batch bt, int V, const float* __restrict__ w, const floa
     __shared__ float s_bs[kPickMaxBlocks];
     __shared__ float s_m[kResBlock];
     __shared__ float s_acc, s_target;
-    __shared__ int s_k, s_pick;
+    __shared__ int s_k, s_pick, s_last;
     const int b = blockIdx.x;
     const int na = n_acc[b];
     if (na < 1 || na > bt.T_max) return;                               // bad tree: already reported
+    const int lane = threadIdx.x & 31;
     const float* bs = block_sum + (size_t)b * n_blocks;
     for (int k = threadIdx.x; k < n_blocks; k += blockDim.x) s_bs[k] = bs[k];
     __syncthreads();
-    if (threadIdx.x == 0) {
-        float total = 0.f;
-        for (int k = 0; k < n_blocks; ++k) total += s_bs[k];
+    if (threadIdx.x < 32) {
+        float total = 0.f;                                             // whole remaining mass, same order of additions
+        warp_find_crossing(s_bs, n_blocks, INFINITY, false, &total, nullptr, lane);
         const float target = w[b] * total;
         float acc = 0.f;
-        int k = 0;
-        for (; k < n_blocks - 1; ++k) {
-            if (acc + s_bs[k] >= target) break;
-            acc += s_bs[k];
-        }
-        s_acc = acc; s_target = target; s_k = k; s_pick = -1;
+        int k = warp_find_crossing(s_bs, n_blocks, target, false, &acc, nullptr, lane);
+        if (k < 0) { k = n_blocks - 1; acc -= s_bs[k]; }               // rounding left the sum short: last block
+        if (lane == 0) { s_acc = acc; s_target = target; s_k = k; s_pick = -1; s_last = -1; }
     }
     __syncthreads();
     const float* m = mass + (size_t)b * V;
-    // (if rounding leaves the sums short, fall through the following blocks to the last token with mass)
-    int last = -1;
+    // (if the chosen block's walk stays short of the target, go on through the following blocks)
     for (int k = s_k; k < n_blocks; ++k) {
         const int t = k * kResBlock + threadIdx.x;
         s_m[threadIdx.x] = t < V ? m[t] : 0.f;
         __syncthreads();
-        if (threadIdx.x == 0) {
+        if (threadIdx.x < 32) {
             float acc = s_acc;
-            const float target = s_target;
-            for (int i = 0; i < kResBlock; ++i) {
-                const float mt = s_m[i];
-                if (mt <= 0.f) continue;
-                last = k * kResBlock + i;
-                if (acc + mt >= target) { s_pick = last; break; }
-                acc += mt;
+            int lastp = -1;
+            const int i = warp_find_crossing(s_m, kResBlock, s_target, true, &acc, &lastp, lane);
+            if (lane == 0) {
+                s_acc = acc;
+                if (lastp >= 0) s_last = k * kResBlock + lastp;
+                if (i >= 0) s_pick = k * kResBlock + i;
             }
-            s_acc = acc;
         }
         __syncthreads();
         if (s_pick >= 0) break;
     }
     if (threadIdx.x == 0) {
-        int pick = s_pick >= 0 ? s_pick : last;
+        int pick = s_pick >= 0 ? s_pick : s_last;
+        if (pick < 0)                                                  // w ~ 1 and nothing left behind the chosen block:
+            for (int t = V - 1; t >= 0 && pick < 0; --t)               // the last token that has mass at all
+                if (m[t] > 0.f) pick = t;
         if (pick < 0) { set_status(status, SD_ERR_BOUNDS); pick = 0; }  // no mass at all: inputs were not finite
         out_tok[(size_t)b * bt.T_max + na - 1] = pick;
     }

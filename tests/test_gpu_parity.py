@@ -462,3 +462,88 @@ def test_full_step_c5_shapes():
         oracle.compact(G, rk, rv, w.k_tree[l], w.v_tree[l], ref_acc[0], ref_acc[1])
         assert np.array_equal(vs.k_cache[l].cpu().numpy().view(np.uint16), rk)
         assert np.array_equal(vs.v_cache[l].cpu().numpy().view(np.uint16), rv)
+
+
+# ------------------------------------------------------------------ several steps in a row: lossless decoding
+def test_speculative_loop_on_gpu_is_lossless():
+    """Twelve verify steps of a toy target (one attention layer + LM head; a token's q/k/v rows depend
+    on the token only) through the library: arbitrary draft trees, attention, fused LM head +
+    acceptance + compaction, lengths advanced from new_len.  The emitted tokens must equal plain
+    sequential greedy decoding computed in fp64 on the host, and the caches must hold exactly the
+    committed tokens' K/V rows (Sec. 4.1 of the paper: verification leaves the target's output
+    unchanged).  Logit gaps of the toy are checked to be far above bf16 rounding first."""
+    D, V, T, B, steps = 128, 40, 8, 2, 12
+    g = np.random.default_rng(10)
+    mk = lambda s: wl.f32_to_bf16_bits((s * g.standard_normal((V, D))).astype(np.float32))
+    Eq, Ek, Ev, W = mk(2.0), mk(1.0), mk(1.0), mk(1.0)
+    f64 = wl.bf16_bits_to_f64
+
+    def greedy(prompt, n_new):
+        toks, min_gap = list(prompt), np.inf
+        for _ in range(n_new):
+            s = f64(Ek[toks]) @ f64(Eq[toks[-1]]) / np.sqrt(D)
+            w = np.exp(s - s.max())
+            hid = wl.f32_to_bf16_bits(((w[:, None] * f64(Ev[toks])).sum(0) / w.sum()).astype(np.float32))
+            lg = f64(W) @ f64(hid)
+            top = np.sort(lg)[-2:]
+            min_gap = min(min_gap, top[1] - top[0])
+            toks.append(int(np.argmax(lg)))
+        return toks, min_gap
+
+    prompts = [[3, 1, 4, 1, 5, 9, 2, 6], [7, 7, 2, 30, 11] + [(5 * i + 3) % V for i in range(60)]]   # the second starts past a block
+    want, gaps = zip(*(greedy(p, 7 * steps) for p in prompts))
+    assert min(gaps) > 0.04, gaps        # bf16 rounding of the hidden state moves a logit by about 0.002
+
+    nblk_per = 4
+    table = np.array([[2, 0, 3, 1], [5, 7, 4, 6]], dtype=np.int32)
+    kc = np.zeros((B * nblk_per, 1, 64, D), dtype=np.uint16); vc = np.zeros_like(kc)
+    committed = [list(p) for p in prompts]
+    for b in range(B):
+        for t, x in enumerate(committed[b][:-1]):
+            kc[table[b, t // 64], 0, t % 64] = Ek[x]; vc[table[b, t // 64], 0, t % 64] = Ev[x]
+    kcd, vcd = to_device(kc), to_device(vc)
+    Wd = to_device(W)
+    st = sd.new_status()
+    emitted = []
+    for step in range(steps):
+        par = np.stack([np.array([-1] + [int(g.integers(0, i)) for i in range(1, T)], dtype=np.int32) for _ in range(B)])
+        tok = np.zeros((B, T), dtype=np.int32)
+        for b in range(B):
+            truth = greedy(committed[b], 7)[0][len(committed[b]):]
+            tok[b, 0] = committed[b][-1]
+            depth = np.zeros(T, dtype=int)
+            for i in range(1, T):
+                depth[i] = depth[par[b, i]] + 1
+                sib = {int(tok[b, j]) for j in range(1, i) if par[b, j] == par[b, i]}
+                cand = truth[depth[i] - 1] if g.random() < 0.6 else int(g.integers(0, V))
+                while cand in sib:                                  # siblings carry distinct tokens
+                    cand = int(g.integers(0, V))
+                tok[b, i] = cand
+        lens = np.array([len(c) - 1 for c in committed], dtype=np.int32)
+        bt = sd.Batch(B, T, 1, 1, D, table, lens, np.full(B, T, np.int32), par)
+        sd.sd_tree_prepare(bt, st)
+        q, kt, vt = to_device(Eq[tok][:, :, None, :]), to_device(Ek[tok][:, :, None, :]), to_device(Ev[tok][:, :, None, :])
+        out = torch.zeros((B, T, 1, D), dtype=torch.bfloat16, device="cuda")
+        ws = torch.empty(sd.sd_workspace_bytes(bt, B * T, V), dtype=torch.uint8, device="cuda")
+        sd.sd_verify_attention(bt, sd.kv_layer(kcd, vcd), q, kt, vt, 1.0 / np.sqrt(D), out, None, ws, st)
+        hidden = out.view(torch.int16).reshape(B * T, D)             # the attention output IS the hidden state
+        am = torch.zeros(B * T, dtype=torch.int32, device="cuda")
+        n_acc = torch.zeros(B, dtype=torch.int32, device="cuda"); new_len = torch.zeros(B, dtype=torch.int32, device="cuda")
+        path = torch.zeros((B, T), dtype=torch.int32, device="cuda"); out_tok = torch.zeros((B, T), dtype=torch.int32, device="cuda")
+        ls = sd.LayerSet([kcd], [vcd], [kt], [vt])
+        sd.sd_lmhead_accept_compact(bt, hidden, Wd, to_device(tok), ls, am, None, n_acc, path, out_tok, new_len, ws, st)
+        torch.cuda.synchronize()
+        assert int(st.item()) == 0
+        na, ot, nl = n_acc.cpu().numpy(), out_tok.cpu().numpy(), new_len.cpu().numpy()
+        for b in range(B):
+            committed[b] += [int(x) for x in ot[b, :na[b]]]
+            assert nl[b] == len(committed[b]) - 1
+        emitted.append(int(na.sum()))
+    for b in range(B):
+        assert committed[b] == want[b][:len(committed[b])]
+    assert max(emitted) > B                                           # speculation accepted drafts
+    kc_after, vc_after = kcd.cpu().numpy().view(np.uint16), vcd.cpu().numpy().view(np.uint16)
+    for b in range(B):
+        for t, x in enumerate(committed[b][:-1]):
+            np.testing.assert_array_equal(kc_after[table[b, t // 64], 0, t % 64], Ek[x])
+            np.testing.assert_array_equal(vc_after[table[b, t // 64], 0, t % 64], Ev[x])
