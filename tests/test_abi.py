@@ -49,3 +49,27 @@ def test_product_code_never_touches_the_checker():
                 text = open(os.path.join(dirpath, f)).read()
                 assert "import oracle" not in text and "from oracle" not in text, f
                 assert "liboracle" not in text and "sd_oracle" not in text, f
+
+
+def test_host_side_refusals_of_the_newer_calls():
+    """Argument checks that need no GPU: every refusal comes back before anything is launched."""
+    from paper_2509_18824_b200 import binding as b
+    L = b.lib
+    f = ctypes.c_float
+    ok = 4096                                               # any 16-byte aligned, non-null stand-in address
+    # draft feature aggregation: at most 8 meta queries, 32 layers, heads of 128
+    assert L.sd_draft_feature_attention(ok, ok, ok, 4, 28, 9, 2, 256, f(1.0), ok, None) == b.SD_ERR_UNSUPPORTED
+    assert L.sd_draft_feature_attention(ok, ok, ok, 4, 33, 4, 2, 256, f(1.0), ok, None) == b.SD_ERR_UNSUPPORTED
+    assert L.sd_draft_feature_attention(ok, ok, ok, 4, 28, 4, 2, 200, f(1.0), ok, None) == b.SD_ERR_UNSUPPORTED
+    assert L.sd_draft_feature_attention(ok, ok, ok, 4, 28, 4, 2, 256, f(0.0), ok, None) == b.SD_ERR_INVALID_ARG
+    assert L.sd_draft_feature_attention(None, ok, ok, 4, 28, 4, 2, 256, f(1.0), ok, None) == b.SD_ERR_INVALID_ARG
+    # soft-max statistics: temperature must be positive, the hidden size a multiple of 64, lse present
+    assert L.sd_lmhead_stats(ok, ok, 8, 128, 100, f(0.0), None, None, ok, ok, 1 << 30, ok, None) == b.SD_ERR_INVALID_ARG
+    assert L.sd_lmhead_stats(ok, ok, 8, 100, 100, f(1.0), None, None, ok, ok, 1 << 30, ok, None) == b.SD_ERR_UNSUPPORTED
+    assert L.sd_lmhead_stats(ok, ok, 8, 128, 100, f(1.0), None, None, None, ok, 1 << 30, ok, None) == b.SD_ERR_INVALID_ARG
+    # the workspace figure covers every call that takes one, and grows with the vocabulary
+    bt = b.sd_batch(8, 60, 28, 4, 128, 64, 66, 16, 16, 16, 16, 16)
+    small = L.sd_workspace_bytes(ctypes.byref(bt), 480, 1024)
+    big = L.sd_workspace_bytes(ctypes.byref(bt), 480, 152064)
+    assert big > small >= L.sd_workspace_bytes(None, 480, 1024) > 0
+    assert big >= 8 * 152064 * 4                            # room for one probability row per sequence
