@@ -54,6 +54,8 @@ struct AttnPlan {
     int n_chunks;      // key chunks per sequence (the last one also takes the tree tile)
     int rows;          // T_max * G
     int row_tiles;
+    int n_layers;      // layers of this launch
+    int ranked;        // dispatch the sequences longest first (only matters when the grid runs in several waves)
 };
 
 static AttnPlan make_plan(const sd_batch& bt, int n_layers, int sms) {
@@ -75,6 +77,8 @@ static AttnPlan make_plan(const sd_batch& bt, int n_layers, int sms) {
         if (cost < best - 1e-9) { best = cost; n = c; }
     }
     p.n_chunks = n;
+    p.n_layers = n_layers;
+    p.ranked = (bt.B > 1 && bt.B <= 64 && (long long)base * n > slots) ? 1 : 0;
     return p;
 }
 
@@ -208,10 +212,32 @@ attn_umma_kernel(const __grid_constant__ AttnLayers<NL> layers, const sd_batch b
     const int lane = threadIdx.x & 31;
     const int chunk = blockIdx.x;
     const int rt = blockIdx.y;
+    // blockIdx.z enumerates (sequence rank, layer, KV head): the CTAs of the longest sequences are
+    // dispatched first, in every layer, so that a ragged batch does not end on a few long stragglers.
+    // The rank -> sequence lookup is done here (up to 64 sequences: each of the first B threads ranks
+    // one sequence by cached length, ties by index); larger batches, and launches that fit the GPU in
+    // one wave, run in index order.
     const int kvh = blockIdx.z % bt.Hkv;
     const int lb = blockIdx.z / bt.Hkv;
-    const int b = lb % bt.B;
-    const AttnLayer& ly = layers.l[lb / bt.B];
+    const int rank_b = lb / plan.n_layers;
+    int b = rank_b;
+    if (plan.ranked) {
+        // (the slot lives in the dynamic shared-memory block: a static variable would push that block's
+        //  1 KiB-aligned start and cost the second resident CTA)
+        int& s_seq = *reinterpret_cast<int*>(bars + 19);
+        if ((int)threadIdx.x < bt.B) {
+            const int mine = __ldg(bt.len + threadIdx.x);
+            int r = 0;
+            for (int j = 0; j < bt.B; ++j) {
+                const int other = __ldg(bt.len + j);
+                r += (other > mine || (other == mine && j < (int)threadIdx.x)) ? 1 : 0;
+            }
+            if (r == rank_b) s_seq = threadIdx.x;
+        }
+        __syncthreads();
+        b = s_seq;
+    }
+    const AttnLayer& ly = layers.l[lb % plan.n_layers];
     const CUtensorMap* const map_kc = &ly.k_cache;
     const CUtensorMap* const map_vc = &ly.v_cache;
     const CUtensorMap* const map_kt = &ly.k_tree;
