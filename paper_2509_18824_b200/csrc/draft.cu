@@ -25,6 +25,9 @@ __device__ __forceinline__ uint32_t pack_bf16(float lo, float hi) {
     return *reinterpret_cast<uint32_t*>(&h);
 }
 
+// SAME: k and v are one buffer (the un-projected reading); every row is then fetched once, into the
+// shared tile, and the K fragments come from that tile too (plain ldmatrix) instead of from global memory.
+template <bool SAME>
 __global__ void __launch_bounds__(kDraftWarps * 32, 3)
 draft_feature_attention_kernel(const uint16_t* __restrict__ qp, const uint16_t* __restrict__ k,
                                const uint16_t* __restrict__ v, int S, int L, int Q, int H, float scale,
@@ -54,16 +57,29 @@ draft_feature_attention_kernel(const uint16_t* __restrict__ qp, const uint16_t* 
                          ::"r"(vs_addr + row * kVRow + c16 * 16), "l"(vh + (size_t)row * D + c16 * 8) : "memory");
         }
         asm volatile("cp.async.commit_group;" ::: "memory");
-        // ---- K rows as B fragments (layer 8 * nt + g, values 16 * ks + 2t .. and + 8): 4-byte loads, all in flight
+        // ---- K rows as B fragments (layer 8 * nt + g, values 16 * ks + 2t .. and + 8)
         uint32_t kb[4][8][2];
+        if (SAME) {
+            asm volatile("cp.async.wait_group 0;" ::: "memory");
+            __syncwarp();
+            const int mi_ = lane >> 3, r_ = lane & 7;
 #pragma unroll
-        for (int nt = 0; nt < 4; ++nt) {
-            const int row = nt * 8 + g;
-            const uint32_t* kr = reinterpret_cast<const uint32_t*>(kh + (size_t)min(row, L - 1) * D) + t;
+            for (int nt = 0; nt < 4; ++nt)
 #pragma unroll
-            for (int ks = 0; ks < 8; ++ks) {
-                kb[nt][ks][0] = __ldg(kr + ks * 8);
-                kb[nt][ks][1] = __ldg(kr + ks * 8 + 4);
+                for (int kp = 0; kp < 4; ++kp)                                      // two k-steps per load
+                    asm volatile("ldmatrix.sync.aligned.m8n8.x4.shared.b16 {%0,%1,%2,%3}, [%4];"
+                                 : "=r"(kb[nt][2 * kp][0]), "=r"(kb[nt][2 * kp][1]), "=r"(kb[nt][2 * kp + 1][0]), "=r"(kb[nt][2 * kp + 1][1])
+                                 : "r"(vs_addr + (nt * 8 + r_) * kVRow + (2 * kp + (mi_ >> 1)) * 32 + (mi_ & 1) * 16) : "memory");
+        } else {                                                                    // 4-byte loads, all in flight
+#pragma unroll
+            for (int nt = 0; nt < 4; ++nt) {
+                const int row = nt * 8 + g;
+                const uint32_t* kr = reinterpret_cast<const uint32_t*>(kh + (size_t)min(row, L - 1) * D) + t;
+#pragma unroll
+                for (int ks = 0; ks < 8; ++ks) {
+                    kb[nt][ks][0] = __ldg(kr + ks * 8);
+                    kb[nt][ks][1] = __ldg(kr + ks * 8 + 4);
+                }
             }
         }
         // ---- meta queries of this head as A fragments (row g; rows >= Q and rows 8..15 are zero)
@@ -149,9 +165,10 @@ sd_status launch_draft_feature_attention(const void* qp, const void* k, const vo
     const long long want = (tasks + kDraftWarps - 1) / kDraftWarps;
     const long long cap = (long long)sms * 6;                        // resident CTAs, grid-stride beyond
     const int grid = (int)(want < cap ? want : cap);
-    if (cudaFuncSetAttribute(draft_feature_attention_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem) != cudaSuccess)
+    auto kern = (k == v) ? draft_feature_attention_kernel<true> : draft_feature_attention_kernel<false>;
+    if (cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem) != cudaSuccess)
         return SD_ERR_CUDA;
-    draft_feature_attention_kernel<<<grid, kDraftWarps * 32, smem, st>>>(
+    kern<<<grid, kDraftWarps * 32, smem, st>>>(
         static_cast<const uint16_t*>(qp), static_cast<const uint16_t*>(k), static_cast<const uint16_t*>(v), S, L, Q, H, scale,
         static_cast<uint16_t*>(out));
     return cuda_ok(cudaGetLastError());
