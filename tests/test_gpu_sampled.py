@@ -30,7 +30,7 @@ def run_stats(hidden, W, inv_temp):
 
 
 @pytest.mark.parametrize("M,Hd,V,inv_temp", [(5, 128, 1000, 1.0), (61, 192, 129, 0.5), (130, 64, 4099, 2.0),
-                                             (600, 128, 2500, 1.0)])
+                                             (600, 128, 2500, 1.0), (3, 64, 100, 1.0), (2, 64, 1, 1.0)])
 def test_lmhead_stats_small_shapes(M, Hd, V, inv_temp):
     g = np.random.default_rng(M + V)
     h = wl.f32_to_bf16_bits((g.standard_normal((M, Hd)) * 2).astype(np.float32))
@@ -94,6 +94,7 @@ def run_sampled(w, tok, inv_temp, u, wv):
     ("c5", dict(L=1, V=8192, Hd=512, prefix=100), 5.0),
     ("c4", dict(L=1, V=4096, Hd=256, prefix_range=(40, 300)), 3.0),          # 16 sequences: two residual passes
     ("chain11", dict(L=1, V=3000, Hd=128, prefix=70), 2.5),
+    ("c1", dict(V=96, Hd=64), 1.5),                                          # vocabulary below one 128-row tile
 ])
 def test_sampled_acceptance_against_the_reference(cfg, over, inv_temp):
     w = wl.make(cfg, attention=False, hidden_gain=24.0, **over)
