@@ -98,7 +98,7 @@ static int sm_count() {
 size_t attention_workspace_bytes(const sd_batch&) { return 256; }
 
 // Everything the CTAs of one layer need.  A launch covers up to kMaxLayersPerLaunch layers (the
-// descriptors travel as kernel parameters); blockIdx.z enumerates (layer, sequence, KV head).
+// descriptors travel as kernel parameters); blockIdx.z enumerates (sequence, layer, KV head).
 struct AttnLayer {
     CUtensorMap k_cache, v_cache;   // 2-D [num_blocks*Hkv*64][128], box 64 x 64
     CUtensorMap k_tree, v_tree;     // 3-D (128, Hkv, B*T_max), box 64 x 1 x 64
