@@ -213,3 +213,40 @@ def test_sampled_full_size_c5():
         assert got == t_ref or margin <= CLOSE, (b, got, t_ref, margin)
         moved += n_acc[b] - 1
     assert moved > 0
+
+
+def test_sampled_gpu_output_frequencies_follow_the_target_distribution():
+    """Losslessness measured on the GPU path itself: 16 identical sequences (root + 3 drafted children)
+    verified with fresh uniforms 300 times; the FIRST emitted token of every sequence must be
+    distributed as the target's p at the root (5 sigma), whichever route produced it (an accepted
+    child or the residual draw)."""
+    B, T, Hd, V, inv_temp, reps = 16, 4, 64, 16, 1.2, 300
+    g = np.random.default_rng(21)
+    bf = lambda a: wl.f32_to_bf16_bits(a.astype(np.float32))
+    hid_one = bf(g.standard_normal((T, Hd)))
+    W = bf(g.standard_normal((V, Hd)) * 0.25)
+
+    class Geo:
+        pass
+    w = Geo()
+    w.B, w.T_max, w.Hq, w.Hkv, w.D = B, T, 4, 1, 128
+    w.block_table = np.arange(B, dtype=np.int32).reshape(B, 1)
+    w.len = np.full(B, 5, np.int32)
+    w.n_nodes = np.full(B, T, np.int32)
+    w.parents = np.tile(np.array([-1, 0, 0, 0], np.int32), (B, 1))
+    w.hidden = np.tile(hid_one, (B, 1))
+    w.W = W
+    lg = oracle.logits(hid_one, W)
+    p, _ = smp.softmax_rows(lg, inv_temp)
+    order = np.argsort(-p[0])
+    tok = np.tile(np.array([0, order[1], order[0], order[3]], np.int32), (B, 1))   # children: 2nd, 1st and 4th most likely
+    counts = np.zeros(V)
+    for rep in range(reps):
+        u = g.random((B, T)).astype(np.float32)
+        wv = g.random(B).astype(np.float32)
+        n_acc, path, out_tok, new_len, _, status = run_sampled(w, tok, inv_temp, u, wv)
+        assert status == 0
+        np.add.at(counts, out_tok[:, 0], 1)
+    n = B * reps
+    sigma = np.sqrt(n * p[0] * (1 - p[0]))
+    assert (np.abs(counts - n * p[0]) <= 5 * sigma + 1).all(), (counts / n, p[0])
