@@ -258,7 +258,7 @@ def main():
     ms_total = e0.elapsed_time(e1)
 
     # per-call durations, same steps, events around every call (same stream)
-    names = ["attention", "attention_single_layer_call", "tail", "lmhead", "accept", "compact"]
+    names = ["attention", "attention_single_layer_call", "tail", "tail_sampled", "lmhead", "accept", "compact"]
     ev = {n: [] for n in names}
     def timed(name, fn):
         a, b = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
@@ -267,7 +267,11 @@ def main():
     for _ in range(args.steps):                           # the same two calls as the timed step
         timed("attention", vs.attention_layers)           # all layers, one library call
         timed("tail", vs.tail)                            # LM head + acceptance + compaction, one call
+    gen = torch.Generator(device="cuda"); gen.manual_seed(rank)
+    u_rand = torch.rand((w.B, w.T_max), device="cuda", generator=gen)
+    w_rand = torch.rand((w.B,), device="cuda", generator=gen)
     for _ in range(max(1, args.steps // 10)):             # for comparison: the tail as three calls,
+        timed("tail_sampled", lambda: vs.tail_sampled(1.0, u_rand, w_rand))   # the tail at temperature 1,
         timed("lmhead", vs.lmhead)                        # attention as one call per layer
         timed("accept", vs.accept)
         timed("compact", vs.compact)
@@ -339,6 +343,7 @@ def main():
                           "attention_ms_per_layer": per_call_ms["attention"] / vs.L,
                           "attention_ms_single_layer_call": per_call_ms["attention_single_layer_call"],
                           "lmhead_accept_compact_ms": per_call_ms["tail"],
+                          "sampled_tail_ms": per_call_ms["tail_sampled"],
                           "lmhead_ms": per_call_ms["lmhead"], "accept_ms": per_call_ms["accept"],
                           "compact_ms": per_call_ms["compact"],
                           "lmhead_tflops": lm_tflops, "lmhead_frac_of_tensor_peak": lm_tflops / peaks["tensor_sustained"],
