@@ -704,6 +704,13 @@ static sd_status launch_lmhead_impl(const void* hidden, const void* W, int M, in
         if (pair) {
             grid &= ~1;
             if (grid > 2 * p.n_tiles) grid = 2 * p.n_tiles;
+            if (p.n_pad > 128) {
+                // Tensor-bound sizes: the slowest pair sets the time (ceil(tiles / pairs) rounds), so use
+                // the fewest pairs that still finish in that many rounds; the SMs left idle cost no time
+                // and leave their share of the power budget to the others.
+                const int rounds = (p.n_tiles + grid / 2 - 1) / (grid / 2);
+                grid = 2 * ((p.n_tiles + rounds - 1) / rounds);
+            }
             auto kern = (bk == 64) ? (p.n_parts == 2 ? lmhead_umma_pair_kernel<64, 2> : lmhead_umma_pair_kernel<64, 1>)
                                    : (p.n_parts == 2 ? lmhead_umma_pair_kernel<32, 2> : lmhead_umma_pair_kernel<32, 1>);
             if (cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)dyn) != cudaSuccess)
