@@ -303,9 +303,10 @@ sd_status sd_lmhead_stats(const void *hidden, const void *W, int32_t M, int32_t 
  *                      among other things, the stop nodes' probabilities over the
  *                      vocabulary (B x V floats) - the only logits-sized data that
  *                      reach memory, for one row per sequence
- * Siblings must carry distinct tokens.  Arithmetic: fp32; a comparison whose two
- * sides differ by less than rounding may fall either way.  A draft token outside
- * [0, V) stores SD_ERR_BOUNDS, a bad tree SD_ERR_INVALID_TREE.
+ * Siblings must carry distinct tokens (a repeated token among the children the
+ * walk looks at stores SD_ERR_INVALID_ARG).  Arithmetic: fp32; a comparison whose
+ * two sides differ by less than rounding may fall either way.  A draft token
+ * outside [0, V) stores SD_ERR_BOUNDS, a bad tree SD_ERR_INVALID_TREE.
  */
 sd_status sd_accept_tree_sampled(const sd_batch *batch, const void *hidden, const void *W,
                                  int32_t Hd, int32_t V, float inv_temp, const float *lse,

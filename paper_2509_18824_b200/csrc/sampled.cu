@@ -118,6 +118,7 @@ __global__ void sampled_walk_kernel(sd_batch bt, const int32_t* __restrict__ dra
     }
     // parent and token of the (up to) two nodes this lane looks after
     const int pa0 = lane < n ? par[lane] : -2, pa1 = lane + 32 < n ? par[lane + 32] : -2;
+    const int tk0 = lane < n ? dt[lane] : -1, tk1 = lane + 32 < n ? dt[lane + 32] : -1;
     int32_t* pth = path + (size_t)b * T;
     int32_t* ot = out_tok + (size_t)b * T;
     int cur = 0, na = 1;
@@ -132,6 +133,10 @@ __global__ void sampled_walk_kernel(sd_batch bt, const int32_t* __restrict__ dra
         while (kids) {                                       // warp-uniform loop
             const int c = __ffsll((long long)kids) - 1;
             kids &= kids - 1;
+            // siblings must carry distinct tokens (an earlier sibling's rejection already removed the mass)
+            const int tc = dt[c];
+            if (__any_sync(0xffffffffu, (pa0 == cur && lane < c && tk0 == tc) || (pa1 == cur && lane + 32 < c && tk1 == tc)))
+                if (lane == 0) set_status(status, SD_ERR_INVALID_ARG);
             const float pc = p_child[(size_t)b * T + c];
             if (u[(size_t)b * T + c] * R < pc) { nxt = c; break; }
             R -= pc;

@@ -167,6 +167,9 @@ def test_sampled_bad_inputs_are_reported():
     u = np.full((1, 8), 0.5, np.float32); wv = np.full(1, 0.5, np.float32)
     *_, status = run_sampled(w, tok, 1.0, u, wv)
     assert status == sd.SD_ERR_BOUNDS
+    dup = np.array([[0, 7, 7, 1, 2, 3, 4, 5]], dtype=np.int32)              # nodes 1 and 2 are siblings with one token
+    *_, status = run_sampled(w, dup, 1.0, np.full((1, 8), 0.999, np.float32), wv)
+    assert status == sd.SD_ERR_INVALID_ARG
     w.parents = w.parents.copy(); w.parents[0, 3] = 6
     *_, status = run_sampled(w, np.arange(8, dtype=np.int32)[None], 1.0, u, wv)
     assert status == sd.SD_ERR_INVALID_TREE
