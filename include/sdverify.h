@@ -275,12 +275,17 @@ sd_status sd_lmhead_accept_compact(const sd_batch *batch, const void *hidden, co
  *   lse[r] = log sum_v exp(logits[r][v] * inv_temp)        (natural log, fp32)
  * accumulated in the same epilogue (running reference and sum per row; logits
  * still never reach memory).  argmax and maxlogit may be NULL.
- *   inv_temp  : 1 / temperature, > 0
- *   workspace : at least sd_workspace_bytes(NULL, M, V)
+ *   inv_temp    : 1 / temperature, > 0
+ *   group_stats : NULL, or dev f32 [ceil(V / 32)][M][2], 8-byte aligned: for every 32
+ *                 consecutive vocabulary rows g and hidden row r the pair (largest
+ *                 logit of the group, sum over the group of exp((logit - largest) *
+ *                 inv_temp)).  sd_accept_tree_sampled uses it to draw its last token
+ *                 without reading W a second time.
+ *   workspace   : at least sd_workspace_bytes(NULL, M, V)
  */
 sd_status sd_lmhead_stats(const void *hidden, const void *W, int32_t M, int32_t Hd, int32_t V,
                           float inv_temp, int32_t *argmax, float *maxlogit, float *lse,
-                          void *workspace, size_t workspace_bytes,
+                          float *group_stats, void *workspace, size_t workspace_bytes,
                           int32_t *dev_status, void *stream);
 
 /*
@@ -299,10 +304,13 @@ sd_status sd_lmhead_stats(const void *hidden, const void *W, int32_t M, int32_t 
  * All random numbers are inputs: u dev f32 [B][T_max] in [0,1), w dev f32 [B].
  *   hidden, W, Hd, V : the LM head's operands (row b * T_max + i = node i of sequence b)
  *   lse              : dev f32 [B * T_max] from sd_lmhead_stats with the same inv_temp
- *   workspace        : at least sd_workspace_bytes(batch, B * T_max, V); it receives,
- *                      among other things, the stop nodes' probabilities over the
- *                      vocabulary (B x V floats) - the only logits-sized data that
- *                      reach memory, for one row per sequence
+ *   group_stats      : the table sd_lmhead_stats filled in the same call as lse, or NULL.
+ *                      With it the last token is found from the per-group masses and
+ *                      32 recomputed logits; without it the stop nodes' rows go
+ *                      through the LM head once more and their probabilities over
+ *                      the vocabulary (B x V floats, in the workspace) are the only
+ *                      logits-sized data that reach memory
+ *   workspace        : at least sd_workspace_bytes(batch, B * T_max, V)
  * Siblings must carry distinct tokens (a repeated token among the children the
  * walk looks at stores SD_ERR_INVALID_ARG).  Arithmetic: fp32; a comparison whose
  * two sides differ by less than rounding may fall either way.  A draft token
@@ -310,6 +318,7 @@ sd_status sd_lmhead_stats(const void *hidden, const void *W, int32_t M, int32_t 
  */
 sd_status sd_accept_tree_sampled(const sd_batch *batch, const void *hidden, const void *W,
                                  int32_t Hd, int32_t V, float inv_temp, const float *lse,
+                                 const float *group_stats,
                                  const int32_t *draft_tok, const float *u, const float *w,
                                  int32_t *n_acc, int32_t *path, int32_t *out_tok, int32_t *new_len,
                                  void *workspace, size_t workspace_bytes,

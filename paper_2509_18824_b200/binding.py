@@ -84,10 +84,11 @@ def _load(path: str = LIB_PATH) -> C.CDLL:
                                              C.c_void_p, C.c_size_t, C.c_void_p, C.c_void_p]
     lib.sd_lmhead_stats.restype = C.c_int
     lib.sd_lmhead_stats.argtypes = [C.c_void_p, C.c_void_p, C.c_int32, C.c_int32, C.c_int32, C.c_float,
-                                    C.c_void_p, C.c_void_p, C.c_void_p, C.c_void_p, C.c_size_t, C.c_void_p, C.c_void_p]
+                                    C.c_void_p, C.c_void_p, C.c_void_p, C.c_void_p, C.c_void_p, C.c_size_t,
+                                    C.c_void_p, C.c_void_p]
     lib.sd_accept_tree_sampled.restype = C.c_int
     lib.sd_accept_tree_sampled.argtypes = [C.c_void_p, C.c_void_p, C.c_void_p, C.c_int32, C.c_int32, C.c_float,
-                                           C.c_void_p, C.c_void_p, C.c_void_p, C.c_void_p,
+                                           C.c_void_p, C.c_void_p, C.c_void_p, C.c_void_p, C.c_void_p,
                                            C.c_void_p, C.c_void_p, C.c_void_p, C.c_void_p,
                                            C.c_void_p, C.c_size_t, C.c_void_p, C.c_void_p]
     lib.sd_draft_feature_attention.restype = C.c_int
@@ -266,24 +267,31 @@ def sd_lmhead_accept_compact(batch: Batch, hidden, W, draft_tok, layers: LayerSe
                                         workspace.numel() * workspace.element_size(), _ptr(status), _stream(stream)))
 
 
-def sd_lmhead_stats(hidden, W, inv_temp: float, argmax, maxlogit, lse, workspace, status, stream=None) -> None:
-    """LM-head arg-max plus lse[r] = log sum_v exp(logit[r][v] * inv_temp)."""
+def group_stats_shape(M: int, V: int):
+    """Shape (float32) of the optional per-group statistics table of sd_lmhead_stats."""
+    return ((V + 31) // 32, M, 2)
+
+
+def sd_lmhead_stats(hidden, W, inv_temp: float, argmax, maxlogit, lse, workspace, status, stream=None,
+                    group_stats=None) -> None:
+    """LM-head arg-max plus lse[r] = log sum_v exp(logit[r][v] * inv_temp); optionally the per-group
+    (maximum, sum) table that lets sd_accept_tree_sampled skip its second pass over W."""
     M, Hd = hidden.shape
     V = W.shape[0]
     assert W.shape[1] == Hd
     _check(lib.sd_lmhead_stats(_ptr(hidden), _ptr(W), int(M), int(Hd), int(V), C.c_float(inv_temp), _ptr(argmax),
-                               _ptr(maxlogit), _ptr(lse), _ptr(workspace),
+                               _ptr(maxlogit), _ptr(lse), _ptr(group_stats), _ptr(workspace),
                                workspace.numel() * workspace.element_size(), _ptr(status), _stream(stream)))
 
 
 def sd_accept_tree_sampled(batch: Batch, hidden, W, inv_temp: float, lse, draft_tok, u, w,
-                           n_acc, path, out_tok, new_len, workspace, status, stream=None) -> None:
+                           n_acc, path, out_tok, new_len, workspace, status, stream=None, group_stats=None) -> None:
     """Acceptance at a sampling temperature (uniforms u [B,T] and w [B] are inputs)."""
     M, Hd = hidden.shape
     V = W.shape[0]
     assert W.shape[1] == Hd and M == batch.B * batch.T_max
     _check(lib.sd_accept_tree_sampled(batch.ref(), _ptr(hidden), _ptr(W), int(Hd), int(V), C.c_float(inv_temp),
-                                      _ptr(lse), _ptr(draft_tok), _ptr(u), _ptr(w), _ptr(n_acc), _ptr(path),
+                                      _ptr(lse), _ptr(group_stats), _ptr(draft_tok), _ptr(u), _ptr(w), _ptr(n_acc), _ptr(path),
                                       _ptr(out_tok), _ptr(new_len), _ptr(workspace),
                                       workspace.numel() * workspace.element_size(), _ptr(status), _stream(stream)))
 

@@ -44,6 +44,10 @@ struct LmParams {
     float* part_sum;   // [gridDim.x][kMaxCols] sum over the CTA's vocabulary rows of 2^((logit - ref) * c2)
     // probability output (residual draw of the sampled acceptance): when mass_out is set, the epilogue
     // stores exp(logit * inv_temp - col_lse[row]) for every (row, vocabulary entry) instead of reducing
+    // per 32 vocabulary rows and hidden row: (group maximum, sum of 2^((logit - maximum) * c2)), optional;
+    // the residual draw of the sampled acceptance finds its token from these without a second pass over W
+    float2* group_stats;    // [ceil(V / 32)][M_total]
+    int M_total;
     float* mass_out;        // [rows of the call][V]
     const float* col_lse;   // [rows of the call]
     float inv_temp;
@@ -319,6 +323,8 @@ lmhead_umma_kernel(const __grid_constant__ CUtensorMap tmW, const __grid_constan
                         float cs;
                         column_argmax_stats32(r, v_ok, v_base, lane, p.c2, cv, ci, cs);
                         merge_sumexp(run_ref[h], run_sum[h], cv, cs, p.c2);
+                        if (p.group_stats && v_base < p.V && c * 32 + lane < p.rows)
+                            p.group_stats[(size_t)(v_base >> 5) * p.M_total + p.row0 + c * 32 + lane] = make_float2(cv, cs);
                     } else {
                         column_argmax32(r, v_ok, v_base, lane, cv, ci);
                     }
@@ -535,6 +541,8 @@ lmhead_umma_pair_kernel(const __grid_constant__ CUtensorMap tmW, const __grid_co
                         float cs;
                         column_argmax_stats32(r, v_ok, v_base, lane, p.c2, cv, ci, cs);
                         merge_sumexp(run_ref[h], run_sum[h], cv, cs, p.c2);
+                        if (p.group_stats && v_base < p.V && c * 32 + lane < p.rows)
+                            p.group_stats[(size_t)(v_base >> 5) * p.M_total + p.row0 + c * 32 + lane] = make_float2(cv, cs);
                     } else {
                         column_argmax32(r, v_ok, v_base, lane, cv, ci);
                     }
@@ -645,7 +653,8 @@ static sd_status launch_lmhead_impl(const void* hidden, const void* W, int M, in
                                     int32_t* argmax, float* maxlogit, void* ws, size_t ws_bytes,
                                     int32_t* dev_status, cudaStream_t st, int* tiles_only_ctas,
                                     float inv_temp = 0.f, float* lse = nullptr,
-                                    float* mass_out = nullptr, const float* col_lse = nullptr) {
+                                    float* mass_out = nullptr, const float* col_lse = nullptr,
+                                    float* group_stats = nullptr) {
     if (ws_bytes < (lse ? stats_workspace_bytes(M, V) : lmhead_workspace_bytes(M, V))) return SD_ERR_WORKSPACE;
     if (tiles_only_ctas && M > kMaxCols) return SD_ERR_UNSUPPORTED;
     int dev = 0, sms = 0;
@@ -692,6 +701,7 @@ static sd_status launch_lmhead_impl(const void* hidden, const void* W, int M, in
         p.part_ref = reinterpret_cast<float*>(static_cast<char*>(ws) + tail_workspace_bytes(M, V));
         p.part_sum = p.part_ref + (size_t)kMaxCtas * kMaxCols;
         p.mass_out = mass_out; p.col_lse = col_lse; p.inv_temp = inv_temp;
+        p.group_stats = reinterpret_cast<float2*>(group_stats); p.M_total = M;
 
         CUtensorMap tmW, tmH;
         if (!encode_tmap_bf16_2d(&tmW, W, (uint64_t)V, (uint64_t)Hd, (uint64_t)Hd * 2, (uint32_t)bk, kBM, bk * 2))
@@ -761,9 +771,10 @@ sd_status launch_lmhead_mass(const void* hidden, const void* W, int M, int Hd, i
 }
 
 sd_status launch_lmhead_stats(const void* hidden, const void* W, int M, int Hd, int V, float inv_temp,
-                              int32_t* argmax, float* maxlogit, float* lse, void* ws, size_t ws_bytes,
-                              int32_t* dev_status, cudaStream_t st) {
-    return launch_lmhead_impl(hidden, W, M, Hd, V, argmax, maxlogit, ws, ws_bytes, dev_status, st, nullptr, inv_temp, lse);
+                              int32_t* argmax, float* maxlogit, float* lse, float* group_stats,
+                              void* ws, size_t ws_bytes, int32_t* dev_status, cudaStream_t st) {
+    return launch_lmhead_impl(hidden, W, M, Hd, V, argmax, maxlogit, ws, ws_bytes, dev_status, st, nullptr, inv_temp, lse,
+                              nullptr, nullptr, group_stats);
 }
 
 sd_status launch_lmhead(const void* hidden, const void* W, int M, int Hd, int V,

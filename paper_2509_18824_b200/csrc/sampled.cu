@@ -20,6 +20,7 @@ struct SampledWs {                     // carved out of the caller's workspace
     int32_t* stop_row;                 // [B]    b * T + stop node
     int32_t* n_excl;                   // [B]
     int32_t* excl;                     // [B][64] drafted tokens of the stop node's children
+    float* excl_p;                     // [B][64] and their probabilities
     float* block_sum;                  // [B][n_blocks]
     float* mass;                       // [B][V]
     uint16_t* stop_hidden;             // [B rounded up to 16][Hd] hidden rows of the stop nodes
@@ -32,7 +33,7 @@ static size_t align256(size_t x) { return (x + 255) & ~(size_t)255; }
 size_t sampled_workspace_bytes(int B, int T, int V, int Hd) {
     const size_t nb = (size_t)(V + kResBlock - 1) / kResBlock;
     const size_t b16 = (size_t)(B + 15) / 16 * 16;
-    return align256((size_t)B * T * 4) + align256((size_t)B * 4) * 3 + align256((size_t)B * 64 * 4) +
+    return align256((size_t)B * T * 4) + align256((size_t)B * 4) * 3 + align256((size_t)B * 64 * 4) * 2 +
            align256((size_t)B * nb * 4) + align256((size_t)B * V * 4) + align256(b16 * Hd * 2) + align256((size_t)B * 4) +
            align256(stats_workspace_bytes(B, V));
 }
@@ -46,6 +47,7 @@ static SampledWs carve(void* ws, int B, int T, int V, int Hd) {
     w.stop_row = reinterpret_cast<int32_t*>(p); p += align256((size_t)B * 4);
     w.n_excl = reinterpret_cast<int32_t*>(p);  p += align256((size_t)B * 4);
     w.excl = reinterpret_cast<int32_t*>(p);    p += align256((size_t)B * 64 * 4);
+    w.excl_p = reinterpret_cast<float*>(p);    p += align256((size_t)B * 64 * 4);
     w.block_sum = reinterpret_cast<float*>(p); p += align256((size_t)B * nb * 4);
     w.mass = reinterpret_cast<float*>(p);      p += align256((size_t)B * V * 4);
     w.stop_hidden = reinterpret_cast<uint16_t*>(p); p += align256((size_t)(B + 15) / 16 * 16 * Hd * 2);
@@ -100,7 +102,7 @@ child_prob_kernel(sd_batch bt, const uint16_t* __restrict__ hidden, const uint16
 __global__ void sampled_walk_kernel(sd_batch bt, const int32_t* __restrict__ draft, const float* __restrict__ p_child,
                                     const float* __restrict__ u, int32_t* n_acc, int32_t* path, int32_t* out_tok,
                                     int32_t* new_len, float* resid, int32_t* stop_row, int32_t* n_excl, int32_t* excl,
-                                    int32_t* status) {
+                                    float* excl_p, int32_t* status) {
     const int b = blockIdx.x, lane = threadIdx.x;
     const int T = bt.T_max;
     const int n = bt.n_nodes[b];
@@ -149,8 +151,8 @@ __global__ void sampled_walk_kernel(sd_batch bt, const int32_t* __restrict__ dra
     // the stop node's drafted tokens carry no mass in the residual
     const uint32_t lo = __ballot_sync(0xffffffffu, pa0 == cur), hi = __ballot_sync(0xffffffffu, pa1 == cur);
     const int rank0 = __popc(lo & ((1u << lane) - 1u)), rank1 = __popc(lo) + __popc(hi & ((1u << lane) - 1u));
-    if (pa0 == cur) excl[(size_t)b * 64 + rank0] = dt[lane];
-    if (pa1 == cur) excl[(size_t)b * 64 + rank1] = dt[lane + 32];
+    if (pa0 == cur) { excl[(size_t)b * 64 + rank0] = dt[lane]; excl_p[(size_t)b * 64 + rank0] = p_child[(size_t)b * T + lane]; }
+    if (pa1 == cur) { excl[(size_t)b * 64 + rank1] = dt[lane + 32]; excl_p[(size_t)b * 64 + rank1] = p_child[(size_t)b * T + lane + 32]; }
     for (int k = na + lane; k < T; k += 32) { pth[k] = -1; ot[k] = -1; }
     if (lane == 0) {
         n_acc[b] = na;
@@ -301,8 +303,101 @@ residual_pick_kernel(sd_batch bt, int V, const float* __restrict__ w, const floa
     }
 }
 
+// Residual draw from the LM-head pass's own statistics.  One CTA per sequence: the masses of the 32-row
+// vocabulary groups of the stop row follow from (group maximum, group sum) and the row's lse; the
+// drafted children's probabilities are taken out of their groups; warp 0 finds the group in which the
+// cumulative mass reaches w * (total); that group's 32 logits are recomputed (32 dot products) and the
+// token is found among them.  W is not streamed a second time and no logits-sized data exist.
+constexpr int kPickMaxGroups = 8192;   // vocabularies up to 262144 tokens
+__global__ void __launch_bounds__(256)
+residual_pick_groups_kernel(sd_batch bt, const uint16_t* __restrict__ hidden, const uint16_t* __restrict__ W, int Hd, int V,
+                            float inv_temp, const float* __restrict__ lse, const float2* __restrict__ group_stats, int n_groups,
+                            const float* __restrict__ w, const int32_t* __restrict__ stop_row, const int32_t* __restrict__ n_excl,
+                            const int32_t* __restrict__ excl, const float* __restrict__ excl_p, const int32_t* __restrict__ n_acc,
+                            int32_t* out_tok, int32_t* status) {
+    __shared__ float s_g[kPickMaxGroups];
+    __shared__ float s_m[32];
+    __shared__ float s_acc, s_target;
+    __shared__ int s_k, s_pick, s_last;
+    const int b = blockIdx.x;
+    const int na = n_acc[b];
+    if (na < 1 || na > bt.T_max) return;                               // bad tree: already reported
+    const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+    const int row = stop_row[b];
+    const int M = bt.B * bt.T_max;
+    const float c2 = inv_temp * 1.4426950408889634f;
+    const float lse2 = lse[row] * 1.4426950408889634f;
+    for (int g = threadIdx.x; g < n_groups; g += blockDim.x) {
+        const float2 st = group_stats[(size_t)g * M + row];
+        s_g[g] = st.y > 0.f ? st.y * exp2f(st.x * c2 - lse2) : 0.f;
+    }
+    __syncthreads();
+    const int ne = n_excl[b];
+    if (threadIdx.x == 0)                                              // drafted children carry no mass (fixed order)
+        for (int e = 0; e < ne; ++e) {
+            const int g = excl[(size_t)b * 64 + e] >> 5;
+            s_g[g] = fmaxf(s_g[g] - excl_p[(size_t)b * 64 + e], 0.f);
+        }
+    __syncthreads();
+    if (threadIdx.x < 32) {
+        float total = 0.f;
+        warp_find_crossing(s_g, n_groups, INFINITY, false, &total, nullptr, lane);
+        const float target = w[b] * total;
+        float acc = 0.f;
+        int k = warp_find_crossing(s_g, n_groups, target, false, &acc, nullptr, lane);
+        if (k < 0) { k = n_groups - 1; acc -= s_g[k]; }
+        if (lane == 0) { s_acc = acc; s_target = target; s_k = k; s_pick = -1; s_last = -1; }
+    }
+    __syncthreads();
+    const uint4* hrow = reinterpret_cast<const uint4*>(hidden + (size_t)row * Hd);
+    // the 32 probabilities of group k, recomputed into s_m: eight warps, four tokens each
+    auto recompute_group = [&](int k) {
+        for (int i = warp * 4; i < warp * 4 + 4; ++i) {
+            const int t = k * 32 + i;
+            float m = 0.f;
+            if (t < V) {
+                const float l = warp_dot_bf16(reinterpret_cast<const uint4*>(W + (size_t)t * Hd), hrow, Hd / 8, lane);
+                bool hit = false;
+                for (int e = lane; e < ne; e += 32) hit |= (excl[(size_t)b * 64 + e] == t);
+                m = __any_sync(0xffffffffu, hit) ? 0.f : __expf(l * inv_temp - lse[row]);
+            }
+            if (lane == 0) s_m[i] = m;
+        }
+        __syncthreads();
+    };
+    for (int k = s_k; k < n_groups; ++k) {
+        recompute_group(k);
+        if (threadIdx.x < 32) {
+            float acc = s_acc;
+            int lastp = -1;
+            const int i = warp_find_crossing(s_m, 32, s_target, true, &acc, &lastp, lane);
+            if (lane == 0) {
+                s_acc = acc;
+                if (lastp >= 0) s_last = k * 32 + lastp;
+                if (i >= 0) s_pick = k * 32 + i;
+            }
+        }
+        __syncthreads();
+        if (s_pick >= 0) break;
+    }
+    // (rounding left the walk short and nothing with mass lay behind the chosen group: the last token
+    //  with mass before it)
+    for (int k = s_k - 1; k >= 0 && s_pick < 0 && s_last < 0; --k) {
+        recompute_group(k);
+        if (threadIdx.x == 0)
+            for (int i = 31; i >= 0; --i)
+                if (s_m[i] > 0.f) { s_last = k * 32 + i; break; }
+        __syncthreads();
+    }
+    if (threadIdx.x == 0) {
+        int pick = s_pick >= 0 ? s_pick : s_last;
+        if (pick < 0) { set_status(status, SD_ERR_BOUNDS); pick = 0; }  // no mass at all: inputs were not finite
+        out_tok[(size_t)b * bt.T_max + na - 1] = pick;
+    }
+}
+
 sd_status launch_accept_sampled(const sd_batch& bt, const void* hidden, const void* W, int Hd, int V, float inv_temp,
-                                const float* lse, const int32_t* draft, const float* u, const float* w,
+                                const float* lse, const float* group_stats, const int32_t* draft, const float* u, const float* w,
                                 int32_t* n_acc, int32_t* path, int32_t* out_tok, int32_t* new_len,
                                 void* ws, size_t ws_bytes, int32_t* dev_status, cudaStream_t st) {
     const int B = bt.B, T = bt.T_max;
@@ -314,7 +409,15 @@ sd_status launch_accept_sampled(const sd_batch& bt, const void* hidden, const vo
     const int n_blocks = (V + kResBlock - 1) / kResBlock;
     child_prob_kernel<<<(B * T * 32 + 127) / 128, 128, 0, st>>>(bt, h, Wp, Hd, V, inv_temp, lse, draft, s.p_child, dev_status);
     sampled_walk_kernel<<<B, 32, 0, st>>>(bt, draft, s.p_child, u, n_acc, path, out_tok, new_len, s.resid, s.stop_row,
-                                         s.n_excl, s.excl, dev_status);
+                                         s.n_excl, s.excl, s.excl_p, dev_status);
+    if (group_stats) {
+        // the LM-head pass left (maximum, sum) of every 32 vocabulary rows: no second pass over W
+        const int n_groups = (V + 31) / 32;
+        if (n_groups > kPickMaxGroups) return SD_ERR_UNSUPPORTED;
+        residual_pick_groups_kernel<<<B, 256, 0, st>>>(bt, h, Wp, Hd, V, inv_temp, lse, reinterpret_cast<const float2*>(group_stats),
+                                                      n_groups, w, s.stop_row, s.n_excl, s.excl, s.excl_p, n_acc, out_tok, dev_status);
+        return cuda_ok(cudaGetLastError());
+    }
     gather_stop_rows_kernel<<<B, 128, 0, st>>>(h, Hd, lse, s.stop_row, s.stop_hidden, s.stop_lse);
     // probabilities of the stop rows over the vocabulary: one more pass of the tensor-core LM-head kernel,
     // its epilogue storing instead of reducing (W is streamed once for all sequences)

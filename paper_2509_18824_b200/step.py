@@ -146,13 +146,16 @@ class VerifyStep:
         given uniforms (u [B,T], w [B], device f32), the residual draw, then compaction."""
         if getattr(self, "lse_rows", None) is None:
             self.lse_rows = torch.zeros(self.w.B * self.w.T_max, dtype=torch.float32, device=self.device)
+            self.group_stats = torch.zeros(sd.group_stats_shape(self.w.B * self.w.T_max, self.w.V),
+                                           dtype=torch.float32, device=self.device)
             need = sd.sd_workspace_bytes(self.batch, self.w.B * self.w.T_max, self.w.V)
             if self.workspace.numel() < need:
                 self.workspace = torch.empty(need, dtype=torch.uint8, device=self.device)
         sd.sd_lmhead_stats(self.hidden, self.W, inv_temp, self.argmax, self.maxlogit, self.lse_rows,
-                           self.workspace, self.status, stream)
+                           self.workspace, self.status, stream, group_stats=self.group_stats)
         sd.sd_accept_tree_sampled(self.batch, self.hidden, self.W, inv_temp, self.lse_rows, self.draft_tok, u, w,
-                                  self.n_acc, self.path, self.out_tok, self.new_len, self.workspace, self.status, stream)
+                                  self.n_acc, self.path, self.out_tok, self.new_len, self.workspace, self.status, stream,
+                                  group_stats=self.group_stats)
         self.compact(stream)
 
     # -- the whole step -------------------------------------------------

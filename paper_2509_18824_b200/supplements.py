@@ -141,16 +141,22 @@ def sampled(cfg="c5", inv_temp=1.0):
     st = vs.status
     flops = 2.0 * M * w.V * w.Hd
     ms_greedy = _time(lambda: sd.sd_lmhead_argmax(vs.hidden, vs.W, vs.argmax, vs.maxlogit, ws, st), 10)
-    ms_stats = _time(lambda: sd.sd_lmhead_stats(vs.hidden, vs.W, inv_temp, vs.argmax, vs.maxlogit, lse, ws, st), 10)
+    gs = torch.zeros(sd.group_stats_shape(M, w.V), dtype=torch.float32, device="cuda")
+    ms_stats0 = _time(lambda: sd.sd_lmhead_stats(vs.hidden, vs.W, inv_temp, vs.argmax, vs.maxlogit, lse, ws, st), 10)
+    ms_stats = _time(lambda: sd.sd_lmhead_stats(vs.hidden, vs.W, inv_temp, vs.argmax, vs.maxlogit, lse, ws, st,
+                                                group_stats=gs), 10)
+    ms_acc0 = _time(lambda: sd.sd_accept_tree_sampled(vs.batch, vs.hidden, vs.W, inv_temp, lse, vs.draft_tok, u, wv,
+                                                      vs.n_acc, vs.path, vs.out_tok, vs.new_len, ws, st), 10)
     ms_acc = _time(lambda: sd.sd_accept_tree_sampled(vs.batch, vs.hidden, vs.W, inv_temp, lse, vs.draft_tok, u, wv,
-                                                     vs.n_acc, vs.path, vs.out_tok, vs.new_len, ws, st), 10)
+                                                     vs.n_acc, vs.path, vs.out_tok, vs.new_len, ws, st, group_stats=gs), 10)
     wbytes = w.V * w.Hd * 2
     print(json.dumps({"call": "sampled tail", "workload": cfg, "rows": M,
                       "sd_lmhead_argmax_us": ms_greedy * 1e3, "sd_lmhead_stats_us": ms_stats * 1e3,
                       "stats_tflops": flops / ms_stats / 1e9, "stats_frac_tensor_burst": flops / ms_stats / 1e9 / tens,
+                      "sd_lmhead_stats_without_group_table_us": ms_stats0 * 1e3,
                       "sd_accept_tree_sampled_us": ms_acc * 1e3,
-                      "accept_weight_stream_gbs": wbytes * ((B + 7) // 8) / ms_acc / 1e6,
-                      "accept_frac_hbm": wbytes * ((B + 7) // 8) / ms_acc / 1e6 / hbm,
+                      "sd_accept_tree_sampled_second_pass_us": ms_acc0 * 1e3,
+                      "second_pass_weight_stream_gbs": wbytes / ms_acc0 / 1e6,
                       "peaks": src, "status": int(st.item())}))
 
 

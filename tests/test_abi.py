@@ -64,9 +64,10 @@ def test_host_side_refusals_of_the_newer_calls():
     assert L.sd_draft_feature_attention(ok, ok, ok, 4, 28, 4, 2, 256, f(0.0), ok, None) == b.SD_ERR_INVALID_ARG
     assert L.sd_draft_feature_attention(None, ok, ok, 4, 28, 4, 2, 256, f(1.0), ok, None) == b.SD_ERR_INVALID_ARG
     # soft-max statistics: temperature must be positive, the hidden size a multiple of 64, lse present
-    assert L.sd_lmhead_stats(ok, ok, 8, 128, 100, f(0.0), None, None, ok, ok, 1 << 30, ok, None) == b.SD_ERR_INVALID_ARG
-    assert L.sd_lmhead_stats(ok, ok, 8, 100, 100, f(1.0), None, None, ok, ok, 1 << 30, ok, None) == b.SD_ERR_UNSUPPORTED
-    assert L.sd_lmhead_stats(ok, ok, 8, 128, 100, f(1.0), None, None, None, ok, 1 << 30, ok, None) == b.SD_ERR_INVALID_ARG
+    assert L.sd_lmhead_stats(ok, ok, 8, 128, 100, f(0.0), None, None, ok, None, ok, 1 << 30, ok, None) == b.SD_ERR_INVALID_ARG
+    assert L.sd_lmhead_stats(ok, ok, 8, 100, 100, f(1.0), None, None, ok, None, ok, 1 << 30, ok, None) == b.SD_ERR_UNSUPPORTED
+    assert L.sd_lmhead_stats(ok, ok, 8, 128, 100, f(1.0), None, None, None, None, ok, 1 << 30, ok, None) == b.SD_ERR_INVALID_ARG
+    assert L.sd_lmhead_stats(ok, ok, 8, 128, 100, f(1.0), None, None, ok, 4100, ok, 1 << 30, ok, None) == b.SD_ERR_INVALID_ARG
     # the workspace figure covers every call that takes one, and grows with the vocabulary
     bt = b.sd_batch(8, 60, 28, 4, 128, 64, 66, 16, 16, 16, 16, 16)
     small = L.sd_workspace_bytes(ctypes.byref(bt), 480, 1024)

@@ -68,7 +68,9 @@ def good_drafts(w, lg, seed):
     return tok
 
 
-def run_sampled(w, tok, inv_temp, u, wv):
+def run_sampled(w, tok, inv_temp, u, wv, groups=True):
+    """groups=True: the LM-head pass also leaves its per-group statistics and the last token is drawn
+    from them; False: the stop rows go through the LM head a second time."""
     bt = sd.Batch.of(w)
     st = sd.new_status()
     h, Wd = to_device(w.hidden), to_device(w.W)
@@ -76,13 +78,14 @@ def run_sampled(w, tok, inv_temp, u, wv):
     B, T = w.B, w.T_max
     ws = torch.zeros(sd.sd_workspace_bytes(bt, M, V), dtype=torch.uint8, device="cuda")
     lse = torch.zeros(M, dtype=torch.float32, device="cuda")
-    sd.sd_lmhead_stats(h, Wd, inv_temp, None, None, lse, ws, st)
+    gs = torch.zeros(sd.group_stats_shape(M, V), dtype=torch.float32, device="cuda") if groups else None
+    sd.sd_lmhead_stats(h, Wd, inv_temp, None, None, lse, ws, st, group_stats=gs)
     n_acc = torch.full((B,), -9, dtype=torch.int32, device="cuda")
     path = torch.full((B, T), -9, dtype=torch.int32, device="cuda")
     out_tok = torch.full((B, T), -9, dtype=torch.int32, device="cuda")
     new_len = torch.full((B,), -9, dtype=torch.int32, device="cuda")
     sd.sd_accept_tree_sampled(bt, h, Wd, inv_temp, lse, to_device(tok), to_device(u), to_device(wv),
-                              n_acc, path, out_tok, new_len, ws, st)
+                              n_acc, path, out_tok, new_len, ws, st, group_stats=gs)
     torch.cuda.synchronize()
     p_child = ws[:B * T * 4].view(torch.float32).cpu().numpy().reshape(B, T)      # first area of the workspace
     return (n_acc.cpu().numpy(), path.cpu().numpy(), out_tok.cpu().numpy(), new_len.cpu().numpy(),
@@ -96,7 +99,8 @@ def run_sampled(w, tok, inv_temp, u, wv):
     ("chain11", dict(L=1, V=3000, Hd=128, prefix=70), 2.5),
     ("c1", dict(V=96, Hd=64), 1.5),                                          # vocabulary below one 128-row tile
 ])
-def test_sampled_acceptance_against_the_reference(cfg, over, inv_temp):
+@pytest.mark.parametrize("groups", [True, False])
+def test_sampled_acceptance_against_the_reference(cfg, over, inv_temp, groups):
     w = wl.make(cfg, attention=False, hidden_gain=24.0, **over)
     B, T, V = w.B, w.T_max, w.W.shape[0]
     lg = oracle.logits(w.hidden, w.W)
@@ -107,7 +111,7 @@ def test_sampled_acceptance_against_the_reference(cfg, over, inv_temp):
     for rep in range(3 if B > 1 else 25):
         u = g.random((B, T)).astype(np.float32)
         wv = g.random(B).astype(np.float32)
-        n_acc, path, out_tok, new_len, p_child, status = run_sampled(w, tok, inv_temp, u, wv)
+        n_acc, path, out_tok, new_len, p_child, status = run_sampled(w, tok, inv_temp, u, wv, groups)
         assert status == 0
         close_calls = 0
         for b in range(B):
@@ -175,7 +179,8 @@ def test_sampled_bad_inputs_are_reported():
     assert status == sd.SD_ERR_INVALID_TREE
 
 
-def test_sampled_full_size_c5():
+@pytest.mark.parametrize("groups", [True, False])
+def test_sampled_full_size_c5(groups):
     """Vocabulary 152064, 8 x 60-node trees: the walk bit for bit on the kernel's own probabilities,
     those probabilities and the drawn tokens against fp64 logits of the rows the walks visited."""
     w = wl.make("c5", attention=False, hidden_gain=40.0)
@@ -193,7 +198,7 @@ def test_sampled_full_size_c5():
     inv_temp = 6.0
     u = g.random((B, T)).astype(np.float32)
     wv = g.random(B).astype(np.float32)
-    n_acc, path, out_tok, new_len, p_child, status = run_sampled(w, tok, inv_temp, u, wv)
+    n_acc, path, out_tok, new_len, p_child, status = run_sampled(w, tok, inv_temp, u, wv, groups)
     assert status == 0
     visited = sorted({b * T + int(path[b, k]) for b in range(B) for k in range(n_acc[b])})
     lg = oracle.logits(w.hidden[visited], w.W)
