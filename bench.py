@@ -270,6 +270,7 @@ def main():
     gen = torch.Generator(device="cuda"); gen.manual_seed(rank)
     u_rand = torch.rand((w.B, w.T_max), device="cuda", generator=gen)
     w_rand = torch.rand((w.B,), device="cuda", generator=gen)
+    vs.tail_sampled(1.0, u_rand, w_rand)                  # untimed: its first call allocates the statistics buffers
     for _ in range(max(1, args.steps // 10)):             # for comparison: the tail as three calls,
         timed("tail_sampled", lambda: vs.tail_sampled(1.0, u_rand, w_rand))   # the tail at temperature 1,
         timed("lmhead", vs.lmhead)                        # attention as one call per layer

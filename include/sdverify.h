@@ -34,7 +34,8 @@
  *   KV cache of one layer, K and V each:  bf16 [num_blocks][Hkv][64][D]
  *       (block = 64 tokens; one (block, head) tile is 16 KiB contiguous)
  *   logical token t of sequence b lives in block block_table[b][t / 64],
- *       slot t % 64.  Slots at or beyond len[b] may hold any finite values.
+ *       slot t % 64.  Slots at or beyond len[b], and the tree K/V rows of nodes at or
+ *       beyond n_nodes[b], may hold any bit pattern (NaN and infinity included): they never reach a sum.
  *   q, out:            bf16 [B][T_max][Hq][D]
  *   tree K, tree V:    bf16 [B][T_max][Hkv][D]
  *   query head h uses KV head h / (Hq / Hkv).

@@ -426,6 +426,27 @@ attn_umma_kernel(const __grid_constant__ AttnLayers<NL> layers, const sd_batch b
         for (int j = 0; j < nt && ok; ++j) {
             const int s = j & 1;
             const uint32_t ph = (uint32_t)(j >> 1) & 1u;
+            const bool tree = (j >= t1 - t0);
+            const int valid = tree ? kKeyTile : len - (t0 + j) * kKeyTile;   // keys of this block inside the prefix
+            // Keys that no row may see (cache slots at and beyond len, rows of unused tree nodes) carry
+            // weight 0, but 0 x NaN or 0 x Inf would still poison the accumulator: their V rows are
+            // cleared in shared memory before P.V reads them (the arrival on p_full below orders the
+            // two), so those slots may hold any bit pattern.  A key row is 128 contiguous bytes in each
+            // of the two D-halves (the swizzle stays inside a row).
+            const int v_rows = tree ? n : valid;
+            if (v_rows < kKeyTile && warp < 2) {                     // threads 0..63 <-> key rows
+                const int vs = j % kVStages;
+                if (!mbar_wait(&v_full[vs], (uint32_t)(j / kVStages) & 1u, abort_flag)) { ok = false; break; }
+                if (row_in_tile >= v_rows) {
+                    uint4* z = reinterpret_cast<uint4*>(v_smem + vs * kKVStage + row_in_tile * 128);
+#pragma unroll
+                    for (int c = 0; c < 8; ++c) {
+                        z[c] = make_uint4(0, 0, 0, 0);
+                        z[c + kSubTile / 16] = make_uint4(0, 0, 0, 0);
+                    }
+                    fence_proxy_async_smem();
+                }
+            }
             if (!mbar_wait(&s_full[s], ph, abort_flag)) { ok = false; break; }
             tc_fence_after_sync();
             // The scores arrive in two halves; the second half is in flight while the first is
@@ -434,8 +455,6 @@ attn_umma_kernel(const __grid_constant__ AttnLayers<NL> layers, const sd_batch b
             tmem_ld32(tmem_s + lane_field + s * kKeyTile, r0);
             tmem_ld_wait();
             tmem_ld32(tmem_s + lane_field + s * kKeyTile + 32, r1);
-            const bool tree = (j >= t1 - t0);
-            const int valid = tree ? kKeyTile : len - (t0 + j) * kKeyTile;   // keys of this block inside the prefix
             const uint32_t mask_lo = tree ? (uint32_t)amask : (valid >= 32 ? ~0u : ((1u << max(valid, 0)) - 1u));
             const uint32_t mask_hi = tree ? (uint32_t)(amask >> 32)
                                           : (valid >= 64 ? ~0u : (valid <= 32 ? 0u : ((1u << (valid - 32)) - 1u)));

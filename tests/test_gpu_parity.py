@@ -153,6 +153,35 @@ def test_attention_planted_key_large_v_and_bad_block_table():
     assert status == sd.SD_ERR_BOUNDS
 
 
+def test_attention_any_bit_pattern_in_invisible_slots():
+    """Cache slots at and beyond len, and the K/V rows of unused tree nodes, may hold NaN and
+    infinity bit patterns (memory that was never written): no key there is visible to any row, so
+    the output must equal the checker's, which never reads them."""
+    p = tiny128(77, B=4, T=16, Hq=14, Hkv=2, lens=(5, 70, 64, 0), gain=3.0)
+    p.n_nodes = np.array([16, 3, 9, 1], dtype=np.int32)
+    junk = np.array([0x7FC0, 0x7F80, 0xFF80, 0xFFFF, 0x7FFF], dtype=np.uint16)
+    for b in range(p.B):
+        P = int(p.len[b])
+        for j in range(P // 64, (P + p.T_max + 63) // 64):      # the sequence's own blocks from slot len on
+            blk = int(p.block_table[b, j])
+            lo = max(0, P - j * 64)
+            for arr in (p.k_cache, p.v_cache):
+                shape = arr[blk, :, lo:].shape
+                arr[blk, :, lo:] = junk[np.arange(int(np.prod(shape))) % len(junk)].reshape(shape)
+        for arr in (p.k_tree, p.v_tree):
+            shape = arr[b, p.n_nodes[b]:].shape
+            arr[b, p.n_nodes[b]:] = junk[np.arange(int(np.prod(shape))) % len(junk)].reshape(shape)
+    out, lse, status = gpu_attention(p)
+    assert status == 0
+    ref, rlse = oracle.attention(oracle.Geometry.of(p), p.k_cache, p.v_cache, p.q, p.k_tree, p.v_tree, p.scale)
+    for b in range(p.B):
+        nb = int(p.n_nodes[b])
+        assert np.isfinite(out[b, :nb]).all() and np.isfinite(ref[b, :nb]).all()
+        check_attention(out[b, :nb], ref[b, :nb], f"sequence {b}")
+        np.testing.assert_allclose(lse[b, :nb], rlse[b, :nb], rtol=2e-3, atol=2e-3)
+        assert (out[b, nb:] == 0).all()
+
+
 @pytest.mark.parametrize("cfg,gain", [("c1", 1.0), ("c1", 45.0), ("c2", 1.0), ("c2", 45.0)])
 def test_attention_configs_full_compare(cfg, gain):
     w = wl.make(cfg, lmhead=False, q_gain=gain)
