@@ -92,6 +92,30 @@ class VerifyStep:
                 path=torch.zeros((B, T), dtype=torch.int32).pin_memory(),
                 out_tok=torch.zeros((B, T), dtype=torch.int32).pin_memory(),
                 new_len=torch.zeros(B, dtype=torch.int32).pin_memory())
+            # The end-to-end path double-buffers the per-step inputs on the device, so that the next
+            # step's copies run while this step still computes.  Slot 0 is the set built above.
+            self._slots = [self._slot_state()]
+            self.batch = sd.Batch.of(w, device=d)
+            self._in_dev = torch.empty_like(self._in_dev)
+            self.q, self.k_tree, self.v_tree = self._layer_views(self._in_dev, w)
+            self.hidden, self.draft_tok = torch.empty_like(self.hidden), torch.empty_like(self.draft_tok)
+            self.layerset = sd.LayerSet(self.k_cache, self.v_cache, self.k_tree, self.v_tree)
+            self.att_all = self._attention_set(0, self.L)
+            self._att_groups = {}
+            self._slots.append(self._slot_state())
+            self._use_slot(0)
+            self._step_no = 0
+
+    _SLOT_FIELDS = ("batch", "_in_dev", "q", "k_tree", "v_tree", "hidden", "draft_tok", "layerset", "att_all",
+                    "_att_groups")
+
+    def _slot_state(self) -> dict:
+        return {k: getattr(self, k) for k in self._SLOT_FIELDS}
+
+    def _use_slot(self, i: int) -> None:
+        """Make input set i the one the call wrappers below hand to the library."""
+        for k, v in self._slots[i].items():
+            setattr(self, k, v)
 
     def _layer_views(self, flat: torch.Tensor, w):
         """Per-layer q / tree K / tree V views of a flat layer-major buffer."""
@@ -196,38 +220,52 @@ class VerifyStep:
         accepted tokens go back to the host; caches and weights stay resident.
         The host-to-device copies run on a second stream, ahead of the compute:
         attention is issued in groups of `group` layers, each group as soon as
-        its layers' copies have landed (an event recorded behind them)."""
+        its layers' copies have landed (an event recorded behind them).  The
+        device-side input buffers exist twice and alternate from step to step,
+        so the copies of step i+1 overlap the last layers and the tail of step i
+        and only wait for step i-1, which read the same buffers."""
         h = self.host
         main = torch.cuda.current_stream()
         if self._copy_stream is None:
             self._copy_stream = torch.cuda.Stream(device=self.device)
-            self._ev_small = torch.cuda.Event()
-            self._ev_layer = [torch.cuda.Event() for _ in range(self.L)]
+            self._ev_small = [torch.cuda.Event() for _ in range(2)]
+            self._ev_layer = [[torch.cuda.Event() for _ in range(self.L)] for _ in range(2)]
+            self._ev_done = [None, None]
+            self._copy_stream.wait_stream(main)     # set-up work on the main stream has finished
         cs = self._copy_stream
-        cs.wait_stream(main)            # the previous step no longer reads the input buffers
+        slot = self._step_no & 1
+        self._step_no += 1
+        self._use_slot(slot)
+        if self._ev_done[slot] is not None:
+            cs.wait_event(self._ev_done[slot])      # the step before last no longer reads this input set
         with torch.cuda.stream(cs):
             self.batch.parents.copy_(h["parents"], non_blocking=True)
             self.batch.n_nodes.copy_(h["n_nodes"], non_blocking=True)
-            self._ev_small.record(cs)
+            self._ev_small[slot].record(cs)
             for l0 in range(0, self.L, group):          # one copy per group of layers
                 l1 = min(l0 + group, self.L)
                 sl = slice(l0 * self._per_layer, l1 * self._per_layer)
                 self._in_dev[sl].copy_(self._in_host[sl], non_blocking=True)
-                self._ev_layer[l1 - 1].record(cs)
+                self._ev_layer[slot][l1 - 1].record(cs)
             self.hidden.copy_(h["hidden"], non_blocking=True)
             self.draft_tok.copy_(h["draft_tok"], non_blocking=True)
-        main.wait_event(self._ev_small)
+            ev_last = torch.cuda.Event()
+            ev_last.record(cs)
+        main.wait_event(self._ev_small[slot])
         sd.sd_tree_prepare(self.batch, self.status)
         for l0 in range(0, self.L, group):
             l1 = min(l0 + group, self.L)
-            main.wait_event(self._ev_layer[l1 - 1])
+            main.wait_event(self._ev_layer[slot][l1 - 1])
             self.attention_layers(l0, l1)
-        main.wait_stream(cs)            # hidden states and draft tokens have arrived
+        main.wait_event(ev_last)        # hidden states and draft tokens have arrived
         self.tail()
         self.host_out["n_acc"].copy_(self.n_acc, non_blocking=True)
         self.host_out["path"].copy_(self.path, non_blocking=True)
         self.host_out["out_tok"].copy_(self.out_tok, non_blocking=True)
         self.host_out["new_len"].copy_(self.new_len, non_blocking=True)
+        if self._ev_done[slot] is None:
+            self._ev_done[slot] = torch.cuda.Event()
+        self._ev_done[slot].record(main)
 
     def check_status(self):
         code = int(self.status.item())

@@ -381,7 +381,7 @@ def test_chained_step_tiny():
     G = oracle.Geometry.of(w)
     ref_acc = oracle.accept(G, w.draft_tok, ram.reshape(w.B, w.T_max))
     vs = VerifyStep(w, keep_host_inputs=True)
-    for mode in ("device", "host"):
+    for mode in ("device", "host", "host", "host"):        # the host path alternates between two input sets
         vs.run() if mode == "device" else vs.run_from_host()
         torch.cuda.synchronize()
         vs.check_status()
