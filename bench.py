@@ -282,6 +282,20 @@ def main():
     clocks = sampler.stop() if rank == 0 else None
     per_call_ms = {n: sum(a.elapsed_time(b) for a, b in ev[n]) / len(ev[n]) for n in names}
 
+    # for comparison: the same step replayed from a CUDA graph (no host work per call)
+    graph = vs.capture()
+    for _ in range(3):
+        graph.replay()
+    g0, g1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    torch.cuda.synchronize()
+    g0.record()
+    for _ in range(args.steps):
+        graph.replay()
+    g1.record()
+    torch.cuda.synchronize()
+    per_call_ms["graph_replay_step"] = g0.elapsed_time(g1) / args.steps
+    del graph
+
     # end to end: this step's inputs from pinned host memory, results back to the host
     for _ in range(2):
         vs.run_from_host()
@@ -345,6 +359,7 @@ def main():
                           "attention_ms_single_layer_call": per_call_ms["attention_single_layer_call"],
                           "lmhead_accept_compact_ms": per_call_ms["tail"],
                           "sampled_tail_ms": per_call_ms["tail_sampled"],
+                          "graph_replay_ms_per_step": per_call_ms["graph_replay_step"],
                           "lmhead_ms": per_call_ms["lmhead"], "accept_ms": per_call_ms["accept"],
                           "compact_ms": per_call_ms["compact"],
                           "lmhead_tflops": lm_tflops, "lmhead_frac_of_tensor_peak": lm_tflops / peaks["tensor_sustained"],

@@ -200,6 +200,17 @@ class VerifyStep:
             self.accept(None, stream)
             self.compact(stream)
 
+    def capture(self, **run_args) -> "torch.cuda.CUDAGraph":
+        """One run() recorded into a CUDA graph (the library calls only enqueue kernels on the stream
+        they are given, so they can be captured); replay() then re-issues the step's launches without
+        any host work per call.  One un-captured run comes first, so that per-kernel set-up is done."""
+        self.run(**run_args)
+        torch.cuda.synchronize()
+        graph = torch.cuda.CUDAGraph()
+        with torch.cuda.graph(graph):
+            self.run(**run_args)
+        return graph
+
     @property
     def launches_per_step(self) -> int:
         """Kernel launches of one run(): attention (one launch per group of up to 32 layers), the
