@@ -371,6 +371,74 @@ def test_compact_bit_exact_and_touches_nothing_else():
         np.testing.assert_array_equal(vc[l].cpu().numpy().view(np.uint16), rv)
 
 
+# ------------------------------------------------------------------ nothing is written outside the outputs
+class Guarded:
+    """Tensors carved out of one device buffer with 4 KiB guard bands of a fixed byte pattern around
+    each; intact() tells whether every guard byte is still there."""
+
+    GUARD, FILL = 4096, 0x5A
+
+    def __init__(self):
+        self.specs, self.total = [], self.GUARD
+
+    def reserve(self, shape, dtype):
+        n = int(np.prod(shape)) * torch.empty(0, dtype=dtype).element_size()
+        self.specs.append((self.total, n, shape, dtype))
+        self.total += (n + 255) // 256 * 256 + self.GUARD
+        return len(self.specs) - 1
+
+    def build(self):
+        self.buf = torch.full((self.total,), self.FILL, dtype=torch.uint8, device="cuda")
+        return [self.buf[o:o + n].view(dt).view(shape) for o, n, shape, dt in self.specs]
+
+    def intact(self):
+        keep = torch.ones(self.total, dtype=torch.bool, device="cuda")
+        for o, n, _, _ in self.specs:
+            keep[o:o + n] = False
+        return bool((self.buf[keep] == self.FILL).all())
+
+
+def test_calls_write_only_their_outputs():
+    """Attention, LM head and acceptance outputs (and the workspace) sit between guard bands; after
+    the calls every guard byte is unchanged, and the results are still the checker's."""
+    g = np.random.default_rng(8)
+    T = 60
+    par = np.stack([np.array([-1] + [int(g.integers(max(0, i - 9), i)) for i in range(1, T)]) for _ in range(2)])
+    p = tiny128(31, B=2, T=T, Hq=28, Hkv=4, lens=(700, 63), parents=par, gain=3.0)
+    p.n_nodes = np.array([60, 41], dtype=np.int32)
+    M, Hd, V = p.B * T, 256, 3000
+    hidden = wl.f32_to_bf16_bits((g.standard_normal((M, Hd)) / 4).astype(np.float32))
+    W = wl.f32_to_bf16_bits((g.standard_normal((V, Hd)) / 4).astype(np.float32))
+    draft = g.integers(0, V, size=(p.B, T)).astype(np.int32)
+    bt = sd.Batch.of(p)
+    st = sd.new_status()
+    sd.sd_tree_prepare(bt, st)
+    gd = Guarded()
+    ws_bytes = sd.sd_workspace_bytes(bt, M, V)
+    for shape, dt in (((p.B, T, p.Hq, p.D), torch.bfloat16), ((p.B, T, p.Hq), torch.float32),
+                      ((M,), torch.int32), ((M,), torch.float32), ((p.B,), torch.int32), ((p.B, T), torch.int32),
+                      ((p.B, T), torch.int32), ((p.B,), torch.int32), ((ws_bytes,), torch.uint8)):
+        gd.reserve(shape, dt)
+    out, lse, am, mx, n_acc, path, out_tok, new_len, ws = gd.build()
+    kc, vc, q, kt, vt = (to_device(x) for x in (p.k_cache, p.v_cache, p.q, p.k_tree, p.v_tree))   # kept alive:
+    hd, Wd, dd = to_device(hidden), to_device(W), to_device(draft)                # the calls only take pointers
+    sd.sd_verify_attention(bt, sd.kv_layer(kc, vc), q, kt, vt, float(p.scale), out, lse, ws, st)
+    sd.sd_lmhead_argmax(hd, Wd, am, mx, ws, st)
+    sd.sd_accept_tree(bt, dd, am.view(p.B, T), n_acc, path, out_tok, new_len, st)
+    torch.cuda.synchronize()
+    assert int(st.item()) == 0
+    assert gd.intact()
+    G = oracle.Geometry.of(p)
+    ref, _ = oracle.attention(G, p.k_cache, p.v_cache, p.q, p.k_tree, p.v_tree, p.scale)
+    for b in range(p.B):
+        check_attention(out.float().cpu().numpy()[b, :p.n_nodes[b]], ref[b, :p.n_nodes[b]], f"sequence {b}")
+    ram, t1, t2 = oracle.lmhead(hidden, W)
+    check_argmax(am.cpu().numpy(), mx.cpu().numpy(), ram, t1, t2)
+    ref_acc = oracle.accept(G, draft, am.cpu().numpy().reshape(p.B, T))
+    for got, want in zip((n_acc, path, out_tok, new_len), ref_acc):
+        np.testing.assert_array_equal(got.cpu().numpy(), want)
+
+
 # ------------------------------------------------------------------ the whole step
 def test_chained_step_tiny():
     """run(): attention -> LM head -> accept -> compact chained on the device, crisp logits."""
