@@ -164,7 +164,11 @@ class Batch:
 
 
 def kv_layer(k_cache: torch.Tensor, v_cache: torch.Tensor) -> sd_kv_layer:
-    return sd_kv_layer(_ptr(k_cache), _ptr(v_cache), int(k_cache.shape[0]))
+    """Descriptor of one layer's paged cache.  The struct only carries addresses, so the returned
+    object also holds on to the two tensors: a descriptor built from temporaries stays valid."""
+    layer = sd_kv_layer(_ptr(k_cache), _ptr(v_cache), int(k_cache.shape[0]))
+    layer._keep = (k_cache, v_cache)
+    return layer
 
 
 def new_status(device="cuda") -> torch.Tensor:
