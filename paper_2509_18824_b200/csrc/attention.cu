@@ -263,6 +263,10 @@ attn_umma_kernel(const __grid_constant__ AttnLayers<NL> layers, const sd_batch b
     // A CTA without key tiles has nothing to compute, but it still takes part in the cluster barriers.
     const bool active = (nt > 0) && aligned;
     const bool clustered = (plan.n_chunks > 1);            // cluster = the chunks of one (b, kvh, row tile)
+    // A last row tile of at most 64 rows (420 rows = 3 x 128 + 36) runs its MMAs with M = 64: the
+    // accumulator rows then sit in lanes 0..15 of each 32-lane TMEM quadrant (row = 16 * quadrant + lane),
+    // the tensor cores work at half width and only 64 rows of Q are staged and re-read per key tile.
+    const bool m64 = (plan.rows - rt * kRowTile) <= 64;
     float m_used = -INFINITY, l = 0.f;                     // softmax state of this thread's row (warps 0-3)
     uint32_t tmem_base = 0;
 
@@ -355,8 +359,8 @@ attn_umma_kernel(const __grid_constant__ AttnLayers<NL> layers, const sd_batch b
         // from uniform registers, and inside a divergent "lane 0 only" region of a full warp every
         // descriptor would first have to be moved there, instruction by instruction.
         {
-            const uint32_t idesc_s = make_idesc_bf16(kRowTile, kKeyTile, false, false);   // S = Q . K^T
-            const uint32_t idesc_o = make_idesc_bf16(kRowTile, kD, false, true);          // O += P . V
+            const uint32_t idesc_s = make_idesc_bf16(m64 ? 64 : kRowTile, kKeyTile, false, false);   // S = Q . K^T
+            const uint32_t idesc_o = make_idesc_bf16(m64 ? 64 : kRowTile, kD, false, true);          // O += P . V
             // k-steps only move the (16-byte granular) start-address field in the low bits
             const uint64_t qdesc_base = make_smem_desc(smem_u32(q_smem), 16, 1024, 128);
             const uint64_t kdesc_base = make_smem_desc(smem_u32(k_smem), 16, 1024, 128);
@@ -402,8 +406,9 @@ attn_umma_kernel(const __grid_constant__ AttnLayers<NL> layers, const sd_batch b
         }
     } else if (warp < 4) {
         // ------------------------------------------------------------ softmax: one thread per row
-        const int row_in_tile = warp * 32 + lane;
-        const int row = rt * kRowTile + row_in_tile;
+        const int tid = warp * 32 + lane;
+        const int row_in_tile = m64 ? (lane < 16 ? warp * 16 + lane : -1) : tid;   // -1: a TMEM lane without a row
+        const int row = (row_in_tile >= 0) ? rt * kRowTile + row_in_tile : plan.rows;
         const int node = row / G;
         const int g = row - node * G;
         const bool row_ok = (row < plan.rows) && (node < n);
@@ -414,7 +419,7 @@ attn_umma_kernel(const __grid_constant__ AttnLayers<NL> layers, const sd_batch b
             for (int c = 0; c < 16; ++c) {
                 uint4 u = row_ok ? __ldg(src + c) : make_uint4(0, 0, 0, 0);
                 uint8_t* dst = q_smem + (c >> 3) * (kRowTile * 128) + row_in_tile * 128 + (((c & 7) ^ (row_in_tile & 7)) << 4);
-                *reinterpret_cast<uint4*>(dst) = u;
+                if (row_in_tile >= 0) *reinterpret_cast<uint4*>(dst) = u;
             }
             fence_proxy_async_smem();
             __syncwarp();
@@ -437,8 +442,8 @@ attn_umma_kernel(const __grid_constant__ AttnLayers<NL> layers, const sd_batch b
             if (v_rows < kKeyTile && warp < 2) {                     // threads 0..63 <-> key rows
                 const int vs = j % kVStages;
                 if (!mbar_wait(&v_full[vs], (uint32_t)(j / kVStages) & 1u, abort_flag)) { ok = false; break; }
-                if (row_in_tile >= v_rows) {
-                    uint4* z = reinterpret_cast<uint4*>(v_smem + vs * kKVStage + row_in_tile * 128);
+                if (tid >= v_rows) {
+                    uint4* z = reinterpret_cast<uint4*>(v_smem + vs * kKVStage + tid * 128);
 #pragma unroll
                     for (int c = 0; c < 8; ++c) {
                         z[c] = make_uint4(0, 0, 0, 0);
@@ -500,7 +505,8 @@ attn_umma_kernel(const __grid_constant__ AttnLayers<NL> layers, const sd_batch b
             }
             const float mt = fmaxf(fmaxf(mx[0], mx[1]), fmaxf(mx[2], mx[3])) * scale_log2;   // scale > 0
             // raise the reference maximum only when it would grow by more than the threshold
-            const bool raise = mt > m_used + kRescaleThreshold;      // true on the first tile (m_used = -inf)
+            // true on the first tile (m_used = -inf); lanes without a row hold stale scores and never ask
+            const bool raise = (row_in_tile >= 0) && (mt > m_used + kRescaleThreshold);
             if (__any_sync(0xffffffffu, raise)) {
                 if (j > 0) {
                     if (!mbar_wait(pv_done, (uint32_t)(j - 1) & 1u, abort_flag)) { ok = false; break; }
@@ -586,13 +592,17 @@ attn_umma_kernel(const __grid_constant__ AttnLayers<NL> layers, const sd_batch b
                 uint32_t o[32];
                 tmem_ld32(tmem_o + lane_field + cc * 32, o);
                 tmem_ld_wait();
+                if (row_in_tile >= 0) {
 #pragma unroll
-                for (int k = 0; k < 8; ++k)
-                    *reinterpret_cast<uint4*>(xo + row_in_tile * kD + (((cc * 8 + k) ^ (row_in_tile & 31)) << 2)) =
-                        make_uint4(o[4 * k], o[4 * k + 1], o[4 * k + 2], o[4 * k + 3]);
+                    for (int k = 0; k < 8; ++k)
+                        *reinterpret_cast<uint4*>(xo + row_in_tile * kD + (((cc * 8 + k) ^ (row_in_tile & 31)) << 2)) =
+                            make_uint4(o[4 * k], o[4 * k + 1], o[4 * k + 2], o[4 * k + 3]);
+                }
             }
-            xs[row_in_tile] = m_used;
-            xs[kRowTile + row_in_tile] = l;
+            if (row_in_tile >= 0) {
+                xs[row_in_tile] = m_used;
+                xs[kRowTile + row_in_tile] = l;
+            }
         } else if (!ok && lane == 0) {
             set_status(status, SD_ERR_TIMEOUT);
         }
