@@ -118,10 +118,11 @@ def test_attention_gqa7_wide_trees_and_unused_nodes():
     np.testing.assert_allclose(lse[ok], rlse[ok], rtol=2e-3, atol=2e-3)
 
 
-@pytest.mark.parametrize("Hq,Hkv,T", [(8, 1, 64), (3, 3, 5), (16, 2, 33), (4, 4, 1)])
+@pytest.mark.parametrize("Hq,Hkv,T", [(8, 1, 64), (3, 3, 5), (16, 2, 33), (4, 4, 1), (8, 1, 8), (5, 1, 13), (6, 1, 32)])
 def test_attention_group_sizes_and_tree_sizes(Hq, Hkv, T):
     """Largest supported shape (64 nodes x 8 grouped heads = 512 rows per KV head), no grouping at
-    all, a single-node tree (plain decoding), odd sizes."""
+    all, a single-node tree (plain decoding), odd sizes; 64 rows exactly (one half-height row tile),
+    65 rows (one full-height tile), 192 rows (a full tile and a half-height one that is full)."""
     g = np.random.default_rng(Hq * 100 + T)
     par = np.stack([np.array([-1] + [int(g.integers(0, i)) for i in range(1, T)]) for _ in range(2)])
     p = tiny128(40 + T, B=2, T=T, Hq=Hq, Hkv=Hkv, lens=(257, 64), parents=par, gain=3.0)
