@@ -458,6 +458,19 @@ def test_chained_step_tiny():
         for got, ref in zip((vs.n_acc, vs.path, vs.out_tok, vs.new_len), ref_acc):
             np.testing.assert_array_equal(got.cpu().numpy(), ref)
     assert vs.host_out["n_acc"][0] == 4
+    # each host-path step uses the inputs that are in pinned memory when it is issued: drafts planted
+    # for another accepted length, two steps (one per device-side input set), then the first again
+    first = w.draft_tok.copy()
+    wl.plant(w, ram.reshape(w.B, w.T_max), np.array([1]))
+    other = w.draft_tok.copy()
+    for drafts, want in ((other, 2), (other, 2), (first, 4)):
+        torch.cuda.synchronize()                  # the previous step has read the pinned buffer
+        vs.host["draft_tok"].copy_(torch.from_numpy(drafts))
+        vs.run_from_host()
+        torch.cuda.synchronize()
+        vs.check_status()
+        assert vs.host_out["n_acc"][0] == want
+    w.draft_tok = first
     rk, rv = w.k_cache[0].copy(), w.v_cache[0].copy()
     oracle.compact(G, rk, rv, w.k_tree[0], w.v_tree[0], ref_acc[0], ref_acc[1])
     np.testing.assert_array_equal(vs.k_cache[0].cpu().numpy().view(np.uint16), rk)
