@@ -92,6 +92,53 @@ __device__ __forceinline__ void compact_sequence(const sd_batch& bt, const Compa
     const int vec_per_node = bt.Hkv * vec_per_head;       // per K or V
     const int per_layer = na * 2 * vec_per_node;
     const int total = per_layer * n_layers;
+    const int per_node = 2 * vec_per_node;                 // K and V vectors of one node
+    if (stride % per_node == 0) {
+        // Every thread keeps its place inside a node (K or V, head, 16-byte piece) and only walks over
+        // the accepted nodes and the layers: no index arithmetic beyond the two table look-ups per vector.
+        const int sub = tid % per_node;
+        const int is_v = sub / vec_per_node;
+        const int kvh = (sub - is_v * vec_per_node) / vec_per_head;
+        const int c = sub - is_v * vec_per_node - kvh * vec_per_head;
+        const int k_step = stride / per_node;
+        constexpr int kUnroll = 4;                         // nodes in flight per thread: loads before stores
+        for (int k0 = tid / per_node; k0 < na; k0 += k_step * kUnroll) {
+            size_t src[kUnroll], dst[kUnroll];
+            int blk[kUnroll];
+#pragma unroll
+            for (int u = 0; u < kUnroll; ++u) {
+                const int k = k0 + u * k_step;
+                blk[u] = -2;                               // -2: no node for this slot
+                if (k >= na) continue;
+                const int node = path[k];
+                const int t = len + k;
+                if (node < 0 || node >= T || t < 0 || t / kBlock >= bt.max_blocks_per_seq) {
+                    set_status(status, SD_ERR_BOUNDS);
+                    continue;
+                }
+                blk[u] = bt.block_table[(size_t)b * bt.max_blocks_per_seq + t / kBlock];
+                src[u] = (((size_t)b * T + node) * bt.Hkv + kvh) * vec_per_head + c;
+                dst[u] = (((size_t)(blk[u] < 0 ? 0 : blk[u]) * bt.Hkv + kvh) * kBlock + (t % kBlock)) * vec_per_head + c;
+            }
+            for (int l = l0; l < l0 + n_layers; ++l) {
+                const uint4* from = is_v ? ly.vt[l] : ly.kt[l];
+                uint4* to = is_v ? ly.vc[l] : ly.kc[l];
+                const int nb = ly.num_blocks[l];
+                uint4 val[kUnroll];
+                bool live[kUnroll];
+#pragma unroll
+                for (int u = 0; u < kUnroll; ++u) {
+                    live[u] = blk[u] >= 0 && blk[u] < nb;
+                    if (blk[u] != -2 && !live[u]) set_status(status, SD_ERR_BOUNDS);
+                    if (live[u]) val[u] = from[src[u]];
+                }
+#pragma unroll
+                for (int u = 0; u < kUnroll; ++u)
+                    if (live[u]) to[dst[u]] = val[u];
+            }
+        }
+        return;
+    }
     for (int idx = tid; idx < total; idx += stride) {
         const int li = idx / per_layer;
         const int l = l0 + li;
