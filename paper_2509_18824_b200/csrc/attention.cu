@@ -38,6 +38,7 @@ constexpr int kTmemCols = 256;                 // O: 0..127, S/P buffers: 128..1
 constexpr float kLog2e = 1.4426950408889634f;
 constexpr float kRescaleThreshold = 8.0f;      // log2 units
 constexpr int kMaxChunks = 8;                  // = portable cluster size
+constexpr int kSplitRounds = 8;                // launches of fewer whole rounds get their remainder as a chunked launch
 
 __device__ __forceinline__ float max3(float a, float b, float c) {
     float d;
@@ -56,6 +57,7 @@ struct AttnPlan {
     int row_tiles;
     int n_layers;      // layers of this launch
     int ranked;        // dispatch the sequences longest first (only matters when the grid runs in several waves)
+    int z0;            // first (sequence rank, layer, KV head) index of this launch: blockIdx.z counts from here
 };
 
 static AttnPlan make_plan(const sd_batch& bt, int n_layers, int sms) {
@@ -72,13 +74,24 @@ static AttnPlan make_plan(const sd_batch& bt, int n_layers, int sms) {
     double best = 1e30;
     for (int c = 1; c <= kMaxChunks && c <= max_tiles; c *= 2) {   // 128 rows split evenly over the chunks
         const double w = (double)base * c / slots;
-        const double waves = (w <= 4.0) ? (double)((base * c + slots - 1) / slots) : w;
-        const double cost = waves * ((max_tiles + c - 1) / c + 3);
+        double waves = (w <= 4.0) ? (double)((base * c + slots - 1) / slots) : w;
+        // Without chunks, and for up to kSplitRounds whole rounds, the CTAs left over after the last whole
+        // round go into a launch of their own, with chunks (launch_group): the partial round then costs
+        // a fraction of a round.  (Longer launches run under the power cap, where this gained nothing.)
+        if (c == 1 && w > 1.0 && base / slots < kSplitRounds) {
+            const int rest = base % slots;
+            int ct = 1;                                    // chunks of the remainder's launch
+            while (2 * ct <= kMaxChunks && 2 * ct <= max_tiles && rest * 2 * ct <= slots) ct *= 2;
+            waves = (double)(base / slots) + (rest == 0 ? 0.0 : (ct > 1 ? 1.0 / ct + 0.1 : 1.0));
+        }
+        // per CTA: its key tiles, a fixed cost of about three tiles, and two more for the in-cluster merge
+        const double cost = waves * ((max_tiles + c - 1) / c + 3 + (c > 1 ? 2 : 0));
         if (cost < best - 1e-9) { best = cost; n = c; }
     }
     p.n_chunks = n;
     p.n_layers = n_layers;
     p.ranked = (bt.B > 1 && bt.B <= 64 && (long long)base * n > slots) ? 1 : 0;
+    p.z0 = 0;
     return p;
 }
 
@@ -217,8 +230,9 @@ attn_umma_kernel(const __grid_constant__ AttnLayers<NL> layers, const sd_batch b
     // The rank -> sequence lookup is done here (up to 64 sequences: each of the first B threads ranks
     // one sequence by cached length, ties by index); larger batches, and launches that fit the GPU in
     // one wave, run in index order.
-    const int kvh = blockIdx.z % bt.Hkv;
-    const int lb = blockIdx.z / bt.Hkv;
+    const int zz = (int)blockIdx.z + plan.z0;
+    const int kvh = zz % bt.Hkv;
+    const int lb = zz / bt.Hkv;
     const int rank_b = lb / plan.n_layers;
     int b = rank_b;
     if (plan.ranked) {
@@ -656,14 +670,13 @@ static bool fill_layer(AttnLayer* ly, const sd_batch& bt, const sd_kv_layer& cac
 }
 
 template <int NL>
-static sd_status launch_group(const AttnLayers<NL>& layers, int n_layers, const sd_batch& bt, float scale,
-                              int32_t* dev_status, cudaStream_t st) {
-    const AttnPlan plan = make_plan(bt, n_layers, sm_count());
+static sd_status launch_plan(const AttnLayers<NL>& layers, const sd_batch& bt, float scale, const AttnPlan& plan,
+                             int z_count, int32_t* dev_status, cudaStream_t st) {
     auto kern = attn_umma_kernel<NL>;
     if (cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, kAttSmem) != cudaSuccess)
         return SD_ERR_CUDA;
     cudaLaunchConfig_t cfg = {};
-    cfg.gridDim = dim3(plan.n_chunks, plan.row_tiles, n_layers * bt.B * bt.Hkv);
+    cfg.gridDim = dim3(plan.n_chunks, plan.row_tiles, z_count);
     cfg.blockDim = dim3(kAttThreads);
     cfg.dynamicSmemBytes = kAttSmem;
     cfg.stream = st;
@@ -677,6 +690,35 @@ static sd_status launch_group(const AttnLayers<NL>& layers, int n_layers, const 
     if (cudaLaunchKernelEx(&cfg, kern, layers, bt, scale * kLog2e, plan, dev_status) != cudaSuccess)
         return SD_ERR_CUDA;
     return SD_OK;
+}
+
+template <int NL>
+static sd_status launch_group(const AttnLayers<NL>& layers, int n_layers, const sd_batch& bt, float scale,
+                              int32_t* dev_status, cudaStream_t st) {
+    AttnPlan plan = make_plan(bt, n_layers, sm_count());
+    const int Z = n_layers * bt.B * bt.Hkv;
+    // A launch of whole-sequence CTAs that runs for more than one round ends on a partial round, in which
+    // the CTAs left over would each work through a whole sequence while most of the GPU idles.  They go
+    // into a second launch of the same kernel with the keys split into chunks (a cluster per row tile),
+    // so that the remainder also spreads over the SMs and takes a fraction of a round.  (In a ranked
+    // launch these are the shortest sequences.)
+    const int slots = 2 * sm_count();
+    const long long ctas = (long long)Z * plan.row_tiles;
+    if (plan.n_chunks == 1 && ctas > slots && ctas / slots < kSplitRounds) {
+        const int z_main = (int)((ctas / slots) * slots / plan.row_tiles);
+        const int z_rest = Z - z_main;
+        int c = 1;
+        while (2 * c <= kMaxChunks && 2 * c <= bt.max_blocks_per_seq &&
+               (long long)z_rest * plan.row_tiles * 2 * c <= slots) c *= 2;
+        if (z_main > 0 && z_rest > 0 && c > 1) {
+            const sd_status s = launch_plan<NL>(layers, bt, scale, plan, z_main, dev_status, st);
+            if (s != SD_OK) return s;
+            plan.z0 = z_main;
+            plan.n_chunks = c;
+            return launch_plan<NL>(layers, bt, scale, plan, z_rest, dev_status, st);
+        }
+    }
+    return launch_plan<NL>(layers, bt, scale, plan, Z, dev_status, st);
 }
 
 // One launch per group of layers: at most kMaxLayersPerLaunch descriptors fit the kernel's
