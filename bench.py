@@ -32,7 +32,7 @@ sys.path.insert(0, ROOT)
 # dram__bytes_read.sum + dram__bytes_write.sum of attn_umma_kernel per layer, from the ncu capture
 # summarised under profiles/.  Set an entry to None whenever the kernel changes until the counters
 # are retaken.
-ATTENTION_DRAM_BYTES_PER_LAYER = {"c5": 72.84e6}
+ATTENTION_DRAM_BYTES_PER_LAYER = {"c5": 72.63e6}
 
 METRIC = "tree_verify_steps_per_s"
 UNIT = "steps/s"
@@ -334,8 +334,8 @@ def main():
                     "peak": peaks["tensor_sustained"], "unit": "TFLOP/s",
                     "frac": att_tflops / peaks["tensor_sustained"],
                     "traffic": traffic * layers_per_launch if traffic else None,
-                    "traffic_unit": "bytes per launch (dram read + write; ncu capture of an 8-layer launch, "
-                                    "scaled by layers per launch)",
+                    "traffic_unit": "bytes per launch (dram read + write; ncu capture of the 6.94-layer main launch of "
+                                    "an 8-layer call, scaled by layers per launch)",
                     "layers_per_launch": layers_per_launch,
                     "algorithmic_bytes_per_launch": work["att_bytes"] * layers_per_launch,
                     "algorithmic_flops_per_launch": work["att_flops"] * layers_per_launch,
