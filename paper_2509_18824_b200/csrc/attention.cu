@@ -447,10 +447,15 @@ attn_umma_kernel(const __grid_constant__ AttnLayers<NL> layers, const sd_batch b
             const uint32_t ph = (uint32_t)(j >> 1) & 1u;
             const bool tree = (j >= t1 - t0);
             const int valid = tree ? kKeyTile : len - (t0 + j) * kKeyTile;   // keys of this block inside the prefix
+            if (!mbar_wait(&s_full[s], ph, abort_flag)) { ok = false; break; }
+            tc_fence_after_sync();
             // Keys that no row may see (cache slots at and beyond len, rows of unused tree nodes) carry
             // weight 0, but 0 x NaN or 0 x Inf would still poison the accumulator: their V rows are
             // cleared in shared memory before P.V reads them (the arrival on p_full below orders the
-            // two), so those slots may hold any bit pattern.  A key row is 128 contiguous bytes in each
+            // two), so those slots may hold any bit pattern.  This comes after the wait for the scores
+            // of tile j: they were issued behind P.V of tile j - 2, which read the V tile that used this
+            // ring slot before, so the slot's barrier is by now in the phase of tile j and the parity
+            // wait below cannot be taken for an earlier phase.  A key row is 128 contiguous bytes in each
             // of the two D-halves (the swizzle stays inside a row).
             const int v_rows = tree ? n : valid;
             if (v_rows < kKeyTile && warp < 2) {                     // threads 0..63 <-> key rows
@@ -466,8 +471,6 @@ attn_umma_kernel(const __grid_constant__ AttnLayers<NL> layers, const sd_batch b
                     fence_proxy_async_smem();
                 }
             }
-            if (!mbar_wait(&s_full[s], ph, abort_flag)) { ok = false; break; }
-            tc_fence_after_sync();
             // The scores arrive in two halves; the second half is in flight while the first is
             // processed.  Raw scores stay unscaled: scale * log2(e) is folded into the exponent's FMA.
             uint32_t r0[32], r1[32];

@@ -264,15 +264,43 @@ def test_attention_layers_call_full_compare(cfg, L, gain):
         np.testing.assert_allclose(got[l][1], rlse, rtol=2e-3, atol=2e-3)
 
 
-def test_attention_layers_call_many_layers_ragged():
-    """More layers than one launch holds (33 > 32), ragged lengths, unused nodes, shuffled blocks:
-    every layer must land in its own output and agree with the checker."""
-    L = 33
+@pytest.mark.parametrize("cfg,L", [("c5", 7), ("chain11", 28)])
+def test_attention_layers_call_full_size_with_remainder_launch(cfg, L):
+    """Full-size calls of a few rounds of CTAs (896 CTAs = 3.03 rounds in both cases), which the library
+    issues as whole-sequence CTAs plus a chunked remainder: sampled rows of every layer against the
+    checker, among them the last sequence's last rows, which the remainder launch computes."""
+    w = wl.make(cfg, lmhead=False, q_gain=45.0, L=L)
+    rows = sample_rows(w, 24, 11)
+    G = oracle.Geometry.of(w)
+    for attempt in range(2):                           # twice: a race would not hit the same rows again
+        got = gpu_attention_layers(w, list(range(L)))
+        for l in range(L):
+            if attempt == 0:
+                ref, rlse = oracle.attention_rows(G, w.k_cache[l], w.v_cache[l], w.q[l], w.k_tree[l], w.v_tree[l],
+                                                  w.scale, rows)
+                check_attention(got[l][0][rows[:, 0], rows[:, 1], rows[:, 2]], ref, f"{cfg} layer {l}")
+                np.testing.assert_allclose(got[l][1][rows[:, 0], rows[:, 1], rows[:, 2]], rlse, rtol=2e-3, atol=2e-3)
+            # every row of the layer against the one-layer call (itself checked against the checker above
+            # and elsewhere): per row, so that one wrong (sequence, KV head) group cannot hide in an average
+            single, _, status = gpu_attention(w, layer=l)
+            assert status == 0
+            d = np.linalg.norm(got[l][0].astype(np.float64) - single, axis=-1)
+            ref_norm = np.linalg.norm(single.astype(np.float64), axis=-1)
+            assert (d <= 1e-2 * ref_norm + 1e-6).all(), f"{cfg} layer {l}: rows differ from the one-layer call"
+
+
+@pytest.mark.parametrize("L,lens,n_nodes", [(33, (130, 61), (24, 9)), (30, (300, 61, 190), (24, 9, 17))])
+def test_attention_layers_call_many_layers_ragged(L, lens, n_nodes):
+    """Ragged lengths, unused nodes, shuffled blocks, every layer against the checker.  First case:
+    more layers than one launch holds (33 > 32).  Second case: 30 layers x 3 sequences x 2 KV heads x
+    2 row tiles = 360 CTAs, more than one round of the 296 resident ones, so the call is issued as a
+    launch of whole-sequence CTAs plus the remainder (the shortest sequence's last layers) in key chunks."""
+    B = len(lens)
     g = np.random.default_rng(21)
     T = 24
-    par = np.stack([np.array([-1] + [int(g.integers(max(0, i - 5), i)) for i in range(1, T)]) for _ in range(2)])
-    w = tiny128(100, B=2, T=T, Hq=14, Hkv=2, lens=(130, 61), parents=par, gain=3.0)
-    w.n_nodes = np.array([24, 9], dtype=np.int32)
+    par = np.stack([np.array([-1] + [int(g.integers(max(0, i - 5), i)) for i in range(1, T)]) for _ in range(B)])
+    w = tiny128(100, B=B, T=T, Hq=14, Hkv=2, lens=lens, parents=par, gain=3.0)
+    w.n_nodes = np.array(n_nodes, dtype=np.int32)
 
     class Layer:
         pass
@@ -299,7 +327,7 @@ def test_attention_layers_call_many_layers_ragged():
         check_attention(got[l][0], ref, f"layer {l}")
         ok = np.isfinite(rlse)
         np.testing.assert_allclose(got[l][1][ok], rlse[ok], rtol=2e-3, atol=2e-3)
-        assert (got[l][0][1, 9:] == 0).all()
+        assert (got[l][0][1, 9:] == 0).all()                     # rows of unused nodes are zeroed
 
 
 # ------------------------------------------------------------------ LM head
