@@ -18,14 +18,15 @@ replacement:
       uniform w:  the first token t whose cumulative remaining mass reaches w * R.
 
 Every random number is an input (u per node, w per sequence).  Plain numpy,
-fp64 unless a dtype is passed; no code shared with the GPU library.  Siblings
-must carry distinct tokens.
+fp64 throughout; no code shared with the GPU library.  Siblings must carry
+distinct tokens.
 
 Parity with the paper's own acceptance statistics is unpinned (they need the
-trained models).  The functions are pinned in tests/test_oracle_sampling.py by
-Monte-Carlo frequencies against p, by the zero-temperature limit (the greedy
-rule), by the single-child case (the textbook accept test) and by numpy's
-cumsum/searchsorted for the inverse CDF.
+trained models).  The functions are pinned in tests/test_oracle_sampling.py:
+softmax_rows against torch's log_softmax / logsumexp in fp64, scipy's softmax
+and a hand-computed case; the rule by Monte-Carlo frequencies against p, by the
+zero-temperature limit (the greedy rule), by the single-child case (the
+textbook accept test) and by numpy's cumsum/searchsorted for the inverse CDF.
 """
 from __future__ import annotations
 
@@ -45,34 +46,35 @@ def children_of(parents: np.ndarray, n: int, i: int):
     return [j for j in range(i + 1, n) if parents[j] == i]
 
 
-def accept_walk(parents, n_nodes, draft_tok, p_child, u, dtype=np.float64):
-    """The acceptance walk of ONE sequence.
+def accept_walk(parents, n_nodes, draft_tok, p_child, u):
+    """The acceptance walk of ONE sequence, fp64.
 
     p_child[j] = probability of draft_tok[j] under the target distribution at parent(j) (j >= 1),
-    u[j] = the uniform drawn for node j.  The comparison u * R < p and the update R -= p are done in
-    `dtype` (fp64 for the definition; float32 reproduces the kernel's arithmetic bit for bit).
-    Returns (path, R): the accepted root path and the residual mass left at its last node.
+    u[j] = the uniform drawn for node j.
+    Returns (path, R, margin): the accepted root path, the residual mass left at its last node, and
+    the smallest |u * R - p| over the comparisons the walk made (how close its closest decision was;
+    infinity when it made none).
     """
     parents = np.asarray(parents)
-    p_child = np.asarray(p_child, dtype=dtype)
-    u = np.asarray(u, dtype=dtype)
+    p_child = np.asarray(p_child, dtype=np.float64)
+    u = np.asarray(u, dtype=np.float64)
     n = int(n_nodes)
     cur, path = 0, [0]
-    one = dtype(1.0)
-    R = one
+    margin = np.inf
     while True:
         nxt = -1
-        R = one
+        R = 1.0
         kids = children_of(parents, n, cur)
         toks = [int(draft_tok[c]) for c in kids]
         assert len(set(toks)) == len(toks), "siblings must carry distinct tokens"
         for c in kids:
-            if dtype(u[c] * R) < p_child[c]:
+            margin = min(margin, abs(u[c] * R - p_child[c]))
+            if u[c] * R < p_child[c]:
                 nxt = c
                 break
-            R = dtype(R - p_child[c])
+            R = R - p_child[c]
         if nxt < 0:
-            return path, R
+            return path, R, margin
         cur = nxt
         path.append(cur)
 
@@ -107,7 +109,7 @@ def verify_sequence(parents, n_nodes, draft_tok, logits, inv_temp, u, w):
     p_child = np.zeros(len(parents))
     for j in range(1, n):
         p_child[j] = p[parents[j], draft_tok[j]]
-    path, R = accept_walk(parents, n, draft_tok, p_child, u)
+    path, R, _ = accept_walk(parents, n, draft_tok, p_child, u)
     last = path[-1]
     excl = [int(draft_tok[c]) for c in children_of(parents, n, last)]
     t, _ = residual_sample(p[last], excl, R, w)

@@ -87,9 +87,7 @@ def run_sampled(w, tok, inv_temp, u, wv, groups=True):
     sd.sd_accept_tree_sampled(bt, h, Wd, inv_temp, lse, to_device(tok), to_device(u), to_device(wv),
                               n_acc, path, out_tok, new_len, ws, st, group_stats=gs)
     torch.cuda.synchronize()
-    p_child = ws[:B * T * 4].view(torch.float32).cpu().numpy().reshape(B, T)      # first area of the workspace
-    return (n_acc.cpu().numpy(), path.cpu().numpy(), out_tok.cpu().numpy(), new_len.cpu().numpy(),
-            p_child, int(st.item()))
+    return (n_acc.cpu().numpy(), path.cpu().numpy(), out_tok.cpu().numpy(), new_len.cpu().numpy(), int(st.item()))
 
 
 @pytest.mark.parametrize("cfg,over,inv_temp", [
@@ -111,30 +109,26 @@ def test_sampled_acceptance_against_the_reference(cfg, over, inv_temp, groups):
     for rep in range(3 if B > 1 else 25):
         u = g.random((B, T)).astype(np.float32)
         wv = g.random(B).astype(np.float32)
-        n_acc, path, out_tok, new_len, p_child, status = run_sampled(w, tok, inv_temp, u, wv, groups)
+        n_acc, path, out_tok, new_len, status = run_sampled(w, tok, inv_temp, u, wv, groups)
         assert status == 0
         close_calls = 0
         for b in range(B):
             n = int(w.n_nodes[b])
             par = w.parents[b]
-            # (1) the probabilities the kernel compared against
-            for j in range(1, n):
-                ref = p64[b * T + par[j], tok[b, j]]
-                assert abs(p_child[b, j] - ref) <= 1e-4 * ref + 1e-7, (b, j, p_child[b, j], ref)
-            # (2) the walk, bit for bit, in the kernel's arithmetic on the kernel's probabilities
-            pth32, R32 = smp.accept_walk(par, n, tok[b], p_child[b], u[b], dtype=np.float32)
-            assert list(path[b, :n_acc[b]]) == pth32 and (path[b, n_acc[b]:] == -1).all()
-            assert new_len[b] == w.len[b] + n_acc[b]
-            assert list(out_tok[b, :n_acc[b] - 1]) == [int(tok[b, j]) for j in pth32[1:]]
-            # (3) against the fp64 definition: same path unless some comparison was a close call
+            # the walk against the fp64 definition: same path unless one of its comparisons was a close call
             pc64 = np.zeros(T)
             for j in range(1, n):
                 pc64[j] = p64[b * T + par[j], tok[b, j]]
-            pth64, R64 = smp.accept_walk(par, n, tok[b], pc64, u[b].astype(np.float64))
-            if pth64 != pth32:
+            pth64, R64, walk_margin = smp.accept_walk(par, n, tok[b], pc64, u[b].astype(np.float64))
+            assert (path[b, n_acc[b]:] == -1).all()
+            assert new_len[b] == w.len[b] + n_acc[b]
+            got_path = [int(x) for x in path[b, :n_acc[b]]]
+            assert list(out_tok[b, :n_acc[b] - 1]) == [int(tok[b, j]) for j in got_path[1:]]
+            if got_path != pth64:
+                assert walk_margin <= CLOSE, (b, got_path, pth64, walk_margin)
                 close_calls += 1
                 continue
-            # (4) the drawn token: inverse CDF over the stop row without its drafted children
+            # the drawn token: inverse CDF over the stop row without its drafted children
             last = pth64[-1]
             excl = [int(tok[b, c]) for c in smp.children_of(par, n, last)]
             t_ref, margin = smp.residual_sample(p64[b * T + last], excl, R64, float(wv[b]))
@@ -159,7 +153,7 @@ def test_sampled_zero_temperature_equals_greedy_acceptance():
     g = np.random.default_rng(3)
     u = (g.random((w.B, w.T_max)) * 0.98 + 0.01).astype(np.float32)
     wv = (g.random(w.B) * 0.98 + 0.01).astype(np.float32)
-    n_acc, path, out_tok, new_len, _, status = run_sampled(w, w.draft_tok, 4000.0, u, wv)
+    n_acc, path, out_tok, new_len, status = run_sampled(w, w.draft_tok, 4000.0, u, wv)
     assert status == 0
     for got, want in zip((n_acc, path, out_tok, new_len), ref):
         np.testing.assert_array_equal(got, want)
@@ -181,8 +175,8 @@ def test_sampled_bad_inputs_are_reported():
 
 @pytest.mark.parametrize("groups", [True, False])
 def test_sampled_full_size_c5(groups):
-    """Vocabulary 152064, 8 x 60-node trees: the walk bit for bit on the kernel's own probabilities,
-    those probabilities and the drawn tokens against fp64 logits of the rows the walks visited."""
+    """Vocabulary 152064, 8 x 60-node trees: the walk and the drawn tokens against the fp64 rule on
+    fp64 logits; a differing decision must be a close call of the fp64 walk, and at most one may occur."""
     w = wl.make("c5", attention=False, hidden_gain=40.0)
     B, T, V = w.B, w.T_max, w.V
     ram, t1, t2 = oracle.lmhead(w.hidden, w.W)                   # good drafts: children get the arg-max first
@@ -198,29 +192,35 @@ def test_sampled_full_size_c5(groups):
     inv_temp = 6.0
     u = g.random((B, T)).astype(np.float32)
     wv = g.random(B).astype(np.float32)
-    n_acc, path, out_tok, new_len, p_child, status = run_sampled(w, tok, inv_temp, u, wv, groups)
+    n_acc, path, out_tok, new_len, status = run_sampled(w, tok, inv_temp, u, wv, groups)
     assert status == 0
-    visited = sorted({b * T + int(path[b, k]) for b in range(B) for k in range(n_acc[b])})
-    lg = oracle.logits(w.hidden[visited], w.W)
-    p64, _ = smp.softmax_rows(lg, inv_temp)
-    row_of = {r: i for i, r in enumerate(visited)}
+    # fp64 probabilities of the rows the rule may look at: every parent (child probabilities) and every
+    # node a walk stopped at (the residual draw)
+    rows = sorted({b * T + int(w.parents[b][j]) for b in range(B) for j in range(1, int(w.n_nodes[b]))}
+                  | {b * T + int(path[b, k]) for b in range(B) for k in range(n_acc[b])})
+    p64, _ = smp.softmax_rows(oracle.logits(w.hidden[rows], w.W), inv_temp)
+    row_of = {r: i for i, r in enumerate(rows)}
     moved = 0
+    close_calls = 0
     for b in range(B):
         n, par = int(w.n_nodes[b]), w.parents[b]
-        pth32, R32 = smp.accept_walk(par, n, tok[b], p_child[b], u[b], dtype=np.float32)
-        assert list(path[b, :n_acc[b]]) == pth32
-        for i in pth32:                                           # children of visited nodes
-            for c in smp.children_of(par, n, i):
-                ref = p64[row_of[b * T + i], tok[b, c]]
-                assert abs(p_child[b, c] - ref) <= 2e-4 * ref + 1e-7
-        last = pth32[-1]
+        pc64 = np.zeros(T)
+        for j in range(1, n):
+            pc64[j] = p64[row_of[b * T + int(par[j])], tok[b, j]]
+        pth64, R64, walk_margin = smp.accept_walk(par, n, tok[b], pc64, u[b].astype(np.float64))
+        got_path = [int(x) for x in path[b, :n_acc[b]]]
+        if got_path != pth64:
+            assert walk_margin <= CLOSE, (b, got_path, pth64, walk_margin)
+            close_calls += 1
+            continue
+        last = pth64[-1]
         excl = [int(tok[b, c]) for c in smp.children_of(par, n, last)]
-        t_ref, margin = smp.residual_sample(p64[row_of[b * T + last]], excl, float(R32), float(wv[b]))
+        t_ref, margin = smp.residual_sample(p64[row_of[b * T + last]], excl, float(R64), float(wv[b]))
         got = int(out_tok[b, n_acc[b] - 1])
         assert got not in excl
         assert got == t_ref or margin <= CLOSE, (b, got, t_ref, margin)
         moved += n_acc[b] - 1
-    assert moved > 0
+    assert moved > 0 and close_calls <= 1
 
 
 def test_sampled_gpu_output_frequencies_follow_the_target_distribution():
@@ -252,7 +252,7 @@ def test_sampled_gpu_output_frequencies_follow_the_target_distribution():
     for rep in range(reps):
         u = g.random((B, T)).astype(np.float32)
         wv = g.random(B).astype(np.float32)
-        n_acc, path, out_tok, new_len, _, status = run_sampled(w, tok, inv_temp, u, wv)
+        n_acc, path, out_tok, new_len, status = run_sampled(w, tok, inv_temp, u, wv)
         assert status == 0
         np.add.at(counts, out_tok[:, 0], 1)
     n = B * reps

@@ -102,16 +102,74 @@ def test_inverse_cdf_against_cumsum_searchsorted():
     assert smp.residual_sample(p, [0], 0.8, 1e-9)[0] == 2
 
 
-def test_walk_in_float32_differs_only_on_close_calls():
-    """The float32 variant (the kernel's arithmetic) takes the same decisions as the fp64 definition
-    except where u * R is within rounding of p."""
+def test_walk_margin_is_the_closest_comparison():
+    """The margin the walk reports bounds how far an input may move before the path changes: shifting
+    every probability by less than the margin leaves the path as it is."""
     g = np.random.default_rng(5)
-    diff = 0
     for seed in range(200):
         t = Tiny(seed, B=1, T=12, lens=(3,))
         pc = g.random(12) * 0.6
         u = g.random(12)
-        a, Ra = smp.accept_walk(t.parents[0], 12, np.arange(12), pc, u)
-        b, Rb = smp.accept_walk(t.parents[0], 12, np.arange(12), pc.astype(np.float32), u.astype(np.float32), dtype=np.float32)
-        diff += (a != b)
-    assert diff <= 1
+        a, Ra, margin = smp.accept_walk(t.parents[0], 12, np.arange(12), pc, u)
+        if not np.isfinite(margin):
+            continue
+        eps = 0.1 * margin          # residuals accumulate at most a handful of shifted probabilities
+        for sign in (-1.0, 1.0):
+            b, _, _ = smp.accept_walk(t.parents[0], 12, np.arange(12), np.clip(pc + sign * eps, 0, 1), u)
+            assert a == b
+
+
+# ---------------------------------------------------------------- the probabilities themselves
+def check_softmax_against_libraries(softmax_rows):
+    """softmax_rows(logits, inv_temp) -> (p, lse) against routines that share nothing with it:
+    torch.log_softmax / torch.logsumexp in fp64, scipy.special.softmax, and a case worked by hand."""
+    import torch
+    from scipy import special
+    g = np.random.default_rng(6)
+    for shape, inv_temp, gain in (((3, 7), 1.0, 1.0), ((5, 129), 0.37, 4.0), ((2, 1000), 6.0, 2.0), ((4, 1), 2.0, 1.0),
+                                  ((2, 33), 40.0, 30.0)):
+        lg = g.standard_normal(shape) * gain
+        p, lse = softmax_rows(lg, inv_temp)
+        z = torch.from_numpy(lg).double() * inv_temp
+        np.testing.assert_allclose(p, torch.log_softmax(z, dim=-1).exp().numpy(), rtol=1e-12, atol=1e-300)
+        np.testing.assert_allclose(lse, torch.logsumexp(z, dim=-1).numpy(), rtol=1e-13, atol=1e-13)
+        np.testing.assert_allclose(p, special.softmax(lg * inv_temp, axis=-1), rtol=1e-12, atol=1e-300)
+        np.testing.assert_allclose(p.sum(-1), 1.0, rtol=1e-13)
+    # by hand: logits (0, 1) at inverse temperature ln 2 are exponents (0, ln 2): weights 1 and 2
+    p, lse = softmax_rows(np.array([[0.0, 1.0]]), np.log(2.0))
+    np.testing.assert_allclose(p, [[1 / 3, 2 / 3]], rtol=1e-15)
+    np.testing.assert_allclose(lse, [np.log(3.0)], rtol=1e-15)
+    # three equal logits: uniform, lse = c * inv_temp + ln 3 (no overflow at a large offset)
+    p, lse = softmax_rows(np.full((1, 3), 800.0), 1.5)
+    np.testing.assert_allclose(p, np.full((1, 3), 1 / 3), rtol=1e-15)
+    np.testing.assert_allclose(lse, [1200.0 + np.log(3.0)], rtol=1e-15)
+
+
+def test_softmax_rows_against_torch_scipy_and_a_hand_case():
+    check_softmax_against_libraries(smp.softmax_rows)
+
+
+def test_softmax_pins_catch_planted_mistakes():
+    """The same checks must reject plausible wrong versions of softmax_rows (planted here, on the CPU)."""
+    import pytest
+
+    def squared_temperature(lg, it):
+        return smp.softmax_rows(lg, it * it)
+
+    def base_two(lg, it):
+        z = np.asarray(lg, dtype=np.float64) * it
+        m = z.max(-1, keepdims=True)
+        e = np.exp2(z - m)
+        s = e.sum(-1, keepdims=True)
+        return e / s, (m + np.log2(s))[..., 0]
+
+    def lse_without_the_maximum(lg, it):
+        p, lse = smp.softmax_rows(lg, it)
+        return p, lse - (np.asarray(lg) * it).max(-1)
+
+    def temperature_divides(lg, it):
+        return smp.softmax_rows(lg, 1.0 / it)
+
+    for wrong in (squared_temperature, base_two, lse_without_the_maximum, temperature_divides):
+        with pytest.raises(AssertionError):
+            check_softmax_against_libraries(wrong)
