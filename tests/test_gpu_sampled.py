@@ -12,7 +12,9 @@ from paper_2509_18824_b200.step import to_device
 
 pytestmark = pytest.mark.gpu
 
-CLOSE = 2e-5          # a comparison u * R < p (or a CDF crossing) nearer than this may fall either way in fp32
+CLOSE = 2e-5          # a CDF crossing nearer than this may fall either way in fp32
+WALK_CLOSE = 2e-4     # a comparison u * R < p nearer than this may fall either way: the kernel's p (fp32 dot product
+                      # of 3584 terms, ex2.approx) is within 1e-4 relative of the fp64 value
 
 
 def run_stats(hidden, W, inv_temp):
@@ -125,7 +127,7 @@ def test_sampled_acceptance_against_the_reference(cfg, over, inv_temp, groups):
             got_path = [int(x) for x in path[b, :n_acc[b]]]
             assert list(out_tok[b, :n_acc[b] - 1]) == [int(tok[b, j]) for j in got_path[1:]]
             if got_path != pth64:
-                assert walk_margin <= CLOSE, (b, got_path, pth64, walk_margin)
+                assert walk_margin <= WALK_CLOSE, (b, got_path, pth64, walk_margin)
                 close_calls += 1
                 continue
             # the drawn token: inverse CDF over the stop row without its drafted children
@@ -210,7 +212,7 @@ def test_sampled_full_size_c5(groups):
         pth64, R64, walk_margin = smp.accept_walk(par, n, tok[b], pc64, u[b].astype(np.float64))
         got_path = [int(x) for x in path[b, :n_acc[b]]]
         if got_path != pth64:
-            assert walk_margin <= CLOSE, (b, got_path, pth64, walk_margin)
+            assert walk_margin <= WALK_CLOSE, (b, got_path, pth64, walk_margin)
             close_calls += 1
             continue
         last = pth64[-1]
