@@ -1,7 +1,19 @@
 // C-ABI entry points: argument validation, then the kernel launchers.
 #include "common.cuh"
 
+#include <stdlib.h>
+
 using namespace sdv;
+
+namespace sdv {
+TestKnobs test_knobs() {
+    TestKnobs k{1ll << 31, 0, 0};
+    if (const char* e = getenv("SDV_TEST_WAIT_CYCLES")) { const long long v = atoll(e); if (v >= 1000) k.wait_cycles = v; }
+    if (const char* e = getenv("SDV_TEST_WITHHOLD")) k.withhold = atoi(e) == 1 ? 1 : 0;
+    if (const char* e = getenv("SDV_TEST_CHUNKS")) { const int v = atoi(e); if (v == 1 || v == 2 || v == 4 || v == 8) k.chunks = v; }
+    return k;
+}
+}  // namespace sdv
 
 namespace {
 

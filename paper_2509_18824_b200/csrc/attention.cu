@@ -17,13 +17,10 @@
 // With one chunk the CTA writes the output itself; otherwise the chunks of a row
 // tile form a thread-block cluster and merge their (max, sum, unnormalised O)
 // through distributed shared memory in a fixed order.
-#include "common.cuh"
-#include "sm100.cuh"
+#include "attention_shared.cuh"
 
 namespace sdv {
-using namespace sm100;
 
-constexpr int kRowTile = 128;                  // query rows per CTA (MMA M)
 constexpr int kKeyTile = 64;                   // keys per tile = one cache block
 constexpr int kAttThreads = 161;               // warps 0-3 softmax, warp 4 TMA, warp 5 = ONE thread: MMA issuer
 constexpr int kTmaWarp = 4, kMmaWarp = 5;
@@ -35,166 +32,6 @@ constexpr int kVStages = 2;
 constexpr int kAttSmem = kQBytes + (kKStages + kVStages) * kKVStage + 256;
 constexpr int kTmemCols = 256;                 // O: 0..127, S/P buffers: 128..191, 192..255
 // P (bf16, two keys per 32-bit column) overwrites the first 32 columns of the S buffer it came from
-constexpr float kLog2e = 1.4426950408889634f;
-constexpr float kRescaleThreshold = 8.0f;      // log2 units
-constexpr int kMaxChunks = 8;                  // = portable cluster size
-constexpr int kSplitRounds = 8;                // launches of fewer whole rounds get their remainder as a chunked launch
-
-__device__ __forceinline__ float max3(float a, float b, float c) {
-    float d;
-    asm("max.f32 %0, %1, %2, %3;" : "=f"(d) : "f"(a), "f"(b), "f"(c));
-    return d;
-}
-__device__ __forceinline__ float ex2_approx(float x) {
-    float y;
-    asm("ex2.approx.ftz.f32 %0, %1;" : "=f"(y) : "f"(x));
-    return y;
-}
-
-struct AttnPlan {
-    int n_chunks;      // key chunks per sequence (the last one also takes the tree tile)
-    int rows;          // T_max * G
-    int row_tiles;
-    int n_layers;      // layers of this launch
-    int ranked;        // dispatch the sequences longest first (only matters when the grid runs in several waves)
-    int z0;            // first (sequence rank, layer, KV head) index of this launch: blockIdx.z counts from here
-};
-
-static AttnPlan make_plan(const sd_batch& bt, int n_layers, int sms) {
-    AttnPlan p;
-    const int G = bt.Hq / bt.Hkv;
-    p.rows = bt.T_max * G;
-    p.row_tiles = (p.rows + kRowTile - 1) / kRowTile;
-    // Pick the chunk count that minimises (waves of CTAs) x (key tiles per CTA + fixed cost),
-    // two CTAs being resident per SM.  Few waves are counted whole; many waves balance out.
-    const int max_tiles = bt.max_blocks_per_seq;
-    const int base = n_layers * bt.B * bt.Hkv * p.row_tiles;
-    const int slots = 2 * sms;
-    int n = 1;
-    double best = 1e30;
-    for (int c = 1; c <= kMaxChunks && c <= max_tiles; c *= 2) {   // 128 rows split evenly over the chunks
-        const double w = (double)base * c / slots;
-        double waves = (w <= 4.0) ? (double)((base * c + slots - 1) / slots) : w;
-        // Without chunks, and for up to kSplitRounds whole rounds, the CTAs left over after the last whole
-        // round go into a launch of their own, with chunks (launch_group): the partial round then costs
-        // a fraction of a round.  (Longer launches run under the power cap, where this gained nothing.)
-        if (c == 1 && w > 1.0 && base / slots < kSplitRounds) {
-            const int rest = base % slots;
-            int ct = 1;                                    // chunks of the remainder's launch
-            while (2 * ct <= kMaxChunks && 2 * ct <= max_tiles && rest * 2 * ct <= slots) ct *= 2;
-            waves = (double)(base / slots) + (rest == 0 ? 0.0 : (ct > 1 ? 1.0 / ct + 0.1 : 1.0));
-        }
-        // per CTA: its key tiles, a fixed cost of about three tiles, and two more for the in-cluster merge
-        const double cost = waves * ((max_tiles + c - 1) / c + 3 + (c > 1 ? 2 : 0));
-        if (cost < best - 1e-9) { best = cost; n = c; }
-    }
-    p.n_chunks = n;
-    p.n_layers = n_layers;
-    p.ranked = (bt.B > 1 && bt.B <= 64 && (long long)base * n > slots) ? 1 : 0;
-    p.z0 = 0;
-    return p;
-}
-
-static int sm_count() {
-    static int sms = 0;
-    if (sms == 0) {
-        int dev = 0;
-        if (cudaGetDevice(&dev) != cudaSuccess ||
-            cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev) != cudaSuccess || sms <= 0)
-            sms = 148;
-    }
-    return sms;
-}
-
-// The chunks of a row tile are merged inside a thread-block cluster, through shared memory:
-// attention needs no global scratch (a nominal size keeps the argument checks uniform).
-size_t attention_workspace_bytes(const sd_batch&) { return 256; }
-
-// Everything the CTAs of one layer need.  A launch covers up to kMaxLayersPerLaunch layers (the
-// descriptors travel as kernel parameters); blockIdx.z enumerates (sequence, layer, KV head).
-struct AttnLayer {
-    CUtensorMap k_cache, v_cache;   // 2-D [num_blocks*Hkv*64][128], box 64 x 64
-    CUtensorMap k_tree, v_tree;     // 3-D (128, Hkv, B*T_max), box 64 x 1 x 64
-    const uint16_t* q;              // bf16 [B][T_max][Hq][D]
-    __nv_bfloat16* out;             // bf16 [B][T_max][Hq][D]
-    float* lse;                     // f32  [B][T_max][Hq] or null
-    int32_t num_blocks;
-};
-constexpr int kMaxLayersPerLaunch = 32;
-template <int NL>
-struct AttnLayers { AttnLayer l[NL]; };
-
-// Final step of a clustered launch.  Each CTA of the cluster finishes 128 / NCH rows of the tile: a
-// warp takes a few rows at a time, every lane four output columns, and adds up the chunks in chunk
-// order (so the result does not depend on timing).  A row of a parked tile is one contiguous
-// 512-byte line of the owning CTA's shared memory; all loads of a batch of rows are issued before
-// any of them is used, so that their latencies overlap.
-struct MergeCtx {
-    const sd_batch& bt; const AttnPlan& plan; __nv_bfloat16* out; float* lse;
-    uint32_t xo_addr, xs_addr;
-    int chunk, rt, b, kvh, n, tpc, tiles_total, warp, lane;
-};
-
-template <int NCH>
-__device__ __forceinline__ void merge_rows(const MergeCtx& x) {
-    constexpr int kRowsPer = kRowTile / NCH;
-    constexpr int kBatch = 16 / NCH;                // rows in flight per warp
-    const int G = x.bt.Hq / x.bt.Hkv;
-    for (int i0 = x.warp * kBatch; i0 < kRowsPer; i0 += 4 * kBatch) {
-        float mc[kBatch][NCH], lc[kBatch][NCH];
-        float4 v[kBatch][NCH];
-#pragma unroll
-        for (int u = 0; u < kBatch; ++u) {
-            const int r = x.chunk * kRowsPer + i0 + u;
-#pragma unroll
-            for (int c = 0; c < NCH; ++c) {
-                const bool live = (c == NCH - 1) || (c * x.tpc < x.tiles_total);   // that chunk had key tiles
-                mc[u][c] = -INFINITY; lc[u][c] = 0.f; v[u][c] = make_float4(0.f, 0.f, 0.f, 0.f);
-                if (live && c == x.chunk) {                  // this CTA's own chunk: plain shared-memory reads
-                    mc[u][c] = ld_smem_f32(x.xs_addr + r * 4);
-                    lc[u][c] = ld_smem_f32(x.xs_addr + (kRowTile + r) * 4);
-                    v[u][c] = ld_smem_v4(x.xo_addr + (uint32_t)(r * kD + ((x.lane ^ (r & 31)) << 2)) * 4);
-                } else if (live) {
-                    mc[u][c] = ld_dsmem_f32(map_dsmem(x.xs_addr + r * 4, c));
-                    lc[u][c] = ld_dsmem_f32(map_dsmem(x.xs_addr + (kRowTile + r) * 4, c));
-                    v[u][c] = ld_dsmem_v4(map_dsmem(x.xo_addr + (uint32_t)(r * kD + ((x.lane ^ (r & 31)) << 2)) * 4, c));
-                }
-            }
-        }
-#pragma unroll
-        for (int u = 0; u < kBatch; ++u) {
-            const int r = x.chunk * kRowsPer + i0 + u;
-            const int row = x.rt * kRowTile + r;
-            if (row >= x.plan.rows) continue;
-            const int node = row / G;
-            const int g = row - node * G;
-            const size_t orow = ((size_t)x.b * x.bt.T_max + node) * x.bt.Hq + x.kvh * G + g;
-            uint2* dst = reinterpret_cast<uint2*>(x.out + orow * kD + x.lane * 4);
-            if (node >= x.n) {                               // unused node: zero row
-                *dst = make_uint2(0, 0);
-                if (x.lse && x.lane == 0) x.lse[orow] = 0.f;
-                continue;
-            }
-            float M = mc[u][0];
-#pragma unroll
-            for (int c = 1; c < NCH; ++c) M = fmaxf(M, mc[u][c]);
-            float den = 0.f;
-            float4 acc = make_float4(0.f, 0.f, 0.f, 0.f);
-#pragma unroll
-            for (int c = 0; c < NCH; ++c) {
-                const float w = exp2f(mc[u][c] - M);         // 0 for a chunk without tiles (m = -inf)
-                den = fmaf(w, lc[u][c], den);
-                acc.x = fmaf(w, v[u][c].x, acc.x); acc.y = fmaf(w, v[u][c].y, acc.y);
-                acc.z = fmaf(w, v[u][c].z, acc.z); acc.w = fmaf(w, v[u][c].w, acc.w);
-            }
-            const float inv = 1.f / den;
-            __nv_bfloat162 h0 = __floats2bfloat162_rn(acc.x * inv, acc.y * inv);
-            __nv_bfloat162 h1 = __floats2bfloat162_rn(acc.z * inv, acc.w * inv);
-            *dst = make_uint2(*reinterpret_cast<uint32_t*>(&h0), *reinterpret_cast<uint32_t*>(&h1));
-            if (x.lse && x.lane == 0) x.lse[orow] = (M + log2f(den)) * 0.6931471805599453f;
-        }
-    }
-}
 
 template <int NL>
 __global__ void __launch_bounds__(kAttThreads, 2)
@@ -266,7 +103,11 @@ attn_umma_kernel(const __grid_constant__ AttnLayers<NL> layers, const sd_batch b
     const int len = max(bt.len[b], 0);
 
     // key tiles of this CTA: cache blocks [t0, t1) and, for the last chunk, the tree tile
-    const int tiles_total = min((len + kKeyTile - 1) / kKeyTile, bt.max_blocks_per_seq);
+    int tiles_total = (len + kKeyTile - 1) / kKeyTile;
+    if (tiles_total > bt.max_blocks_per_seq) {             // the block table does not cover this length
+        if (threadIdx.x == 0) set_status(status, SD_ERR_BOUNDS);
+        tiles_total = bt.max_blocks_per_seq;
+    }
     const int tpc = (tiles_total + plan.n_chunks - 1) / plan.n_chunks;
     const int t0 = min(chunk * tpc, tiles_total);
     const int t1 = min(t0 + tpc, tiles_total);
@@ -356,7 +197,7 @@ attn_umma_kernel(const __grid_constant__ AttnLayers<NL> layers, const sd_batch b
                 }
                 if (progress) {
                     t_last = clock64();
-                } else if (*reinterpret_cast<volatile int*>(abort_flag) || clock64() - t_last > kWaitCycles) {
+                } else if (*reinterpret_cast<volatile int*>(abort_flag) || clock64() - t_last > plan.wait_cycles) {
                     *reinterpret_cast<volatile int*>(abort_flag) = 1;
                     ok = false;
                 }
@@ -380,11 +221,11 @@ attn_umma_kernel(const __grid_constant__ AttnLayers<NL> layers, const sd_batch b
             const uint64_t kdesc_base = make_smem_desc(smem_u32(k_smem), 16, 1024, 128);
             // V is stored [key][d]: N (= d) contiguous; D-halves kSubTile apart, 8-key groups 1 KiB apart
             const uint64_t vdesc_base = make_smem_desc(smem_u32(v_smem), kSubTile, 1024, 128);
-            bool ok = mbar_wait(q_full, 0, abort_flag);
+            bool ok = mbar_wait(q_full, 0, abort_flag, plan.wait_cycles);
             auto issue_s = [&](int j) -> bool {
                 const int s = j & 1;                               // score buffer
                 const int ks = j % kKStages;                       // K ring slot
-                if (!mbar_wait(&k_full[ks], (uint32_t)(j / kKStages) & 1u, abort_flag)) return false;
+                if (!mbar_wait(&k_full[ks], (uint32_t)(j / kKStages) & 1u, abort_flag, plan.wait_cycles)) return false;
                 tc_fence_after_sync();
                 const uint64_t kd = kdesc_base + (uint64_t)(ks * (kKVStage >> 4));
                 const uint32_t d = tmem_s + s * kKeyTile;
@@ -402,9 +243,9 @@ attn_umma_kernel(const __grid_constant__ AttnLayers<NL> layers, const sd_batch b
                 if (!ok) break;
                 const int s = j & 1;
                 const uint32_t ph = (uint32_t)(j >> 1) & 1u;
-                if (!mbar_wait(&p_full[s], ph, abort_flag)) { ok = false; break; }
+                if (!mbar_wait(&p_full[s], ph, abort_flag, plan.wait_cycles)) { ok = false; break; }
                 const int vs = j % kVStages;
-                if (!mbar_wait(&v_full[vs], (uint32_t)(j / kVStages) & 1u, abort_flag)) { ok = false; break; }
+                if (!mbar_wait(&v_full[vs], (uint32_t)(j / kVStages) & 1u, abort_flag, plan.wait_cycles)) { ok = false; break; }
                 tc_fence_after_sync();
                 const uint64_t vd = vdesc_base + (uint64_t)(vs * (kKVStage >> 4));
                 const uint32_t pa = tmem_s + s * kKeyTile;        // P comes straight from TMEM: 16 keys = 8 columns
@@ -415,8 +256,12 @@ attn_umma_kernel(const __grid_constant__ AttnLayers<NL> layers, const sd_batch b
                 mma_commit(&v_empty[vs]);
                 mma_commit(pv_done);
             }
-            if (ok) mma_commit(o_full);
-            if (!ok) set_status(status, SD_ERR_TIMEOUT);
+            mma_commit(o_full);
+            if (!ok) {
+                // unwinding: nothing may give tensor memory back while an MMA issued above still runs
+                set_status(status, SD_ERR_TIMEOUT);
+                mbar_wait_plain(o_full, 0, plan.wait_cycles);
+            }
         }
     } else if (warp < 4) {
         // ------------------------------------------------------------ softmax: one thread per row
@@ -447,7 +292,7 @@ attn_umma_kernel(const __grid_constant__ AttnLayers<NL> layers, const sd_batch b
             const uint32_t ph = (uint32_t)(j >> 1) & 1u;
             const bool tree = (j >= t1 - t0);
             const int valid = tree ? kKeyTile : len - (t0 + j) * kKeyTile;   // keys of this block inside the prefix
-            if (!mbar_wait(&s_full[s], ph, abort_flag)) { ok = false; break; }
+            if (!mbar_wait(&s_full[s], ph, abort_flag, plan.wait_cycles)) { ok = false; break; }
             tc_fence_after_sync();
             // Keys that no row may see (cache slots at and beyond len, rows of unused tree nodes) carry
             // weight 0, but 0 x NaN or 0 x Inf would still poison the accumulator: their V rows are
@@ -460,7 +305,7 @@ attn_umma_kernel(const __grid_constant__ AttnLayers<NL> layers, const sd_batch b
             const int v_rows = tree ? n : valid;
             if (v_rows < kKeyTile && warp < 2) {                     // threads 0..63 <-> key rows
                 const int vs = j % kVStages;
-                if (!mbar_wait(&v_full[vs], (uint32_t)(j / kVStages) & 1u, abort_flag)) { ok = false; break; }
+                if (!mbar_wait(&v_full[vs], (uint32_t)(j / kVStages) & 1u, abort_flag, plan.wait_cycles)) { ok = false; break; }
                 if (tid >= v_rows) {
                     uint4* z = reinterpret_cast<uint4*>(v_smem + vs * kKVStage + tid * 128);
 #pragma unroll
@@ -526,7 +371,7 @@ attn_umma_kernel(const __grid_constant__ AttnLayers<NL> layers, const sd_batch b
             const bool raise = (row_in_tile >= 0) && (mt > m_used + kRescaleThreshold);
             if (__any_sync(0xffffffffu, raise)) {
                 if (j > 0) {
-                    if (!mbar_wait(pv_done, (uint32_t)(j - 1) & 1u, abort_flag)) { ok = false; break; }
+                    if (!mbar_wait(pv_done, (uint32_t)(j - 1) & 1u, abort_flag, plan.wait_cycles)) { ok = false; break; }
                     tc_fence_after_sync();
                     const float alpha = raise ? exp2f(m_used - mt) : 1.f;
 #pragma unroll
@@ -565,11 +410,11 @@ attn_umma_kernel(const __grid_constant__ AttnLayers<NL> layers, const sd_batch b
             tmem_st_wait();
             tc_fence_before_sync();
             __syncwarp();
-            if (lane == 0) mbar_arrive(&p_full[s]);
+            if (lane == 0 && !(plan.withhold && j == 0)) mbar_arrive(&p_full[s]);
         }
         // ------------------------------------------------------------ epilogue
         // (a parity wait on pv_done would be ambiguous here: the softmax may be two phases ahead of it)
-        if (ok) ok = mbar_wait(o_full, 0, abort_flag);
+        if (ok) ok = mbar_wait(o_full, 0, abort_flag, plan.wait_cycles);
         if (ok && !clustered) {
             // single chunk: normalise and write bf16 output
             tc_fence_after_sync();
@@ -673,13 +518,13 @@ static bool fill_layer(AttnLayer* ly, const sd_batch& bt, const sd_kv_layer& cac
 }
 
 template <int NL>
-static sd_status launch_plan(const AttnLayers<NL>& layers, const sd_batch& bt, float scale, const AttnPlan& plan,
-                             int z_count, int32_t* dev_status, cudaStream_t st) {
+sd_status launch_rows1(const AttnLayers<NL>& layers, const sd_batch& bt, float scale, const AttnPlan& plan,
+                       int z_count, int32_t* dev_status, cudaStream_t st) {
     auto kern = attn_umma_kernel<NL>;
     if (cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, kAttSmem) != cudaSuccess)
         return SD_ERR_CUDA;
     cudaLaunchConfig_t cfg = {};
-    cfg.gridDim = dim3(plan.n_chunks, plan.row_tiles, z_count);
+    cfg.gridDim = dim3(plan.n_chunks, plan.ctas_per_group, z_count);
     cfg.blockDim = dim3(kAttThreads);
     cfg.dynamicSmemBytes = kAttSmem;
     cfg.stream = st;
@@ -694,34 +539,100 @@ static sd_status launch_plan(const AttnLayers<NL>& layers, const sd_batch& bt, f
         return SD_ERR_CUDA;
     return SD_OK;
 }
+template sd_status launch_rows1<1>(const AttnLayers<1>&, const sd_batch&, float, const AttnPlan&, int, int32_t*,
+                                   cudaStream_t);
+template sd_status launch_rows1<kMaxLayersPerLaunch>(const AttnLayers<kMaxLayersPerLaunch>&, const sd_batch&, float,
+                                                     const AttnPlan&, int, int32_t*, cudaStream_t);
+
+// SM count of the current device (cached per device ordinal)
+static int sm_count() {
+    constexpr int kDevs = 64;
+    static int cache[kDevs];
+    int dev = 0, sms = 0;
+    if (cudaGetDevice(&dev) != cudaSuccess || dev < 0) return 148;
+    if (dev < kDevs && cache[dev] > 0) return cache[dev];
+    if (cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev) != cudaSuccess || sms <= 0) sms = 148;
+    if (dev < kDevs) cache[dev] = sms;
+    return sms;
+}
+
+// The chunks of a row tile are merged inside a thread-block cluster, through shared memory:
+// attention needs no global scratch (a nominal size keeps the argument checks uniform).
+size_t attention_workspace_bytes(const sd_batch&) { return 256; }
+
+// Which kernel, and how many key chunks.  Up to 128 query rows per KV head (chains, small trees or
+// few grouped heads) run one row tile per CTA, two CTAs per SM; more rows run two row tiles per CTA
+// (one CTA per SM), which shares every K/V tile between the two and uses full-width score MMAs.
+static AttnPlan make_plan(const sd_batch& bt, int n_layers, int sms, bool* two_tiles) {
+    AttnPlan p;
+    const int G = bt.Hq / bt.Hkv;
+    p.rows = bt.T_max * G;
+    p.row_tiles = (p.rows + kRowTile - 1) / kRowTile;
+    *two_tiles = p.row_tiles >= 2;
+    p.ctas_per_group = *two_tiles ? (p.row_tiles + 1) / 2 : p.row_tiles;
+    // Pick the chunk count that minimises (waves of CTAs) x (key tiles per CTA + fixed cost).
+    // Few waves are counted whole; many waves balance out.
+    const int max_tiles = bt.max_blocks_per_seq;
+    const int base = n_layers * bt.B * bt.Hkv * p.ctas_per_group;
+    const int slots = *two_tiles ? sms : 2 * sms;
+    int n = 1;
+    double best = 1e30;
+    for (int c = 1; c <= kMaxChunks && c <= max_tiles; c *= 2) {   // 128 rows split evenly over the chunks
+        const double w = (double)base * c / slots;
+        double waves = (w <= 4.0) ? (double)((base * c + slots - 1) / slots) : w;
+        // Without chunks, and for up to kSplitRounds whole rounds, the CTAs left over after the last whole
+        // round go into a launch of their own, with chunks (launch_group): the partial round then costs
+        // a fraction of a round.  (Longer launches run under the power cap, where this gained nothing.)
+        if (c == 1 && w > 1.0 && base / slots < kSplitRounds) {
+            const int rest = base % slots;
+            int ct = 1;                                    // chunks of the remainder's launch
+            while (2 * ct <= kMaxChunks && 2 * ct <= max_tiles && rest * 2 * ct <= slots) ct *= 2;
+            waves = (double)(base / slots) + (rest == 0 ? 0.0 : (ct > 1 ? 1.0 / ct + 0.1 : 1.0));
+        }
+        // per CTA: its key tiles, a fixed cost of about three tiles, and two more for the in-cluster merge
+        const double cost = waves * ((max_tiles + c - 1) / c + 3 + (c > 1 ? 2 : 0));
+        if (cost < best - 1e-9) { best = cost; n = c; }
+    }
+    const TestKnobs knobs = test_knobs();
+    if (knobs.chunks > 0 && knobs.chunks <= max_tiles) n = knobs.chunks;
+    p.n_chunks = n;
+    p.n_layers = n_layers;
+    p.ranked = (bt.B > 1 && bt.B <= 64 && (long long)base * n > slots) ? 1 : 0;
+    p.z0 = 0;
+    p.wait_cycles = knobs.wait_cycles;
+    p.withhold = knobs.withhold;
+    return p;
+}
 
 template <int NL>
 static sd_status launch_group(const AttnLayers<NL>& layers, int n_layers, const sd_batch& bt, float scale,
                               int32_t* dev_status, cudaStream_t st) {
-    AttnPlan plan = make_plan(bt, n_layers, sm_count());
+    bool two_tiles = false;
+    AttnPlan plan = make_plan(bt, n_layers, sm_count(), &two_tiles);
+    auto launch = two_tiles ? launch_rows2<NL> : launch_rows1<NL>;
     const int Z = n_layers * bt.B * bt.Hkv;
     // A launch of whole-sequence CTAs that runs for more than one round ends on a partial round, in which
     // the CTAs left over would each work through a whole sequence while most of the GPU idles.  They go
     // into a second launch of the same kernel with the keys split into chunks (a cluster per row tile),
     // so that the remainder also spreads over the SMs and takes a fraction of a round.  (In a ranked
     // launch these are the shortest sequences.)
-    const int slots = 2 * sm_count();
-    const long long ctas = (long long)Z * plan.row_tiles;
-    if (plan.n_chunks == 1 && ctas > slots && ctas / slots < kSplitRounds) {
-        const int z_main = (int)((ctas / slots) * slots / plan.row_tiles);
+    const int slots = two_tiles ? sm_count() : 2 * sm_count();
+    const long long ctas = (long long)Z * plan.ctas_per_group;
+    if (plan.n_chunks == 1 && ctas > slots && ctas / slots < kSplitRounds && test_knobs().chunks == 0) {
+        const int z_main = (int)((ctas / slots) * slots / plan.ctas_per_group);
         const int z_rest = Z - z_main;
         int c = 1;
         while (2 * c <= kMaxChunks && 2 * c <= bt.max_blocks_per_seq &&
-               (long long)z_rest * plan.row_tiles * 2 * c <= slots) c *= 2;
+               (long long)z_rest * plan.ctas_per_group * 2 * c <= slots) c *= 2;
         if (z_main > 0 && z_rest > 0 && c > 1) {
-            const sd_status s = launch_plan<NL>(layers, bt, scale, plan, z_main, dev_status, st);
+            const sd_status s = launch(layers, bt, scale, plan, z_main, dev_status, st);
             if (s != SD_OK) return s;
             plan.z0 = z_main;
             plan.n_chunks = c;
-            return launch_plan<NL>(layers, bt, scale, plan, z_rest, dev_status, st);
+            return launch(layers, bt, scale, plan, z_rest, dev_status, st);
         }
     }
-    return launch_plan<NL>(layers, bt, scale, plan, Z, dev_status, st);
+    return launch(layers, bt, scale, plan, Z, dev_status, st);
 }
 
 // One launch per group of layers: at most kMaxLayersPerLaunch descriptors fit the kernel's

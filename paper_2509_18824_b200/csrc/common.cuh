@@ -26,6 +26,14 @@ inline bool aligned16(const void* p) { return (reinterpret_cast<uintptr_t>(p) & 
 
 inline sd_status cuda_ok(cudaError_t e) { return e == cudaSuccess ? SD_OK : SD_ERR_CUDA; }
 
+// Test hooks, read from the environment at every launch (unset in normal use):
+//   SDV_TEST_WAIT_CYCLES  bound of the kernels' barrier waits in SM cycles (default: about a second)
+//   SDV_TEST_WITHHOLD     1: one role of the tensor-core kernels withholds its first arrival, so that
+//                         a bounded wait runs out and the launch ends with SD_ERR_TIMEOUT
+//   SDV_TEST_CHUNKS       1, 2, 4 or 8: key chunks per sequence of single-launch attention calls
+struct TestKnobs { long long wait_cycles; int withhold; int chunks; };
+TestKnobs test_knobs();
+
 // launch-side entry points implemented in the kernel files
 sd_status launch_tree_prepare(const sd_batch& bt, int32_t* dev_status, cudaStream_t st);
 sd_status launch_accept(const sd_batch& bt, const int32_t* draft, const int32_t* target,

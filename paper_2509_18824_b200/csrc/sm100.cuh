@@ -47,22 +47,31 @@ __device__ __forceinline__ bool mbar_try_wait(uint64_t* bar, uint32_t parity) {
     return ok != 0;
 }
 
-// Bounded wait: gives up after ~kWaitCycles SM cycles, or as soon as another
-// thread of the CTA has raised *abort_flag.  Returns false when it gave up
-// (and raises the flag itself), so that callers can unwind instead of hanging.
+// Bounded wait: gives up after `limit` SM cycles (about a second by default), or as soon as another
+// thread of the CTA has raised *abort_flag.  Returns false when it gave up (and raises the flag
+// itself), so that callers can unwind instead of hanging.
 constexpr long long kWaitCycles = 1ll << 31;   // about a second
 
-__device__ __forceinline__ bool mbar_wait(uint64_t* bar, uint32_t parity, volatile int* abort_flag) {
+__device__ __forceinline__ bool mbar_wait(uint64_t* bar, uint32_t parity, volatile int* abort_flag,
+                                          long long limit = kWaitCycles) {
     if (mbar_try_wait(bar, parity)) return true;
     const long long t0 = clock64();
     while (true) {
         if (mbar_try_wait(bar, parity)) return true;
         if (*abort_flag) return false;
-        if (clock64() - t0 > kWaitCycles) {
+        if (clock64() - t0 > limit) {
             *abort_flag = 1;
             return false;
         }
     }
+}
+// The same wait without the abort flag, for the unwinding path itself (e.g. "every MMA issued so far
+// has completed" before tensor memory is given back).
+__device__ __forceinline__ bool mbar_wait_plain(uint64_t* bar, uint32_t parity, long long limit) {
+    const long long t0 = clock64();
+    while (!mbar_try_wait(bar, parity))
+        if (clock64() - t0 > limit) return false;
+    return true;
 }
 
 // ---------------------------------------------------------------- thread-block clusters
