@@ -11,7 +11,7 @@ CSRC = os.path.join(HERE, "csrc")
 INCLUDE = os.path.join(os.path.dirname(HERE), "include")
 OBJ = os.path.join(HERE, "_build")
 LIB = os.path.join(HERE, "libsdverify.so")
-SOURCES = ["api.cu", "tree.cu", "compact.cu", "attention.cu", "attention_pingpong.cu", "lmhead.cu", "sampled.cu", "draft.cu", "tmap.cu"]
+SOURCES = ["api.cu", "tree.cu", "compact.cu", "attention.cu", "lmhead.cu", "sampled.cu", "draft.cu", "tmap.cu"]
 NVCC_FLAGS = ["-gencode", "arch=compute_100a,code=sm_100a", "-lineinfo", "-O3", "-std=c++17",
               "-Xcompiler", "-fPIC", "-I", INCLUDE, "-I", CSRC]
 

@@ -560,21 +560,18 @@ static int sm_count() {
 // attention needs no global scratch (a nominal size keeps the argument checks uniform).
 size_t attention_workspace_bytes(const sd_batch&) { return 256; }
 
-// Which kernel, and how many key chunks.  Up to 128 query rows per KV head (chains, small trees or
-// few grouped heads) run one row tile per CTA, two CTAs per SM; more rows run two row tiles per CTA
-// (one CTA per SM), which shares every K/V tile between the two and uses full-width score MMAs.
-static AttnPlan make_plan(const sd_batch& bt, int n_layers, int sms, bool* two_tiles) {
+// How many key chunks per sequence.
+static AttnPlan make_plan(const sd_batch& bt, int n_layers, int sms) {
     AttnPlan p;
     const int G = bt.Hq / bt.Hkv;
     p.rows = bt.T_max * G;
     p.row_tiles = (p.rows + kRowTile - 1) / kRowTile;
-    *two_tiles = p.row_tiles >= 2;
-    p.ctas_per_group = *two_tiles ? (p.row_tiles + 1) / 2 : p.row_tiles;
-    // Pick the chunk count that minimises (waves of CTAs) x (key tiles per CTA + fixed cost).
-    // Few waves are counted whole; many waves balance out.
+    p.ctas_per_group = p.row_tiles;
+    // Pick the chunk count that minimises (waves of CTAs) x (key tiles per CTA + fixed cost),
+    // two CTAs being resident per SM.  Few waves are counted whole; many waves balance out.
     const int max_tiles = bt.max_blocks_per_seq;
-    const int base = n_layers * bt.B * bt.Hkv * p.ctas_per_group;
-    const int slots = *two_tiles ? sms : 2 * sms;
+    const int base = n_layers * bt.B * bt.Hkv * p.row_tiles;
+    const int slots = 2 * sms;
     int n = 1;
     double best = 1e30;
     for (int c = 1; c <= kMaxChunks && c <= max_tiles; c *= 2) {   // 128 rows split evenly over the chunks
@@ -594,7 +591,7 @@ static AttnPlan make_plan(const sd_batch& bt, int n_layers, int sms, bool* two_t
         if (cost < best - 1e-9) { best = cost; n = c; }
     }
     const TestKnobs knobs = test_knobs();
-    if (knobs.chunks > 0 && knobs.chunks <= max_tiles) n = knobs.chunks;
+    if (knobs.chunks > 0 && knobs.chunks <= max_tiles) n = knobs.chunks;     // test hook
     p.n_chunks = n;
     p.n_layers = n_layers;
     p.ranked = (bt.B > 1 && bt.B <= 64 && (long long)base * n > slots) ? 1 : 0;
@@ -607,32 +604,30 @@ static AttnPlan make_plan(const sd_batch& bt, int n_layers, int sms, bool* two_t
 template <int NL>
 static sd_status launch_group(const AttnLayers<NL>& layers, int n_layers, const sd_batch& bt, float scale,
                               int32_t* dev_status, cudaStream_t st) {
-    bool two_tiles = false;
-    AttnPlan plan = make_plan(bt, n_layers, sm_count(), &two_tiles);
-    auto launch = two_tiles ? launch_rows2<NL> : launch_rows1<NL>;
+    AttnPlan plan = make_plan(bt, n_layers, sm_count());
     const int Z = n_layers * bt.B * bt.Hkv;
     // A launch of whole-sequence CTAs that runs for more than one round ends on a partial round, in which
     // the CTAs left over would each work through a whole sequence while most of the GPU idles.  They go
     // into a second launch of the same kernel with the keys split into chunks (a cluster per row tile),
     // so that the remainder also spreads over the SMs and takes a fraction of a round.  (In a ranked
     // launch these are the shortest sequences.)
-    const int slots = two_tiles ? sm_count() : 2 * sm_count();
-    const long long ctas = (long long)Z * plan.ctas_per_group;
+    const int slots = 2 * sm_count();
+    const long long ctas = (long long)Z * plan.row_tiles;
     if (plan.n_chunks == 1 && ctas > slots && ctas / slots < kSplitRounds && test_knobs().chunks == 0) {
-        const int z_main = (int)((ctas / slots) * slots / plan.ctas_per_group);
+        const int z_main = (int)((ctas / slots) * slots / plan.row_tiles);
         const int z_rest = Z - z_main;
         int c = 1;
         while (2 * c <= kMaxChunks && 2 * c <= bt.max_blocks_per_seq &&
-               (long long)z_rest * plan.ctas_per_group * 2 * c <= slots) c *= 2;
+               (long long)z_rest * plan.row_tiles * 2 * c <= slots) c *= 2;
         if (z_main > 0 && z_rest > 0 && c > 1) {
-            const sd_status s = launch(layers, bt, scale, plan, z_main, dev_status, st);
+            const sd_status s = launch_rows1<NL>(layers, bt, scale, plan, z_main, dev_status, st);
             if (s != SD_OK) return s;
             plan.z0 = z_main;
             plan.n_chunks = c;
-            return launch(layers, bt, scale, plan, z_rest, dev_status, st);
+            return launch_rows1<NL>(layers, bt, scale, plan, z_rest, dev_status, st);
         }
     }
-    return launch(layers, bt, scale, plan, Z, dev_status, st);
+    return launch_rows1<NL>(layers, bt, scale, plan, Z, dev_status, st);
 }
 
 // One launch per group of layers: at most kMaxLayersPerLaunch descriptors fit the kernel's

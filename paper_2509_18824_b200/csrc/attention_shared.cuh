@@ -1,6 +1,5 @@
-// Pieces shared by the two tree-attention kernels (one row tile per CTA with 64-key tiles; two row
-// tiles per CTA with 128-key tiles): launch plan, per-layer descriptors, and the in-cluster merge of
-// key chunks through distributed shared memory.
+// Pieces of the tree-attention kernel that its launcher shares with it: launch plan, per-layer
+// descriptors, and the in-cluster merge of key chunks through distributed shared memory.
 #pragma once
 #include <stdlib.h>
 #include "common.cuh"
@@ -129,8 +128,5 @@ __device__ __forceinline__ void merge_rows(const MergeCtx& x) {
 template <int NL>
 sd_status launch_rows1(const AttnLayers<NL>& layers, const sd_batch& bt, float scale, const AttnPlan& plan,
                        int z_count, int32_t* dev_status, cudaStream_t st);     // one row tile per CTA, 64-key tiles
-template <int NL>
-sd_status launch_rows2(const AttnLayers<NL>& layers, const sd_batch& bt, float scale, const AttnPlan& plan,
-                       int z_count, int32_t* dev_status, cudaStream_t st);     // two row tiles per CTA, 128-key tiles
 
 }  // namespace sdv

@@ -551,7 +551,9 @@ lmhead_umma_pair_kernel(const __grid_constant__ CUtensorMap tmW, const __grid_co
             }
             tc_fence_before_sync();
             __syncwarp();
-            if (lane == 0) mbar_arrive_remote(map_dsmem(smem_u32(&tmem_empty[buf]), 0));
+            // (the accumulator reads above have completed: tcgen05.wait::ld; a CTA-scope release is enough,
+            //  and a cluster-scope one costs on the order of a thousand cycles per arrival)
+            if (lane == 0) mbar_arrive_remote_light(map_dsmem(smem_u32(&tmem_empty[buf]), 0));
         }
         asm volatile("bar.sync 1, %0;" ::"n"(kEpiWarps * 32) : "memory");
         int32_t* red_key = reinterpret_cast<int32_t*>(smem);

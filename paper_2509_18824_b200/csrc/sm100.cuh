@@ -116,9 +116,17 @@ __device__ __forceinline__ uint32_t cluster_ctarank() {
     asm volatile("mov.u32 %0, %%cluster_ctarank;" : "=r"(r));
     return r;
 }
-// arrive on an mbarrier that lives in another CTA of the cluster (address from map_dsmem)
+// arrive on an mbarrier that lives in another CTA of the cluster (address from map_dsmem), with a
+// release at cluster scope: everything this thread wrote before becomes visible to the waiting CTA
+// (costs on the order of a thousand cycles)
 __device__ __forceinline__ void mbar_arrive_remote(uint32_t cluster_addr) {
     asm volatile("mbarrier.arrive.release.cluster.shared::cluster.b64 _, [%0];" ::"r"(cluster_addr) : "memory");
+}
+// the same arrival with the default (CTA-scope) release: for signals whose payload is ordered by other
+// means (tensor-memory stores completed with tcgen05.wait::st, shared-memory writes made visible to
+// the async proxy with fence.proxy.async)
+__device__ __forceinline__ void mbar_arrive_remote_light(uint32_t cluster_addr) {
+    asm volatile("mbarrier.arrive.shared::cluster.b64 _, [%0];" ::"r"(cluster_addr) : "memory");
 }
 
 // ---------------------------------------------------------------- TMA
