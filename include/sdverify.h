@@ -122,8 +122,9 @@ sd_status sd_tree_prepare(const sd_batch *batch, int32_t *dev_status, void *stre
  *   workspace         : dev scratch of at least sd_workspace_bytes(batch, 0, 0)
  * Arithmetic: bf16 inputs, fp32 accumulation, bf16 output (round to nearest even).
  * Needs batch->anc_mask filled.  Errors: SD_ERR_INVALID_ARG, SD_ERR_UNSUPPORTED,
- * SD_ERR_WORKSPACE on the host; SD_ERR_BOUNDS (block-table entry outside
- * [0, num_blocks)) or SD_ERR_TIMEOUT through *dev_status.
+ * SD_ERR_WORKSPACE (workspace_bytes below sd_workspace_bytes) on the host;
+ * SD_ERR_BOUNDS (block-table entry outside [0, num_blocks), or len[b] needs
+ * more than max_blocks_per_seq blocks) or SD_ERR_TIMEOUT through *dev_status.
  */
 sd_status sd_verify_attention(const sd_batch *batch, const sd_kv_layer *cache,
                               const void *q, const void *k_tree, const void *v_tree,
@@ -195,7 +196,8 @@ sd_status sd_lmhead_argmax(const void *hidden, const void *W,
  *     number the built-in table holds; larger M returns SD_ERR_UNSUPPORTED and
  *     launches nothing (call it once per slice of rows instead).
  *   - The first call on each device looks up the table's device address.
- *     Make that first call during start-up, before any stream capture begins.
+ *     Make that first call during start-up, before any stream capture begins,
+ *     and from one host thread (later calls may come from any thread).
  *   - All calls on a device share the one table, and it keeps whatever the
  *     previous call left in it.  No entry needs clearing between calls (each
  *     call overwrites every entry it later reads), but two calls whose kernels
@@ -252,8 +254,9 @@ sd_status sd_compact_kv(const sd_batch *batch, const sd_kv_layer *layers, int32_
  *     sd_lmhead_argmax(hidden, W, M = B * T_max, ...)      row b * T_max + i = node i of sequence b
  *     sd_accept_tree(batch, draft_tok, argmax, ...)
  *     sd_compact_kv(batch, layers, L, ..., n_acc, path)
- * but after the LM-head tiles a single kernel (one CTA per sequence) merges the
- * arg-max candidates, picks the accepted path and copies the accepted K/V rows,
+ * but after the LM-head tiles a single kernel (one CTA per sequence and layer;
+ * every CTA repeats the merge and the acceptance of its sequence, the CTAs of
+ * layer 0 write the outputs) merges the arg-max candidates, picks the accepted path and copies the accepted K/V rows,
  * instead of three launches of a few microseconds each.  Arguments as in the three
  * calls; argmax [B * T_max] and maxlogit (nullable) are outputs as well.
  * B * T_max > 512 or L > 64 falls back to the three separate steps internally.

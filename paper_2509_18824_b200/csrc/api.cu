@@ -107,7 +107,7 @@ sd_status sd_verify_attention_layers(const sd_batch* batch, const sd_kv_layer* c
             return SD_ERR_INVALID_ARG;
         if (lse_layers && lse_layers[l] && (reinterpret_cast<uintptr_t>(lse_layers[l]) & 3u)) return SD_ERR_INVALID_ARG;
     }
-    (void)workspace_bytes;
+    if (workspace_bytes < attention_workspace_bytes(*batch)) return SD_ERR_WORKSPACE;
     return launch_attention_layers(*batch, caches, L, q_layers, k_tree_layers, v_tree_layers, scale, out_layers,
                                    lse_layers, dev_status, static_cast<cudaStream_t>(stream));
 }

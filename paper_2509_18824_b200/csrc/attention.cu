@@ -665,7 +665,8 @@ sd_status launch_attention_layers(const sd_batch& bt, const sd_kv_layer* caches,
 sd_status launch_attention(const sd_batch& bt, const sd_kv_layer& cache, const void* q,
                            const void* kt, const void* vt, float scale, void* out, float* lse,
                            void* ws, size_t ws_bytes, int32_t* dev_status, cudaStream_t st) {
-    (void)ws; (void)ws_bytes;
+    (void)ws;
+    if (ws_bytes < attention_workspace_bytes(bt)) return SD_ERR_WORKSPACE;
     return launch_attention_layers(bt, &cache, 1, &q, &kt, &vt, scale, &out, &lse, dev_status, st);
 }
 

@@ -7,6 +7,7 @@
 // leaves TMEM: the epilogue warps reduce each column over the 128 vocabulary
 // lanes (max + lowest index) and keep a running best per hidden row; only
 // (max, index) pairs per CTA reach memory, and a tiny kernel merges them.
+#include <atomic>
 #include "tree_device.cuh"
 #include "sm100.cuh"
 
@@ -891,7 +892,7 @@ constexpr size_t kStaticScratchBytes = (size_t)kMaxCtas * kMaxCols * 2 * sizeof(
 static __device__ __align__(256) unsigned char g_lmhead_scratch[kStaticScratchBytes];
 
 constexpr int kMaxDevices = 64;
-static void* g_scratch_addr[kMaxDevices];     // device address of the array, per device ordinal
+static std::atomic<void*> g_scratch_addr[kMaxDevices];     // device address of the array, per device ordinal
 
 // The array's name is only a host-side handle here; the device address has to be
 // asked for, once per device, with that device current.
@@ -899,12 +900,13 @@ static sd_status static_scratch(void** ptr) {
     int dev = 0;
     if (cudaGetDevice(&dev) != cudaSuccess) return SD_ERR_CUDA;
     if (dev < 0 || dev >= kMaxDevices) return SD_ERR_UNSUPPORTED;
-    if (!g_scratch_addr[dev]) {
-        void* p = nullptr;
+    void* p = g_scratch_addr[dev].load(std::memory_order_relaxed);
+    if (!p) {
+        // (two threads that both find the slot empty look the same address up twice: harmless)
         if (cudaGetSymbolAddress(&p, g_lmhead_scratch) != cudaSuccess || !p) return SD_ERR_CUDA;
-        g_scratch_addr[dev] = p;
+        g_scratch_addr[dev].store(p, std::memory_order_relaxed);
     }
-    *ptr = g_scratch_addr[dev];
+    *ptr = p;
     return SD_OK;
 }
 

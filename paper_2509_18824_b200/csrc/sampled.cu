@@ -402,6 +402,9 @@ sd_status launch_accept_sampled(const sd_batch& bt, const void* hidden, const vo
                                 void* ws, size_t ws_bytes, int32_t* dev_status, cudaStream_t st) {
     const int B = bt.B, T = bt.T_max;
     if (Hd > 16384) return SD_ERR_UNSUPPORTED;
+    // vocabulary limits of the residual draw, checked before anything is launched
+    if (group_stats ? ((V + 31) / 32 > kPickMaxGroups) : ((V + kResBlock - 1) / kResBlock > kPickMaxBlocks))
+        return SD_ERR_UNSUPPORTED;
     if (ws_bytes < sampled_workspace_bytes(B, T, V, 16384)) return SD_ERR_WORKSPACE;
     const SampledWs s = carve(ws, B, T, V, 16384);
     const uint16_t* h = static_cast<const uint16_t*>(hidden);
@@ -413,7 +416,6 @@ sd_status launch_accept_sampled(const sd_batch& bt, const void* hidden, const vo
     if (group_stats) {
         // the LM-head pass left (maximum, sum) of every 32 vocabulary rows: no second pass over W
         const int n_groups = (V + 31) / 32;
-        if (n_groups > kPickMaxGroups) return SD_ERR_UNSUPPORTED;
         residual_pick_groups_kernel<<<B, 256, 0, st>>>(bt, h, Wp, Hd, V, inv_temp, lse, reinterpret_cast<const float2*>(group_stats),
                                                       n_groups, w, s.stop_row, s.n_excl, s.excl, s.excl_p, n_acc, out_tok, dev_status);
         return cuda_ok(cudaGetLastError());
@@ -425,7 +427,6 @@ sd_status launch_accept_sampled(const sd_batch& bt, const void* hidden, const vo
                                       stats_workspace_bytes(B, V), dev_status, st);
     if (ls != SD_OK) return ls;
     residual_blocksum_kernel<<<dim3(n_blocks, B), kResBlock, 0, st>>>(V, s.n_excl, s.excl, s.mass, s.block_sum, n_blocks);
-    if (n_blocks > kPickMaxBlocks) return SD_ERR_UNSUPPORTED;
     residual_pick_kernel<<<B, kResBlock, 0, st>>>(bt, V, w, s.mass, s.block_sum, n_blocks, n_acc, out_tok, dev_status);
     return cuda_ok(cudaGetLastError());
 }

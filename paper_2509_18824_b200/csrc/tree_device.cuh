@@ -105,10 +105,12 @@ __device__ __forceinline__ void compact_sequence(const sd_batch& bt, const Compa
         for (int k0 = tid / per_node; k0 < na; k0 += k_step * kUnroll) {
             size_t src[kUnroll], dst[kUnroll];
             int blk[kUnroll];
+            bool has[kUnroll];                             // this slot holds an accepted node
 #pragma unroll
             for (int u = 0; u < kUnroll; ++u) {
                 const int k = k0 + u * k_step;
-                blk[u] = -2;                               // -2: no node for this slot
+                blk[u] = -1;
+                has[u] = false;
                 if (k >= na) continue;
                 const int node = path[k];
                 const int t = len + k;
@@ -116,6 +118,7 @@ __device__ __forceinline__ void compact_sequence(const sd_batch& bt, const Compa
                     set_status(status, SD_ERR_BOUNDS);
                     continue;
                 }
+                has[u] = true;
                 blk[u] = bt.block_table[(size_t)b * bt.max_blocks_per_seq + t / kBlock];
                 src[u] = (((size_t)b * T + node) * bt.Hkv + kvh) * vec_per_head + c;
                 dst[u] = (((size_t)(blk[u] < 0 ? 0 : blk[u]) * bt.Hkv + kvh) * kBlock + (t % kBlock)) * vec_per_head + c;
@@ -128,8 +131,8 @@ __device__ __forceinline__ void compact_sequence(const sd_batch& bt, const Compa
                 bool live[kUnroll];
 #pragma unroll
                 for (int u = 0; u < kUnroll; ++u) {
-                    live[u] = blk[u] >= 0 && blk[u] < nb;
-                    if (blk[u] != -2 && !live[u]) set_status(status, SD_ERR_BOUNDS);
+                    live[u] = has[u] && blk[u] >= 0 && blk[u] < nb;
+                    if (has[u] && !live[u]) set_status(status, SD_ERR_BOUNDS);
                     if (live[u]) val[u] = from[src[u]];
                 }
 #pragma unroll

@@ -74,3 +74,31 @@ def test_host_side_refusals_of_the_newer_calls():
     big = L.sd_workspace_bytes(ctypes.byref(bt), 480, 152064)
     assert big > small >= L.sd_workspace_bytes(None, 480, 1024) > 0
     assert big >= 8 * 152064 * 4                            # room for one probability row per sequence
+
+
+def test_host_side_refusals_come_before_any_launch():
+    """Host-detectable problems of the attention and the sampled-acceptance calls return their status with
+    nothing enqueued (there is no GPU here: a launch attempt would come back as SD_ERR_CUDA instead)."""
+    from paper_2509_18824_b200 import binding as b
+    L = b.lib
+    f = ctypes.c_float
+    ok = 4096
+    bt = b.sd_batch(2, 8, 4, 1, 128, 64, 4, ok, ok, ok, ok, ok)
+    cache = b.sd_kv_layer(ok, ok, 8)
+    need = L.sd_workspace_bytes(ctypes.byref(bt), 0, 0)
+    assert need > 0
+    # workspace smaller than sd_workspace_bytes: refused, for the one-layer and the all-layers call
+    assert L.sd_verify_attention(ctypes.byref(bt), ctypes.byref(cache), ok, ok, ok, f(0.1), ok, None,
+                                 ok, need - 1, ok, None) == b.SD_ERR_WORKSPACE
+    ptrs = (ctypes.c_void_p * 1)(ok)
+    assert L.sd_verify_attention_layers(ctypes.byref(bt), ctypes.byref(cache), 1, ptrs, ptrs, ptrs, f(0.1), ptrs, None,
+                                        ok, need - 1, ok, None) == b.SD_ERR_WORKSPACE
+    # sampled acceptance: a vocabulary beyond the residual draw's tables (8192 groups of 32 with the
+    # group statistics, 4096 blocks of 256 without) is refused before the first kernel
+    big = 1 << 40
+    assert L.sd_accept_tree_sampled(ctypes.byref(bt), ok, ok, 128, 8192 * 32 + 1, f(1.0), ok, ok, ok, ok, ok,
+                                    ok, ok, ok, ok, ok, big, ok, None) == b.SD_ERR_UNSUPPORTED
+    assert L.sd_accept_tree_sampled(ctypes.byref(bt), ok, ok, 128, 4096 * 256 + 1, f(1.0), ok, None, ok, ok, ok,
+                                    ok, ok, ok, ok, ok, big, ok, None) == b.SD_ERR_UNSUPPORTED
+    assert L.sd_accept_tree_sampled(ctypes.byref(bt), ok, ok, 128, 1000, f(1.0), ok, None, ok, ok, ok,
+                                    ok, ok, ok, ok, ok, 16, ok, None) == b.SD_ERR_WORKSPACE

@@ -70,3 +70,25 @@ def test_static_scratch_variant_refuses_too_many_rows():
     assert e.value.code == sd.SD_ERR_UNSUPPORTED
     torch.cuda.synchronize()
     assert (am.cpu().numpy() == -1).all() and int(st.item()) == 0
+
+
+def test_static_scratch_variant_leaves_free_memory_alone():
+    """The property the entry point is named for: once the first call on the device is behind us (it
+    resolves the table's address, and the kernels' code may still have to be loaded before it), a call
+    does not move the device's free memory: nothing is allocated, nothing is freed.  (Free memory is a
+    device-wide figure; the measurement is repeated so that a change from outside is not mistaken for one.)"""
+    h, W = _inputs(5, 300, 256, 9000)
+    am = torch.full((300,), -1, dtype=torch.int32, device="cuda")
+    st = sd.new_status()
+    sd.sd_lmhead_argmax_static(h, W, am, None, st)
+    torch.cuda.synchronize()
+    moved = []
+    for _ in range(3):
+        before = torch.cuda.mem_get_info()[0]
+        sd.sd_lmhead_argmax_static(h, W, am, None, st)
+        torch.cuda.synchronize()
+        moved.append(torch.cuda.mem_get_info()[0] - before)
+        if moved[-1] == 0:
+            break
+    assert moved[-1] == 0, moved
+    assert int(st.item()) == 0
