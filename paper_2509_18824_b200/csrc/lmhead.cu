@@ -52,6 +52,8 @@ struct LmParams {
     float* mass_out;        // [rows of the call][V]
     const float* col_lse;   // [rows of the call]
     float inv_temp;
+    long long wait_cycles;  // bound of every barrier wait, in SM cycles
+    int withhold;           // test hook (single-CTA kernel): the first tile's "accumulator complete" is never signalled
 };
 
 size_t lmhead_workspace_bytes(int M, int V) {
@@ -193,6 +195,7 @@ lmhead_umma_kernel(const __grid_constant__ CUtensorMap tmW, const __grid_constan
     __shared__ __align__(8) uint64_t empty_bar[kMaxStages];
     __shared__ __align__(8) uint64_t tmem_full[2];
     __shared__ __align__(8) uint64_t tmem_empty[2];
+    __shared__ __align__(8) uint64_t mma_idle;               // unwinding only: every MMA issued so far has completed
     __shared__ uint32_t tmem_base_slot;
     __shared__ int abort_flag;
 
@@ -205,6 +208,7 @@ lmhead_umma_kernel(const __grid_constant__ CUtensorMap tmW, const __grid_constan
         abort_flag = 0;
         for (int s = 0; s < p.stages; ++s) { mbar_init(&full_bar[s], 1); mbar_init(&empty_bar[s], 1); }
         for (int b = 0; b < 2; ++b) { mbar_init(&tmem_full[b], 1); mbar_init(&tmem_empty[b], kEpiWarps); }
+        mbar_init(&mma_idle, 1);
         fence_barrier_init();
     }
     if (warp == kTmaWarpLm) {          // a full warp
@@ -229,7 +233,7 @@ lmhead_umma_kernel(const __grid_constant__ CUtensorMap tmW, const __grid_constan
                 for (int kb = 0; kb < kblocks; ++kb, ++it) {
                     const int s = it % p.stages;
                     const uint32_t ph = (uint32_t)(it / p.stages) & 1u;
-                    if (!mbar_wait(&empty_bar[s], ph ^ 1u, &abort_flag)) { ok = false; break; }
+                    if (!mbar_wait(&empty_bar[s], ph ^ 1u, &abort_flag, p.wait_cycles)) { ok = false; break; }
                     uint8_t* a = smem + (size_t)s * stage_bytes;
                     mbar_arrive_expect_tx(&full_bar[s], (uint32_t)stage_bytes);
                     tma_load_2d(a, &tmW, kb * BK, v0, &full_bar[s], pol_w);
@@ -252,13 +256,13 @@ lmhead_umma_kernel(const __grid_constant__ CUtensorMap tmW, const __grid_constan
             for (int t = 0; t < my_tiles && ok; ++t) {
                 const int buf = t % p.acc_bufs;
                 const uint32_t use = (uint32_t)(t / p.acc_bufs);
-                if (!mbar_wait(&tmem_empty[buf], (use & 1u) ^ 1u, &abort_flag)) { ok = false; break; }
+                if (!mbar_wait(&tmem_empty[buf], (use & 1u) ^ 1u, &abort_flag, p.wait_cycles)) { ok = false; break; }
                 tc_fence_after_sync();
                 const uint32_t d0 = tmem_base + (uint32_t)(buf * p.buf_stride);
                 for (int kb = 0; kb < kblocks; ++kb, ++it) {
                     const int s = it % p.stages;
                     const uint32_t ph = (uint32_t)(it / p.stages) & 1u;
-                    if (!mbar_wait(&full_bar[s], ph, &abort_flag)) { ok = false; break; }
+                    if (!mbar_wait(&full_bar[s], ph, &abort_flag, p.wait_cycles)) { ok = false; break; }
                     tc_fence_after_sync();
                     const uint32_t a_addr = smem_u32(smem + (size_t)s * stage_bytes);
                     const uint32_t b_addr = a_addr + (uint32_t)a_bytes;
@@ -273,9 +277,14 @@ lmhead_umma_kernel(const __grid_constant__ CUtensorMap tmW, const __grid_constan
                     }
                     mma_commit(&empty_bar[s]);            // stage reusable once these MMAs have read it
                 }
-                if (ok) mma_commit(&tmem_full[buf]);       // accumulator complete
+                if (ok && !(p.withhold && t == 0)) mma_commit(&tmem_full[buf]);       // accumulator complete
             }
-            if (!ok) set_status(status, SD_ERR_TIMEOUT);
+            if (!ok || p.withhold) {
+                // unwinding: nothing may give tensor memory back while an MMA issued above still runs
+                if (!ok) set_status(status, SD_ERR_TIMEOUT);
+                mma_commit(&mma_idle);
+                mbar_wait_plain(&mma_idle, 0, p.wait_cycles);
+            }
         }
     } else {
         // ------------------------------------------------ epilogue warps 0..7
@@ -294,7 +303,7 @@ lmhead_umma_kernel(const __grid_constant__ CUtensorMap tmW, const __grid_constan
         for (int t = 0; t < my_tiles && ok; ++t) {
             const int buf = t % p.acc_bufs;
             const uint32_t use = (uint32_t)(t / p.acc_bufs);
-            if (!mbar_wait(&tmem_full[buf], use & 1u, &abort_flag)) { ok = false; break; }
+            if (!mbar_wait(&tmem_full[buf], use & 1u, &abort_flag, p.wait_cycles)) { ok = false; break; }
             tc_fence_after_sync();
             const int v_base = ((int)blockIdx.x + t * (int)gridDim.x) * kBM + quad * 32;
             const bool v_ok = (v_base + lane) < p.V;
@@ -360,6 +369,7 @@ lmhead_umma_kernel(const __grid_constant__ CUtensorMap tmW, const __grid_constan
                 const int32_t k2 = red_key[w * kMaxCols + col], i2 = red_idx[w * kMaxCols + col];
                 if (k2 > k || (k2 == k && i2 < i)) { k = k2; i = i2; }
             }
+            if (!ok && col == (int)threadIdx.x) set_status(status, SD_ERR_TIMEOUT);
             p.part_key[(size_t)blockIdx.x * kMaxCols + col] = ok ? k : INT32_MIN;
             p.part_idx[(size_t)blockIdx.x * kMaxCols + col] = i;
             if (stats) {
@@ -443,7 +453,7 @@ lmhead_umma_pair_kernel(const __grid_constant__ CUtensorMap tmW, const __grid_co
                 for (int kb = 0; kb < kblocks; ++kb, ++it) {
                     const int s = it % p.stages;
                     const uint32_t ph = (uint32_t)(it / p.stages) & 1u;
-                    if (!mbar_wait(&empty_bar[s], ph ^ 1u, &abort_flag)) { ok = false; break; }
+                    if (!mbar_wait(&empty_bar[s], ph ^ 1u, &abort_flag, p.wait_cycles)) { ok = false; break; }
                     uint8_t* a = smem + (size_t)s * stage_bytes;
                     if (rank == 0) mbar_arrive_expect_tx(&full_bar[s], 2u * (uint32_t)stage_bytes);
                     const uint32_t bar = map_dsmem(smem_u32(&full_bar[s]), 0);     // the leader's barrier
@@ -468,13 +478,13 @@ lmhead_umma_pair_kernel(const __grid_constant__ CUtensorMap tmW, const __grid_co
             for (int t = 0; t < my_tiles && ok; ++t) {
                 const int buf = t % p.acc_bufs;
                 const uint32_t use = (uint32_t)(t / p.acc_bufs);
-                if (!mbar_wait(&tmem_empty[buf], (use & 1u) ^ 1u, &abort_flag)) { ok = false; break; }
+                if (!mbar_wait(&tmem_empty[buf], (use & 1u) ^ 1u, &abort_flag, p.wait_cycles)) { ok = false; break; }
                 tc_fence_after_sync();
                 const uint32_t d0 = tmem_base + (uint32_t)(buf * p.buf_stride);
                 for (int kb = 0; kb < kblocks; ++kb, ++it) {
                     const int s = it % p.stages;
                     const uint32_t ph = (uint32_t)(it / p.stages) & 1u;
-                    if (!mbar_wait(&full_bar[s], ph, &abort_flag)) { ok = false; break; }
+                    if (!mbar_wait(&full_bar[s], ph, &abort_flag, p.wait_cycles)) { ok = false; break; }
                     tc_fence_after_sync();
                     // descriptors of the stage; k-steps and parts only move the 16-byte-granular start address
                     const uint32_t a_addr = smem_u32(smem + (size_t)s * stage_bytes);
@@ -512,7 +522,7 @@ lmhead_umma_pair_kernel(const __grid_constant__ CUtensorMap tmW, const __grid_co
         for (int t = 0; t < my_tiles && ok; ++t) {
             const int buf = t % p.acc_bufs;
             const uint32_t use = (uint32_t)(t / p.acc_bufs);
-            if (!mbar_wait(&tmem_full[buf], use & 1u, &abort_flag)) { ok = false; break; }
+            if (!mbar_wait(&tmem_full[buf], use & 1u, &abort_flag, p.wait_cycles)) { ok = false; break; }
             tc_fence_after_sync();
             const int v_base = ((pair + t * n_pairs) * 2 + (int)rank) * kBM + quad * 32;
             const bool v_ok = (v_base + lane) < p.V;
@@ -578,6 +588,7 @@ lmhead_umma_pair_kernel(const __grid_constant__ CUtensorMap tmW, const __grid_co
                 const int32_t k2 = red_key[w * kMaxCols + col], i2 = red_idx[w * kMaxCols + col];
                 if (k2 > k || (k2 == k && i2 < i)) { k = k2; i = i2; }
             }
+            if (!ok && col == (int)threadIdx.x) set_status(status, SD_ERR_TIMEOUT);
             p.part_key[(size_t)blockIdx.x * kMaxCols + col] = ok ? k : INT32_MIN;
             p.part_idx[(size_t)blockIdx.x * kMaxCols + col] = i;
             if (stats) {
@@ -704,6 +715,9 @@ static sd_status launch_lmhead_impl(const void* hidden, const void* W, int M, in
         p.part_ref = reinterpret_cast<float*>(static_cast<char*>(ws) + tail_workspace_bytes(M, V));
         p.part_sum = p.part_ref + (size_t)kMaxCtas * kMaxCols;
         p.mass_out = mass_out; p.col_lse = col_lse; p.inv_temp = inv_temp;
+        const TestKnobs knobs = test_knobs();
+        p.wait_cycles = knobs.wait_cycles;
+        p.withhold = knobs.withhold;
         p.group_stats = reinterpret_cast<float2*>(group_stats); p.M_total = M;
 
         CUtensorMap tmW, tmH;
