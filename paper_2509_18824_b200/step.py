@@ -183,11 +183,12 @@ class VerifyStep:
         self.compact(stream)
 
     # -- the whole step -------------------------------------------------
-    def run(self, stream=None, per_layer=False, fused_tail=True):
-        """All layers' attention in one call (the step's q and tree K/V are all present up front), then
-        LM head + acceptance + compaction in one call.  per_layer=True issues one attention call per
-        layer, as a decoder that interleaves its own layers would; fused_tail=False issues the three
-        tail calls separately."""
+    def run(self, stream=None, per_layer=True, fused_tail=True):
+        """One attention call per layer, as a decoder issues them (layer l + 1's q, k and v depend on
+        layer l's attention output), then LM head + acceptance + compaction in one call.
+        per_layer=False puts all layers' attention into ONE call, which is only possible when every
+        layer's q and tree K/V exist up front (an upper bound for a real decoder); fused_tail=False
+        issues the three tail calls separately."""
         if per_layer:
             for l in range(self.L):
                 self.attention(l, stream)
@@ -211,12 +212,11 @@ class VerifyStep:
             self.run(**run_args)
         return graph
 
-    @property
-    def launches_per_step(self) -> int:
-        """Kernel launches of one run(): attention (one launch per group of up to 32 layers), the
-        LM-head tiles and the fused merge/acceptance/compaction kernel."""
-        return ((self.L + sd.ATTENTION_LAYERS_PER_LAUNCH - 1) // sd.ATTENTION_LAYERS_PER_LAUNCH
-                + sd.KERNELS_PER_TAIL)
+    def launches_per_step(self, per_layer: bool = True) -> int:
+        """Kernel launches of one run(): attention (one launch per layer, or per group of up to 32 layers
+        in the all-layers call), the LM-head tiles and the fused merge/acceptance/compaction kernel."""
+        att = self.L if per_layer else (self.L + sd.ATTENTION_LAYERS_PER_LAUNCH - 1) // sd.ATTENTION_LAYERS_PER_LAUNCH
+        return att * sd.KERNELS_PER_ATTENTION + sd.KERNELS_PER_TAIL
 
     def h2d_bytes(self) -> int:
         h = self.host
@@ -226,7 +226,7 @@ class VerifyStep:
     def d2h_bytes(self) -> int:
         return sum(t.numel() * t.element_size() for t in self.host_out.values())
 
-    def run_from_host(self, group: int = 7):
+    def run_from_host(self, group: int = 7, per_layer: bool = True):
         """End-to-end step: this step's inputs come from pinned host memory, the
         accepted tokens go back to the host; caches and weights stay resident.
         The host-to-device copies run on a second stream, ahead of the compute:
@@ -234,7 +234,9 @@ class VerifyStep:
         its layers' copies have landed (an event recorded behind them).  The
         device-side input buffers exist twice and alternate from step to step,
         so the copies of step i+1 overlap the last layers and the tail of step i
-        and only wait for step i-1, which read the same buffers."""
+        and only wait for step i-1, which read the same buffers.  per_layer: one attention call
+        per layer (a decoder computes layer l + 1's q, k, v from layer l's output) instead of one
+        call per group of layers."""
         h = self.host
         main = torch.cuda.current_stream()
         if self._copy_stream is None:
@@ -267,7 +269,11 @@ class VerifyStep:
         for l0 in range(0, self.L, group):
             l1 = min(l0 + group, self.L)
             main.wait_event(self._ev_layer[slot][l1 - 1])
-            self.attention_layers(l0, l1)
+            if per_layer:
+                for l in range(l0, l1):
+                    self.attention(l)
+            else:
+                self.attention_layers(l0, l1)
         main.wait_event(ev_last)        # hidden states and draft tokens have arrived
         self.tail()
         self.host_out["n_acc"].copy_(self.n_acc, non_blocking=True)

@@ -76,8 +76,14 @@ def attention(configs=("c2", "c3", "c4", "c5", "chain11")):
 
 
 def attention_layers(configs=("c5", "chain11", "c4"), L=28):
+    for r in measure_attention_layers(configs, L):
+        print(json.dumps(r))
+
+
+def measure_attention_layers(configs=("c5", "chain11", "c4"), L=28, reps=20):
     """All L layers through sd_verify_attention_layers (one launch): the regime of a whole verify
-    step, where per-launch costs are paid once.  chain11 is the bandwidth-bound case."""
+    step, where per-launch costs are paid once.  chain11 is the bandwidth-bound case.  Yields one
+    record per workload."""
     hbm, tens, src = _peaks()
     for cfg in configs:
         sp = wl.spec(cfg)
@@ -92,19 +98,20 @@ def attention_layers(configs=("c5", "chain11", "c4"), L=28):
         out = [torch.zeros((w.B, w.T_max, w.Hq, w.D), dtype=torch.bfloat16, device="cuda") for _ in range(w.L)]
         ws = torch.empty(sd.sd_workspace_bytes(bt), dtype=torch.uint8, device="cuda")
         ls = sd.AttentionLayerSet(kc, vc, q, kt, vt, out)
-        ms = _time(lambda: sd.sd_verify_attention_layers(bt, ls, w.scale, ws, st), 20)
+        ms = _time(lambda: sd.sd_verify_attention_layers(bt, ls, w.scale, ws, st), reps)
         vis = sum(int((int(w.len[b]) + wl.node_depths(w.parents[b]) + 1).sum()) for b in range(w.B))
         flops = 4.0 * w.D * w.Hq * vis * w.L
         nbytes = (sum(int(w.len[b]) + w.T_max for b in range(w.B)) * w.Hkv * w.D * 4
                   + 2 * w.B * w.T_max * w.Hq * w.D * 2) * w.L
-        print(json.dumps({"call": "sd_verify_attention_layers", "workload": cfg, "layers": w.L, "us": ms * 1e3,
-                          "us_per_layer": ms * 1e3 / w.L,
-                          "tflops": flops / ms / 1e9, "frac_tensor_burst": flops / ms / 1e9 / tens,
-                          "gbs": nbytes / ms / 1e6, "frac_hbm": nbytes / ms / 1e6 / hbm,
-                          "frac_hbm_nominal_8TBs": nbytes / ms / 1e6 / 8000.0,
-                          "flop_per_byte": flops / nbytes, "peaks": src, "status": int(st.item())}))
+        rec = {"call": "sd_verify_attention_layers", "workload": cfg, "layers": w.L, "us": ms * 1e3,
+               "us_per_layer": ms * 1e3 / w.L,
+               "tflops": flops / ms / 1e9, "frac_tensor_burst": flops / ms / 1e9 / tens,
+               "algorithmic_bytes": nbytes, "gbs": nbytes / ms / 1e6, "frac_hbm": nbytes / ms / 1e6 / hbm,
+               "frac_hbm_nominal_8TBs": nbytes / ms / 1e6 / 8000.0,
+               "flop_per_byte": flops / nbytes, "peaks": src, "status": int(st.item())}
         del kc, vc, q, kt, vt, out, ls
         torch.cuda.empty_cache()
+        yield rec
 
 
 def lmhead(rows=(60, 240, 480, 960), V=152064, Hd=3584):
@@ -177,7 +184,11 @@ def draft(S=4096, L=28, Q=4, H=28):
                           "frac_hbm_nominal_8TBs": nbytes / ms / 1e6 / 8000.0, "bytes": nbytes, "peaks": src}))
 
 
-def compact(B=1024, L=8, T=64, Hkv=4, D=128):
+def compact(**kw):
+    print(json.dumps(measure_compact(**kw)))
+
+
+def measure_compact(B=1024, L=8, T=64, Hkv=4, D=128):
     """Stress shape for compaction: every node of every tree accepted (a 64-node chain), 1024
     sequences, 8 layers: 2 x 1.07 GB moved per call."""
     hbm, _, src = _peaks()
@@ -200,10 +211,10 @@ def compact(B=1024, L=8, T=64, Hkv=4, D=128):
     moved = 2.0 * B * T * Hkv * D * 2 * 2 * L          # read + write, K and V
     ok = all(torch.equal(kc[l][2 * b + (int(lens[b]) + 5) // 64, :, (int(lens[b]) + 5) % 64], kt[l][b, 5])
              for l in (0, L - 1) for b in (0, B - 1))
-    print(json.dumps({"call": "sd_compact_kv", "workload": f"stress B={B} L={L} all {T} nodes accepted",
-                      "us": ms * 1e3, "gbs": moved / ms / 1e6, "frac_hbm": moved / ms / 1e6 / hbm,
-                      "frac_hbm_nominal_8TBs": moved / ms / 1e6 / 8000.0, "bytes": moved, "peaks": src,
-                      "spot_check": bool(ok), "status": int(st.item())}))
+    return {"call": "sd_compact_kv", "workload": f"stress B={B} L={L} all {T} nodes accepted",
+            "us": ms * 1e3, "gbs": moved / ms / 1e6, "frac_hbm": moved / ms / 1e6 / hbm,
+            "frac_hbm_nominal_8TBs": moved / ms / 1e6 / 8000.0, "bytes": moved, "peaks": src,
+            "spot_check": bool(ok), "status": int(st.item())}
 
 
 if __name__ == "__main__":

@@ -554,26 +554,30 @@ def test_chained_step_tiny():
     np.testing.assert_array_equal(vs.v_cache[0].cpu().numpy().view(np.uint16), rv)
 
 
-def test_step_replayed_from_a_cuda_graph():
-    """The step's library calls recorded into a CUDA graph and replayed: same outputs and the same
-    cache bytes as the directly issued step (the checker's, via test_chained_step_tiny's route)."""
-    w = wl.make("c1", hidden_gain=16.0)
+@pytest.mark.parametrize("per_layer", [True, False])
+def test_step_replayed_from_a_cuda_graph(per_layer):
+    """The step's library calls (one attention call per layer, or all three layers in one call) recorded
+    into a CUDA graph and replayed: same outputs and the same cache bytes as the directly issued step
+    (the checker's, via test_chained_step_tiny's route)."""
+    w = wl.make("c1", hidden_gain=16.0, L=3)
     ram, _, _ = oracle.lmhead(w.hidden, w.W)
     wl.plant(w, ram.reshape(w.B, w.T_max), np.array([2]))
     ref_acc = oracle.accept(oracle.Geometry.of(w), w.draft_tok, ram.reshape(w.B, w.T_max))
     vs = VerifyStep(w)
-    graph = vs.capture()
+    graph = vs.capture(per_layer=per_layer)
     outs = (vs.n_acc, vs.path, vs.out_tok, vs.new_len, vs.argmax)
-    direct = [t.clone() for t in outs] + [vs.out[0].clone(), vs.k_cache[0].clone(), vs.v_cache[0].clone()]
+    state = list(vs.out) + list(vs.k_cache) + list(vs.v_cache)
+    direct = [t.clone() for t in outs] + [t.clone() for t in state]
     for t in outs:
         t.fill_(-3)
-    vs.out[0].fill_(7.0)
-    vs.k_cache[0].copy_(to_device(w.k_cache[0])); vs.v_cache[0].copy_(to_device(w.v_cache[0]))   # undo the compaction
+    for l in range(vs.L):
+        vs.out[l].fill_(7.0)
+        vs.k_cache[l].copy_(to_device(w.k_cache[l])); vs.v_cache[l].copy_(to_device(w.v_cache[l]))   # undo the compaction
     for _ in range(2):
         graph.replay()
     torch.cuda.synchronize()
     vs.check_status()
-    for got, ref in zip(list(outs) + [vs.out[0], vs.k_cache[0], vs.v_cache[0]], direct):
+    for got, ref in zip(list(outs) + state, direct):
         assert torch.equal(got, ref)
     for got, ref in zip((vs.n_acc, vs.path, vs.out_tok, vs.new_len), ref_acc):
         np.testing.assert_array_equal(got.cpu().numpy(), ref)
