@@ -15,8 +15,12 @@
 // is only raised when it grows by more than 2^8, so the accumulator in TMEM is
 // rescaled rarely.  P goes back into TMEM and feeds the second MMA from there.
 // With one chunk the CTA writes the output itself; otherwise the chunks of a row
-// tile form a thread-block cluster and merge their (max, sum, unnormalised O)
-// through distributed shared memory in a fixed order.
+// tile form a thread-block cluster: every CTA pushes its (max, sum, unnormalised
+// O) rows into the shared memory of the CTA that finishes them (remote stores),
+// and each CTA merges its share of the rows locally, in chunk order.
+// The launch is a programmatic dependent launch: barriers, tensor memory and
+// tensor-map prefetch are set up before the kernel waits for the kernel ahead of
+// it in the stream, so consecutive per-layer calls overlap their ends.
 #include "attention_shared.cuh"
 
 namespace sdv {
@@ -71,6 +75,42 @@ attn_umma_kernel(const __grid_constant__ AttnLayers<NL> layers, const sd_batch b
     const int kvh = zz % bt.Hkv;
     const int lb = zz / bt.Hkv;
     const int rank_b = lb / plan.n_layers;
+    const AttnLayer& ly = layers.l[lb % plan.n_layers];
+    const CUtensorMap* const map_kc = &ly.k_cache;
+    const CUtensorMap* const map_vc = &ly.v_cache;
+    const CUtensorMap* const map_kt = &ly.k_tree;
+    const CUtensorMap* const map_vt = &ly.v_tree;
+
+    // Set-up that touches no global memory comes first: when the launch is allowed to start before the
+    // kernel ahead of it in the stream has finished (programmatic dependent launch: one attention call
+    // per layer, back to back), it overlaps that kernel's tail.  The kernel behind this one may start
+    // its own set-up as soon as every CTA of this grid is running.
+    griddep_launch_dependents();
+    const bool aligned = (smem_u32(smem) & 1023u) == 0;    // swizzled tiles need 1 KiB alignment
+    uint32_t tmem_base = 0;
+    if (aligned) {
+        if (warp == kMmaWarp) {                            // (a thread with nothing else to do at this point)
+            *abort_flag = 0;
+            for (int i = 0; i < kKStages; ++i) { mbar_init(&k_full[i], 1); mbar_init(&k_empty[i], 1); }
+            for (int i = 0; i < kVStages; ++i) { mbar_init(&v_full[i], 1); mbar_init(&v_empty[i], 1); }
+            for (int i = 0; i < 2; ++i) { mbar_init(&s_full[i], 1); mbar_init(&p_full[i], 4); }
+            mbar_init(pv_done, 1); mbar_init(q_full, 4); mbar_init(o_full, 1);
+            fence_barrier_init();
+        }
+        if (warp == kTmaWarp) {                            // a full warp (the MMA warp is a single thread)
+            tmem_alloc(tmem_slot, kTmemCols);
+            tmem_relinquish();
+        }
+        if (warp == kTmaWarp && lane == 0) {
+            prefetch_tensormap(map_kc); prefetch_tensormap(map_vc);
+            prefetch_tensormap(map_kt); prefetch_tensormap(map_vt);
+        }
+    } else if (threadIdx.x == 0) {
+        set_status(status, SD_ERR_UNSUPPORTED);
+    }
+    // everything below reads (or writes) global memory that the kernel ahead may still be working on
+    griddep_wait();
+
     int b = rank_b;
     if (plan.ranked) {
         // (the slot lives in the dynamic shared-memory block: a static variable would push that block's
@@ -88,19 +128,32 @@ attn_umma_kernel(const __grid_constant__ AttnLayers<NL> layers, const sd_batch b
         __syncthreads();
         b = s_seq;
     }
-    const AttnLayer& ly = layers.l[lb % plan.n_layers];
-    const CUtensorMap* const map_kc = &ly.k_cache;
-    const CUtensorMap* const map_vc = &ly.v_cache;
-    const CUtensorMap* const map_kt = &ly.k_tree;
-    const CUtensorMap* const map_vt = &ly.v_tree;
     const uint16_t* __restrict__ q = ly.q;
     __nv_bfloat16* __restrict__ out = ly.out;
     float* __restrict__ lse = ly.lse;
     const int num_blocks = ly.num_blocks;
     const int G = bt.Hq / bt.Hkv;
     const int T = bt.T_max;
-    const int n = min(max(bt.n_nodes[b], 0), T);
-    const int len = max(bt.len[b], 0);
+    // A last row tile of at most 64 rows (420 rows = 3 x 128 + 36) runs its MMAs with M = 64: the
+    // accumulator rows then sit in lanes 0..15 of each 32-lane TMEM quadrant (row = 16 * quadrant + lane),
+    // the tensor cores work at half width and only 64 rows of Q are staged and re-read per key tile.
+    const bool m64 = (plan.rows - rt * kRowTile) <= 64;
+    // The softmax threads request their row of Q together with the lengths, before anything waits for
+    // either.  A node index below T_max always addresses memory of q; rows of unused nodes are replaced
+    // by zeros when staged.
+    const int q_tid = warp * 32 + lane;
+    const int q_row_in_tile = (warp >= 4) ? -1 : (m64 ? (lane < 16 ? warp * 16 + lane : -1) : q_tid);   // -1: no row
+    const int q_row = (q_row_in_tile >= 0) ? rt * kRowTile + q_row_in_tile : plan.rows;
+    const int n = min(max(__ldg(bt.n_nodes + b), 0), T);      // (requested before the row, needed before it)
+    const int len = max(__ldg(bt.len + b), 0);
+    uint4 q_regs[16];
+    if (q_row < plan.rows) {
+        const int node = q_row / G;
+        const uint4* src = reinterpret_cast<const uint4*>(
+            q + (((size_t)b * T + node) * bt.Hq + kvh * G + (q_row - node * G)) * kD);
+#pragma unroll
+        for (int c = 0; c < 16; ++c) q_regs[c] = __ldg(src + c);
+    }
 
     // key tiles of this CTA: cache blocks [t0, t1) and, for the last chunk, the tree tile
     int tiles_total = (len + kKeyTile - 1) / kKeyTile;
@@ -113,42 +166,21 @@ attn_umma_kernel(const __grid_constant__ AttnLayers<NL> layers, const sd_batch b
     const int t1 = min(t0 + tpc, tiles_total);
     const bool has_tree = (chunk == plan.n_chunks - 1);
     const int nt = (t1 - t0) + (has_tree ? 1 : 0);
-    const bool aligned = (smem_u32(smem) & 1023u) == 0;    // swizzled tiles need 1 KiB alignment
-    if (!aligned && threadIdx.x == 0) set_status(status, SD_ERR_UNSUPPORTED);
     // A CTA without key tiles has nothing to compute, but it still takes part in the cluster barriers.
     const bool active = (nt > 0) && aligned;
     const bool clustered = (plan.n_chunks > 1);            // cluster = the chunks of one (b, kvh, row tile)
-    // A last row tile of at most 64 rows (420 rows = 3 x 128 + 36) runs its MMAs with M = 64: the
-    // accumulator rows then sit in lanes 0..15 of each 32-lane TMEM quadrant (row = 16 * quadrant + lane),
-    // the tensor cores work at half width and only 64 rows of Q are staged and re-read per key tile.
-    const bool m64 = (plan.rows - rt * kRowTile) <= 64;
     float m_used = -INFINITY, l = 0.f;                     // softmax state of this thread's row (warps 0-3)
-    uint32_t tmem_base = 0;
+    bool rows_ready = false;                               // ... and whether it completed (clustered launches)
 
-    if (active) {
-    if (threadIdx.x == 0) {
-        *abort_flag = 0;
-        for (int i = 0; i < kKStages; ++i) { mbar_init(&k_full[i], 1); mbar_init(&k_empty[i], 1); }
-        for (int i = 0; i < kVStages; ++i) { mbar_init(&v_full[i], 1); mbar_init(&v_empty[i], 1); }
-        for (int i = 0; i < 2; ++i) { mbar_init(&s_full[i], 1); mbar_init(&p_full[i], 4); }
-        mbar_init(pv_done, 1); mbar_init(q_full, 4); mbar_init(o_full, 1);
-        fence_barrier_init();
-    }
-    if (warp == kTmaWarp) {                                // a full warp (the MMA warp is a single thread)
-        tmem_alloc(tmem_slot, kTmemCols);
-        tmem_relinquish();
-    }
-    if (warp == kTmaWarp && lane == 0) {
-        prefetch_tensormap(map_kc); prefetch_tensormap(map_vc);
-        prefetch_tensormap(map_kt); prefetch_tensormap(map_vt);
-    }
+    // the set-up at the top (barriers, tensor memory) is visible to every thread from here on
     tc_fence_before_sync();
     __syncthreads();
     tc_fence_after_sync();
-    tmem_base = *tmem_slot;
+    if (aligned) tmem_base = *tmem_slot;
     const uint32_t tmem_o = tmem_base;
     const uint32_t tmem_s = tmem_base + 128;
 
+    if (active) {
     if (warp == kTmaWarp) {
         // ------------------------------------------------------------ TMA producer (one thread)
         // K and V tiles travel through separate rings and are issued independently, whichever slot
@@ -272,11 +304,9 @@ attn_umma_kernel(const __grid_constant__ AttnLayers<NL> layers, const sd_batch b
         const int g = row - node * G;
         const bool row_ok = (row < plan.rows) && (node < n);
         {   // stage this row of Q (zeros for padding rows) in the swizzled K-major layout
-            const uint4* src = reinterpret_cast<const uint4*>(
-                q + (((size_t)b * T + (row_ok ? node : 0)) * bt.Hq + kvh * G + (row_ok ? g : 0)) * kD);
 #pragma unroll
             for (int c = 0; c < 16; ++c) {
-                uint4 u = row_ok ? __ldg(src + c) : make_uint4(0, 0, 0, 0);
+                uint4 u = row_ok ? q_regs[c] : make_uint4(0, 0, 0, 0);
                 uint8_t* dst = q_smem + (c >> 3) * (kRowTile * 128) + row_in_tile * 128 + (((c & 7) ^ (row_in_tile & 7)) << 4);
                 if (row_in_tile >= 0) *reinterpret_cast<uint4*>(dst) = u;
             }
@@ -442,29 +472,7 @@ attn_umma_kernel(const __grid_constant__ AttnLayers<NL> layers, const sd_batch b
             }
             if (row < plan.rows && lse) lse[orow] = row_ok ? (m_used + log2f(l)) * 0.6931471805599453f : 0.f;
         } else if (ok) {
-            // several chunks: park (m, l, unnormalised O) in this CTA's own shared memory, where the
-            // CTAs of the cluster read it.  The K/V rings are idle by now (every MMA has completed).
-            // 16-byte pieces of a row are XOR-swizzled by the row index so that the per-row accesses
-            // of a warp spread over the banks.
-            tc_fence_after_sync();
-            float* xo = reinterpret_cast<float*>(k_smem);
-            float* xs = xo + kRowTile * kD;
-#pragma unroll
-            for (int cc = 0; cc < 4; ++cc) {
-                uint32_t o[32];
-                tmem_ld32(tmem_o + lane_field + cc * 32, o);
-                tmem_ld_wait();
-                if (row_in_tile >= 0) {
-#pragma unroll
-                    for (int k = 0; k < 8; ++k)
-                        *reinterpret_cast<uint4*>(xo + row_in_tile * kD + (((cc * 8 + k) ^ (row_in_tile & 31)) << 2)) =
-                            make_uint4(o[4 * k], o[4 * k + 1], o[4 * k + 2], o[4 * k + 3]);
-                }
-            }
-            if (row_in_tile >= 0) {
-                xs[row_in_tile] = m_used;
-                xs[kRowTile + row_in_tile] = l;
-            }
+            rows_ready = true;         // several chunks: the rows leave for their finishing CTAs below
         } else if (!ok && lane == 0) {
             set_status(status, SD_ERR_TIMEOUT);
         }
@@ -472,7 +480,42 @@ attn_umma_kernel(const __grid_constant__ AttnLayers<NL> layers, const sd_batch b
     }   // active
 
     if (clustered) {
-        // every thread of every CTA of the cluster: exchange areas are complete and visible
+        // every thread of every CTA of the cluster: all MMAs and copies of the cluster have completed, so
+        // every CTA's K/V rings are free to receive rows
+        __syncwarp();
+        cluster_arrive_release();
+        cluster_wait_acquire();
+        if (active && warp < 4) {
+            // Each row (maximum, sum, unnormalised O) goes straight from tensor memory into the shared
+            // memory of the CTA that finishes it: remote stores stream, remote loads would each cost a
+            // round trip.  Row r of the tile is finished by the CTA of chunk r / (128 / n_chunks).
+            const int rows_per = kRowTile / plan.n_chunks;
+            const int tid = warp * 32 + lane;
+            const int row_in_tile = m64 ? (lane < 16 ? warp * 16 + lane : -1) : tid;
+            const int rr = max(row_in_tile, 0);
+            const int slot = chunk * rows_per + rr % rows_per;
+            const uint32_t xo_remote = map_dsmem(smem_u32(k_smem), (uint32_t)(rr / rows_per));
+            const uint32_t xs_remote = xo_remote + kRowTile * kD * 4;
+            const bool mine = rows_ready && row_in_tile >= 0;
+            tc_fence_after_sync();
+#pragma unroll
+            for (int cc = 0; cc < 4; ++cc) {
+                uint32_t o[32];
+                tmem_ld32(tmem_base + ((uint32_t)(warp * 32) << 16) + cc * 32, o);
+                tmem_ld_wait();
+                if (mine) {
+#pragma unroll
+                    for (int k = 0; k < 8; ++k)
+                        st_dsmem_v4(xo_remote + (uint32_t)(slot * kD + (((cc * 8 + k) ^ (slot & 31)) << 2)) * 4,
+                                    o[4 * k], o[4 * k + 1], o[4 * k + 2], o[4 * k + 3]);
+                }
+            }
+            if (mine) {
+                st_dsmem_f32(xs_remote + slot * 4, m_used);
+                st_dsmem_f32(xs_remote + (kRowTile + slot) * 4, l);
+            }
+        }
+        // all rows have landed where they are finished
         __syncwarp();
         cluster_arrive_release();
         cluster_wait_acquire();
@@ -484,12 +527,8 @@ attn_umma_kernel(const __grid_constant__ AttnLayers<NL> layers, const sd_batch b
             else if (plan.n_chunks == 4) merge_rows<4>(mc);
             else merge_rows<8>(mc);
         }
-        // every CTA keeps its shared memory alive until all the others have read it
-        __syncwarp();
-        cluster_arrive_release();
-        cluster_wait_acquire();
     }
-    if (!active) return;
+    if (!aligned) return;
     tc_fence_before_sync();
     __syncthreads();
     if (warp == kTmaWarp) {
@@ -528,13 +567,18 @@ sd_status launch_rows1(const AttnLayers<NL>& layers, const sd_batch& bt, float s
     cfg.blockDim = dim3(kAttThreads);
     cfg.dynamicSmemBytes = kAttSmem;
     cfg.stream = st;
-    cudaLaunchAttribute attr[1];
+    cudaLaunchAttribute attr[2];
     attr[0].id = cudaLaunchAttributeClusterDimension;      // the chunks of one row tile form a cluster
     attr[0].val.clusterDim.x = plan.n_chunks;
     attr[0].val.clusterDim.y = 1;
     attr[0].val.clusterDim.z = 1;
+    // The launch may begin while the kernel before it in the stream is still running (its CTAs take the
+    // SM slots that one frees and do their set-up); the kernel waits for that kernel's completion before
+    // it touches global memory.  Consecutive attention calls - one per layer - overlap their ends this way.
+    attr[1].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+    attr[1].val.programmaticStreamSerializationAllowed = 1;
     cfg.attrs = attr;
-    cfg.numAttrs = 1;
+    cfg.numAttrs = 2;
     if (cudaLaunchKernelEx(&cfg, kern, layers, bt, scale * kLog2e, plan, dev_status) != cudaSuccess)
         return SD_ERR_CUDA;
     return SD_OK;

@@ -51,78 +51,86 @@ constexpr int kMaxLayersPerLaunch = 32;
 template <int NL>
 struct AttnLayers { AttnLayer l[NL]; };
 
-// Final step of a clustered launch.  Each CTA of the cluster finishes 128 / NCH rows of the tile: a
-// warp takes a few rows at a time, every lane four output columns, and adds up the chunks in chunk
-// order (so the result does not depend on timing).  A row of a parked tile is one contiguous
-// 512-byte line of the owning CTA's shared memory; all loads of a batch of rows are issued before
-// any of them is used, so that their latencies overlap.
+// Final step of a clustered launch.  Chunk c's CTA has PUSHED its unnormalised rows (and their
+// maximum and sum) into the shared memory of the CTA that finishes them: the CTA of chunk o owns rows
+// o * 128 / NCH .. of the tile and holds, for each of its rows, one slot per chunk (slot = c * rows
+// per CTA + local row).  Every read here is local.  A warp takes a few rows at a time, every lane
+// four output columns, and adds up the chunks in chunk order (so the result does not depend on
+// timing).  A slot is one contiguous 512-byte line whose 16-byte pieces are XOR-swizzled by the slot
+// index (the pushing threads write one row each: without the swizzle a warp's stores would meet in
+// one bank group).
 struct MergeCtx {
     const sd_batch& bt; const AttnPlan& plan; __nv_bfloat16* out; float* lse;
-    uint32_t xo_addr, xs_addr;
+    uint32_t xo_addr, xs_addr;          // this CTA's exchange area: rows, then maxima [128] and sums [128]
     int chunk, rt, b, kvh, n, tpc, tiles_total, warp, lane;
 };
 
 template <int NCH>
 __device__ __forceinline__ void merge_rows(const MergeCtx& x) {
-    constexpr int kRowsPer = kRowTile / NCH;
-    constexpr int kBatch = 16 / NCH;                // rows in flight per warp
+    // Eight lanes per row (16 output columns each), four rows per warp at a time; the warp's rows are
+    // consecutive, so node and head within the group are counted up instead of divided out.
+    constexpr int kRowsPer = kRowTile / NCH;        // rows this CTA finishes
+    constexpr int kPerWarp = kRowsPer / 4;          // ... and each of its four warps (a multiple of 4)
     const int G = x.bt.Hq / x.bt.Hkv;
-    for (int i0 = x.warp * kBatch; i0 < kRowsPer; i0 += 4 * kBatch) {
-        float mc[kBatch][NCH], lc[kBatch][NCH];
-        float4 v[kBatch][NCH];
+    const int sub = x.lane >> 3, ql = x.lane & 7;
+    const int first = x.rt * kRowTile + x.chunk * kRowsPer + x.warp * kPerWarp + sub;   // this lane's first row
+    int node = first / G;
+    int g = first - node * G;
+#pragma unroll 1
+    for (int i = 0; i < kPerWarp; i += 4) {
+        const int rl = x.warp * kPerWarp + i + sub;             // row among this CTA's rows
+        const int row = first + i;
+        float mc[NCH];
+        float M = -INFINITY;
 #pragma unroll
-        for (int u = 0; u < kBatch; ++u) {
-            const int r = x.chunk * kRowsPer + i0 + u;
+        for (int c = 0; c < NCH; ++c) {
+            const bool live = (c == NCH - 1) || (c * x.tpc < x.tiles_total);   // that chunk had key tiles
+            mc[c] = live ? ld_smem_f32(x.xs_addr + (c * kRowsPer + rl) * 4) : -INFINITY;
+            M = fmaxf(M, mc[c]);
+        }
+        float den = 0.f;
+        float4 acc[4];
 #pragma unroll
-            for (int c = 0; c < NCH; ++c) {
-                const bool live = (c == NCH - 1) || (c * x.tpc < x.tiles_total);   // that chunk had key tiles
-                mc[u][c] = -INFINITY; lc[u][c] = 0.f; v[u][c] = make_float4(0.f, 0.f, 0.f, 0.f);
-                if (live && c == x.chunk) {                  // this CTA's own chunk: plain shared-memory reads
-                    mc[u][c] = ld_smem_f32(x.xs_addr + r * 4);
-                    lc[u][c] = ld_smem_f32(x.xs_addr + (kRowTile + r) * 4);
-                    v[u][c] = ld_smem_v4(x.xo_addr + (uint32_t)(r * kD + ((x.lane ^ (r & 31)) << 2)) * 4);
-                } else if (live) {
-                    mc[u][c] = ld_dsmem_f32(map_dsmem(x.xs_addr + r * 4, c));
-                    lc[u][c] = ld_dsmem_f32(map_dsmem(x.xs_addr + (kRowTile + r) * 4, c));
-                    v[u][c] = ld_dsmem_v4(map_dsmem(x.xo_addr + (uint32_t)(r * kD + ((x.lane ^ (r & 31)) << 2)) * 4, c));
-                }
+        for (int p = 0; p < 4; ++p) acc[p] = make_float4(0.f, 0.f, 0.f, 0.f);
+#pragma unroll
+        for (int c = 0; c < NCH; ++c) {
+            if (mc[c] == -INFINITY) continue;                    // a chunk without tiles
+            const int slot = c * kRowsPer + rl;
+            const float w = ex2_approx(mc[c] - M);
+            den = fmaf(w, ld_smem_f32(x.xs_addr + (kRowTile + slot) * 4), den);
+#pragma unroll
+            for (int p = 0; p < 4; ++p) {
+                const float4 v = ld_smem_v4(x.xo_addr + (uint32_t)(slot * kD + (((ql * 4 + p) ^ (slot & 31)) << 2)) * 4);
+                acc[p].x = fmaf(w, v.x, acc[p].x); acc[p].y = fmaf(w, v.y, acc[p].y);
+                acc[p].z = fmaf(w, v.z, acc[p].z); acc[p].w = fmaf(w, v.w, acc[p].w);
             }
         }
-#pragma unroll
-        for (int u = 0; u < kBatch; ++u) {
-            const int r = x.chunk * kRowsPer + i0 + u;
-            const int row = x.rt * kRowTile + r;
-            if (row >= x.plan.rows) continue;
-            const int node = row / G;
-            const int g = row - node * G;
+        if (row < x.plan.rows) {
             const size_t orow = ((size_t)x.b * x.bt.T_max + node) * x.bt.Hq + x.kvh * G + g;
-            uint2* dst = reinterpret_cast<uint2*>(x.out + orow * kD + x.lane * 4);
-            if (node >= x.n) {                               // unused node: zero row
-                *dst = make_uint2(0, 0);
-                if (x.lse && x.lane == 0) x.lse[orow] = 0.f;
-                continue;
-            }
-            float M = mc[u][0];
+            uint4* dst = reinterpret_cast<uint4*>(x.out + orow * kD + ql * 16);
+            if (node >= x.n) {                                   // unused node: zero row
+                dst[0] = make_uint4(0, 0, 0, 0);
+                dst[1] = make_uint4(0, 0, 0, 0);
+                if (x.lse && ql == 0) x.lse[orow] = 0.f;
+            } else {
+                const float inv = __frcp_rn(den);
+                uint32_t w[8];
 #pragma unroll
-            for (int c = 1; c < NCH; ++c) M = fmaxf(M, mc[u][c]);
-            float den = 0.f;
-            float4 acc = make_float4(0.f, 0.f, 0.f, 0.f);
-#pragma unroll
-            for (int c = 0; c < NCH; ++c) {
-                const float w = exp2f(mc[u][c] - M);         // 0 for a chunk without tiles (m = -inf)
-                den = fmaf(w, lc[u][c], den);
-                acc.x = fmaf(w, v[u][c].x, acc.x); acc.y = fmaf(w, v[u][c].y, acc.y);
-                acc.z = fmaf(w, v[u][c].z, acc.z); acc.w = fmaf(w, v[u][c].w, acc.w);
+                for (int p = 0; p < 4; ++p) {
+                    __nv_bfloat162 h0 = __floats2bfloat162_rn(acc[p].x * inv, acc[p].y * inv);
+                    __nv_bfloat162 h1 = __floats2bfloat162_rn(acc[p].z * inv, acc[p].w * inv);
+                    w[2 * p] = *reinterpret_cast<uint32_t*>(&h0);
+                    w[2 * p + 1] = *reinterpret_cast<uint32_t*>(&h1);
+                }
+                dst[0] = make_uint4(w[0], w[1], w[2], w[3]);
+                dst[1] = make_uint4(w[4], w[5], w[6], w[7]);
+                if (x.lse && ql == 0) x.lse[orow] = (M + __log2f(den)) * 0.6931471805599453f;
             }
-            const float inv = 1.f / den;
-            __nv_bfloat162 h0 = __floats2bfloat162_rn(acc.x * inv, acc.y * inv);
-            __nv_bfloat162 h1 = __floats2bfloat162_rn(acc.z * inv, acc.w * inv);
-            *dst = make_uint2(*reinterpret_cast<uint32_t*>(&h0), *reinterpret_cast<uint32_t*>(&h1));
-            if (x.lse && x.lane == 0) x.lse[orow] = (M + log2f(den)) * 0.6931471805599453f;
         }
+        g += 4;                                                  // the next group's row: four further on
+        while (g >= G) { g -= G; ++node; }
     }
 }
-
 
 // one launch of `z_count` (sequence rank, layer, KV head) groups starting at plan.z0
 template <int NL>
