@@ -244,6 +244,8 @@ def main():
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--no-supplements", action="store_true",
                     help="skip the chain-decoding and compaction-stress measurements (profiler captures)")
+    ap.add_argument("--repeats", type=int, default=0,
+                    help="measurements of K steps each (default: as many as make about a second of timed work)")
     ap.add_argument("--layers", type=int, default=0,
                     help="override the number of layers (small cases for profiler captures only)")
     args = ap.parse_args()
@@ -307,7 +309,7 @@ def main():
     barrier()
     vs.check_status()
     probe = timed_repeats(graph.replay, 1)[0]                    # untimed estimate: how many repeats make a second
-    repeats = int(min(50, max(1, math.ceil(1000.0 / max(probe, 1e-3)))))
+    repeats = args.repeats if args.repeats > 0 else int(min(50, max(1, math.ceil(1000.0 / max(probe, 1e-3)))))
     if rank == 0:
         sampler.wait_first()
     m0 = sampler.mark() if rank == 0 else 0

@@ -3,6 +3,7 @@ the LM head at several row counts, and the bandwidth-regime cases (chain
 decoding, a compaction stress shape).  One JSON line per measurement.
 
     python -m paper_2509_18824_b200.supplements [attention] [attention_layers] [lmhead] [lmhead480] [sampled] [draft] [compact]
+                                                [chain8] [compact512]        (small cases for profiler captures)
 
 Timing: CUDA events on the launching stream, >= 3 warm-up calls, inputs rotated
 over several layers so that the working set exceeds L2.
@@ -233,3 +234,8 @@ if __name__ == "__main__":
         draft()
     if "compact" in what:
         compact()
+    if "chain8" in what:                   # chain decoding, 8 layers in one call (0.55 GB of K/V)
+        for r in measure_attention_layers(("chain11",), L=8, reps=3):
+            print(json.dumps(r))
+    if "compact512" in what:               # half the stress shape: 1.07 GB moved per call
+        compact(B=512)

@@ -154,6 +154,49 @@ def test_attention_planted_key_large_v_and_bad_block_table():
     assert status == sd.SD_ERR_BOUNDS
 
 
+def test_attention_length_beyond_the_block_table_is_reported():
+    """A cached length that needs more blocks than max_blocks_per_seq is an error (SD_ERR_BOUNDS in the
+    status word), not a silently shortened sequence."""
+    p = tiny128(7, B=2, T=8, Hq=4, Hkv=2, lens=(100, 40), gain=2.0)
+    _, _, status = gpu_attention(p)
+    assert status == 0
+    p.len = p.len.copy(); p.len[1] = 64 * p.block_table.shape[1] + 1
+    _, _, status = gpu_attention(p)
+    assert status == sd.SD_ERR_BOUNDS
+
+
+def test_compaction_reports_a_corrupt_block_table_entry():
+    """Block-table entries of -2 (and any other value outside [0, num_blocks)) under an accepted node are
+    reported as SD_ERR_BOUNDS and nothing is written through them."""
+    sp = wl.spec("c5"); sp.L = 2; sp.prefix = 100; sp.B = 3
+    w = wl.make_geometry(sp)
+    wl.fill_attention(w)
+    g = np.random.default_rng(6)
+    target = g.integers(0, 5, size=(w.B, w.T_max)).astype(np.int32)
+    wl.plant(w, target, np.array([3, 2, 4]))
+    n_acc, path, _, _ = oracle.accept(oracle.Geometry.of(w), w.draft_tok, target)
+    for bad in (-2, -1, 10 ** 6):
+        w2_table = w.block_table.copy()
+        w2_table[1, int(w.len[1]) // 64] = bad            # the block that sequence 1's accepted rows go to
+        geo = type("G", (), dict(B=w.B, T_max=w.T_max, Hq=w.Hq, Hkv=w.Hkv, D=w.D, block_table=w2_table,
+                                 len=w.len, n_nodes=w.n_nodes, parents=w.parents))
+        bt = sd.Batch.of(geo)
+        st = sd.new_status()
+        kc = [to_device(x) for x in w.k_cache]; vc = [to_device(x) for x in w.v_cache]
+        kt = [to_device(x) for x in w.k_tree]; vt = [to_device(x) for x in w.v_tree]
+        sd.sd_compact_kv(bt, sd.LayerSet(kc, vc, kt, vt), to_device(n_acc), to_device(path), st)
+        torch.cuda.synchronize()
+        assert int(st.item()) == sd.SD_ERR_BOUNDS, bad
+        # sequences 0 and 2 were compacted as usual, sequence 1 wrote nothing
+        G2 = oracle.Geometry(w.B, w.T_max, w.Hq, w.Hkv, w.D, w.block_table, w.len, w.n_nodes, w.parents)
+        na2 = n_acc.copy(); na2[1] = 0
+        for l in range(w.L):
+            rk, rv = w.k_cache[l].copy(), w.v_cache[l].copy()
+            oracle.compact(G2, rk, rv, w.k_tree[l], w.v_tree[l], na2, path)
+            np.testing.assert_array_equal(kc[l].cpu().numpy().view(np.uint16), rk)
+            np.testing.assert_array_equal(vc[l].cpu().numpy().view(np.uint16), rv)
+
+
 def test_attention_any_bit_pattern_in_invisible_slots():
     """Cache slots at and beyond len, and the K/V rows of unused tree nodes, may hold NaN and
     infinity bit patterns (memory that was never written): no key there is visible to any row, so
