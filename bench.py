@@ -39,7 +39,7 @@ sys.path.insert(0, ROOT)
 # dram__bytes_read.sum + dram__bytes_write.sum of one single-layer launch of attn_umma_kernel, from the ncu
 # capture summarised under profiles/.  Set an entry to None whenever the kernel changes until the counters
 # are retaken.
-ATTENTION_DRAM_BYTES_PER_LAUNCH = {"c5": None}
+ATTENTION_DRAM_BYTES_PER_LAUNCH = {"c5": 75.0e6}
 
 METRIC = "tree_verify_steps_per_s"
 UNIT = "steps/s"
