@@ -76,7 +76,9 @@ __device__ __forceinline__ void merge_rows(const MergeCtx& x) {
     const int first = x.rt * kRowTile + x.chunk * kRowsPer + x.warp * kPerWarp + sub;   // this lane's first row
     int node = first / G;
     int g = first - node * G;
-#pragma unroll 1
+    // (unrolled: the groups are independent, and one warp per scheduler partition has nothing else to
+    //  hide the latency of a group's dependent loads, exponentials and stores behind)
+#pragma unroll
     for (int i = 0; i < kPerWarp; i += 4) {
         const int rl = x.warp * kPerWarp + i + sub;             // row among this CTA's rows
         const int row = first + i;
