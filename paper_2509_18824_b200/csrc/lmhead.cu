@@ -180,6 +180,105 @@ __device__ __forceinline__ void merge_sumexp(float& ref, float& sum, float ref2,
     else            { sum += sum2 * ex2_lm((ref2 - ref) * c2); }
 }
 
+// ---------------------------------------------------------------------------
+// Epilogue shared by the one-CTA and the two-CTA kernel.  Warp w of the eight epilogue warps works on
+// TMEM lanes 32 * (w & 3) .. +31 (the only ones it may read) and on the 32-column chunks of parity
+// w >> 2; per (warp, column) it keeps a running best (value, vocabulary row) and, for the soft-max
+// statistics, a running (reference, sum).
+// ---------------------------------------------------------------------------
+struct EpiState {
+    float best_val[kMaxCols / 64];
+    int32_t best_idx[kMaxCols / 64];
+    float run_ref[kMaxCols / 64], run_sum[kMaxCols / 64];
+};
+
+__device__ __forceinline__ void epi_init(EpiState& e) {
+#pragma unroll
+    for (int c = 0; c < kMaxCols / 64; ++c) {
+        e.best_val[c] = -INFINITY; e.best_idx[c] = 0x7fffffff; e.run_ref[c] = -INFINITY; e.run_sum[c] = 0.f;
+    }
+}
+
+// one accumulator tile (128 vocabulary rows from v_base - 32 * quad on; this warp's 32 of them start at v_base)
+__device__ __forceinline__ void epi_tile(const LmParams& p, EpiState& e, uint32_t taddr, int v_base, int lane, int par) {
+    const bool stats = p.c2 > 0.f;
+    const bool v_ok = (v_base + lane) < p.V;
+#pragma unroll
+    for (int h = 0; h < kMaxCols / 64; ++h) {
+        const int c = 2 * h + par;                 // this warp's chunk of the pair (2h, 2h + 1)
+        if (c * 32 < p.n_pad) {
+            uint32_t r[32];
+            tmem_ld32(taddr + c * 32, r);
+            tmem_ld_wait();
+            float cv;
+            int32_t ci;
+            if (p.mass_out) {
+                if (v_ok) {
+#pragma unroll
+                    for (int j = 0; j < 32; ++j) {
+                        const int row = c * 32 + j;
+                        if (row < p.rows)
+                            p.mass_out[(size_t)(p.row0 + row) * p.V + v_base + lane] =
+                                __expf(__uint_as_float(r[j]) * p.inv_temp - __ldg(p.col_lse + p.row0 + row));
+                    }
+                }
+                continue;
+            }
+            if (stats) {
+                float cs;
+                column_argmax_stats32(r, v_ok, v_base, lane, p.c2, cv, ci, cs);
+                merge_sumexp(e.run_ref[h], e.run_sum[h], cv, cs, p.c2);
+                if (p.group_stats && v_base < p.V && c * 32 + lane < p.rows)
+                    p.group_stats[(size_t)(v_base >> 5) * p.M_total + p.row0 + c * 32 + lane] = make_float2(cv, cs);
+            } else {
+                column_argmax32(r, v_ok, v_base, lane, cv, ci);
+            }
+            if (cv > e.best_val[h]) { e.best_val[h] = cv; e.best_idx[h] = ci; }
+        }
+    }
+}
+
+// After the last tile: the four lane quadrants' results are merged through shared memory (the pipeline
+// stages are idle by now: the last accumulator was complete, so every copy has landed and every MMA has
+// read it) and this CTA's row of the candidate tables is written.
+__device__ __forceinline__ void epi_finish(const LmParams& p, const EpiState& e, uint8_t* smem, int quad, int par,
+                                           int lane, bool ok, int32_t* status) {
+    const bool stats = p.c2 > 0.f;
+    asm volatile("bar.sync 1, %0;" ::"n"(kEpiWarps * 32) : "memory");
+    int32_t* red_key = reinterpret_cast<int32_t*>(smem);
+    int32_t* red_idx = red_key + 4 * kMaxCols;
+    float* red_ref = reinterpret_cast<float*>(red_idx + 4 * kMaxCols);
+    float* red_sum = red_ref + 4 * kMaxCols;
+#pragma unroll
+    for (int h = 0; h < kMaxCols / 64; ++h) {
+        red_key[quad * kMaxCols + (2 * h + par) * 32 + lane] = ordered_key(__float_as_uint(e.best_val[h]));
+        red_idx[quad * kMaxCols + (2 * h + par) * 32 + lane] = e.best_idx[h];
+        if (stats) {
+            red_ref[quad * kMaxCols + (2 * h + par) * 32 + lane] = e.run_ref[h];
+            red_sum[quad * kMaxCols + (2 * h + par) * 32 + lane] = e.run_sum[h];
+        }
+    }
+    asm volatile("bar.sync 1, %0;" ::"n"(kEpiWarps * 32) : "memory");
+    for (int col = threadIdx.x; col < kMaxCols; col += kEpiWarps * 32) {
+        int32_t k = red_key[col], i = red_idx[col];
+#pragma unroll
+        for (int w = 1; w < 4; ++w) {
+            const int32_t k2 = red_key[w * kMaxCols + col], i2 = red_idx[w * kMaxCols + col];
+            if (k2 > k || (k2 == k && i2 < i)) { k = k2; i = i2; }
+        }
+        if (!ok && col == (int)threadIdx.x) set_status(status, SD_ERR_TIMEOUT);
+        p.part_key[(size_t)blockIdx.x * kMaxCols + col] = ok ? k : INT32_MIN;
+        p.part_idx[(size_t)blockIdx.x * kMaxCols + col] = i;
+        if (stats) {
+            float rf = red_ref[col], sm = red_sum[col];
+#pragma unroll
+            for (int w = 1; w < 4; ++w) merge_sumexp(rf, sm, red_ref[w * kMaxCols + col], red_sum[w * kMaxCols + col], p.c2);
+            p.part_ref[(size_t)blockIdx.x * kMaxCols + col] = rf;
+            p.part_sum[(size_t)blockIdx.x * kMaxCols + col] = sm;
+        }
+    }
+}
+
 template <int BK>
 __global__ void __launch_bounds__(kLmThreads, 1)
 lmhead_umma_kernel(const __grid_constant__ CUtensorMap tmW, const __grid_constant__ CUtensorMap tmH,
@@ -288,17 +387,9 @@ lmhead_umma_kernel(const __grid_constant__ CUtensorMap tmW, const __grid_constan
         }
     } else {
         // ------------------------------------------------ epilogue warps 0..7
-        // warp w works on TMEM lanes 32 * (w & 3) .. +31 (the only ones it may read) and on the
-        // 32-column chunks of parity w >> 2
         const int quad = warp & 3, par = warp >> 2;
-        float best_val[kMaxCols / 64];
-        int32_t best_idx[kMaxCols / 64];
-        float run_ref[kMaxCols / 64], run_sum[kMaxCols / 64];
-#pragma unroll
-        for (int c = 0; c < kMaxCols / 64; ++c) {
-            best_val[c] = -INFINITY; best_idx[c] = 0x7fffffff; run_ref[c] = -INFINITY; run_sum[c] = 0.f;
-        }
-        const bool stats = p.c2 > 0.f;
+        EpiState e;
+        epi_init(e);
         bool ok = true;
         for (int t = 0; t < my_tiles && ok; ++t) {
             const int buf = t % p.acc_bufs;
@@ -306,80 +397,12 @@ lmhead_umma_kernel(const __grid_constant__ CUtensorMap tmW, const __grid_constan
             if (!mbar_wait(&tmem_full[buf], use & 1u, &abort_flag, p.wait_cycles)) { ok = false; break; }
             tc_fence_after_sync();
             const int v_base = ((int)blockIdx.x + t * (int)gridDim.x) * kBM + quad * 32;
-            const bool v_ok = (v_base + lane) < p.V;
-            const uint32_t taddr = tmem_base + ((uint32_t)(quad * 32) << 16) + (uint32_t)(buf * p.buf_stride);
-#pragma unroll
-            for (int h = 0; h < kMaxCols / 64; ++h) {
-                const int c = 2 * h + par;                 // this warp's chunk of the pair (2h, 2h + 1)
-                if (c * 32 < p.n_pad) {
-                    uint32_t r[32];
-                    tmem_ld32(taddr + c * 32, r);
-                    tmem_ld_wait();
-                    float cv;
-                    int32_t ci;
-                    if (p.mass_out) {
-                        if (v_ok) {
-#pragma unroll
-                            for (int j = 0; j < 32; ++j) {
-                                const int row = c * 32 + j;
-                                if (row < p.rows)
-                                    p.mass_out[(size_t)(p.row0 + row) * p.V + v_base + lane] =
-                                        __expf(__uint_as_float(r[j]) * p.inv_temp - __ldg(p.col_lse + p.row0 + row));
-                            }
-                        }
-                        continue;
-                    }
-                    if (stats) {
-                        float cs;
-                        column_argmax_stats32(r, v_ok, v_base, lane, p.c2, cv, ci, cs);
-                        merge_sumexp(run_ref[h], run_sum[h], cv, cs, p.c2);
-                        if (p.group_stats && v_base < p.V && c * 32 + lane < p.rows)
-                            p.group_stats[(size_t)(v_base >> 5) * p.M_total + p.row0 + c * 32 + lane] = make_float2(cv, cs);
-                    } else {
-                        column_argmax32(r, v_ok, v_base, lane, cv, ci);
-                    }
-                    if (cv > best_val[h]) { best_val[h] = cv; best_idx[h] = ci; }
-                }
-            }
+            epi_tile(p, e, tmem_base + ((uint32_t)(quad * 32) << 16) + (uint32_t)(buf * p.buf_stride), v_base, lane, par);
             tc_fence_before_sync();
             __syncwarp();
             if (lane == 0) mbar_arrive(&tmem_empty[buf]);
         }
-        // merge the four warps through shared memory (the pipeline stages are idle by now:
-        // the last accumulator was complete, so every copy has landed and every MMA has read it)
-        asm volatile("bar.sync 1, %0;" ::"n"(kEpiWarps * 32) : "memory");
-        int32_t* red_key = reinterpret_cast<int32_t*>(smem);
-        int32_t* red_idx = red_key + 4 * kMaxCols;
-        float* red_ref = reinterpret_cast<float*>(red_idx + 4 * kMaxCols);
-        float* red_sum = red_ref + 4 * kMaxCols;
-#pragma unroll
-        for (int h = 0; h < kMaxCols / 64; ++h) {
-            red_key[quad * kMaxCols + (2 * h + par) * 32 + lane] = ordered_key(__float_as_uint(best_val[h]));
-            red_idx[quad * kMaxCols + (2 * h + par) * 32 + lane] = best_idx[h];
-            if (stats) {
-                red_ref[quad * kMaxCols + (2 * h + par) * 32 + lane] = run_ref[h];
-                red_sum[quad * kMaxCols + (2 * h + par) * 32 + lane] = run_sum[h];
-            }
-        }
-        asm volatile("bar.sync 1, %0;" ::"n"(kEpiWarps * 32) : "memory");
-        for (int col = threadIdx.x; col < kMaxCols; col += kEpiWarps * 32) {
-            int32_t k = red_key[col], i = red_idx[col];
-#pragma unroll
-            for (int w = 1; w < 4; ++w) {
-                const int32_t k2 = red_key[w * kMaxCols + col], i2 = red_idx[w * kMaxCols + col];
-                if (k2 > k || (k2 == k && i2 < i)) { k = k2; i = i2; }
-            }
-            if (!ok && col == (int)threadIdx.x) set_status(status, SD_ERR_TIMEOUT);
-            p.part_key[(size_t)blockIdx.x * kMaxCols + col] = ok ? k : INT32_MIN;
-            p.part_idx[(size_t)blockIdx.x * kMaxCols + col] = i;
-            if (stats) {
-                float rf = red_ref[col], sm = red_sum[col];
-#pragma unroll
-                for (int w = 1; w < 4; ++w) merge_sumexp(rf, sm, red_ref[w * kMaxCols + col], red_sum[w * kMaxCols + col], p.c2);
-                p.part_ref[(size_t)blockIdx.x * kMaxCols + col] = rf;
-                p.part_sum[(size_t)blockIdx.x * kMaxCols + col] = sm;
-            }
-        }
+        epi_finish(p, e, smem, quad, par, lane, ok, status);
     }
     tc_fence_before_sync();
     __syncthreads();
@@ -507,17 +530,9 @@ lmhead_umma_pair_kernel(const __grid_constant__ CUtensorMap tmW, const __grid_co
         }
     } else {
         // ------------------------------------------------ epilogue warps 0..7
-        // warp w works on TMEM lanes 32 * (w & 3) .. +31 (the only ones it may read) and on the
-        // 32-column chunks of parity w >> 2
         const int quad = warp & 3, par = warp >> 2;
-        float best_val[kMaxCols / 64];
-        int32_t best_idx[kMaxCols / 64];
-        float run_ref[kMaxCols / 64], run_sum[kMaxCols / 64];
-#pragma unroll
-        for (int c = 0; c < kMaxCols / 64; ++c) {
-            best_val[c] = -INFINITY; best_idx[c] = 0x7fffffff; run_ref[c] = -INFINITY; run_sum[c] = 0.f;
-        }
-        const bool stats = p.c2 > 0.f;
+        EpiState e;
+        epi_init(e);
         bool ok = true;
         for (int t = 0; t < my_tiles && ok; ++t) {
             const int buf = t % p.acc_bufs;
@@ -525,80 +540,14 @@ lmhead_umma_pair_kernel(const __grid_constant__ CUtensorMap tmW, const __grid_co
             if (!mbar_wait(&tmem_full[buf], use & 1u, &abort_flag, p.wait_cycles)) { ok = false; break; }
             tc_fence_after_sync();
             const int v_base = ((pair + t * n_pairs) * 2 + (int)rank) * kBM + quad * 32;
-            const bool v_ok = (v_base + lane) < p.V;
-            const uint32_t taddr = tmem_base + ((uint32_t)(quad * 32) << 16) + (uint32_t)(buf * p.buf_stride);
-#pragma unroll
-            for (int h = 0; h < kMaxCols / 64; ++h) {
-                const int c = 2 * h + par;                 // this warp's chunk of the pair (2h, 2h + 1)
-                if (c * 32 < p.n_pad) {
-                    uint32_t r[32];
-                    tmem_ld32(taddr + c * 32, r);
-                    tmem_ld_wait();
-                    float cv;
-                    int32_t ci;
-                    if (p.mass_out) {
-                        if (v_ok) {
-#pragma unroll
-                            for (int j = 0; j < 32; ++j) {
-                                const int row = c * 32 + j;
-                                if (row < p.rows)
-                                    p.mass_out[(size_t)(p.row0 + row) * p.V + v_base + lane] =
-                                        __expf(__uint_as_float(r[j]) * p.inv_temp - __ldg(p.col_lse + p.row0 + row));
-                            }
-                        }
-                        continue;
-                    }
-                    if (stats) {
-                        float cs;
-                        column_argmax_stats32(r, v_ok, v_base, lane, p.c2, cv, ci, cs);
-                        merge_sumexp(run_ref[h], run_sum[h], cv, cs, p.c2);
-                        if (p.group_stats && v_base < p.V && c * 32 + lane < p.rows)
-                            p.group_stats[(size_t)(v_base >> 5) * p.M_total + p.row0 + c * 32 + lane] = make_float2(cv, cs);
-                    } else {
-                        column_argmax32(r, v_ok, v_base, lane, cv, ci);
-                    }
-                    if (cv > best_val[h]) { best_val[h] = cv; best_idx[h] = ci; }
-                }
-            }
+            epi_tile(p, e, tmem_base + ((uint32_t)(quad * 32) << 16) + (uint32_t)(buf * p.buf_stride), v_base, lane, par);
             tc_fence_before_sync();
             __syncwarp();
             // (the accumulator reads above have completed: tcgen05.wait::ld; a CTA-scope release is enough,
             //  and a cluster-scope one costs on the order of a thousand cycles per arrival)
             if (lane == 0) mbar_arrive_remote_light(map_dsmem(smem_u32(&tmem_empty[buf]), 0));
         }
-        asm volatile("bar.sync 1, %0;" ::"n"(kEpiWarps * 32) : "memory");
-        int32_t* red_key = reinterpret_cast<int32_t*>(smem);
-        int32_t* red_idx = red_key + 4 * kMaxCols;
-        float* red_ref = reinterpret_cast<float*>(red_idx + 4 * kMaxCols);
-        float* red_sum = red_ref + 4 * kMaxCols;
-#pragma unroll
-        for (int h = 0; h < kMaxCols / 64; ++h) {
-            red_key[quad * kMaxCols + (2 * h + par) * 32 + lane] = ordered_key(__float_as_uint(best_val[h]));
-            red_idx[quad * kMaxCols + (2 * h + par) * 32 + lane] = best_idx[h];
-            if (stats) {
-                red_ref[quad * kMaxCols + (2 * h + par) * 32 + lane] = run_ref[h];
-                red_sum[quad * kMaxCols + (2 * h + par) * 32 + lane] = run_sum[h];
-            }
-        }
-        asm volatile("bar.sync 1, %0;" ::"n"(kEpiWarps * 32) : "memory");
-        for (int col = threadIdx.x; col < kMaxCols; col += kEpiWarps * 32) {
-            int32_t k = red_key[col], i = red_idx[col];
-#pragma unroll
-            for (int w = 1; w < 4; ++w) {
-                const int32_t k2 = red_key[w * kMaxCols + col], i2 = red_idx[w * kMaxCols + col];
-                if (k2 > k || (k2 == k && i2 < i)) { k = k2; i = i2; }
-            }
-            if (!ok && col == (int)threadIdx.x) set_status(status, SD_ERR_TIMEOUT);
-            p.part_key[(size_t)blockIdx.x * kMaxCols + col] = ok ? k : INT32_MIN;
-            p.part_idx[(size_t)blockIdx.x * kMaxCols + col] = i;
-            if (stats) {
-                float rf = red_ref[col], sm = red_sum[col];
-#pragma unroll
-                for (int w = 1; w < 4; ++w) merge_sumexp(rf, sm, red_ref[w * kMaxCols + col], red_sum[w * kMaxCols + col], p.c2);
-                p.part_ref[(size_t)blockIdx.x * kMaxCols + col] = rf;
-                p.part_sum[(size_t)blockIdx.x * kMaxCols + col] = sm;
-            }
-        }
+        epi_finish(p, e, smem, quad, par, lane, ok, status);
     }
     tc_fence_before_sync();
     __syncthreads();
