@@ -416,7 +416,7 @@ def main():
                     "attention_frac_of_burst_peak": work["att_flops"] * vs.L / (per_call_ms["attention_all_layers_call"] * 1e-3) / 1e12 / peaks["tensor_burst"]},
                 "calls": {"attention_ms_single_layer_call": per_call_ms["attention_single_layer_call"],
                           "lmhead_accept_compact_ms": per_call_ms["tail"],
-                          "sampled_tail_ms": per_call_ms["tail_sampled"],
+                          "lmhead_accept_sampled_compact_ms": per_call_ms["tail_sampled"],
                           "lmhead_ms": per_call_ms["lmhead"], "accept_ms": per_call_ms["accept"],
                           "compact_ms": per_call_ms["compact"],
                           "lmhead_tflops": lm_tflops,

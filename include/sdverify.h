@@ -329,6 +329,35 @@ sd_status sd_accept_tree_sampled(const sd_batch *batch, const void *hidden, cons
                                  int32_t *dev_status, void *stream);
 
 /*
+ * LM head, acceptance at a sampling temperature and compaction in one call (Sec. 1:
+ * lossless validation; Sec. 4.1: the survivors' KV joins the context).  Equivalent,
+ * output for output and byte for byte, to
+ *     sd_lmhead_stats(hidden, W, M = B * T_max, ..., argmax = NULL, maxlogit = NULL, lse, group_stats)
+ *     sd_accept_tree_sampled(batch, hidden, W, ..., lse, group_stats, draft_tok, u, w, ...)
+ *     sd_compact_kv(batch, layers, L, ..., n_acc, path)
+ * but behind the LM-head tiles a single kernel does the rest: one cluster of eight
+ * CTAs per sequence merges the rows' soft-max statistics, computes the drafted
+ * tokens' probabilities, walks the tree, draws the last token from the group table
+ * and copies the accepted K/V rows (each CTA a share of the layers) - two launches
+ * instead of six.  Arguments as in the three calls:
+ *   lse         : dev f32 [B * T_max], output
+ *   group_stats : dev f32 [ceil(V / 32)][B * T_max][2], 8-byte aligned, scratch that the
+ *                 call fills and reads (required here)
+ *   workspace   : at least sd_workspace_bytes(batch, B * T_max, V)
+ * V > 262144 returns SD_ERR_UNSUPPORTED before anything is launched; B * T_max > 512
+ * or L > 64 falls back to the separate steps internally.
+ */
+sd_status sd_lmhead_accept_sampled_compact(const sd_batch *batch, const void *hidden, const void *W,
+                                           int32_t Hd, int32_t V, float inv_temp,
+                                           const int32_t *draft_tok, const float *u, const float *w,
+                                           const sd_kv_layer *layers, int32_t L,
+                                           const void *const *k_tree_layers, const void *const *v_tree_layers,
+                                           float *lse, float *group_stats,
+                                           int32_t *n_acc, int32_t *path, int32_t *out_tok, int32_t *new_len,
+                                           void *workspace, size_t workspace_bytes,
+                                           int32_t *dev_status, void *stream);
+
+/*
  * Draft-side feature aggregation (Sec. 3.1.1, f_c^i = Flatten(CrossAttention(f_q, f_i, f_i))):
  * Q meta queries, shared by all tokens, attend over the L target-layer features
  * of every token.  This is the attention core for H heads of size 128

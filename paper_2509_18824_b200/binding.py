@@ -29,10 +29,12 @@ KERNELS_PER_ATTENTION = 1      # split-KV chunks merge inside the kernel (thread
 ATTENTION_LAYERS_PER_LAUNCH = 32   # sd_verify_attention_layers: layers sharing one launch
 KERNELS_PER_TAIL = 2               # sd_lmhead_accept_compact: LM-head tiles + fused tail kernel
 KERNELS_PER_LMHEAD = 2         # tiles + cross-slab reduce
+KERNELS_PER_SAMPLED_TAIL = 2       # sd_lmhead_accept_sampled_compact: LM-head tiles + one cluster kernel
 
 EXPORTS = ["sd_version", "sd_status_string", "sd_workspace_bytes", "sd_tree_prepare",
            "sd_verify_attention", "sd_verify_attention_layers", "sd_lmhead_argmax", "sd_lmhead_argmax_static", "sd_accept_tree",
-           "sd_compact_kv", "sd_lmhead_accept_compact", "sd_lmhead_stats", "sd_accept_tree_sampled", "sd_draft_feature_attention"]
+           "sd_compact_kv", "sd_lmhead_accept_compact", "sd_lmhead_stats", "sd_accept_tree_sampled", "sd_lmhead_accept_sampled_compact",
+           "sd_draft_feature_attention"]
 
 
 class sd_kv_layer(C.Structure):
@@ -91,6 +93,13 @@ def _load(path: str = LIB_PATH) -> C.CDLL:
                                            C.c_void_p, C.c_void_p, C.c_void_p, C.c_void_p, C.c_void_p,
                                            C.c_void_p, C.c_void_p, C.c_void_p, C.c_void_p,
                                            C.c_void_p, C.c_size_t, C.c_void_p, C.c_void_p]
+    lib.sd_lmhead_accept_sampled_compact.restype = C.c_int
+    lib.sd_lmhead_accept_sampled_compact.argtypes = [C.c_void_p, C.c_void_p, C.c_void_p, C.c_int32, C.c_int32, C.c_float,
+                                                     C.c_void_p, C.c_void_p, C.c_void_p,
+                                                     C.c_void_p, C.c_int32, C.c_void_p, C.c_void_p,
+                                                     C.c_void_p, C.c_void_p,
+                                                     C.c_void_p, C.c_void_p, C.c_void_p, C.c_void_p,
+                                                     C.c_void_p, C.c_size_t, C.c_void_p, C.c_void_p]
     lib.sd_draft_feature_attention.restype = C.c_int
     lib.sd_draft_feature_attention.argtypes = [C.c_void_p, C.c_void_p, C.c_void_p, C.c_int32, C.c_int32, C.c_int32,
                                                C.c_int32, C.c_int32, C.c_float, C.c_void_p, C.c_void_p]
@@ -298,6 +307,22 @@ def sd_accept_tree_sampled(batch: Batch, hidden, W, inv_temp: float, lse, draft_
                                       _ptr(lse), _ptr(group_stats), _ptr(draft_tok), _ptr(u), _ptr(w), _ptr(n_acc), _ptr(path),
                                       _ptr(out_tok), _ptr(new_len), _ptr(workspace),
                                       workspace.numel() * workspace.element_size(), _ptr(status), _stream(stream)))
+
+
+def sd_lmhead_accept_sampled_compact(batch: Batch, hidden, W, inv_temp: float, draft_tok, u, w, layers: LayerSet,
+                                     lse, group_stats, n_acc, path, out_tok, new_len, workspace, status,
+                                     stream=None) -> None:
+    """LM-head statistics, acceptance at a sampling temperature and KV compaction in all layers: the
+    LM-head tiles and one tail kernel."""
+    M, Hd = hidden.shape
+    V = W.shape[0]
+    assert W.shape[1] == Hd and M == batch.B * batch.T_max
+    _check(lib.sd_lmhead_accept_sampled_compact(batch.ref(), _ptr(hidden), _ptr(W), int(Hd), int(V), C.c_float(inv_temp),
+                                                _ptr(draft_tok), _ptr(u), _ptr(w), layers.layers, layers.L, layers.kt,
+                                                layers.vt, _ptr(lse), _ptr(group_stats), _ptr(n_acc), _ptr(path),
+                                                _ptr(out_tok), _ptr(new_len), _ptr(workspace),
+                                                workspace.numel() * workspace.element_size(), _ptr(status),
+                                                _stream(stream)))
 
 
 def sd_draft_feature_attention(qp, k, v, H: int, scale: float, out, stream=None) -> None:

@@ -196,6 +196,30 @@ sd_status sd_accept_tree_sampled(const sd_batch* batch, const void* hidden, cons
                                  new_len, workspace, workspace_bytes, dev_status, static_cast<cudaStream_t>(stream));
 }
 
+sd_status sd_lmhead_accept_sampled_compact(const sd_batch* batch, const void* hidden, const void* W, int32_t Hd, int32_t V,
+                                           float inv_temp, const int32_t* draft_tok, const float* u, const float* w,
+                                           const sd_kv_layer* layers, int32_t L,
+                                           const void* const* k_tree_layers, const void* const* v_tree_layers,
+                                           float* lse, float* group_stats,
+                                           int32_t* n_acc, int32_t* path, int32_t* out_tok, int32_t* new_len,
+                                           void* workspace, size_t workspace_bytes, int32_t* dev_status, void* stream) {
+    sd_status s = check_geometry(batch, true);
+    if (s != SD_OK) return s;
+    if (!ok_ptr(hidden) || !ok_ptr(W) || !lse || !group_stats || !draft_tok || !u || !w) return SD_ERR_INVALID_ARG;
+    if (reinterpret_cast<uintptr_t>(group_stats) & 7u) return SD_ERR_INVALID_ARG;
+    if (!n_acc || !path || !out_tok || !new_len || !ok_ptr(workspace) || !dev_status) return SD_ERR_INVALID_ARG;
+    if (V < 1 || Hd < 1 || !(inv_temp > 0.f)) return SD_ERR_INVALID_ARG;
+    if (Hd % 64 != 0) return SD_ERR_UNSUPPORTED;
+    if (!layers || L < 1 || !k_tree_layers || !v_tree_layers) return SD_ERR_INVALID_ARG;
+    for (int l = 0; l < L; ++l) {
+        if (!ok_ptr(layers[l].k) || !ok_ptr(layers[l].v) || layers[l].num_blocks < 1) return SD_ERR_INVALID_ARG;
+        if (!ok_ptr(k_tree_layers[l]) || !ok_ptr(v_tree_layers[l])) return SD_ERR_INVALID_ARG;
+    }
+    return launch_lmhead_accept_sampled_compact(*batch, hidden, W, Hd, V, inv_temp, draft_tok, u, w, layers, L, k_tree_layers,
+                                                v_tree_layers, lse, group_stats, n_acc, path, out_tok, new_len, workspace,
+                                                workspace_bytes, dev_status, static_cast<cudaStream_t>(stream));
+}
+
 sd_status sd_draft_feature_attention(const void* qp, const void* k, const void* v, int32_t S, int32_t L, int32_t Q,
                                      int32_t H, int32_t D, float scale, void* out, void* stream) {
     if (!ok_ptr(qp) || !ok_ptr(k) || !ok_ptr(v) || !ok_ptr(out)) return SD_ERR_INVALID_ARG;

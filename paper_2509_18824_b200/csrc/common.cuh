@@ -72,10 +72,22 @@ sd_status launch_lmhead_stats(const void* hidden, const void* W, int M, int Hd, 
 sd_status launch_lmhead_mass(const void* hidden, const void* W, int M, int Hd, int V, float inv_temp,
                              const float* row_lse, float* mass, void* ws, size_t ws_bytes,
                              int32_t* dev_status, cudaStream_t st);
+// per-CTA tables the LM-head tiles of a statistics pass leave in the workspace (row stride 512 entries)
+struct LmTables { const int32_t* part_key; const int32_t* part_idx; const float* part_ref; const float* part_sum; int n_ctas; };
+sd_status launch_lmhead_stats_tiles(const void* hidden, const void* W, int M, int Hd, int V, float inv_temp,
+                                    float* lse, float* group_stats, void* ws, size_t ws_bytes,
+                                    int32_t* dev_status, cudaStream_t st, LmTables* tables);
 size_t sampled_workspace_bytes(int B, int T, int V, int Hd);
 sd_status launch_accept_sampled(const sd_batch& bt, const void* hidden, const void* W, int Hd, int V, float inv_temp,
                                 const float* lse, const float* group_stats, const int32_t* draft, const float* u,
                                 const float* w, int32_t* n_acc, int32_t* path, int32_t* out_tok, int32_t* new_len,
                                 void* ws, size_t ws_bytes, int32_t* dev_status, cudaStream_t st);
+
+sd_status launch_lmhead_accept_sampled_compact(const sd_batch& bt, const void* hidden, const void* W, int Hd, int V,
+                                               float inv_temp, const int32_t* draft, const float* u, const float* w,
+                                               const sd_kv_layer* layers, int L, const void* const* kt, const void* const* vt,
+                                               float* lse, float* group_stats, int32_t* n_acc, int32_t* path,
+                                               int32_t* out_tok, int32_t* new_len, void* ws, size_t ws_bytes,
+                                               int32_t* dev_status, cudaStream_t st);
 
 }  // namespace sdv

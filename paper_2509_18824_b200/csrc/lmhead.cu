@@ -118,12 +118,6 @@ __device__ __forceinline__ void column_argmax32(const uint32_t (&r)[32], bool v_
     ci = v_base + (__ffs(pick_lane(who, lane)) - 1);
 }
 
-__device__ __forceinline__ float ex2_lm(float x) {
-    float y;
-    asm("ex2.approx.ftz.f32 %0, %1;" : "=f"(y) : "f"(x));
-    return y;
-}
-
 // Sum over the 32 lanes of each of 32 per-lane values: lane j receives sum_lanes x[j].  Five
 // exchange steps; in each a lane keeps the half of its values whose column index has the step's
 // bit equal to its own lane bit and hands the other half to its partner (fixed order of additions).
@@ -171,13 +165,6 @@ __device__ __forceinline__ void column_argmax_stats32(const uint32_t (&r)[32], b
 #pragma unroll
     for (int j = 0; j < 32; ++j) e[j] = (v[j] == -INFINITY) ? 0.f : ex2_lm((v[j] - mx[j]) * c2);
     cs = transpose_sum32(e, lane);
-}
-
-// running (reference, sum) of a column takes in a new partial (ref2, sum2)
-__device__ __forceinline__ void merge_sumexp(float& ref, float& sum, float ref2, float sum2, float c2) {
-    if (!(sum2 > 0.f)) return;
-    if (ref2 > ref) { sum = sum * ex2_lm((ref - ref2) * c2) + sum2; ref = ref2; }
-    else            { sum += sum2 * ex2_lm((ref2 - ref) * c2); }
 }
 
 // ---------------------------------------------------------------------------
@@ -582,29 +569,12 @@ lmhead_merge_stats_kernel(const int32_t* __restrict__ part_key, const int32_t* _
                           int n_ctas, int rows, int row0, float c2, int32_t* __restrict__ argmax,
                           float* __restrict__ maxlogit, float* __restrict__ lse) {
     const int col = blockIdx.x * 32 + (threadIdx.x >> 3), sub = threadIdx.x & 7;
-    int32_t k = INT32_MIN, i = 0x7fffffff;
-    float rf = -INFINITY, sm = 0.f;
-    if (col < rows) {
-        for (int c = sub; c < n_ctas; c += 8) {
-            take_better(k, i, __ldg(part_key + (size_t)c * kMaxCols + col), __ldg(part_idx + (size_t)c * kMaxCols + col));
-            merge_sumexp(rf, sm, __ldg(part_ref + (size_t)c * kMaxCols + col), __ldg(part_sum + (size_t)c * kMaxCols + col), c2);
-        }
-    }
-#pragma unroll
-    for (int d = 1; d <= 4; d <<= 1) {
-        const int32_t k2 = __shfl_xor_sync(0xffffffffu, k, d), i2 = __shfl_xor_sync(0xffffffffu, i, d);
-        const float rf2 = __shfl_xor_sync(0xffffffffu, rf, d), sm2 = __shfl_xor_sync(0xffffffffu, sm, d);
-        take_better(k, i, k2, i2);
-        // both partners must end with the same bits: combine in the order (lower lane, higher lane)
-        float ra = (threadIdx.x & d) ? rf2 : rf, sa = (threadIdx.x & d) ? sm2 : sm;
-        const float rb = (threadIdx.x & d) ? rf : rf2, sb = (threadIdx.x & d) ? sm : sm2;
-        merge_sumexp(ra, sa, rb, sb, c2);
-        rf = ra; sm = sa;
-    }
+    int32_t k, i;
+    const float row_lse = merge_row_stats(part_key, part_idx, part_ref, part_sum, n_ctas, kMaxCols, col, col < rows, sub, c2, k, i);
     if (col < rows && sub == 0) {
         if (argmax) argmax[row0 + col] = i;
         if (maxlogit) maxlogit[row0 + col] = key_to_float(k);
-        lse[row0 + col] = (rf * c2 + log2f(sm)) * 0.6931471805599453f;
+        lse[row0 + col] = row_lse;
     }
 }
 
@@ -743,6 +713,22 @@ sd_status launch_lmhead_stats(const void* hidden, const void* W, int M, int Hd, 
                               nullptr, nullptr, group_stats);
 }
 
+// only the tiles of the statistics pass (M <= 512): the caller's own kernel merges the per-CTA tables
+sd_status launch_lmhead_stats_tiles(const void* hidden, const void* W, int M, int Hd, int V, float inv_temp,
+                                    float* lse, float* group_stats, void* ws, size_t ws_bytes,
+                                    int32_t* dev_status, cudaStream_t st, LmTables* tables) {
+    int n_ctas = 0;
+    const sd_status s = launch_lmhead_impl(hidden, W, M, Hd, V, nullptr, nullptr, ws, ws_bytes, dev_status, st, &n_ctas,
+                                           inv_temp, lse, nullptr, nullptr, group_stats);
+    if (s != SD_OK) return s;
+    tables->part_key = static_cast<const int32_t*>(ws);
+    tables->part_idx = tables->part_key + (size_t)kMaxCtas * kMaxCols;
+    tables->part_ref = reinterpret_cast<const float*>(static_cast<const char*>(ws) + tail_workspace_bytes(M, V));
+    tables->part_sum = tables->part_ref + (size_t)kMaxCtas * kMaxCols;
+    tables->n_ctas = n_ctas;
+    return SD_OK;
+}
+
 sd_status launch_lmhead(const void* hidden, const void* W, int M, int Hd, int V,
                         int32_t* argmax, float* maxlogit, void* ws, size_t ws_bytes,
                         int32_t* dev_status, cudaStream_t st) {
@@ -810,9 +796,6 @@ tail_kernel(sd_batch bt, const __grid_constant__ CompactLayers ly,
     // 3. accepted rows into this layer's cache
     compact_sequence(bt, ly, layer, 1, b, s_na, s_path, threadIdx.x, blockDim.x, status);
 }
-
-void fill_compact_layers(CompactLayers* ly, const sd_kv_layer* layers, const void* const* kt, const void* const* vt,
-                         int l0, int nl);
 
 sd_status launch_lmhead_accept_compact(const sd_batch& bt, const void* hidden, const void* W, int Hd, int V,
                                        const int32_t* draft, const sd_kv_layer* layers, int L,

@@ -2,13 +2,18 @@
 // rejection without replacement along the tree, then one token from the residual distribution at
 // the node where the walk stops.  All random numbers are inputs.
 //
-//   child_prob_kernel      p[b][j] = exp(logit(parent(j), token(j)) / temperature - lse(parent(j)))
-//   sampled_walk_kernel    the walk: accepted path, residual mass, the stop node's drafted tokens
+// The steps are device functions, used by the stand-alone kernels behind sd_accept_tree_sampled and by
+// the one tail kernel behind sd_lmhead_accept_sampled_compact:
+//   child_prob             p[b][j] = exp(logit(parent(j), token(j)) / temperature - lse(parent(j)))
+//   sampled_walk           the walk: accepted path, residual mass, the stop node's drafted tokens
+//   residual_pick_groups   the last token from the LM-head pass's per-group (maximum, sum) table
+// Without that table the stand-alone call goes over W a second time:
 //   gather_stop_rows_kernel + the LM-head tcgen05 kernel in its store mode
 //                          exp(logit / temperature - lse) of the stop node's row over the whole vocabulary
 //   residual_blocksum_kernel  drafted tokens of the stop node zeroed, sums per 256-token block
 //   residual_pick_kernel   inverse CDF in vocabulary order; writes the final token
 #include "tree_device.cuh"
+#include "sm100.cuh"
 
 namespace sdv {
 
@@ -56,23 +61,72 @@ static SampledWs carve(void* ws, int B, int T, int V, int Hd) {
     return w;
 }
 
-// dot product of two bf16 rows of length Hd (multiple of 64) by one warp, fp32, fixed order:
-// lane l takes the 16-byte pieces l, l + 32, ...; lanes are combined by a butterfly
-__device__ __forceinline__ float warp_dot_bf16(const uint4* __restrict__ a, const uint4* __restrict__ b, int n_vec, int lane) {
-    float acc = 0.f;
-    for (int i = lane; i < n_vec; i += 32) {
-        const uint4 x = __ldg(a + i), y = b[i];
-        acc = fmaf(bf16lo(x.x), bf16lo(y.x), acc); acc = fmaf(bf16hi(x.x), bf16hi(y.x), acc);
-        acc = fmaf(bf16lo(x.y), bf16lo(y.y), acc); acc = fmaf(bf16hi(x.y), bf16hi(y.y), acc);
-        acc = fmaf(bf16lo(x.z), bf16lo(y.z), acc); acc = fmaf(bf16hi(x.z), bf16hi(y.z), acc);
-        acc = fmaf(bf16lo(x.w), bf16lo(y.w), acc); acc = fmaf(bf16hi(x.w), bf16hi(y.w), acc);
-    }
-#pragma unroll
-    for (int d = 16; d >= 1; d >>= 1) acc += __shfl_xor_sync(0xffffffffu, acc, d);
+__device__ __forceinline__ float fma8_bf16(const uint4& x, const uint4& y, float acc) {
+    acc = fmaf(bf16lo(x.x), bf16lo(y.x), acc); acc = fmaf(bf16hi(x.x), bf16hi(y.x), acc);
+    acc = fmaf(bf16lo(x.y), bf16lo(y.y), acc); acc = fmaf(bf16hi(x.y), bf16hi(y.y), acc);
+    acc = fmaf(bf16lo(x.z), bf16lo(y.z), acc); acc = fmaf(bf16hi(x.z), bf16hi(y.z), acc);
+    acc = fmaf(bf16lo(x.w), bf16lo(y.w), acc); acc = fmaf(bf16hi(x.w), bf16hi(y.w), acc);
     return acc;
 }
 
-// one warp per (sequence, node >= 1)
+// Dot products of NR bf16 rows a[0..NR) with one bf16 row b, all of length 8 * n_vec (Hd, a multiple of
+// 64), by one warp, fp32, fixed order: lane l takes the 16-byte pieces l, l + 32, ... in that order;
+// lanes are combined by a butterfly.  The loads of a batch of pieces are issued before its arithmetic
+// (latency-bound: every load in flight at once), which does not change the order of the additions.
+template <int NR>
+__device__ __forceinline__ void warp_dots_bf16(const uint4* (&a)[NR], const uint4* b, int n_vec, int lane, float (&out)[NR]) {
+    constexpr int kAhead = NR >= 4 ? 4 : 8;            // pieces per lane in flight, per row (more did not help: one SM's load path is the limit)
+    float acc[NR];
+#pragma unroll
+    for (int r = 0; r < NR; ++r) acc[r] = 0.f;
+    for (int i0 = lane; i0 < n_vec; i0 += 32 * kAhead) {
+        uint4 x[NR][kAhead], y[kAhead];
+#pragma unroll
+        for (int k = 0; k < kAhead; ++k) {
+            const int i = i0 + 32 * k;
+            if (i < n_vec) {
+                y[k] = b[i];
+#pragma unroll
+                for (int r = 0; r < NR; ++r) x[r][k] = __ldg(a[r] + i);
+            }
+        }
+#pragma unroll
+        for (int k = 0; k < kAhead; ++k)
+            if (i0 + 32 * k < n_vec) {
+#pragma unroll
+                for (int r = 0; r < NR; ++r) acc[r] = fma8_bf16(x[r][k], y[k], acc[r]);
+            }
+    }
+#pragma unroll
+    for (int r = 0; r < NR; ++r) {
+#pragma unroll
+        for (int d = 16; d >= 1; d >>= 1) acc[r] += __shfl_xor_sync(0xffffffffu, acc[r], d);
+        out[r] = acc[r];
+    }
+}
+
+// Probability, under its parent's target distribution, of the token drafted at node j of sequence b
+// (0 for the root and for unused nodes); one warp.  lse: log sum exp of the LM-head rows.
+__device__ __forceinline__ float child_prob(const sd_batch& bt, int b, int j, int lane, const uint16_t* __restrict__ hidden,
+                                            const uint16_t* __restrict__ W, int Hd, int V, float inv_temp, const float* lse,
+                                            const int32_t* __restrict__ draft, int32_t* status) {
+    const int T = bt.T_max;
+    const int n = bt.n_nodes[b];
+    if (!(j >= 1 && j < n && n <= T)) return 0.f;
+    const int par = bt.parents[(size_t)b * T + j];
+    const int tok = draft[(size_t)b * T + j];
+    if (par < 0 || par >= j || tok < 0 || tok >= V) {
+        if (lane == 0) set_status(status, par < 0 || par >= j ? SD_ERR_INVALID_TREE : SD_ERR_BOUNDS);
+        return 0.f;
+    }
+    const int row = b * T + par;
+    const uint4* wrow[1] = {reinterpret_cast<const uint4*>(W + (size_t)tok * Hd)};
+    float l[1];
+    warp_dots_bf16<1>(wrow, reinterpret_cast<const uint4*>(hidden + (size_t)row * Hd), Hd / 8, lane, l);
+    return __expf(l[0] * inv_temp - lse[row]);
+}
+
+// one warp per (sequence, node)
 __global__ void __launch_bounds__(128)
 child_prob_kernel(sd_batch bt, const uint16_t* __restrict__ hidden, const uint16_t* __restrict__ W, int Hd, int V,
                   float inv_temp, const float* __restrict__ lse, const int32_t* __restrict__ draft,
@@ -81,29 +135,21 @@ child_prob_kernel(sd_batch bt, const uint16_t* __restrict__ hidden, const uint16
     const int T = bt.T_max;
     if (warp >= bt.B * T) return;
     const int b = warp / T, j = warp - b * T;
-    float p = 0.f;
-    const int n = bt.n_nodes[b];
-    if (j >= 1 && j < n && n <= T) {
-        const int par = bt.parents[(size_t)b * T + j];
-        const int tok = draft[(size_t)b * T + j];
-        if (par < 0 || par >= j || tok < 0 || tok >= V) {
-            if (lane == 0) set_status(status, par < 0 || par >= j ? SD_ERR_INVALID_TREE : SD_ERR_BOUNDS);
-        } else {
-            const int row = b * T + par;
-            const float l = warp_dot_bf16(reinterpret_cast<const uint4*>(W + (size_t)tok * Hd),
-                                          reinterpret_cast<const uint4*>(hidden + (size_t)row * Hd), Hd / 8, lane);
-            p = __expf(l * inv_temp - lse[row]);
-        }
-    }
+    const float p = child_prob(bt, b, j, lane, hidden, W, Hd, V, inv_temp, lse, draft, status);
     if (lane == 0) p_child[(size_t)b * T + j] = p;
 }
 
-// one warp per sequence
-__global__ void sampled_walk_kernel(sd_batch bt, const int32_t* __restrict__ draft, const float* __restrict__ p_child,
-                                    const float* __restrict__ u, int32_t* n_acc, int32_t* path, int32_t* out_tok,
-                                    int32_t* new_len, float* resid, int32_t* stop_row, int32_t* n_excl, int32_t* excl,
-                                    float* excl_p, int32_t* status) {
-    const int b = blockIdx.x, lane = threadIdx.x;
+// The rejection walk of one sequence, by one warp.  Results go where `o` points (global or shared
+// memory): the accepted path and the drafted tokens along it (entries beyond: -1; the slot of the
+// token still to be drawn: -1), the drafted tokens of the stop node's children and their
+// probabilities.  Returns, in every lane: accepted nodes (0: bad tree, reported, nothing written), the
+// stop node, the number of its children, the residual mass left there.
+struct WalkOut { int32_t* path; int32_t* out_tok; int32_t* excl; float* excl_p; };
+struct WalkEnd { int na, stop, n_excl; float R; };
+
+__device__ __forceinline__ WalkEnd sampled_walk(const sd_batch& bt, int b, int lane, const int32_t* __restrict__ draft,
+                                                const float* p_child, const float* __restrict__ u, const WalkOut& o,
+                                                int32_t* status) {
     const int T = bt.T_max;
     const int n = bt.n_nodes[b];
     const int32_t* par = bt.parents + (size_t)b * T;
@@ -115,52 +161,65 @@ __global__ void sampled_walk_kernel(sd_batch bt, const int32_t* __restrict__ dra
             if (i == 0 ? (p != -1) : (p < 0 || p >= i)) bad = true;
         }
     if (__any_sync(0xffffffffu, bad)) {
-        if (lane == 0) { set_status(status, SD_ERR_INVALID_TREE); n_acc[b] = 0; n_excl[b] = 0; stop_row[b] = b * T; resid[b] = 0.f; }
-        return;
+        if (lane == 0) set_status(status, SD_ERR_INVALID_TREE);
+        return WalkEnd{0, 0, 0, 0.f};
     }
-    // parent and token of the (up to) two nodes this lane looks after
-    const int pa0 = lane < n ? par[lane] : -2, pa1 = lane + 32 < n ? par[lane + 32] : -2;
-    const int tk0 = lane < n ? dt[lane] : -1, tk1 = lane + 32 < n ? dt[lane + 32] : -1;
-    int32_t* pth = path + (size_t)b * T;
-    int32_t* ot = out_tok + (size_t)b * T;
+    // parent, token, probability and uniform number of the (up to) two nodes this lane looks after
+    const bool has0 = lane < n, has1 = lane + 32 < n;
+    const int pa0 = has0 ? par[lane] : -2, pa1 = has1 ? par[lane + 32] : -2;
+    const int tk0 = has0 ? dt[lane] : -1, tk1 = has1 ? dt[lane + 32] : -1;
+    const float pc0 = has0 ? p_child[(size_t)b * T + lane] : 0.f, pc1 = has1 ? p_child[(size_t)b * T + lane + 32] : 0.f;
+    const float u0 = has0 ? u[(size_t)b * T + lane] : 0.f, u1 = has1 ? u[(size_t)b * T + lane + 32] : 0.f;
     int cur = 0, na = 1;
     float R = 1.f;
-    if (lane == 0) pth[0] = 0;
+    if (lane == 0) o.path[0] = 0;
     while (true) {
         // children of cur, as a 64-bit mask in node order
         const uint32_t lo = __ballot_sync(0xffffffffu, pa0 == cur), hi = __ballot_sync(0xffffffffu, pa1 == cur);
         uint64_t kids = ((uint64_t)hi << 32) | lo;
         R = 1.f;
-        int nxt = -1;
+        int nxt = -1, nxt_tok = -1;
         while (kids) {                                       // warp-uniform loop
             const int c = __ffsll((long long)kids) - 1;
             kids &= kids - 1;
+            const int tc = __shfl_sync(0xffffffffu, c < 32 ? tk0 : tk1, c & 31);
+            const float pc = __shfl_sync(0xffffffffu, c < 32 ? pc0 : pc1, c & 31);
+            const float uc = __shfl_sync(0xffffffffu, c < 32 ? u0 : u1, c & 31);
             // siblings must carry distinct tokens (an earlier sibling's rejection already removed the mass)
-            const int tc = dt[c];
             if (__any_sync(0xffffffffu, (pa0 == cur && lane < c && tk0 == tc) || (pa1 == cur && lane + 32 < c && tk1 == tc)))
                 if (lane == 0) set_status(status, SD_ERR_INVALID_ARG);
-            const float pc = p_child[(size_t)b * T + c];
-            if (u[(size_t)b * T + c] * R < pc) { nxt = c; break; }
+            if (uc * R < pc) { nxt = c; nxt_tok = tc; break; }
             R -= pc;
         }
         if (nxt < 0) break;
-        if (lane == 0) { pth[na] = nxt; ot[na - 1] = dt[nxt]; }
+        if (lane == 0) { o.path[na] = nxt; o.out_tok[na - 1] = nxt_tok; }
         cur = nxt;
         ++na;
     }
     // the stop node's drafted tokens carry no mass in the residual
     const uint32_t lo = __ballot_sync(0xffffffffu, pa0 == cur), hi = __ballot_sync(0xffffffffu, pa1 == cur);
     const int rank0 = __popc(lo & ((1u << lane) - 1u)), rank1 = __popc(lo) + __popc(hi & ((1u << lane) - 1u));
-    if (pa0 == cur) { excl[(size_t)b * 64 + rank0] = dt[lane]; excl_p[(size_t)b * 64 + rank0] = p_child[(size_t)b * T + lane]; }
-    if (pa1 == cur) { excl[(size_t)b * 64 + rank1] = dt[lane + 32]; excl_p[(size_t)b * 64 + rank1] = p_child[(size_t)b * T + lane + 32]; }
-    for (int k = na + lane; k < T; k += 32) { pth[k] = -1; ot[k] = -1; }
+    if (pa0 == cur) { o.excl[rank0] = tk0; o.excl_p[rank0] = pc0; }
+    if (pa1 == cur) { o.excl[rank1] = tk1; o.excl_p[rank1] = pc1; }
+    for (int k = na - 1 + lane; k < T; k += 32) { if (k >= na) o.path[k] = -1; o.out_tok[k] = -1; }
+    return WalkEnd{na, cur, __popc(lo) + __popc(hi), R};
+}
+
+// one warp per sequence
+__global__ void sampled_walk_kernel(sd_batch bt, const int32_t* __restrict__ draft, const float* __restrict__ p_child,
+                                    const float* __restrict__ u, int32_t* n_acc, int32_t* path, int32_t* out_tok,
+                                    int32_t* new_len, float* resid, int32_t* stop_row, int32_t* n_excl, int32_t* excl,
+                                    float* excl_p, int32_t* status) {
+    const int b = blockIdx.x, lane = threadIdx.x;
+    const int T = bt.T_max;
+    const WalkOut o{path + (size_t)b * T, out_tok + (size_t)b * T, excl + (size_t)b * 64, excl_p + (size_t)b * 64};
+    const WalkEnd e = sampled_walk(bt, b, lane, draft, p_child, u, o, status);
     if (lane == 0) {
-        n_acc[b] = na;
-        new_len[b] = bt.len[b] + na;
-        resid[b] = R;
-        stop_row[b] = b * T + cur;
-        n_excl[b] = __popc(lo) + __popc(hi);
-        ot[na - 1] = -1;                                     // filled by residual_pick_kernel
+        n_acc[b] = e.na;
+        n_excl[b] = e.n_excl;
+        stop_row[b] = b * T + e.stop;
+        resid[b] = e.R;
+        if (e.na > 0) new_len[b] = bt.len[b] + e.na;
     }
 }
 
@@ -201,49 +260,51 @@ residual_blocksum_kernel(int V, const int32_t* __restrict__ n_excl, const int32_
     if (threadIdx.x == 0) block_sum[(size_t)b * n_blocks + blockIdx.x] = s_v[0];
 }
 
-// First index i in [0, n) at which base + v[0] + ... + v[i] reaches target, found by one warp: every
-// lane sums a contiguous chunk, an inclusive scan over the lanes gives each chunk's starting value,
-// and the first lane whose chunk contains the crossing walks it element by element (fixed order of
-// additions).  positive_only: elements <= 0 cannot be the answer (tokens without mass).  Returns -1
-// when the sum stays short; *acc_io then holds base + the whole sum; *last_pos the last index with v > 0.
-__device__ __forceinline__ int warp_find_crossing(const float* v, int n, float target, bool positive_only,
-                                                  float* acc_io, int* last_pos, int lane) {
-    const int chunk = (n + 31) / 32;
-    const int i0 = min(n, lane * chunk), i1 = min(n, i0 + chunk);
-    float sum = 0.f;
-    int lastp = -1;
-    for (int i = i0; i < i1; ++i) { sum += v[i]; if (v[i] > 0.f) lastp = i; }
-    float incl = sum;
-#pragma unroll
-    for (int d = 1; d < 32; d <<= 1) {
-        const float y = __shfl_up_sync(0xffffffffu, incl, d);
-        if (lane >= d) incl += y;
-    }
-    const float before = *acc_io + (incl - sum);
-    int found = -1;
-    float acc_at = 0.f;
-    // lanes in order: the first chunk in which the walk actually reaches the target
-    uint32_t cand = __ballot_sync(0xffffffffu, i0 < i1 && before + sum >= target);
-    while (cand && found < 0) {
-        const int L0 = __ffs(cand) - 1;
-        cand &= cand - 1;
-        int idx = -1;
-        float acc = before;
-        if (lane == L0) {
-            for (int i = i0; i < i1; ++i) {
-                if (positive_only && !(v[i] > 0.f)) continue;
-                if (acc + v[i] >= target) { idx = i; break; }
-                acc += v[i];
-            }
+// Where the running sum *acc_io + v[0] + v[1] + ... first reaches `target`, among the elements with
+// v > 0 (all v >= 0), found by one warp in a few rounds: the range is cut into 32 consecutive pieces,
+// every lane sums one, an inclusive scan over the lanes gives each piece's end value, and the search
+// goes on inside the first piece that has mass and whose end value reaches the target, until the
+// pieces are single elements.  Every addition happens in a fixed order, so the answer is the same in
+// every run.  Returns the index, or -1 when the whole sum stays short; *acc_io then holds the running
+// sum in front of the returned element (all of it for -1); *last_pos the last index with v > 0, if any.
+// One level down the same elements are added in smaller pieces: where that leaves the refined search
+// a rounding short of the target, the piece's last element with mass is the answer.
+__device__ __forceinline__ int warp_find_crossing(const float* v, int n, float target, float* acc_io, int* last_pos, int lane) {
+    int lo = 0, hi = n;
+    float base = *acc_io;
+    for (bool top = true;; top = false) {
+        const int chunk = (hi - lo + 31) / 32;
+        const int i0 = min(hi, lo + lane * chunk), i1 = min(hi, i0 + chunk);
+        float sum = 0.f;
+        int lastp = -1;
+        for (int i = i0; i < i1; ++i) {
+            const float x = v[i];
+            sum += x;
+            if (x > 0.f) lastp = i;
         }
-        found = __shfl_sync(0xffffffffu, idx, L0);
-        acc_at = __shfl_sync(0xffffffffu, acc, L0);
+        float incl = sum;
+#pragma unroll
+        for (int d = 1; d < 32; d <<= 1) {
+            const float y = __shfl_up_sync(0xffffffffu, incl, d);
+            if (lane >= d) incl += y;
+        }
+        float excl = __shfl_up_sync(0xffffffffu, incl, 1);
+        if (lane == 0) excl = 0.f;
+        const int lp = __reduce_max_sync(0xffffffffu, lastp);
+        if (top && last_pos && lp >= 0) *last_pos = lp;
+        const uint32_t cand = __ballot_sync(0xffffffffu, sum > 0.f && base + incl >= target);
+        if (!cand) {
+            const float all = base + __shfl_sync(0xffffffffu, incl, 31);
+            if (top) { *acc_io = all; return -1; }
+            *acc_io = all - v[lp];                                   // (lp >= 0: the piece was chosen for having mass)
+            return lp;
+        }
+        const int L0 = __ffs(cand) - 1;
+        base += __shfl_sync(0xffffffffu, excl, L0);
+        lo = __shfl_sync(0xffffffffu, i0, L0);
+        hi = __shfl_sync(0xffffffffu, i1, L0);
+        if (chunk == 1) { *acc_io = base; return lo; }
     }
-    const float total = __shfl_sync(0xffffffffu, incl, 31);
-    const int lp = __reduce_max_sync(0xffffffffu, lastp);
-    if (last_pos && lp >= 0) *last_pos = lp;
-    *acc_io = found >= 0 ? acc_at : *acc_io + total;
-    return found;
 }
 
 // One CTA per sequence.  The block sums, then the masses of one block at a time, are brought into
@@ -266,10 +327,10 @@ residual_pick_kernel(sd_batch bt, int V, const float* __restrict__ w, const floa
     __syncthreads();
     if (threadIdx.x < 32) {
         float total = 0.f;                                             // whole remaining mass, same order of additions
-        warp_find_crossing(s_bs, n_blocks, INFINITY, false, &total, nullptr, lane);
+        warp_find_crossing(s_bs, n_blocks, INFINITY, &total, nullptr, lane);
         const float target = w[b] * total;
         float acc = 0.f;
-        int k = warp_find_crossing(s_bs, n_blocks, target, false, &acc, nullptr, lane);
+        int k = warp_find_crossing(s_bs, n_blocks, target, &acc, nullptr, lane);
         if (k < 0) { k = n_blocks - 1; acc -= s_bs[k]; }               // rounding left the sum short: last block
         if (lane == 0) { s_acc = acc; s_target = target; s_k = k; s_pick = -1; s_last = -1; }
     }
@@ -283,7 +344,7 @@ residual_pick_kernel(sd_batch bt, int V, const float* __restrict__ w, const floa
         if (threadIdx.x < 32) {
             float acc = s_acc;
             int lastp = -1;
-            const int i = warp_find_crossing(s_m, kResBlock, s_target, true, &acc, &lastp, lane);
+            const int i = warp_find_crossing(s_m, kResBlock, s_target, &acc, &lastp, lane);
             if (lane == 0) {
                 s_acc = acc;
                 if (lastp >= 0) s_last = k * kResBlock + lastp;
@@ -303,65 +364,115 @@ residual_pick_kernel(sd_batch bt, int V, const float* __restrict__ w, const floa
     }
 }
 
-// Residual draw from the LM-head pass's own statistics.  One CTA per sequence: the masses of the 32-row
-// vocabulary groups of the stop row follow from (group maximum, group sum) and the row's lse; the
-// drafted children's probabilities are taken out of their groups; warp 0 finds the group in which the
-// cumulative mass reaches w * (total); that group's 32 logits are recomputed (32 dot products) and the
-// token is found among them.  W is not streamed a second time and no logits-sized data exist.
+// Residual draw from the LM-head pass's own statistics, by one CTA of 256 threads for one sequence.
+// The masses of the 32-row vocabulary groups of the stop row follow from (group maximum, group sum)
+// and the row's lse; the drafted children's probabilities are taken out of their groups; warp 0 finds
+// the group in which the cumulative mass reaches w * (total); that group's 32 logits are recomputed
+// (32 dot products) and the token is found among them.  W is not streamed a second time and no
+// logits-sized data exist.  row: LM-head row of the stop node; excl / excl_p: its ne drafted children.
 constexpr int kPickMaxGroups = 8192;   // vocabularies up to 262144 tokens
-__global__ void __launch_bounds__(256)
-residual_pick_groups_kernel(sd_batch bt, const uint16_t* __restrict__ hidden, const uint16_t* __restrict__ W, int Hd, int V,
-                            float inv_temp, const float* __restrict__ lse, const float2* __restrict__ group_stats, int n_groups,
-                            const float* __restrict__ w, const int32_t* __restrict__ stop_row, const int32_t* __restrict__ n_excl,
-                            const int32_t* __restrict__ excl, const float* __restrict__ excl_p, const int32_t* __restrict__ n_acc,
-                            int32_t* out_tok, int32_t* status) {
+// kClusterCtas > 1: the CTAs of the cluster share the reading of the table (each entry sits in a
+// sector of its own, so one SM's load path is the limit) and push the masses into the shared memory
+// of the cluster's first CTA, which alone goes on; every CTA of the cluster must make the call.
+template <int kClusterCtas>
+__device__ __forceinline__ void residual_pick_groups(const uint16_t* __restrict__ hidden, const uint16_t* __restrict__ W,
+                                                     int Hd, int V, float inv_temp, float row_lse, int M, int row,
+                                                     const float2* __restrict__ group_stats, int n_groups, float wb,
+                                                     int ne, const int32_t* excl, const float* excl_p,
+                                                     int32_t* out_slot, int32_t* status) {
     __shared__ float s_g[kPickMaxGroups];
+    __shared__ float s_part[256];                                      // sums of the threads' runs of groups
     __shared__ float s_m[32];
+    __shared__ int32_t s_ex[64];                                       // the stop node's drafted tokens ...
+    __shared__ float s_exp[64];                                        // ... and their probabilities
     __shared__ float s_acc, s_target;
     __shared__ int s_k, s_pick, s_last;
-    const int b = blockIdx.x;
-    const int na = n_acc[b];
-    if (na < 1 || na > bt.T_max) return;                               // bad tree: already reported
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
-    const int row = stop_row[b];
-    const int M = bt.B * bt.T_max;
     const float c2 = inv_temp * 1.4426950408889634f;
-    const float lse2 = lse[row] * 1.4426950408889634f;
-    for (int g = threadIdx.x; g < n_groups; g += blockDim.x) {
-        const float2 st = group_stats[(size_t)g * M + row];
-        s_g[g] = st.y > 0.f ? st.y * exp2f(st.x * c2 - lse2) : 0.f;
+    const float lse2 = row_lse * 1.4426950408889634f;
+    {
+        // (one 8-byte entry per group, a table row apart: the loads of a batch are issued together)
+        const int rank = kClusterCtas > 1 ? (int)sm100::cluster_ctarank() : 0;
+        const int per_cta = (n_groups + kClusterCtas - 1) / kClusterCtas;
+        const int g_end = min(n_groups, (rank + 1) * per_cta);
+        const uint32_t dst = kClusterCtas > 1 ? sm100::map_dsmem(sm100::smem_u32(s_g), 0) : 0;
+        constexpr int kAhead = 8;
+        for (int g0 = rank * per_cta + threadIdx.x; g0 < g_end; g0 += (int)blockDim.x * kAhead) {
+            float2 st[kAhead];
+#pragma unroll
+            for (int a = 0; a < kAhead; ++a) {
+                const int g = g0 + (int)blockDim.x * a;
+                if (g < g_end) st[a] = __ldg(group_stats + (size_t)g * M + row);
+            }
+#pragma unroll
+            for (int a = 0; a < kAhead; ++a) {
+                const int g = g0 + (int)blockDim.x * a;
+                if (g < g_end) {
+                    const float m = st[a].y > 0.f ? st[a].y * exp2f(st[a].x * c2 - lse2) : 0.f;
+                    if (kClusterCtas > 1) sm100::st_dsmem_f32(dst + g * 4, m);
+                    else s_g[g] = m;
+                }
+            }
+        }
+        if (kClusterCtas > 1) {
+            sm100::cluster_arrive_release();
+            sm100::cluster_wait_acquire();
+            if (rank != 0) return;
+        }
     }
+    if (threadIdx.x < ne) { s_ex[threadIdx.x] = excl[threadIdx.x]; s_exp[threadIdx.x] = excl_p[threadIdx.x]; }
     __syncthreads();
-    const int ne = n_excl[b];
     if (threadIdx.x == 0)                                              // drafted children carry no mass (fixed order)
         for (int e = 0; e < ne; ++e) {
-            const int g = excl[(size_t)b * 64 + e] >> 5;
-            s_g[g] = fmaxf(s_g[g] - excl_p[(size_t)b * 64 + e], 0.f);
+            const int g = s_ex[e] >> 5;
+            s_g[g] = fmaxf(s_g[g] - s_exp[e], 0.f);
         }
+    __syncthreads();
+    // every thread sums a run of consecutive groups; the search goes over the 256 sums, then inside one run
+    const int run = (n_groups + (int)blockDim.x - 1) / (int)blockDim.x;
+    {
+        const int g0 = min(n_groups, (int)threadIdx.x * run), g1 = min(n_groups, g0 + run);
+        float sum = 0.f;
+        for (int g = g0; g < g1; ++g) sum += s_g[g];
+        s_part[threadIdx.x] = sum;
+    }
     __syncthreads();
     if (threadIdx.x < 32) {
         float total = 0.f;
-        warp_find_crossing(s_g, n_groups, INFINITY, false, &total, nullptr, lane);
-        const float target = w[b] * total;
+        warp_find_crossing(s_part, (int)blockDim.x, INFINITY, &total, nullptr, lane);
+        const float target = wb * total;
         float acc = 0.f;
-        int k = warp_find_crossing(s_g, n_groups, target, false, &acc, nullptr, lane);
-        if (k < 0) { k = n_groups - 1; acc -= s_g[k]; }
+        int k = -1;
+        const int t = warp_find_crossing(s_part, (int)blockDim.x, target, &acc, nullptr, lane);
+        if (t >= 0) {
+            const int g0 = t * run, len = min(n_groups, g0 + run) - g0;
+            int lastp = -1;
+            k = warp_find_crossing(s_g + g0, len, target, &acc, &lastp, lane);
+            if (k < 0) { k = max(lastp, 0); acc -= s_g[g0 + k]; }      // a rounding short inside the run: its last group with mass
+            k += g0;
+        } else {                                                       // no mass anywhere (reported below), or w * total rounded up
+            k = n_groups - 1;
+            acc -= s_g[k];
+        }
         if (lane == 0) { s_acc = acc; s_target = target; s_k = k; s_pick = -1; s_last = -1; }
     }
     __syncthreads();
     const uint4* hrow = reinterpret_cast<const uint4*>(hidden + (size_t)row * Hd);
     // the 32 probabilities of group k, recomputed into s_m: eight warps, four tokens each
     auto recompute_group = [&](int k) {
-        for (int i = warp * 4; i < warp * 4 + 4; ++i) {
-            const int t = k * 32 + i;
-            float m = 0.f;
-            if (t < V) {
-                const float l = warp_dot_bf16(reinterpret_cast<const uint4*>(W + (size_t)t * Hd), hrow, Hd / 8, lane);
-                bool hit = false;
-                for (int e = lane; e < ne; e += 32) hit |= (excl[(size_t)b * 64 + e] == t);
-                m = __any_sync(0xffffffffu, hit) ? 0.f : __expf(l * inv_temp - lse[row]);
-            }
-            if (lane == 0) s_m[i] = m;
+        const int t0 = k * 32 + warp * 4;
+        const uint4* wrow[4];
+#pragma unroll
+        for (int i = 0; i < 4; ++i) wrow[i] = reinterpret_cast<const uint4*>(W + (size_t)min(t0 + i, V - 1) * Hd);
+        float l[4];
+        warp_dots_bf16<4>(wrow, hrow, Hd / 8, lane, l);
+#pragma unroll
+        for (int i = 0; i < 4; ++i) {
+            const int t = t0 + i;
+            bool hit = false;
+            for (int e = lane; e < ne; e += 32) hit |= (s_ex[e] == t);
+            const float m = (t >= V || __any_sync(0xffffffffu, hit)) ? 0.f : __expf(l[i] * inv_temp - row_lse);
+            if (lane == 0) s_m[warp * 4 + i] = m;
         }
         __syncthreads();
     };
@@ -370,7 +481,7 @@ residual_pick_groups_kernel(sd_batch bt, const uint16_t* __restrict__ hidden, co
         if (threadIdx.x < 32) {
             float acc = s_acc;
             int lastp = -1;
-            const int i = warp_find_crossing(s_m, 32, s_target, true, &acc, &lastp, lane);
+            const int i = warp_find_crossing(s_m, 32, s_target, &acc, &lastp, lane);
             if (lane == 0) {
                 s_acc = acc;
                 if (lastp >= 0) s_last = k * 32 + lastp;
@@ -392,8 +503,144 @@ residual_pick_groups_kernel(sd_batch bt, const uint16_t* __restrict__ hidden, co
     if (threadIdx.x == 0) {
         int pick = s_pick >= 0 ? s_pick : s_last;
         if (pick < 0) { set_status(status, SD_ERR_BOUNDS); pick = 0; }  // no mass at all: inputs were not finite
-        out_tok[(size_t)b * bt.T_max + na - 1] = pick;
+        *out_slot = pick;
     }
+}
+
+// one CTA per sequence
+__global__ void __launch_bounds__(256)
+residual_pick_groups_kernel(sd_batch bt, const uint16_t* __restrict__ hidden, const uint16_t* __restrict__ W, int Hd, int V,
+                            float inv_temp, const float* __restrict__ lse, const float2* __restrict__ group_stats, int n_groups,
+                            const float* __restrict__ w, const int32_t* __restrict__ stop_row, const int32_t* __restrict__ n_excl,
+                            const int32_t* __restrict__ excl, const float* __restrict__ excl_p, const int32_t* __restrict__ n_acc,
+                            int32_t* out_tok, int32_t* status) {
+    const int b = blockIdx.x;
+    const int na = n_acc[b];
+    if (na < 1 || na > bt.T_max) return;                               // bad tree: already reported
+    const int row = stop_row[b];
+    residual_pick_groups<1>(hidden, W, Hd, V, inv_temp, lse[row], bt.B * bt.T_max, row, group_stats, n_groups, w[b], n_excl[b],
+                            excl + (size_t)b * 64, excl_p + (size_t)b * 64, out_tok + (size_t)b * bt.T_max + na - 1, status);
+}
+
+// ---------------------------------------------------------------------------
+// Tail of a verify step at a sampling temperature, behind the LM-head tiles of a statistics pass: one
+// cluster of eight CTAs per sequence.
+//   1. every CTA merges the per-CTA soft-max partials of eight of the sequence's LM-head rows -> lse
+//   2. every warp of the cluster computes one node's probability under its parent's distribution
+//   3. every CTA repeats the (cheap) rejection walk into its own shared memory
+//   4. the cluster's first CTA writes the outputs and draws the last token from the group table
+//   5. every CTA copies the accepted nodes' K/V into the caches of its share of the layers
+// Steps 1 and 2 hand their results on through global memory across a cluster barrier.  The arithmetic
+// is that of the stand-alone kernels (the same device functions), so the results are the same bits.
+// ---------------------------------------------------------------------------
+constexpr int kTailCluster = 8;
+__global__ void __launch_bounds__(256)
+sampled_tail_kernel(sd_batch bt, const __grid_constant__ CompactLayers ly, int L, LmTables tb, float c2,
+                    const uint16_t* __restrict__ hidden, const uint16_t* __restrict__ W, int Hd, int V, float inv_temp,
+                    const float2* __restrict__ group_stats, int n_groups, const int32_t* __restrict__ draft,
+                    const float* __restrict__ u, const float* __restrict__ w, float* lse, float* p_child,
+                    int32_t* n_acc, int32_t* path, int32_t* out_tok, int32_t* new_len, int32_t* status) {
+    __shared__ int32_t s_path[kMaxT], s_tok[kMaxT], s_excl[64];
+    __shared__ float s_excl_p[64];
+    __shared__ WalkEnd s_end;
+    const int b = blockIdx.x / kTailCluster;
+    const int rank = (int)sm100::cluster_ctarank();
+    const int T = bt.T_max, warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+    // 1. lse of rows rank * 8 .. + 7 (of every 64): eight lanes per row, the first two warps
+    if (warp < 2)
+        for (int r0 = 0; r0 < T; r0 += 8 * kTailCluster) {
+            const int node = r0 + rank * 8 + (threadIdx.x >> 3), sub = threadIdx.x & 7;
+            int32_t k, i;
+            const float row_lse = merge_row_stats(tb.part_key, tb.part_idx, tb.part_ref, tb.part_sum, tb.n_ctas, kLmMaxCols,
+                                                  b * T + node, node < T, sub, c2, k, i);
+            if (node < T && sub == 0) lse[b * T + node] = row_lse;
+        }
+    sm100::cluster_arrive_release();
+    sm100::cluster_wait_acquire();
+    // 2. probabilities of the drafted tokens: node rank * 8 + warp (of every 64)
+    for (int j0 = 0; j0 < T; j0 += 8 * kTailCluster) {
+        const int j = j0 + rank * 8 + warp;
+        if (j < T) {
+            const float p = child_prob(bt, b, j, lane, hidden, W, Hd, V, inv_temp, lse, draft, status);
+            if (lane == 0) p_child[(size_t)b * T + j] = p;
+        }
+    }
+    sm100::cluster_arrive_release();
+    sm100::cluster_wait_acquire();
+    // 3. the walk
+    if (warp == 0) {
+        const WalkOut o{s_path, s_tok, s_excl, s_excl_p};
+        const WalkEnd e = sampled_walk(bt, b, lane, draft, p_child, u, o, status);
+        if (lane == 0) s_end = e;
+    }
+    __syncthreads();
+    const WalkEnd e = s_end;
+    // 4. outputs and the last token (the whole cluster reads the group table, the first CTA draws)
+    if (rank == 0 && threadIdx.x == 0) {
+        n_acc[b] = e.na;
+        if (e.na > 0) new_len[b] = bt.len[b] + e.na;
+    }
+    if (e.na > 0) {                                                    // (the same in every CTA of the cluster)
+        if (rank == 0)
+            for (int k = threadIdx.x; k < T; k += blockDim.x) {
+                path[(size_t)b * T + k] = s_path[k];
+                if (k != e.na - 1) out_tok[(size_t)b * T + k] = s_tok[k];
+            }
+        const int row = b * T + e.stop;
+        residual_pick_groups<kTailCluster>(hidden, W, Hd, V, inv_temp, lse[row], bt.B * T, row, group_stats, n_groups, w[b],
+                                           e.n_excl, s_excl, s_excl_p, out_tok + (size_t)b * T + e.na - 1, status);
+    }
+    // 5. accepted rows into the caches; the first CTA, busy with the draw, takes the smallest share
+    for (int l = kTailCluster - 1 - rank; l < L; l += kTailCluster)
+        compact_sequence(bt, ly, l, 1, b, e.na, s_path, threadIdx.x, blockDim.x, status);
+}
+
+sd_status launch_lmhead_accept_sampled_compact(const sd_batch& bt, const void* hidden, const void* W, int Hd, int V,
+                                               float inv_temp, const int32_t* draft, const float* u, const float* w,
+                                               const sd_kv_layer* layers, int L, const void* const* kt, const void* const* vt,
+                                               float* lse, float* group_stats, int32_t* n_acc, int32_t* path,
+                                               int32_t* out_tok, int32_t* new_len, void* ws, size_t ws_bytes,
+                                               int32_t* dev_status, cudaStream_t st) {
+    const int B = bt.B, T = bt.T_max, M = B * T;
+    if (Hd > 16384 || (V + 31) / 32 > kPickMaxGroups) return SD_ERR_UNSUPPORTED;
+    if (ws_bytes < sampled_workspace_bytes(B, T, V, 16384)) return SD_ERR_WORKSPACE;
+    const SampledWs s = carve(ws, B, T, V, 16384);
+    const size_t lm_bytes = stats_workspace_bytes(M, V);
+    if (M > kLmMaxCols || L > kLayersPerLaunch) {
+        // shapes beyond one pass of the candidate tables or one set of layer descriptors: the same steps
+        // as separate launches
+        sd_status r = launch_lmhead_stats(hidden, W, M, Hd, V, inv_temp, nullptr, nullptr, lse, group_stats, s.lm_ws, lm_bytes,
+                                          dev_status, st);
+        if (r != SD_OK) return r;
+        r = launch_accept_sampled(bt, hidden, W, Hd, V, inv_temp, lse, group_stats, draft, u, w, n_acc, path, out_tok, new_len,
+                                  ws, ws_bytes, dev_status, st);
+        if (r != SD_OK) return r;
+        return launch_compact(bt, layers, L, kt, vt, n_acc, path, dev_status, st);
+    }
+    LmTables tb;
+    const sd_status r = launch_lmhead_stats_tiles(hidden, W, M, Hd, V, inv_temp, lse, group_stats, s.lm_ws, lm_bytes,
+                                                  dev_status, st, &tb);
+    if (r != SD_OK) return r;
+    CompactLayers ly;
+    fill_compact_layers(&ly, layers, kt, vt, 0, L);
+    cudaLaunchConfig_t cfg = {};
+    cfg.gridDim = dim3(B * kTailCluster);
+    cfg.blockDim = dim3(256);
+    cfg.stream = st;
+    cudaLaunchAttribute attr[1];
+    attr[0].id = cudaLaunchAttributeClusterDimension;
+    attr[0].val.clusterDim.x = kTailCluster;
+    attr[0].val.clusterDim.y = 1;
+    attr[0].val.clusterDim.z = 1;
+    cfg.attrs = attr;
+    cfg.numAttrs = 1;
+    const float c2 = inv_temp * 1.4426950408889634f;
+    const int n_groups = (V + 31) / 32;
+    if (cudaLaunchKernelEx(&cfg, sampled_tail_kernel, bt, ly, L, tb, c2, static_cast<const uint16_t*>(hidden),
+                           static_cast<const uint16_t*>(W), Hd, V, inv_temp, reinterpret_cast<const float2*>(group_stats),
+                           n_groups, draft, u, w, lse, s.p_child, n_acc, path, out_tok, new_len, dev_status) != cudaSuccess)
+        return SD_ERR_CUDA;
+    return SD_OK;
 }
 
 sd_status launch_accept_sampled(const sd_batch& bt, const void* hidden, const void* W, int Hd, int V, float inv_temp,

@@ -16,6 +16,10 @@ struct CompactLayers {
     int32_t num_blocks[kLayersPerLaunch];
 };
 
+// descriptors of layers [l0, l0 + nl) (implemented beside the compaction kernel)
+void fill_compact_layers(CompactLayers* ly, const sd_kv_layer* layers, const void* const* kt, const void* const* vt,
+                         int l0, int nl);
+
 __device__ __forceinline__ float key_to_float(int32_t k) {
     return __int_as_float(k < 0 ? (k ^ 0x7fffffff) : k);
 }
@@ -23,6 +27,68 @@ __device__ __forceinline__ float key_to_float(int32_t k) {
 // (key, index) candidates: larger key wins, lower index among equal keys
 __device__ __forceinline__ void take_better(int32_t& k, int32_t& i, int32_t k2, int32_t i2) {
     if (k2 > k || (k2 == k && i2 < i)) { k = k2; i = i2; }
+}
+
+__device__ __forceinline__ float ex2_lm(float x) {
+    float y;
+    asm("ex2.approx.ftz.f32 %0, %1;" : "=f"(y) : "f"(x));
+    return y;
+}
+
+// running (reference, sum) of a row's soft-max statistics takes in a new partial (ref2, sum2):
+// sum counts 2^((logit - ref) * c2)
+__device__ __forceinline__ void merge_sumexp(float& ref, float& sum, float ref2, float sum2, float c2) {
+    if (!(sum2 > 0.f)) return;
+    if (ref2 > ref) { sum = sum * ex2_lm((ref - ref2) * c2) + sum2; ref = ref2; }
+    else            { sum += sum2 * ex2_lm((ref2 - ref) * c2); }
+}
+
+// Candidates and soft-max partials of one hidden row (column `col` of the per-CTA tables), merged by the
+// eight consecutive lanes that share the row: lane `sub` takes the CTAs sub, sub + 8, ..., then three
+// exchange steps combine the eight (always lower lane first, so all eight end with the same bits).
+// Every lane of the warp must call this; rows beyond the problem pass active = false.  Returns the
+// row's log sum exp(logit / temperature) (natural log); k, i: the arg-max candidate (key, index).
+__device__ __forceinline__ float merge_row_stats(const int32_t* __restrict__ part_key, const int32_t* __restrict__ part_idx,
+                                                 const float* __restrict__ part_ref, const float* __restrict__ part_sum,
+                                                 int n_ctas, int row_stride, int col, bool active, int sub, float c2,
+                                                 int32_t& k, int32_t& i) {
+    k = INT32_MIN; i = 0x7fffffff;
+    float rf = -INFINITY, sm = 0.f;
+    if (active) {
+        // (the loads of a batch are issued together, then merged in CTA order: latency-bound)
+        constexpr int kAhead = 20;                  // 148 CTAs: 19 per lane
+        for (int c0 = sub; c0 < n_ctas; c0 += 8 * kAhead) {
+            int32_t pk[kAhead], pi[kAhead];
+            float pr[kAhead], ps[kAhead];
+#pragma unroll
+            for (int a = 0; a < kAhead; ++a) {
+                const int c = c0 + 8 * a;
+                if (c < n_ctas) {
+                    pk[a] = __ldg(part_key + (size_t)c * row_stride + col);
+                    pi[a] = __ldg(part_idx + (size_t)c * row_stride + col);
+                    pr[a] = __ldg(part_ref + (size_t)c * row_stride + col);
+                    ps[a] = __ldg(part_sum + (size_t)c * row_stride + col);
+                }
+            }
+#pragma unroll
+            for (int a = 0; a < kAhead; ++a)
+                if (c0 + 8 * a < n_ctas) {
+                    take_better(k, i, pk[a], pi[a]);
+                    merge_sumexp(rf, sm, pr[a], ps[a], c2);
+                }
+        }
+    }
+#pragma unroll
+    for (int d = 1; d <= 4; d <<= 1) {
+        const int32_t k2 = __shfl_xor_sync(0xffffffffu, k, d), i2 = __shfl_xor_sync(0xffffffffu, i, d);
+        const float rf2 = __shfl_xor_sync(0xffffffffu, rf, d), sm2 = __shfl_xor_sync(0xffffffffu, sm, d);
+        take_better(k, i, k2, i2);
+        float ra = (sub & d) ? rf2 : rf, sa = (sub & d) ? sm2 : sm;
+        const float rb = (sub & d) ? rf : rf2, sb = (sub & d) ? sm : sm2;
+        merge_sumexp(ra, sa, rb, sb, c2);
+        rf = ra; sm = sa;
+    }
+    return (rf * c2 + log2f(sm)) * 0.6931471805599453f;
 }
 
 // Greedy acceptance for one sequence, executed by one warp.  par/dt/tg point at the sequence's

@@ -165,9 +165,10 @@ class VerifyStep:
                                     self.maxlogit, self.n_acc, self.path, self.out_tok, self.new_len,
                                     self.workspace, self.status, stream)
 
-    def tail_sampled(self, inv_temp: float, u: torch.Tensor, w: torch.Tensor, stream=None):
+    def tail_sampled(self, inv_temp: float, u: torch.Tensor, w: torch.Tensor, stream=None, fused=True):
         """The tail at a sampling temperature: LM head with log-sum-exp, the rejection walk with the
-        given uniforms (u [B,T], w [B], device f32), the residual draw, then compaction."""
+        given uniforms (u [B,T], w [B], device f32), the residual draw, then compaction; through the one
+        fused call, or (fused=False) as the three separate calls it stands for."""
         if getattr(self, "lse_rows", None) is None:
             self.lse_rows = torch.zeros(self.w.B * self.w.T_max, dtype=torch.float32, device=self.device)
             self.group_stats = torch.zeros(sd.group_stats_shape(self.w.B * self.w.T_max, self.w.V),
@@ -175,7 +176,12 @@ class VerifyStep:
             need = sd.sd_workspace_bytes(self.batch, self.w.B * self.w.T_max, self.w.V)
             if self.workspace.numel() < need:
                 self.workspace = torch.empty(need, dtype=torch.uint8, device=self.device)
-        sd.sd_lmhead_stats(self.hidden, self.W, inv_temp, self.argmax, self.maxlogit, self.lse_rows,
+        if fused:
+            sd.sd_lmhead_accept_sampled_compact(self.batch, self.hidden, self.W, inv_temp, self.draft_tok, u, w,
+                                                self.layerset, self.lse_rows, self.group_stats, self.n_acc, self.path,
+                                                self.out_tok, self.new_len, self.workspace, self.status, stream)
+            return
+        sd.sd_lmhead_stats(self.hidden, self.W, inv_temp, None, None, self.lse_rows,
                            self.workspace, self.status, stream, group_stats=self.group_stats)
         sd.sd_accept_tree_sampled(self.batch, self.hidden, self.W, inv_temp, self.lse_rows, self.draft_tok, u, w,
                                   self.n_acc, self.path, self.out_tok, self.new_len, self.workspace, self.status, stream,

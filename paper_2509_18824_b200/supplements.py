@@ -157,8 +157,12 @@ def sampled(cfg="c5", inv_temp=1.0):
                                                       vs.n_acc, vs.path, vs.out_tok, vs.new_len, ws, st), 10)
     ms_acc = _time(lambda: sd.sd_accept_tree_sampled(vs.batch, vs.hidden, vs.W, inv_temp, lse, vs.draft_tok, u, wv,
                                                      vs.n_acc, vs.path, vs.out_tok, vs.new_len, ws, st, group_stats=gs), 10)
+    ms_sep = _time(lambda: vs.tail_sampled(inv_temp, u, wv, fused=False), 10)
+    ms_fused = _time(lambda: vs.tail_sampled(inv_temp, u, wv, fused=True), 10)
     wbytes = w.V * w.Hd * 2
     print(json.dumps({"call": "sampled tail", "workload": cfg, "rows": M,
+                      "whole_tail_fused_call_us": ms_fused * 1e3, "whole_tail_separate_calls_us": ms_sep * 1e3,
+                      "layers_compacted": vs.L,
                       "sd_lmhead_argmax_us": ms_greedy * 1e3, "sd_lmhead_stats_us": ms_stats * 1e3,
                       "stats_tflops": flops / ms_stats / 1e9, "stats_frac_tensor_burst": flops / ms_stats / 1e9 / tens,
                       "sd_lmhead_stats_without_group_table_us": ms_stats0 * 1e3,

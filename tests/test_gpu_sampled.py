@@ -1,5 +1,6 @@
-"""GPU parity of verification at a sampling temperature: sd_lmhead_stats and sd_accept_tree_sampled
-against oracle/sampling.py on the same seeded inputs (uniform numbers are inputs on both sides)."""
+"""GPU parity of verification at a sampling temperature: sd_lmhead_stats, sd_accept_tree_sampled and
+the fused sd_lmhead_accept_sampled_compact against oracle/sampling.py on the same seeded inputs
+(uniform numbers are inputs on both sides)."""
 import numpy as np
 import pytest
 import torch
@@ -8,7 +9,7 @@ import oracle
 from oracle import sampling as smp
 from paper_2509_18824_b200 import binding as sd
 from paper_2509_18824_b200 import workloads as wl
-from paper_2509_18824_b200.step import to_device
+from paper_2509_18824_b200.step import VerifyStep, to_device
 
 pytestmark = pytest.mark.gpu
 
@@ -260,3 +261,157 @@ def test_sampled_gpu_output_frequencies_follow_the_target_distribution():
     n = B * reps
     sigma = np.sqrt(n * p[0] * (1 - p[0]))
     assert (np.abs(counts - n * p[0]) <= 5 * sigma + 1).all(), (counts / n, p[0])
+
+
+def decisive_uniforms(w, tok, p64_of_row, g, floor=20 * WALK_CLOSE):
+    """Uniform numbers under which no comparison of the fp64 walk is a close call (redrawn per
+    sequence until the smallest |u * R - p| on its walk exceeds `floor`), with the fp64 walk's results."""
+    B, T = w.B, w.T_max
+    u = np.zeros((B, T), np.float32)
+    n_acc = np.zeros(B, np.int32)
+    path = np.full((B, T), -1, np.int32)
+    stop_R = np.zeros(B)
+    for b in range(B):
+        n, par = int(w.n_nodes[b]), w.parents[b]
+        pc64 = np.zeros(T)
+        for j in range(1, n):
+            pc64[j] = p64_of_row(b * T + int(par[j]))[tok[b, j]]
+        for _ in range(200):
+            u[b] = g.random(T).astype(np.float32)
+            pth, R, margin = smp.accept_walk(par, n, tok[b], pc64, u[b].astype(np.float64))
+            if margin > floor:
+                break
+        else:
+            raise AssertionError("no decisive uniforms found")
+        n_acc[b] = len(pth)
+        path[b, :len(pth)] = pth
+        stop_R[b] = R
+    return u, n_acc, path, stop_R
+
+
+def step_outputs(vs):
+    return dict(lse=vs.lse_rows.cpu().numpy(), n_acc=vs.n_acc.cpu().numpy(), path=vs.path.cpu().numpy(),
+                out_tok=vs.out_tok.cpu().numpy(), new_len=vs.new_len.cpu().numpy(),
+                k=[x.cpu().numpy() for x in vs.k_cache], v=[x.cpu().numpy() for x in vs.v_cache])
+
+
+@pytest.mark.parametrize("cfg,over,inv_temp", [
+    ("c1", dict(L=1), 2.0),
+    ("c2", dict(L=3, V=5000, Hd=256), 3.0),
+    ("c5", dict(L=9, V=8192, Hd=512, prefix=200), 5.0),                      # nine layers over eight CTAs
+    ("c4", dict(L=2, V=4096, Hd=256, prefix_range=(40, 300)), 3.0),          # 960 rows: the internal fall-back
+    ("chain11", dict(L=4, V=3000, Hd=128, prefix=70), 2.5),
+])
+def test_fused_sampled_tail_equals_the_separate_calls_and_the_reference(cfg, over, inv_temp):
+    """sd_lmhead_accept_sampled_compact against sd_lmhead_stats + sd_accept_tree_sampled +
+    sd_compact_kv: every output and every cache byte identical.  Against the checker: with uniforms
+    under which the fp64 walk has no close call the path must be the fp64 path, the drawn token the
+    fp64 token (or a close call of the CDF), and the caches those the checker's compaction leaves."""
+    w = wl.make(cfg, hidden_gain=24.0, **over)
+    B, T, V, L = w.B, w.T_max, w.W.shape[0], w.L
+    lg = oracle.logits(w.hidden, w.W)
+    p64, lse64 = smp.softmax_rows(lg, inv_temp)
+    tok = good_drafts(w, lg, 5)
+    w.draft_tok = tok
+    g = np.random.default_rng(17)
+    u, ref_n_acc, ref_path, stop_R = decisive_uniforms(w, tok, lambda r: p64[r], g)
+    wv = g.random(B).astype(np.float32)
+    res = []
+    for fused in (False, True):
+        vs = VerifyStep(w)
+        vs.tail_sampled(inv_temp, to_device(u), to_device(wv), fused=fused)
+        torch.cuda.synchronize()
+        vs.check_status()
+        res.append(step_outputs(vs))
+    for key in ("lse", "n_acc", "path", "out_tok", "new_len"):
+        np.testing.assert_array_equal(res[0][key], res[1][key], err_msg=key)
+    for l in range(L):
+        np.testing.assert_array_equal(res[0]["k"][l], res[1]["k"][l])
+        np.testing.assert_array_equal(res[0]["v"][l], res[1]["v"][l])
+    got = res[1]
+    np.testing.assert_allclose(got["lse"], lse64, rtol=0, atol=5e-4)
+    np.testing.assert_array_equal(got["n_acc"], ref_n_acc)
+    np.testing.assert_array_equal(got["path"], ref_path)
+    np.testing.assert_array_equal(got["new_len"], w.len + ref_n_acc)
+    close_calls = 0
+    for b in range(B):
+        n, par, na = int(w.n_nodes[b]), w.parents[b], int(ref_n_acc[b])
+        assert list(got["out_tok"][b, :na - 1]) == [int(tok[b, j]) for j in ref_path[b, 1:na]]
+        assert (got["out_tok"][b, na:] == -1).all()
+        last = int(ref_path[b, na - 1])
+        excl = [int(tok[b, c]) for c in smp.children_of(par, n, last)]
+        t_ref, margin = smp.residual_sample(p64[b * T + last], excl, float(stop_R[b]), float(wv[b]))
+        t_got = int(got["out_tok"][b, na - 1])
+        assert t_got not in excl and 0 <= t_got < V
+        if t_got != t_ref:
+            assert margin <= CLOSE * max(float(stop_R[b]), 1e-3), (b, t_got, t_ref, margin)
+            close_calls += 1
+    assert close_calls <= max(1, B // 8)
+    assert B == 1 or (ref_n_acc > 1).any()                                   # some walk moved
+    G = oracle.Geometry.of(w)
+    for l in range(L):
+        rk, rv = w.k_cache[l].copy(), w.v_cache[l].copy()
+        oracle.compact(G, rk, rv, w.k_tree[l], w.v_tree[l], ref_n_acc, ref_path)
+        np.testing.assert_array_equal(got["k"][l].view(np.uint16), rk)
+        np.testing.assert_array_equal(got["v"][l].view(np.uint16), rv)
+
+
+def test_fused_sampled_tail_bad_tree_touches_no_cache():
+    w = wl.make("c1", hidden_gain=16.0)
+    w.parents = w.parents.copy(); w.parents[0, 3] = 5
+    vs = VerifyStep(w)
+    before_k, before_v = vs.k_cache[0].clone(), vs.v_cache[0].clone()
+    vs.status.zero_()
+    vs.tail_sampled(1.0, to_device(np.full((1, 8), 0.5, np.float32)), to_device(np.full(1, 0.5, np.float32)))
+    torch.cuda.synchronize()
+    assert int(vs.status.item()) == sd.SD_ERR_INVALID_TREE
+    assert int(vs.n_acc[0].item()) == 0
+    assert torch.equal(before_k, vs.k_cache[0]) and torch.equal(before_v, vs.v_cache[0])
+
+
+def test_fused_sampled_tail_full_vocabulary():
+    """Batch 8, 60-node trees, vocabulary 152064, four layers: the fused call against the fp64 rule on
+    the rows the rule looks at, and against the checker's compaction."""
+    w = wl.make("c5", hidden_gain=40.0, L=4, prefix=300)
+    B, T, V, L = w.B, w.T_max, w.V, w.L
+    ram, t1, t2 = oracle.lmhead(w.hidden, w.W)
+    g = np.random.default_rng(12)
+    tok = g.integers(0, V, size=(B, T)).astype(np.int32)
+    for b in range(B):
+        for i in range(int(w.n_nodes[b])):
+            kids = smp.children_of(w.parents[b], int(w.n_nodes[b]), i)
+            if kids:
+                tok[b, kids[0]] = ram[b * T + i]
+                for k, c in enumerate(kids[1:]):
+                    tok[b, c] = (ram[b * T + i] + 1 + k) % V
+    w.draft_tok = tok
+    inv_temp = 6.0
+    rows = sorted({b * T + int(w.parents[b][j]) for b in range(B) for j in range(1, int(w.n_nodes[b]))}
+                  | {b * T + j for b in range(B) for j in range(int(w.n_nodes[b]))})
+    p64, lse64 = smp.softmax_rows(oracle.logits(w.hidden[rows], w.W), inv_temp)
+    row_of = {r: i for i, r in enumerate(rows)}
+    u, ref_n_acc, ref_path, stop_R = decisive_uniforms(w, tok, lambda r: p64[row_of[r]], g)
+    wv = g.random(B).astype(np.float32)
+    vs = VerifyStep(w)
+    vs.tail_sampled(inv_temp, to_device(u), to_device(wv))
+    torch.cuda.synchronize()
+    vs.check_status()
+    got = step_outputs(vs)
+    np.testing.assert_allclose(got["lse"][rows], lse64, rtol=0, atol=5e-4)
+    np.testing.assert_array_equal(got["n_acc"], ref_n_acc)
+    np.testing.assert_array_equal(got["path"], ref_path)
+    for b in range(B):
+        n, par, na = int(w.n_nodes[b]), w.parents[b], int(ref_n_acc[b])
+        last = int(ref_path[b, na - 1])
+        excl = [int(tok[b, c]) for c in smp.children_of(par, n, last)]
+        t_ref, margin = smp.residual_sample(p64[row_of[b * T + last]], excl, float(stop_R[b]), float(wv[b]))
+        t_got = int(got["out_tok"][b, na - 1])
+        assert t_got not in excl
+        assert t_got == t_ref or margin <= CLOSE, (b, t_got, t_ref, margin)
+    assert (ref_n_acc > 1).any()
+    G = oracle.Geometry.of(w)
+    for l in range(L):
+        rk, rv = w.k_cache[l].copy(), w.v_cache[l].copy()
+        oracle.compact(G, rk, rv, w.k_tree[l], w.v_tree[l], ref_n_acc, ref_path)
+        np.testing.assert_array_equal(got["k"][l].view(np.uint16), rk)
+        np.testing.assert_array_equal(got["v"][l].view(np.uint16), rv)
