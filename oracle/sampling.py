@@ -21,12 +21,24 @@ Every random number is an input (u per node, w per sequence).  Plain numpy,
 fp64 throughout; no code shared with the GPU library.  Siblings must carry
 distinct tokens.
 
+For a CHAIN whose tokens were sampled from draft distributions (node j's token x_j drawn from q_{j-1},
+the draft model's distribution behind node j-1) the rule keeps its general form (accept_chain_q,
+residual_sample_q, verify_chain_q below):
+
+    walking down the chain from the root, accept x_j  iff  u[j] * q_{j-1}(x_j) < p_{j-1}(x_j),
+    i.e. with probability min(1, p/q); at the first rejection, behind node i = j - 1, emit one token
+    from the normalised positive part of p_i - q_i; if every draft was accepted emit one token from
+    p_leaf.  Inverse CDF in vocabulary order with the uniform w, as above.
+
 Parity with the paper's own acceptance statistics is unpinned (they need the
 trained models).  The functions are pinned in tests/test_oracle_sampling.py:
 softmax_rows against torch's log_softmax / logsumexp in fp64, scipy's softmax
 and a hand-computed case; the rule by Monte-Carlo frequencies against p, by the
 zero-temperature limit (the greedy rule), by the single-child case (the
-textbook accept test) and by numpy's cumsum/searchsorted for the inverse CDF.
+textbook accept test) and by numpy's cumsum/searchsorted for the inverse CDF;
+the general-q chain rule by Monte-Carlo frequencies against p, by the point-mass
+case (where it must reproduce verify_sequence), by q = p (everything accepted)
+and by a hand-computed case.
 """
 from __future__ import annotations
 
@@ -114,3 +126,53 @@ def verify_sequence(parents, n_nodes, draft_tok, logits, inv_temp, u, w):
     excl = [int(draft_tok[c]) for c in children_of(parents, n, last)]
     t, _ = residual_sample(p[last], excl, R, w)
     return path, [int(draft_tok[j]) for j in path[1:]] + [t]
+
+
+def accept_chain_q(n_nodes, p_tok, q_tok, u):
+    """Acceptance along a chain drafted by sampling, fp64.
+
+    p_tok[j], q_tok[j] = probability of node j's token under the target's and under the draft's
+    distribution behind node j - 1 (j >= 1); u[j] the uniform drawn for node j.
+    Returns (n_acc, margin): accepted nodes including the root, and the smallest |u * q - p| compared."""
+    p_tok = np.asarray(p_tok, dtype=np.float64)
+    q_tok = np.asarray(q_tok, dtype=np.float64)
+    u = np.asarray(u, dtype=np.float64)
+    n_acc, margin = 1, np.inf
+    for j in range(1, int(n_nodes)):
+        margin = min(margin, abs(u[j] * q_tok[j] - p_tok[j]))
+        if not (u[j] * q_tok[j] < p_tok[j]):
+            break
+        n_acc += 1
+    return n_acc, margin
+
+
+def residual_sample_q(p_row, q_row, w):
+    """One token from the normalised positive part of p - q (from p itself when q_row is None): the
+    first token, in vocabulary order, at which the cumulative mass reaches w times the total mass; the
+    last token with mass if rounding leaves the sum short.  Returns (t, margin, total): margin as in
+    residual_sample, total = the mass that was normalised by."""
+    r = np.array(p_row, dtype=np.float64)
+    if q_row is not None:
+        r = np.maximum(r - np.asarray(q_row, dtype=np.float64), 0.0)
+    total = float(r.sum())
+    t, margin = residual_sample(r, [], total, w)
+    return t, margin, total
+
+
+def verify_chain_q(n_nodes, draft_tok, logits, inv_temp, q_rows, u, w):
+    """Whole rule for one chain (node j's parent is node j - 1) from the target's logits [T, V] and the
+    draft's distributions q_rows [T, V] (row i = the distribution node i + 1's token was drawn from).
+    Returns (n_acc, out_tok): out_tok = the accepted drafts, then the token drawn where the walk stopped."""
+    p, _ = softmax_rows(logits, inv_temp)
+    n = int(n_nodes)
+    q_rows = np.asarray(q_rows, dtype=np.float64)
+    p_tok = np.zeros(n)
+    q_tok = np.zeros(n)
+    for j in range(1, n):
+        p_tok[j] = p[j - 1, draft_tok[j]]
+        q_tok[j] = q_rows[j - 1, draft_tok[j]]
+    n_acc, _ = accept_chain_q(n, p_tok, q_tok, u)
+    stop = n_acc - 1
+    rejected = n_acc < n
+    t, _, _ = residual_sample_q(p[stop], q_rows[stop] if rejected else None, w)
+    return n_acc, [int(draft_tok[j]) for j in range(1, n_acc)] + [t]

@@ -173,3 +173,106 @@ def test_softmax_pins_catch_planted_mistakes():
     for wrong in (squared_temperature, base_two, lse_without_the_maximum, temperature_divides):
         with pytest.raises(AssertionError):
             check_softmax_against_libraries(wrong)
+
+
+# ---------------------------------------------------------------------------------------------------
+# chains drafted by sampling from a draft distribution q (the rule in its general form)
+# ---------------------------------------------------------------------------------------------------
+def chain_q_pins(verify_chain_q):
+    """Everything that fixes the general-q chain rule; raises AssertionError on the first pin that fails."""
+    g = np.random.default_rng(5)
+    V, T = 6, 3
+    # (1) Monte Carlo: drafts really drawn from q; the first emitted token must follow p_0 and, given that
+    # the first draft was accepted, the second must follow p_1 - for a draft far from and one close to p
+    for spread in (2.0, 0.3):
+        logits = g.standard_normal((T, V)) * 1.5
+        p, _ = smp.softmax_rows(logits, 1.1)
+        q, _ = smp.softmax_rows(logits + g.standard_normal((T, V)) * spread, 0.9)
+        n_draw = 60000
+        first, second = np.zeros(V), np.zeros(V)
+        cdf = np.cumsum(q, axis=1)
+        for _ in range(n_draw):
+            tok = np.zeros(T, dtype=np.int64)
+            for j in range(1, T):
+                tok[j] = min(int(np.searchsorted(cdf[j - 1], g.random(), side="right")), V - 1)
+            n_acc, out = verify_chain_q(T, tok, logits, 1.1, q, g.random(T), g.random())
+            assert len(out) == n_acc
+            first[out[0]] += 1
+            if n_acc >= 2:
+                second[out[1]] += 1
+        for counts, target in ((first, p[0]), (second, p[1])):
+            n = counts.sum()
+            sigma = np.sqrt(n * target * (1 - target))
+            assert (np.abs(counts - n * target) <= 5 * sigma + 1).all(), (spread, counts / n, target)
+    # (2) point-mass drafts: the tree rule on a chain, already pinned, must come out
+    for seed in range(30):
+        g2 = np.random.default_rng(100 + seed)
+        T2 = 5
+        logits = g2.standard_normal((T2, V)) * 2.0
+        tok = g2.integers(0, V, size=T2)
+        q = np.zeros((T2, V))
+        for j in range(1, T2):
+            q[j - 1, tok[j]] = 1.0
+        u, w = g2.random(T2), g2.random()
+        parents = np.arange(-1, T2 - 1)
+        path, out_ref = smp.verify_sequence(parents, T2, tok, logits, 1.4, u, w)
+        n_acc, out = verify_chain_q(T2, tok, logits, 1.4, q, u, w)
+        assert n_acc == len(path) and out == out_ref, (seed, out, out_ref)
+    # (3) q = p: every draft is accepted whatever u < 1 is, and the last token comes from p_leaf by the
+    # library's inverse CDF
+    logits = g.standard_normal((4, V))
+    p, _ = smp.softmax_rows(logits, 1.0)
+    tok = np.array([0, 2, 5, 1])
+    for w in (0.0, 0.31, 0.77, 0.999):
+        n_acc, out = verify_chain_q(4, tok, logits, 1.0, p, np.full(4, 0.999999), w)
+        assert n_acc == 4 and out[:3] == [2, 5, 1]
+        assert out[3] == int(np.searchsorted(np.cumsum(p[3]), w * p[3].sum(), side="left"))
+    # (4) by hand: p = (0.5, 0.3, 0.2), q = (0.2, 0.7, 0.1), draft token 1: kept iff u < 3/7; otherwise the
+    # residual is (0.3, 0, 0.1) / 0.4 = (0.75, 0, 0.25)
+    logits = np.log(np.array([[0.5, 0.3, 0.2], [0.2, 0.2, 0.6]]))
+    q = np.array([[0.2, 0.7, 0.1], [1 / 3, 1 / 3, 1 / 3]])
+    tok = np.array([0, 1])
+    assert verify_chain_q(2, tok, logits, 1.0, q, [0.0, 0.42], 0.7)[0] == 2          # 0.42 < 3/7: accepted
+    assert verify_chain_q(2, tok, logits, 1.0, q, [0.0, 0.42], 0.5)[1] == [1, 2]     # then from p_1 = (.2, .2, .6): 0.5 -> token 2
+    assert verify_chain_q(2, tok, logits, 1.0, q, [0.0, 0.43], 0.7) == (1, [0])      # 0.43 > 3/7: rejected; 0.7 < 0.75 -> token 0
+    assert verify_chain_q(2, tok, logits, 1.0, q, [0.0, 0.43], 0.8) == (1, [2])      # 0.8 > 0.75 -> token 2
+
+
+def test_chain_rule_with_a_general_draft_distribution():
+    chain_q_pins(smp.verify_chain_q)
+
+
+def test_chain_q_pins_catch_planted_mistakes():
+    """Each plausible mistake in the general-q rule must trip at least one pin."""
+    import pytest
+
+    def mutant(accept=None, residual=None, use_q_after_full_accept=False):
+        def f(n_nodes, draft_tok, logits, inv_temp, q_rows, u, w):
+            p, _ = smp.softmax_rows(logits, inv_temp)
+            n = int(n_nodes)
+            q_rows = np.asarray(q_rows, dtype=np.float64)
+            n_acc = 1
+            for j in range(1, n):
+                pt, qt = p[j - 1, draft_tok[j]], q_rows[j - 1, draft_tok[j]]
+                ok = accept(u[j], pt, qt) if accept else (u[j] * qt < pt)
+                if not ok:
+                    break
+                n_acc += 1
+            stop = n_acc - 1
+            if n_acc < n or use_q_after_full_accept:
+                r = residual(p[stop], q_rows[stop]) if residual else np.maximum(p[stop] - q_rows[stop], 0)
+            else:
+                r = p[stop]
+            t, _ = smp.residual_sample(r, [], float(r.sum()), w)
+            return n_acc, [int(draft_tok[j]) for j in range(1, n_acc)] + [t]
+        return f
+
+    chain_q_pins(mutant())                                            # the harness itself is sound
+    for bad in (mutant(accept=lambda u, p, q: u * p < q),             # ratio upside down
+                mutant(accept=lambda u, p, q: u < p),                 # q forgotten in the test
+                mutant(residual=lambda p, q: np.maximum(q - p, 0)),   # sign of the residual
+                mutant(residual=lambda p, q: p),                      # no residual correction at all
+                mutant(residual=lambda p, q: np.abs(p - q)),          # not clipped
+                mutant(use_q_after_full_accept=True)):                # residual applied although nothing was rejected
+        with pytest.raises(AssertionError):
+            chain_q_pins(bad)
