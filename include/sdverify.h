@@ -329,6 +329,43 @@ sd_status sd_accept_tree_sampled(const sd_batch *batch, const void *hidden, cons
                                  int32_t *dev_status, void *stream);
 
 /*
+ * Acceptance at a sampling temperature for CHAINS whose tokens were drawn from the
+ * draft model's own distributions (Sec. 1, lossless validation; the cited
+ * speculative-sampling rule in its general form).  Every tree must be a chain
+ * (parents[b][j] == j - 1).  With p_i = softmax(logits_i * inv_temp) the target's and
+ * q_i the draft's distribution behind node i (node i + 1's token was drawn from q_i):
+ *   walking down from the root, node j is accepted iff
+ *       u[b][j] * q_{j-1}(draft_tok[j]) < p_{j-1}(draft_tok[j])          (probability min(1, p/q))
+ *   at the first rejection, behind node i = j - 1, one token is drawn from the
+ *   normalised positive part of p_i - q_i; if every draft is accepted, from p_leaf:
+ *   the first token, in vocabulary order, at which the cumulative mass reaches
+ *   w[b] times the total mass.
+ * Outputs as sd_accept_tree (path[b][k] = k; out_tok = accepted drafts, then the drawn token).
+ *   lse    : dev f32 [B * T_max] from sd_lmhead_stats with the same inv_temp
+ *   q_tok  : dev f32 [B][T_max], q_tok[b][j] = q_{j-1}(draft_tok[b][j]) for j >= 1
+ *   q_rows : dev f32 [B][T_max][V], row [b][i] = q_i; only the row of the node where a
+ *            sequence's walk stops is read, and only if a draft was rejected there
+ *   u, w   : dev f32 [B][T_max] and [B], uniform numbers in [0, 1)
+ *   workspace : at least sd_workspace_bytes(batch, B * T_max, V)
+ * The stop nodes' rows go through the LM head once more (their probabilities over
+ * the vocabulary, B x V floats in the workspace, are the only logits-sized data that
+ * reach memory).  A tree that branches stores SD_ERR_UNSUPPORTED, a bad tree
+ * SD_ERR_INVALID_TREE, a draft token outside [0, V) SD_ERR_BOUNDS (through
+ * *dev_status; n_acc[b] = 0 for the first two).  V > 1048576 returns SD_ERR_UNSUPPORTED
+ * before anything is launched.  Drafted trees that branch AND were sampled from a
+ * distribution are not covered (their rule renormalises over the vocabulary after
+ * every rejected sibling); deterministic (top-k) trees go through
+ * sd_accept_tree_sampled.
+ */
+sd_status sd_accept_chain_sampled(const sd_batch *batch, const void *hidden, const void *W,
+                                  int32_t Hd, int32_t V, float inv_temp, const float *lse,
+                                  const int32_t *draft_tok, const float *q_tok, const float *q_rows,
+                                  const float *u, const float *w,
+                                  int32_t *n_acc, int32_t *path, int32_t *out_tok, int32_t *new_len,
+                                  void *workspace, size_t workspace_bytes,
+                                  int32_t *dev_status, void *stream);
+
+/*
  * LM head, acceptance at a sampling temperature and compaction in one call (Sec. 1:
  * lossless validation; Sec. 4.1: the survivors' KV joins the context).  Equivalent,
  * output for output and byte for byte, to

@@ -196,6 +196,22 @@ sd_status sd_accept_tree_sampled(const sd_batch* batch, const void* hidden, cons
                                  new_len, workspace, workspace_bytes, dev_status, static_cast<cudaStream_t>(stream));
 }
 
+sd_status sd_accept_chain_sampled(const sd_batch* batch, const void* hidden, const void* W, int32_t Hd, int32_t V,
+                                  float inv_temp, const float* lse, const int32_t* draft_tok, const float* q_tok,
+                                  const float* q_rows, const float* u, const float* w,
+                                  int32_t* n_acc, int32_t* path, int32_t* out_tok, int32_t* new_len,
+                                  void* workspace, size_t workspace_bytes, int32_t* dev_status, void* stream) {
+    sd_status s = check_geometry(batch, true);
+    if (s != SD_OK) return s;
+    if (!ok_ptr(hidden) || !ok_ptr(W) || !lse || !draft_tok || !q_tok || !q_rows || !u || !w) return SD_ERR_INVALID_ARG;
+    if (!n_acc || !path || !out_tok || !new_len || !ok_ptr(workspace) || !dev_status) return SD_ERR_INVALID_ARG;
+    if (V < 1 || Hd < 1 || !(inv_temp > 0.f)) return SD_ERR_INVALID_ARG;
+    if (Hd % 64 != 0) return SD_ERR_UNSUPPORTED;
+    return launch_accept_chain_sampled(*batch, hidden, W, Hd, V, inv_temp, lse, draft_tok, q_tok, q_rows, u, w, n_acc, path,
+                                       out_tok, new_len, workspace, workspace_bytes, dev_status,
+                                       static_cast<cudaStream_t>(stream));
+}
+
 sd_status sd_lmhead_accept_sampled_compact(const sd_batch* batch, const void* hidden, const void* W, int32_t Hd, int32_t V,
                                            float inv_temp, const int32_t* draft_tok, const float* u, const float* w,
                                            const sd_kv_layer* layers, int32_t L,

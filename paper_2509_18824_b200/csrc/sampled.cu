@@ -235,10 +235,14 @@ __global__ void gather_stop_rows_kernel(const uint16_t* __restrict__ hidden, int
     if (threadIdx.x == 0) stop_lse[b] = lse[row];
 }
 
-// grid (blocks of 256 tokens, sequences): drafted tokens of the stop node lose their mass, then the
-// block's masses are summed in a fixed order (pairwise tree over the 256 positions)
+// grid (blocks of 256 tokens, sequences): the stop node's row becomes the residual it is drawn from, then
+// the block's masses are summed in a fixed order (pairwise tree over the 256 positions).  Point-mass
+// drafts (q_rows null): the drafted tokens of the stop node lose their mass.  Drafts sampled from a
+// distribution (chains): where a draft was rejected (n_excl[b] != 0) the mass becomes
+// max(p - q, 0) with q = the draft's distribution behind the stop node, row stop_row[b] of q_rows.
 __global__ void __launch_bounds__(kResBlock)
 residual_blocksum_kernel(int V, const int32_t* __restrict__ n_excl, const int32_t* __restrict__ excl,
+                         const float* __restrict__ q_rows, const int32_t* __restrict__ stop_row,
                          float* __restrict__ mass, float* __restrict__ block_sum, int n_blocks) {
     __shared__ float s_v[kResBlock];
     const int b = blockIdx.y;
@@ -247,9 +251,16 @@ residual_blocksum_kernel(int V, const int32_t* __restrict__ n_excl, const int32_
     if (t < V) {
         m = mass[(size_t)b * V + t];
         const int ne = n_excl[b];
-        bool hit = false;
-        for (int e = 0; e < ne; ++e) hit |= (__ldg(excl + (size_t)b * 64 + e) == t);
-        if (hit) { m = 0.f; mass[(size_t)b * V + t] = 0.f; }
+        if (q_rows) {
+            if (ne) {
+                m = fmaxf(m - __ldg(q_rows + (size_t)stop_row[b] * V + t), 0.f);
+                mass[(size_t)b * V + t] = m;
+            }
+        } else {
+            bool hit = false;
+            for (int e = 0; e < ne; ++e) hit |= (__ldg(excl + (size_t)b * 64 + e) == t);
+            if (hit) { m = 0.f; mass[(size_t)b * V + t] = 0.f; }
+        }
     }
     s_v[threadIdx.x] = m;
     __syncthreads();
@@ -522,6 +533,85 @@ residual_pick_groups_kernel(sd_batch bt, const uint16_t* __restrict__ hidden, co
                             excl + (size_t)b * 64, excl_p + (size_t)b * 64, out_tok + (size_t)b * bt.T_max + na - 1, status);
 }
 
+// Chains drafted by SAMPLING from a draft distribution (one warp per sequence): node j's token is kept
+// iff u * q(token) < p(token), q and p the draft's and the target's probability of that token behind
+// node j - 1; the walk stops at the first rejection.  Leaves the accepted prefix, the stop node's
+// LM-head row and whether a draft was rejected there (the residual then is max(p - q, 0), else p).
+__global__ void chain_walk_q_kernel(sd_batch bt, const int32_t* __restrict__ draft, const float* __restrict__ p_child,
+                                    const float* __restrict__ q_tok, const float* __restrict__ u, int32_t* n_acc,
+                                    int32_t* path, int32_t* out_tok, int32_t* new_len, int32_t* stop_row, int32_t* rejected,
+                                    int32_t* status) {
+    const int b = blockIdx.x, lane = threadIdx.x;
+    const int T = bt.T_max;
+    const int n = bt.n_nodes[b];
+    const int32_t* par = bt.parents + (size_t)b * T;
+    const int32_t* dt = draft + (size_t)b * T;
+    bool bad = (n < 1 || n > T), branching = false;
+    if (!bad)
+        for (int i = lane; i < n; i += 32) {
+            const int p = par[i];
+            if (i == 0 ? (p != -1) : (p < 0 || p >= i)) bad = true;
+            else if (i > 0 && p != i - 1) branching = true;
+        }
+    bad = __any_sync(0xffffffffu, bad);
+    branching = __any_sync(0xffffffffu, branching);
+    if (bad || branching) {
+        if (lane == 0) {
+            set_status(status, bad ? SD_ERR_INVALID_TREE : SD_ERR_UNSUPPORTED);
+            n_acc[b] = 0; stop_row[b] = b * T; rejected[b] = 0;
+        }
+        return;
+    }
+    bool keep[2];
+#pragma unroll
+    for (int h = 0; h < 2; ++h) {
+        const int j = lane + 32 * h;
+        keep[h] = true;
+        if (j >= 1 && j < n) {
+            const size_t at = (size_t)b * T + j;
+            keep[h] = u[at] * q_tok[at] < p_child[at];
+        }
+    }
+    const uint32_t lo = __ballot_sync(0xffffffffu, !keep[0]), hi = __ballot_sync(0xffffffffu, !keep[1]);
+    const int na = lo ? __ffs(lo) - 1 : (hi ? 32 + __ffs(hi) - 1 : n);      // the first rejected node, or all
+    for (int k = lane; k < T; k += 32) {
+        path[(size_t)b * T + k] = k < na ? k : -1;
+        out_tok[(size_t)b * T + k] = k + 1 < na ? dt[k + 1] : -1;            // slot na - 1: the token still to be drawn
+    }
+    if (lane == 0) {
+        n_acc[b] = na;
+        new_len[b] = bt.len[b] + na;
+        stop_row[b] = b * T + na - 1;
+        rejected[b] = na < n ? 1 : 0;
+    }
+}
+
+sd_status launch_accept_chain_sampled(const sd_batch& bt, const void* hidden, const void* W, int Hd, int V, float inv_temp,
+                                      const float* lse, const int32_t* draft, const float* q_tok, const float* q_rows,
+                                      const float* u, const float* w, int32_t* n_acc, int32_t* path, int32_t* out_tok,
+                                      int32_t* new_len, void* ws, size_t ws_bytes, int32_t* dev_status, cudaStream_t st) {
+    const int B = bt.B, T = bt.T_max;
+    if (Hd > 16384 || (V + kResBlock - 1) / kResBlock > kPickMaxBlocks) return SD_ERR_UNSUPPORTED;
+    if (ws_bytes < sampled_workspace_bytes(B, T, V, 16384)) return SD_ERR_WORKSPACE;
+    const SampledWs s = carve(ws, B, T, V, 16384);
+    const uint16_t* h = static_cast<const uint16_t*>(hidden);
+    const uint16_t* Wp = static_cast<const uint16_t*>(W);
+    const int n_blocks = (V + kResBlock - 1) / kResBlock;
+    child_prob_kernel<<<(B * T * 32 + 127) / 128, 128, 0, st>>>(bt, h, Wp, Hd, V, inv_temp, lse, draft, s.p_child, dev_status);
+    chain_walk_q_kernel<<<B, 32, 0, st>>>(bt, draft, s.p_child, q_tok, u, n_acc, path, out_tok, new_len, s.stop_row, s.n_excl,
+                                         dev_status);
+    gather_stop_rows_kernel<<<B, 128, 0, st>>>(h, Hd, lse, s.stop_row, s.stop_hidden, s.stop_lse);
+    // the stop rows' probabilities over the vocabulary (the LM-head kernel in its store mode), turned into
+    // the residual max(p - q, 0) where a draft was rejected
+    const sd_status ls = launch_lmhead_mass(s.stop_hidden, W, B, Hd, V, inv_temp, s.stop_lse, s.mass, s.lm_ws,
+                                            stats_workspace_bytes(B, V), dev_status, st);
+    if (ls != SD_OK) return ls;
+    residual_blocksum_kernel<<<dim3(n_blocks, B), kResBlock, 0, st>>>(V, s.n_excl, s.excl, q_rows, s.stop_row, s.mass,
+                                                                      s.block_sum, n_blocks);
+    residual_pick_kernel<<<B, kResBlock, 0, st>>>(bt, V, w, s.mass, s.block_sum, n_blocks, n_acc, out_tok, dev_status);
+    return cuda_ok(cudaGetLastError());
+}
+
 // ---------------------------------------------------------------------------
 // Tail of a verify step at a sampling temperature, behind the LM-head tiles of a statistics pass: one
 // cluster of eight CTAs per sequence.
@@ -673,7 +763,8 @@ sd_status launch_accept_sampled(const sd_batch& bt, const void* hidden, const vo
     sd_status ls = launch_lmhead_mass(s.stop_hidden, W, B, Hd, V, inv_temp, s.stop_lse, s.mass, s.lm_ws,
                                       stats_workspace_bytes(B, V), dev_status, st);
     if (ls != SD_OK) return ls;
-    residual_blocksum_kernel<<<dim3(n_blocks, B), kResBlock, 0, st>>>(V, s.n_excl, s.excl, s.mass, s.block_sum, n_blocks);
+    residual_blocksum_kernel<<<dim3(n_blocks, B), kResBlock, 0, st>>>(V, s.n_excl, s.excl, nullptr, nullptr, s.mass, s.block_sum,
+                                                                      n_blocks);
     residual_pick_kernel<<<B, kResBlock, 0, st>>>(bt, V, w, s.mass, s.block_sum, n_blocks, n_acc, out_tok, dev_status);
     return cuda_ok(cudaGetLastError());
 }

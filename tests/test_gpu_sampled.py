@@ -415,3 +415,205 @@ def test_fused_sampled_tail_full_vocabulary():
         oracle.compact(G, rk, rv, w.k_tree[l], w.v_tree[l], ref_n_acc, ref_path)
         np.testing.assert_array_equal(got["k"][l].view(np.uint16), rk)
         np.testing.assert_array_equal(got["v"][l].view(np.uint16), rv)
+
+
+# ---------------------------------------------------------------------------------------------------
+# chains drafted by sampling from the draft model's own distributions: sd_accept_chain_sampled
+# ---------------------------------------------------------------------------------------------------
+def drafted_chain(w, lg, inv_temp, spread, seed):
+    """A drafter close to, but not, the target: q[b][i] = softmax of the target's logits behind node i
+    plus noise (float32, the array both sides read); node i + 1's token is drawn from it."""
+    g = np.random.default_rng(seed)
+    B, T, V = w.B, w.T_max, lg.shape[1]
+    q64, _ = smp.softmax_rows(lg + g.standard_normal(lg.shape) * spread, inv_temp * 0.8)
+    q = np.ascontiguousarray(q64.astype(np.float32).reshape(B, T, V))
+    tok = np.zeros((B, T), dtype=np.int32)
+    for b in range(B):
+        for j in range(1, int(w.n_nodes[b])):
+            cdf = np.cumsum(q[b, j - 1].astype(np.float64))
+            tok[b, j] = min(int(np.searchsorted(cdf, g.random() * cdf[-1], side="right")), V - 1)
+    q_tok = np.zeros((B, T), dtype=np.float32)
+    for b in range(B):
+        for j in range(1, int(w.n_nodes[b])):
+            q_tok[b, j] = q[b, j - 1, tok[b, j]]
+    return q, tok, q_tok
+
+
+def run_chain_q(w, tok, q, q_tok, inv_temp, u, wv):
+    bt = sd.Batch.of(w)
+    st = sd.new_status()
+    h, Wd = to_device(w.hidden), to_device(w.W)
+    M, V = w.hidden.shape[0], w.W.shape[0]
+    B, T = w.B, w.T_max
+    ws = torch.zeros(sd.sd_workspace_bytes(bt, M, V), dtype=torch.uint8, device="cuda")
+    lse = torch.zeros(M, dtype=torch.float32, device="cuda")
+    sd.sd_lmhead_stats(h, Wd, inv_temp, None, None, lse, ws, st)
+    n_acc = torch.full((B,), -9, dtype=torch.int32, device="cuda")
+    path = torch.full((B, T), -9, dtype=torch.int32, device="cuda")
+    out_tok = torch.full((B, T), -9, dtype=torch.int32, device="cuda")
+    new_len = torch.full((B,), -9, dtype=torch.int32, device="cuda")
+    sd.sd_accept_chain_sampled(bt, h, Wd, inv_temp, lse, to_device(tok), to_device(q_tok), to_device(q),
+                               to_device(u), to_device(wv), n_acc, path, out_tok, new_len, ws, st)
+    torch.cuda.synchronize()
+    return (n_acc.cpu().numpy(), path.cpu().numpy(), out_tok.cpu().numpy(), new_len.cpu().numpy(), int(st.item()))
+
+
+def decisive_chain_inputs(w, tok, q, p64_of_row, g, floor=20 * WALK_CLOSE, floor_w=2e-3):
+    """Uniforms under which neither an accept test (u * q against p, the two further apart than `floor`
+    times p: the kernel's p is within 1e-4 relative of the fp64 value) nor the last token's CDF crossing
+    of the fp64 rule is a close call, with the fp64 rule's results (n_acc and the emitted tokens)."""
+    B, T = w.B, w.T_max
+    u = np.zeros((B, T), np.float32)
+    wv = np.zeros(B, np.float32)
+    ref_n, ref_out = np.zeros(B, np.int32), np.full((B, T), -1, np.int32)
+    for b in range(B):
+        n = int(w.n_nodes[b])
+        p_tok, q_tok = np.zeros(n), np.zeros(n)
+        for j in range(1, n):
+            p_tok[j] = p64_of_row(b * T + j - 1)[tok[b, j]]
+            q_tok[j] = q[b, j - 1, tok[b, j]]
+        for _ in range(400):
+            u[b] = g.random(T).astype(np.float32)
+            na, _ = smp.accept_chain_q(n, p_tok, q_tok, u[b].astype(np.float64))
+            looked_at = range(1, min(na + 1, n))             # the accepted nodes and the rejected one
+            if all(abs(u[b, j] * q_tok[j] - p_tok[j]) > floor * p_tok[j] for j in looked_at):
+                break
+        else:
+            raise AssertionError("no decisive uniforms found")
+        stop = na - 1
+        for _ in range(400):
+            wv[b] = np.float32(g.random())
+            t, margin, total = smp.residual_sample_q(p64_of_row(b * T + stop), q[b, stop] if na < n else None, float(wv[b]))
+            if margin > floor_w * total:
+                break
+        else:
+            raise AssertionError("no decisive w found")
+        ref_n[b] = na
+        ref_out[b, :na - 1] = tok[b, 1:na]
+        ref_out[b, na - 1] = t
+    return u, wv, ref_n, ref_out
+
+
+@pytest.mark.parametrize("cfg,over,inv_temp,spread", [
+    ("chain11", dict(L=1, V=3000, Hd=128, prefix=70), 2.5, 0.6),
+    ("chain11", dict(L=1, V=3000, Hd=128, prefix=70), 2.5, 0.05),            # a drafter very close to the target
+    ("chain11", dict(L=1, V=96, Hd=64, prefix=70), 1.5, 1.0),                # vocabulary below one 128-row tile
+    ("chain11", dict(L=1, V=8192, Hd=512, prefix=100, B=16), 4.0, 0.4),      # 16 sequences
+])
+def test_chain_acceptance_with_a_draft_distribution_against_the_reference(cfg, over, inv_temp, spread):
+    w = wl.make(cfg, attention=False, hidden_gain=24.0, **over)
+    B, T, V = w.B, w.T_max, w.W.shape[0]
+    lg = oracle.logits(w.hidden, w.W)
+    p64, _ = smp.softmax_rows(lg, inv_temp)
+    q, tok, q_tok = drafted_chain(w, lg, inv_temp, spread, 3)
+    g = np.random.default_rng(8)
+    moved = rejected = 0
+    for rep in range(3):
+        u, wv, ref_n, ref_out = decisive_chain_inputs(w, tok, q, lambda r: p64[r], g)
+        n_acc, path, out_tok, new_len, status = run_chain_q(w, tok, q, q_tok, inv_temp, u, wv)
+        assert status == 0
+        np.testing.assert_array_equal(n_acc, ref_n)
+        np.testing.assert_array_equal(out_tok, ref_out)
+        np.testing.assert_array_equal(new_len, w.len + ref_n)
+        for b in range(B):
+            assert list(path[b, :ref_n[b]]) == list(range(ref_n[b])) and (path[b, ref_n[b]:] == -1).all()
+        moved += int((ref_n > 1).sum())
+        rejected += int((ref_n < w.n_nodes).sum())
+    assert moved > 0 and rejected > 0                       # both branches of the rule were exercised
+
+
+def test_chain_acceptance_draft_equal_to_the_target_accepts_everything():
+    w = wl.make("chain11", attention=False, hidden_gain=24.0, L=1, V=3000, Hd=128, prefix=70)
+    B, T, V = w.B, w.T_max, w.W.shape[0]
+    inv_temp = 2.0
+    lg = oracle.logits(w.hidden, w.W)
+    p64, _ = smp.softmax_rows(lg, inv_temp)
+    q = np.ascontiguousarray(p64.astype(np.float32).reshape(B, T, V))
+    g = np.random.default_rng(4)
+    tok = np.zeros((B, T), np.int32)
+    for b in range(B):
+        for j in range(1, T):
+            tok[b, j] = np.argsort(-p64[b * T + j - 1])[g.integers(0, 3)]       # a likely token (any token works)
+    q_tok = np.zeros((B, T), np.float32)
+    for b in range(B):
+        q_tok[b, 1:] = q[b, np.arange(T - 1), tok[b, 1:]]
+    u = (g.random((B, T)) * 0.98).astype(np.float32)
+    wv = g.random(B).astype(np.float32)
+    n_acc, path, out_tok, new_len, status = run_chain_q(w, tok, q, q_tok, inv_temp, u, wv)
+    assert status == 0
+    np.testing.assert_array_equal(n_acc, w.n_nodes)
+    for b in range(B):
+        n = int(w.n_nodes[b])
+        assert list(out_tok[b, :n - 1]) == list(tok[b, 1:n])
+        t_ref, margin, total = smp.residual_sample_q(p64[b * T + n - 1], None, float(wv[b]))
+        assert out_tok[b, n - 1] == t_ref or margin <= CLOSE
+
+
+def test_chain_acceptance_refuses_trees_that_branch():
+    w = wl.make("c1", attention=False, hidden_gain=16.0)                    # an 8-node tree with branches
+    V = w.W.shape[0]
+    q = np.full((1, 8, V), 1.0 / V, np.float32)
+    tok = np.arange(8, dtype=np.int32)[None]
+    half = np.full((1, 8), 0.5, np.float32)
+    n_acc, *_, status = run_chain_q(w, tok, q, np.full((1, 8), 1.0 / V, np.float32), 1.0, half, np.full(1, 0.5, np.float32))
+    assert status == sd.SD_ERR_UNSUPPORTED and n_acc[0] == 0
+
+
+def test_chain_acceptance_full_vocabulary():
+    """Root + 10 drafts, 8 sequences, vocabulary 152064, draft distributions of the full width."""
+    w = wl.make("chain11", attention=False, hidden_gain=40.0)
+    B, T, V = w.B, w.T_max, w.V
+    inv_temp = 6.0
+    lg = oracle.logits(w.hidden, w.W)
+    p64, _ = smp.softmax_rows(lg, inv_temp)
+    q, tok, q_tok = drafted_chain(w, lg, inv_temp, 0.15, 9)
+    g = np.random.default_rng(10)
+    u, wv, ref_n, ref_out = decisive_chain_inputs(w, tok, q, lambda r: p64[r], g)
+    n_acc, path, out_tok, new_len, status = run_chain_q(w, tok, q, q_tok, inv_temp, u, wv)
+    assert status == 0
+    np.testing.assert_array_equal(n_acc, ref_n)
+    np.testing.assert_array_equal(out_tok, ref_out)
+    assert (ref_n > 1).any() and (ref_n < w.n_nodes).any()
+
+
+def test_chain_acceptance_gpu_output_frequencies_follow_the_target_distribution():
+    """Losslessness of the general rule measured on the GPU path: 16 identical chains (root + 2 drafts)
+    whose drafts are drawn afresh from q 300 times; the first emitted token of every sequence must be
+    distributed as the target's p at the root (5 sigma), whether it was an accepted draft or a redraw."""
+    B, T, Hd, V, inv_temp, reps = 16, 3, 64, 16, 1.2, 300
+    g = np.random.default_rng(22)
+    bf = lambda a: wl.f32_to_bf16_bits(a.astype(np.float32))
+    hid_one = bf(g.standard_normal((T, Hd)))
+    W = bf(g.standard_normal((V, Hd)) * 0.25)
+
+    class Geo:
+        pass
+    w = Geo()
+    w.B, w.T_max, w.Hq, w.Hkv, w.D = B, T, 4, 1, 128
+    w.block_table = np.arange(B, dtype=np.int32).reshape(B, 1)
+    w.len = np.full(B, 5, np.int32)
+    w.n_nodes = np.full(B, T, np.int32)
+    w.parents = np.tile(np.array([-1, 0, 1], np.int32), (B, 1))
+    w.hidden = np.tile(hid_one, (B, 1))
+    w.W = W
+    lg = oracle.logits(hid_one, W)
+    p, _ = smp.softmax_rows(lg, inv_temp)
+    q_one, _ = smp.softmax_rows(lg + g.standard_normal(lg.shape) * 0.8, 1.0)
+    q = np.ascontiguousarray(np.tile(q_one.astype(np.float32)[None], (B, 1, 1)))
+    cdf = np.cumsum(q_one.astype(np.float32).astype(np.float64), axis=1)
+    counts = np.zeros(V)
+    for rep in range(reps):
+        tok = np.zeros((B, T), np.int32)
+        q_tok = np.zeros((B, T), np.float32)
+        for b in range(B):
+            for j in range(1, T):
+                tok[b, j] = min(int(np.searchsorted(cdf[j - 1], g.random() * cdf[j - 1, -1], side="right")), V - 1)
+                q_tok[b, j] = q[b, j - 1, tok[b, j]]
+        u = g.random((B, T)).astype(np.float32)
+        wv = g.random(B).astype(np.float32)
+        n_acc, path, out_tok, new_len, status = run_chain_q(w, tok, q, q_tok, inv_temp, u, wv)
+        assert status == 0
+        np.add.at(counts, out_tok[:, 0], 1)
+    n = B * reps
+    sigma = np.sqrt(n * p[0] * (1 - p[0]))
+    assert (np.abs(counts - n * p[0]) <= 5 * sigma + 1).all(), (counts / n, p[0])
