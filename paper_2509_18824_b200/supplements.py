@@ -172,6 +172,32 @@ def sampled(cfg="c5", inv_temp=1.0):
                       "peaks": src, "status": int(st.item())}))
 
 
+def chain_sampled(inv_temp=1.0):
+    """sd_accept_chain_sampled on chain decoding shapes (root + 10 drafts, 8 sequences, vocabulary 152064):
+    drafts and draft distributions are random here, which does not change the work."""
+    from .step import VerifyStep
+    w = wl.make("chain11", attention=False, L=1)
+    wl.fill_attention(w, [0])
+    vs = VerifyStep(w)
+    B, T, M, V = w.B, w.T_max, w.B * w.T_max, w.V
+    g = torch.Generator(device="cuda"); g.manual_seed(0)
+    u = torch.rand((B, T), device="cuda", generator=g)
+    wv = torch.rand((B,), device="cuda", generator=g)
+    q = torch.rand((B, T, V), device="cuda", generator=g)
+    q /= q.sum(dim=-1, keepdim=True)
+    q_tok = torch.gather(q[:, : T - 1], 2, vs.draft_tok[:, 1:].long().unsqueeze(-1)).squeeze(-1)
+    q_tok = torch.cat([torch.zeros((B, 1), device="cuda"), q_tok], dim=1).contiguous()
+    lse = torch.zeros(M, dtype=torch.float32, device="cuda")
+    ws = torch.empty(sd.sd_workspace_bytes(vs.batch, M, V), dtype=torch.uint8, device="cuda")
+    st = vs.status
+    ms_stats = _time(lambda: sd.sd_lmhead_stats(vs.hidden, vs.W, inv_temp, None, None, lse, ws, st), 10)
+    ms_acc = _time(lambda: sd.sd_accept_chain_sampled(vs.batch, vs.hidden, vs.W, inv_temp, lse, vs.draft_tok, q_tok, q, u, wv,
+                                                      vs.n_acc, vs.path, vs.out_tok, vs.new_len, ws, st), 10)
+    print(json.dumps({"call": "sd_accept_chain_sampled", "workload": "chain11", "rows": M,
+                      "sd_lmhead_stats_us": ms_stats * 1e3, "sd_accept_chain_sampled_us": ms_acc * 1e3,
+                      "second_pass_weight_stream_gbs": V * w.Hd * 2 / ms_acc / 1e6, "status": int(st.item())}))
+
+
 def draft(S=4096, L=28, Q=4, H=28):
     """Draft-side feature aggregation on a 7B-shaped prefill: S tokens x 28 layer features of width 3584."""
     hbm, _, src = _peaks()
@@ -234,6 +260,7 @@ if __name__ == "__main__":
         lmhead(rows=(480,))
     if "sampled" in what:
         sampled()
+        chain_sampled()
     if "draft" in what:
         draft()
     if "compact" in what:
