@@ -76,12 +76,12 @@ def attention(configs=("c2", "c3", "c4", "c5", "chain11")):
         torch.cuda.empty_cache()
 
 
-def attention_layers(configs=("c5", "chain11", "c4"), L=28):
+def attention_layers(configs=("c5", "chain11", "tree28", "c4"), L=28):
     for r in measure_attention_layers(configs, L):
         print(json.dumps(r))
 
 
-def measure_attention_layers(configs=("c5", "chain11", "c4"), L=28, reps=20):
+def measure_attention_layers(configs=("c5", "chain11", "tree28", "c4"), L=28, reps=20):
     """All L layers through sd_verify_attention_layers (one launch): the regime of a whole verify
     step, where per-launch costs are paid once.  chain11 is the bandwidth-bound case.  Yields one
     record per workload."""

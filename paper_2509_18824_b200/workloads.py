@@ -204,6 +204,8 @@ def spec(config: str) -> Spec:
         return Spec("c5", 4, 8, 28, 4, 128, 60, "eagle", 6, prefix=4096, L=28, plant=True)
     if c == "chain11":   # the paper's own setting: 10 drafted tokens in a chain
         return Spec("chain11", 5, 8, 28, 4, 128, 11, "chain", 10, prefix=4096, L=1)
+    if c == "tree28":    # a short tree (root + 27 drafts, depth 5): 196 query rows per KV head, near the ridge point
+        return Spec("tree28", 6, 8, 28, 4, 128, 28, "eagle", 5, prefix=4096, L=1)
     raise KeyError(config)
 
 

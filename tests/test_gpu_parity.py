@@ -274,11 +274,12 @@ def check_every_row(got, ref, what):
 
 
 @pytest.mark.parametrize("cfg,gain", [("c3", 1.0), ("c3", 45.0), ("c4", 1.0), ("c4", 45.0),
-                                      ("chain11", 1.0), ("chain11", 45.0)])
+                                      ("chain11", 1.0), ("chain11", 45.0), ("tree28", 1.0), ("tree28", 45.0)])
 def test_attention_full_size_every_row(cfg, gain):
     """The configured shapes in full (c3: 4 x 8192 prefix; c4: 16 ragged sequences through the shuffled
-    block table; chain11: the paper's chain setting), at unit scale and with peaked scores: every row
-    of the one-layer call against the checker."""
+    block table; chain11: the paper's chain setting; tree28: a short tree, one full and one partly
+    filled row tile), at unit scale and with peaked scores: every row of the one-layer call against the
+    checker."""
     w = wl.make(cfg, lmhead=False, q_gain=gain)
     out, lse, status = gpu_attention(w, layer=0)
     assert status == 0

@@ -36,6 +36,9 @@ def test_trees_are_valid_and_reach_their_depth():
     np.testing.assert_array_equal(w.parents[0], [-1, 0, 0, 1, 1, 2, 3, 3])
     w = wl.make_geometry(wl.spec("chain11"))
     np.testing.assert_array_equal(w.parents[0], np.arange(-1, 10))
+    w = wl.make_geometry(wl.spec("tree28"))
+    assert w.T_max == 28 and (w.n_nodes == 28).all()
+    assert [int(wl.node_depths(w.parents[b]).max()) for b in range(w.B)] == [5] * w.B
 
 
 def test_generation_is_deterministic_and_scaled():
