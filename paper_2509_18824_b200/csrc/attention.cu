@@ -630,8 +630,11 @@ static AttnPlan make_plan(const sd_batch& bt, int n_layers, int sms) {
             while (2 * ct <= kMaxChunks && 2 * ct <= max_tiles && rest * 2 * ct <= slots) ct *= 2;
             waves = (double)(base / slots) + (rest == 0 ? 0.0 : (ct > 1 ? 1.0 / ct + 0.1 : 1.0));
         }
-        // per CTA: its key tiles, a fixed cost of about three tiles, and two more for the in-cluster merge
-        const double cost = waves * ((max_tiles + c - 1) / c + 3 + (c > 1 ? 2 : 0));
+        // per CTA: its key tiles, a fixed cost of about three tiles, and the in-cluster merge: two to three
+        // tiles' worth for clusters of two and four, about eleven for clusters of eight (measured: with
+        // eight chunks a launch gains nothing over four unless it saves more than eight tiles per CTA)
+        const int merge = (c == 1) ? 0 : (c == 2 ? 2 : (c == 4 ? 3 : 11));
+        const double cost = waves * ((max_tiles + c - 1) / c + 3 + merge);
         if (cost < best - 1e-9) { best = cost; n = c; }
     }
     const TestKnobs knobs = test_knobs();
