@@ -496,7 +496,10 @@ attn_umma_kernel(const __grid_constant__ AttnLayers<NL> layers, const sd_batch b
             const int slot = chunk * rows_per + rr % rows_per;
             const uint32_t xo_remote = map_dsmem(smem_u32(k_smem), (uint32_t)(rr / rows_per));
             const uint32_t xs_remote = xo_remote + kRowTile * kD * 4;
-            const bool mine = rows_ready && row_in_tile >= 0;
+            // rows beyond the tile's last query row and rows of unused nodes are not exchanged: the merge
+            // writes zeros for the latter without reading anything
+            const int push_row = rt * kRowTile + rr;
+            const bool mine = rows_ready && row_in_tile >= 0 && push_row < plan.rows && push_row / G < n;
             tc_fence_after_sync();
 #pragma unroll
             for (int cc = 0; cc < 4; ++cc) {

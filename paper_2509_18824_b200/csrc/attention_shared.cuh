@@ -82,11 +82,12 @@ __device__ __forceinline__ void merge_rows(const MergeCtx& x) {
     for (int i = 0; i < kPerWarp; i += 4) {
         const int rl = x.warp * kPerWarp + i + sub;             // row among this CTA's rows
         const int row = first + i;
+        const bool has_data = row < x.plan.rows && node < x.n;  // only such rows were pushed
         float mc[NCH];
         float M = -INFINITY;
 #pragma unroll
         for (int c = 0; c < NCH; ++c) {
-            const bool live = (c == NCH - 1) || (c * x.tpc < x.tiles_total);   // that chunk had key tiles
+            const bool live = has_data && ((c == NCH - 1) || (c * x.tpc < x.tiles_total));   // that chunk had key tiles
             mc[c] = live ? ld_smem_f32(x.xs_addr + (c * kRowsPer + rl) * 4) : -INFINITY;
             M = fmaxf(M, mc[c]);
         }
