@@ -293,6 +293,19 @@ sd_status sd_lmhead_stats(const void *hidden, const void *W, int32_t M, int32_t 
                           int32_t *dev_status, void *stream);
 
 /*
+ * sd_lmhead_stats that also keeps the raw logits (Sec. 1 / Sec. 4.2: chain decoding,
+ * where a step verifies few rows).  For M rows the logits are M x V floats - 53 MB for
+ * root + 10 drafts of 8 sequences at V = 152064, a twentieth of W - and keeping them
+ * lets sd_accept_chain_sampled draw its last token without streaming W again.
+ *   logits : dev f32 [M][V], logits[r][v] = sum_k hidden[r][k] * W[v][k] (fp32 accumulation)
+ * Everything else as sd_lmhead_stats (no group table).
+ */
+sd_status sd_lmhead_stats_logits(const void *hidden, const void *W, int32_t M, int32_t Hd, int32_t V,
+                                 float inv_temp, int32_t *argmax, float *maxlogit, float *lse,
+                                 float *logits, void *workspace, size_t workspace_bytes,
+                                 int32_t *dev_status, void *stream);
+
+/*
  * Acceptance at a sampling temperature for a deterministically drafted tree
  * (Sec. 1, lossless validation; rule of the cited speculative-sampling work with
  * a point-mass draft distribution).  With p_i = softmax(logits_i * inv_temp) the
@@ -342,14 +355,17 @@ sd_status sd_accept_tree_sampled(const sd_batch *batch, const void *hidden, cons
  *   w[b] times the total mass.
  * Outputs as sd_accept_tree (path[b][k] = k; out_tok = accepted drafts, then the drawn token).
  *   lse    : dev f32 [B * T_max] from sd_lmhead_stats with the same inv_temp
+ *   logits : NULL, or dev f32 [B * T_max][V] as sd_lmhead_stats_logits left them in the same
+ *            pass as lse: the stop rows' probabilities are then formed from them and W is
+ *            not read a second time
  *   q_tok  : dev f32 [B][T_max], q_tok[b][j] = q_{j-1}(draft_tok[b][j]) for j >= 1
  *   q_rows : dev f32 [B][T_max][V], row [b][i] = q_i; only the row of the node where a
  *            sequence's walk stops is read, and only if a draft was rejected there
  *   u, w   : dev f32 [B][T_max] and [B], uniform numbers in [0, 1)
  *   workspace : at least sd_workspace_bytes(batch, B * T_max, V)
- * The stop nodes' rows go through the LM head once more (their probabilities over
- * the vocabulary, B x V floats in the workspace, are the only logits-sized data that
- * reach memory).  A tree that branches stores SD_ERR_UNSUPPORTED, a bad tree
+ * Without `logits` the stop nodes' rows go through the LM head once more (their
+ * probabilities over the vocabulary, B x V floats in the workspace, are then the only
+ * logits-sized data that reach memory).  A tree that branches stores SD_ERR_UNSUPPORTED, a bad tree
  * SD_ERR_INVALID_TREE, a draft token outside [0, V) SD_ERR_BOUNDS (through
  * *dev_status; n_acc[b] = 0 for the first two).  V > 1048576 returns SD_ERR_UNSUPPORTED
  * before anything is launched.  Drafted trees that branch AND were sampled from a
@@ -359,6 +375,7 @@ sd_status sd_accept_tree_sampled(const sd_batch *batch, const void *hidden, cons
  */
 sd_status sd_accept_chain_sampled(const sd_batch *batch, const void *hidden, const void *W,
                                   int32_t Hd, int32_t V, float inv_temp, const float *lse,
+                                  const float *logits,
                                   const int32_t *draft_tok, const float *q_tok, const float *q_rows,
                                   const float *u, const float *w,
                                   int32_t *n_acc, int32_t *path, int32_t *out_tok, int32_t *new_len,

@@ -33,7 +33,7 @@ KERNELS_PER_SAMPLED_TAIL = 2       # sd_lmhead_accept_sampled_compact: LM-head t
 
 EXPORTS = ["sd_version", "sd_status_string", "sd_workspace_bytes", "sd_tree_prepare",
            "sd_verify_attention", "sd_verify_attention_layers", "sd_lmhead_argmax", "sd_lmhead_argmax_static", "sd_accept_tree",
-           "sd_compact_kv", "sd_lmhead_accept_compact", "sd_lmhead_stats", "sd_accept_tree_sampled", "sd_lmhead_accept_sampled_compact", "sd_accept_chain_sampled",
+           "sd_compact_kv", "sd_lmhead_accept_compact", "sd_lmhead_stats", "sd_accept_tree_sampled", "sd_lmhead_accept_sampled_compact", "sd_accept_chain_sampled", "sd_lmhead_stats_logits",
            "sd_draft_feature_attention"]
 
 
@@ -94,8 +94,13 @@ def _load(path: str = LIB_PATH) -> C.CDLL:
                                            C.c_void_p, C.c_void_p, C.c_void_p, C.c_void_p,
                                            C.c_void_p, C.c_size_t, C.c_void_p, C.c_void_p]
     lib.sd_accept_chain_sampled.restype = C.c_int
+    lib.sd_lmhead_stats_logits.restype = C.c_int
+    lib.sd_lmhead_stats_logits.argtypes = [C.c_void_p, C.c_void_p, C.c_int32, C.c_int32, C.c_int32, C.c_float,
+                                           C.c_void_p, C.c_void_p, C.c_void_p, C.c_void_p, C.c_void_p, C.c_size_t,
+                                           C.c_void_p, C.c_void_p]
     lib.sd_accept_chain_sampled.argtypes = [C.c_void_p, C.c_void_p, C.c_void_p, C.c_int32, C.c_int32, C.c_float,
-                                            C.c_void_p, C.c_void_p, C.c_void_p, C.c_void_p, C.c_void_p, C.c_void_p,
+                                            C.c_void_p, C.c_void_p,
+                                            C.c_void_p, C.c_void_p, C.c_void_p, C.c_void_p, C.c_void_p,
                                             C.c_void_p, C.c_void_p, C.c_void_p, C.c_void_p,
                                             C.c_void_p, C.c_size_t, C.c_void_p, C.c_void_p]
     lib.sd_lmhead_accept_sampled_compact.restype = C.c_int
@@ -314,16 +319,28 @@ def sd_accept_tree_sampled(batch: Batch, hidden, W, inv_temp: float, lse, draft_
                                       workspace.numel() * workspace.element_size(), _ptr(status), _stream(stream)))
 
 
+def sd_lmhead_stats_logits(hidden, W, inv_temp: float, argmax, maxlogit, lse, logits, workspace, status,
+                           stream=None) -> None:
+    """sd_lmhead_stats that also keeps the raw logits [M,V] (device f32)."""
+    M, Hd = hidden.shape
+    V = W.shape[0]
+    assert W.shape[1] == Hd and tuple(logits.shape) == (M, V) and logits.dtype == torch.float32 and logits.is_contiguous()
+    _check(lib.sd_lmhead_stats_logits(_ptr(hidden), _ptr(W), int(M), int(Hd), int(V), C.c_float(inv_temp), _ptr(argmax),
+                                      _ptr(maxlogit), _ptr(lse), _ptr(logits), _ptr(workspace),
+                                      workspace.numel() * workspace.element_size(), _ptr(status), _stream(stream)))
+
+
 def sd_accept_chain_sampled(batch: Batch, hidden, W, inv_temp: float, lse, draft_tok, q_tok, q_rows, u, w,
-                            n_acc, path, out_tok, new_len, workspace, status, stream=None) -> None:
+                            n_acc, path, out_tok, new_len, workspace, status, stream=None, logits=None) -> None:
     """Acceptance at a sampling temperature for chains drafted by sampling: q_tok [B,T] the draft's
-    probability of every drafted token, q_rows [B,T,V] its distributions (device f32)."""
+    probability of every drafted token, q_rows [B,T,V] its distributions (device f32); logits: what
+    sd_lmhead_stats_logits kept, or None (the stop rows then go through the LM head once more)."""
     M, Hd = hidden.shape
     V = W.shape[0]
     assert W.shape[1] == Hd and M == batch.B * batch.T_max
     assert tuple(q_rows.shape) == (batch.B, batch.T_max, V) and q_rows.dtype == torch.float32 and q_rows.is_contiguous()
     _check(lib.sd_accept_chain_sampled(batch.ref(), _ptr(hidden), _ptr(W), int(Hd), int(V), C.c_float(inv_temp),
-                                       _ptr(lse), _ptr(draft_tok), _ptr(q_tok), _ptr(q_rows), _ptr(u), _ptr(w),
+                                       _ptr(lse), _ptr(logits), _ptr(draft_tok), _ptr(q_tok), _ptr(q_rows), _ptr(u), _ptr(w),
                                        _ptr(n_acc), _ptr(path), _ptr(out_tok), _ptr(new_len), _ptr(workspace),
                                        workspace.numel() * workspace.element_size(), _ptr(status), _stream(stream)))
 

@@ -196,8 +196,20 @@ sd_status sd_accept_tree_sampled(const sd_batch* batch, const void* hidden, cons
                                  new_len, workspace, workspace_bytes, dev_status, static_cast<cudaStream_t>(stream));
 }
 
+sd_status sd_lmhead_stats_logits(const void* hidden, const void* W, int32_t M, int32_t Hd, int32_t V, float inv_temp,
+                                 int32_t* argmax, float* maxlogit, float* lse, float* logits,
+                                 void* workspace, size_t workspace_bytes, int32_t* dev_status, void* stream) {
+    if (!ok_ptr(hidden) || !ok_ptr(W) || !lse || !logits || !ok_ptr(workspace) || !dev_status) return SD_ERR_INVALID_ARG;
+    if (reinterpret_cast<uintptr_t>(logits) & 3u) return SD_ERR_INVALID_ARG;
+    if (M < 1 || V < 1 || Hd < 1 || !(inv_temp > 0.f)) return SD_ERR_INVALID_ARG;
+    if (Hd % 64 != 0) return SD_ERR_UNSUPPORTED;
+    return launch_lmhead_stats(hidden, W, M, Hd, V, inv_temp, argmax, maxlogit, lse, nullptr, workspace, workspace_bytes,
+                               dev_status, static_cast<cudaStream_t>(stream), logits);
+}
+
 sd_status sd_accept_chain_sampled(const sd_batch* batch, const void* hidden, const void* W, int32_t Hd, int32_t V,
-                                  float inv_temp, const float* lse, const int32_t* draft_tok, const float* q_tok,
+                                  float inv_temp, const float* lse, const float* logits,
+                                  const int32_t* draft_tok, const float* q_tok,
                                   const float* q_rows, const float* u, const float* w,
                                   int32_t* n_acc, int32_t* path, int32_t* out_tok, int32_t* new_len,
                                   void* workspace, size_t workspace_bytes, int32_t* dev_status, void* stream) {
@@ -207,7 +219,7 @@ sd_status sd_accept_chain_sampled(const sd_batch* batch, const void* hidden, con
     if (!n_acc || !path || !out_tok || !new_len || !ok_ptr(workspace) || !dev_status) return SD_ERR_INVALID_ARG;
     if (V < 1 || Hd < 1 || !(inv_temp > 0.f)) return SD_ERR_INVALID_ARG;
     if (Hd % 64 != 0) return SD_ERR_UNSUPPORTED;
-    return launch_accept_chain_sampled(*batch, hidden, W, Hd, V, inv_temp, lse, draft_tok, q_tok, q_rows, u, w, n_acc, path,
+    return launch_accept_chain_sampled(*batch, hidden, W, Hd, V, inv_temp, lse, logits, draft_tok, q_tok, q_rows, u, w, n_acc, path,
                                        out_tok, new_len, workspace, workspace_bytes, dev_status,
                                        static_cast<cudaStream_t>(stream));
 }

@@ -68,7 +68,7 @@ sd_status launch_draft_feature_attention(const void* qp, const void* k, const vo
 size_t stats_workspace_bytes(int M, int V);
 sd_status launch_lmhead_stats(const void* hidden, const void* W, int M, int Hd, int V, float inv_temp,
                               int32_t* argmax, float* maxlogit, float* lse, float* group_stats,
-                              void* ws, size_t ws_bytes, int32_t* dev_status, cudaStream_t st);
+                              void* ws, size_t ws_bytes, int32_t* dev_status, cudaStream_t st, float* logits = nullptr);
 sd_status launch_lmhead_mass(const void* hidden, const void* W, int M, int Hd, int V, float inv_temp,
                              const float* row_lse, float* mass, void* ws, size_t ws_bytes,
                              int32_t* dev_status, cudaStream_t st);
@@ -84,9 +84,10 @@ sd_status launch_accept_sampled(const sd_batch& bt, const void* hidden, const vo
                                 void* ws, size_t ws_bytes, int32_t* dev_status, cudaStream_t st);
 
 sd_status launch_accept_chain_sampled(const sd_batch& bt, const void* hidden, const void* W, int Hd, int V, float inv_temp,
-                                      const float* lse, const int32_t* draft, const float* q_tok, const float* q_rows,
-                                      const float* u, const float* w, int32_t* n_acc, int32_t* path, int32_t* out_tok,
-                                      int32_t* new_len, void* ws, size_t ws_bytes, int32_t* dev_status, cudaStream_t st);
+                                      const float* lse, const float* logits, const int32_t* draft, const float* q_tok,
+                                      const float* q_rows, const float* u, const float* w, int32_t* n_acc, int32_t* path,
+                                      int32_t* out_tok, int32_t* new_len, void* ws, size_t ws_bytes, int32_t* dev_status,
+                                      cudaStream_t st);
 sd_status launch_lmhead_accept_sampled_compact(const sd_batch& bt, const void* hidden, const void* W, int Hd, int V,
                                                float inv_temp, const int32_t* draft, const float* u, const float* w,
                                                const sd_kv_layer* layers, int L, const void* const* kt, const void* const* vt,

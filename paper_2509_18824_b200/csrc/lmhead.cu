@@ -50,6 +50,7 @@ struct LmParams {
     float2* group_stats;    // [ceil(V / 32)][M_total]
     int M_total;
     float* mass_out;        // [rows of the call][V]
+    float* logit_out;       // statistics pass only, optional: the raw logits, [M_total][V] (small M: chain decoding)
     const float* col_lse;   // [rows of the call]
     float inv_temp;
     long long wait_cycles;  // bound of every barrier wait, in SM cycles
@@ -217,6 +218,12 @@ __device__ __forceinline__ void epi_tile(const LmParams& p, EpiState& e, uint32_
                 merge_sumexp(e.run_ref[h], e.run_sum[h], cv, cs, p.c2);
                 if (p.group_stats && v_base < p.V && c * 32 + lane < p.rows)
                     p.group_stats[(size_t)(v_base >> 5) * p.M_total + p.row0 + c * 32 + lane] = make_float2(cv, cs);
+                if (p.logit_out && v_ok) {
+#pragma unroll
+                    for (int j = 0; j < 32; ++j)
+                        if (c * 32 + j < p.rows)
+                            p.logit_out[(size_t)(p.row0 + c * 32 + j) * p.V + v_base + lane] = __uint_as_float(r[j]);
+                }
             } else {
                 column_argmax32(r, v_ok, v_base, lane, cv, ci);
             }
@@ -587,7 +594,7 @@ static sd_status launch_lmhead_impl(const void* hidden, const void* W, int M, in
                                     int32_t* dev_status, cudaStream_t st, int* tiles_only_ctas,
                                     float inv_temp = 0.f, float* lse = nullptr,
                                     float* mass_out = nullptr, const float* col_lse = nullptr,
-                                    float* group_stats = nullptr) {
+                                    float* group_stats = nullptr, float* logit_out = nullptr) {
     if (ws_bytes < (lse ? stats_workspace_bytes(M, V) : lmhead_workspace_bytes(M, V))) return SD_ERR_WORKSPACE;
     if (tiles_only_ctas && M > kMaxCols) return SD_ERR_UNSUPPORTED;
     int dev = 0, sms = 0;
@@ -638,6 +645,7 @@ static sd_status launch_lmhead_impl(const void* hidden, const void* W, int M, in
         p.wait_cycles = knobs.wait_cycles;
         p.withhold = knobs.withhold;
         p.group_stats = reinterpret_cast<float2*>(group_stats); p.M_total = M;
+        p.logit_out = logit_out;
 
         CUtensorMap tmW, tmH;
         if (!encode_tmap_bf16_2d(&tmW, W, (uint64_t)V, (uint64_t)Hd, (uint64_t)Hd * 2, (uint32_t)bk, kBM, bk * 2))
@@ -708,9 +716,9 @@ sd_status launch_lmhead_mass(const void* hidden, const void* W, int M, int Hd, i
 
 sd_status launch_lmhead_stats(const void* hidden, const void* W, int M, int Hd, int V, float inv_temp,
                               int32_t* argmax, float* maxlogit, float* lse, float* group_stats,
-                              void* ws, size_t ws_bytes, int32_t* dev_status, cudaStream_t st) {
+                              void* ws, size_t ws_bytes, int32_t* dev_status, cudaStream_t st, float* logits) {
     return launch_lmhead_impl(hidden, W, M, Hd, V, argmax, maxlogit, ws, ws_bytes, dev_status, st, nullptr, inv_temp, lse,
-                              nullptr, nullptr, group_stats);
+                              nullptr, nullptr, group_stats, logits);
 }
 
 // only the tiles of the statistics pass (M <= 512): the caller's own kernel merges the per-CTA tables

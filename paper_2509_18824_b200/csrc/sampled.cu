@@ -240,16 +240,25 @@ __global__ void gather_stop_rows_kernel(const uint16_t* __restrict__ hidden, int
 // drafts (q_rows null): the drafted tokens of the stop node lose their mass.  Drafts sampled from a
 // distribution (chains): where a draft was rejected (n_excl[b] != 0) the mass becomes
 // max(p - q, 0) with q = the draft's distribution behind the stop node, row stop_row[b] of q_rows.
+// With `logits` (the LM-head pass kept its raw logits: chain decoding, few rows) the stop row's
+// probabilities are formed here, exp(logit / temperature - lse), instead of by a second pass over W.
 __global__ void __launch_bounds__(kResBlock)
 residual_blocksum_kernel(int V, const int32_t* __restrict__ n_excl, const int32_t* __restrict__ excl,
                          const float* __restrict__ q_rows, const int32_t* __restrict__ stop_row,
+                         const float* __restrict__ logits, const float* __restrict__ lse, float inv_temp,
                          float* __restrict__ mass, float* __restrict__ block_sum, int n_blocks) {
     __shared__ float s_v[kResBlock];
     const int b = blockIdx.y;
     const int t = blockIdx.x * kResBlock + threadIdx.x;
     float m = 0.f;
     if (t < V) {
-        m = mass[(size_t)b * V + t];
+        if (logits) {
+            const int row = stop_row[b];
+            m = __expf(__ldg(logits + (size_t)row * V + t) * inv_temp - __ldg(lse + row));
+            if (!q_rows || !n_excl[b]) mass[(size_t)b * V + t] = m;
+        } else {
+            m = mass[(size_t)b * V + t];
+        }
         const int ne = n_excl[b];
         if (q_rows) {
             if (ne) {
@@ -587,9 +596,10 @@ __global__ void chain_walk_q_kernel(sd_batch bt, const int32_t* __restrict__ dra
 }
 
 sd_status launch_accept_chain_sampled(const sd_batch& bt, const void* hidden, const void* W, int Hd, int V, float inv_temp,
-                                      const float* lse, const int32_t* draft, const float* q_tok, const float* q_rows,
-                                      const float* u, const float* w, int32_t* n_acc, int32_t* path, int32_t* out_tok,
-                                      int32_t* new_len, void* ws, size_t ws_bytes, int32_t* dev_status, cudaStream_t st) {
+                                      const float* lse, const float* logits, const int32_t* draft, const float* q_tok,
+                                      const float* q_rows, const float* u, const float* w, int32_t* n_acc, int32_t* path,
+                                      int32_t* out_tok, int32_t* new_len, void* ws, size_t ws_bytes, int32_t* dev_status,
+                                      cudaStream_t st) {
     const int B = bt.B, T = bt.T_max;
     if (Hd > 16384 || (V + kResBlock - 1) / kResBlock > kPickMaxBlocks) return SD_ERR_UNSUPPORTED;
     if (ws_bytes < sampled_workspace_bytes(B, T, V, 16384)) return SD_ERR_WORKSPACE;
@@ -600,14 +610,17 @@ sd_status launch_accept_chain_sampled(const sd_batch& bt, const void* hidden, co
     child_prob_kernel<<<(B * T * 32 + 127) / 128, 128, 0, st>>>(bt, h, Wp, Hd, V, inv_temp, lse, draft, s.p_child, dev_status);
     chain_walk_q_kernel<<<B, 32, 0, st>>>(bt, draft, s.p_child, q_tok, u, n_acc, path, out_tok, new_len, s.stop_row, s.n_excl,
                                          dev_status);
-    gather_stop_rows_kernel<<<B, 128, 0, st>>>(h, Hd, lse, s.stop_row, s.stop_hidden, s.stop_lse);
-    // the stop rows' probabilities over the vocabulary (the LM-head kernel in its store mode), turned into
-    // the residual max(p - q, 0) where a draft was rejected
-    const sd_status ls = launch_lmhead_mass(s.stop_hidden, W, B, Hd, V, inv_temp, s.stop_lse, s.mass, s.lm_ws,
-                                            stats_workspace_bytes(B, V), dev_status, st);
-    if (ls != SD_OK) return ls;
-    residual_blocksum_kernel<<<dim3(n_blocks, B), kResBlock, 0, st>>>(V, s.n_excl, s.excl, q_rows, s.stop_row, s.mass,
-                                                                      s.block_sum, n_blocks);
+    if (!logits) {
+        // the stop rows' probabilities over the vocabulary: the LM-head kernel once more, in its store mode
+        gather_stop_rows_kernel<<<B, 128, 0, st>>>(h, Hd, lse, s.stop_row, s.stop_hidden, s.stop_lse);
+        const sd_status ls = launch_lmhead_mass(s.stop_hidden, W, B, Hd, V, inv_temp, s.stop_lse, s.mass, s.lm_ws,
+                                                stats_workspace_bytes(B, V), dev_status, st);
+        if (ls != SD_OK) return ls;
+    }
+    // ... turned into the residual max(p - q, 0) where a draft was rejected (with the kept logits of the
+    // LM-head pass the probabilities themselves are formed here as well)
+    residual_blocksum_kernel<<<dim3(n_blocks, B), kResBlock, 0, st>>>(V, s.n_excl, s.excl, q_rows, s.stop_row, logits, lse,
+                                                                      inv_temp, s.mass, s.block_sum, n_blocks);
     residual_pick_kernel<<<B, kResBlock, 0, st>>>(bt, V, w, s.mass, s.block_sum, n_blocks, n_acc, out_tok, dev_status);
     return cuda_ok(cudaGetLastError());
 }
@@ -763,8 +776,8 @@ sd_status launch_accept_sampled(const sd_batch& bt, const void* hidden, const vo
     sd_status ls = launch_lmhead_mass(s.stop_hidden, W, B, Hd, V, inv_temp, s.stop_lse, s.mass, s.lm_ws,
                                       stats_workspace_bytes(B, V), dev_status, st);
     if (ls != SD_OK) return ls;
-    residual_blocksum_kernel<<<dim3(n_blocks, B), kResBlock, 0, st>>>(V, s.n_excl, s.excl, nullptr, nullptr, s.mass, s.block_sum,
-                                                                      n_blocks);
+    residual_blocksum_kernel<<<dim3(n_blocks, B), kResBlock, 0, st>>>(V, s.n_excl, s.excl, nullptr, nullptr, nullptr, nullptr, 0.f,
+                                                                      s.mass, s.block_sum, n_blocks);
     residual_pick_kernel<<<B, kResBlock, 0, st>>>(bt, V, w, s.mass, s.block_sum, n_blocks, n_acc, out_tok, dev_status);
     return cuda_ok(cudaGetLastError());
 }

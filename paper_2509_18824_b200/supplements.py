@@ -193,7 +193,12 @@ def chain_sampled(inv_temp=1.0):
     ms_stats = _time(lambda: sd.sd_lmhead_stats(vs.hidden, vs.W, inv_temp, None, None, lse, ws, st), 10)
     ms_acc = _time(lambda: sd.sd_accept_chain_sampled(vs.batch, vs.hidden, vs.W, inv_temp, lse, vs.draft_tok, q_tok, q, u, wv,
                                                       vs.n_acc, vs.path, vs.out_tok, vs.new_len, ws, st), 10)
+    logits = torch.empty((M, V), dtype=torch.float32, device="cuda")
+    ms_stats_lg = _time(lambda: sd.sd_lmhead_stats_logits(vs.hidden, vs.W, inv_temp, None, None, lse, logits, ws, st), 10)
+    ms_acc_lg = _time(lambda: sd.sd_accept_chain_sampled(vs.batch, vs.hidden, vs.W, inv_temp, lse, vs.draft_tok, q_tok, q, u, wv,
+                                                         vs.n_acc, vs.path, vs.out_tok, vs.new_len, ws, st, logits=logits), 10)
     print(json.dumps({"call": "sd_accept_chain_sampled", "workload": "chain11", "rows": M,
+                      "sd_lmhead_stats_logits_us": ms_stats_lg * 1e3, "sd_accept_chain_sampled_from_logits_us": ms_acc_lg * 1e3,
                       "sd_lmhead_stats_us": ms_stats * 1e3, "sd_accept_chain_sampled_us": ms_acc * 1e3,
                       "second_pass_weight_stream_gbs": V * w.Hd * 2 / ms_acc / 1e6, "status": int(st.item())}))
 

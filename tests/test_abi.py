@@ -104,10 +104,12 @@ def test_host_side_refusals_come_before_any_launch():
                                     ok, ok, ok, ok, ok, 16, ok, None) == b.SD_ERR_WORKSPACE
     # chains drafted by sampling: the vocabulary limit of the block-wise draw, the distributions are required
     chain = lambda V, q_rows, ws_bytes: L.sd_accept_chain_sampled(
-        ctypes.byref(bt), ok, ok, 128, V, f(1.0), ok, ok, ok, q_rows, ok, ok, ok, ok, ok, ok, ok, ws_bytes, ok, None)
+        ctypes.byref(bt), ok, ok, 128, V, f(1.0), ok, None, ok, ok, q_rows, ok, ok, ok, ok, ok, ok, ok, ws_bytes, ok, None)
     assert chain(4096 * 256 + 1, ok, big) == b.SD_ERR_UNSUPPORTED
     assert chain(1000, None, big) == b.SD_ERR_INVALID_ARG
     assert chain(1000, ok, 16) == b.SD_ERR_WORKSPACE
+    assert L.sd_lmhead_stats_logits(ok, ok, 8, 128, 100, f(1.0), None, None, ok, None, ok, 1 << 30, ok, None) == b.SD_ERR_INVALID_ARG
+    assert L.sd_lmhead_stats_logits(ok, ok, 8, 100, 100, f(1.0), None, None, ok, ok, ok, 1 << 30, ok, None) == b.SD_ERR_UNSUPPORTED
     # the fused call at a temperature: the same vocabulary limit, the group table is required, workspace
     fused = lambda V, gs, ws_bytes: L.sd_lmhead_accept_sampled_compact(
         ctypes.byref(bt), ok, ok, 128, V, f(1.0), ok, ok, ok, ctypes.byref(cache), 1, ptrs, ptrs, ok, gs,

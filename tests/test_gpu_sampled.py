@@ -439,7 +439,9 @@ def drafted_chain(w, lg, inv_temp, spread, seed):
     return q, tok, q_tok
 
 
-def run_chain_q(w, tok, q, q_tok, inv_temp, u, wv):
+def run_chain_q(w, tok, q, q_tok, inv_temp, u, wv, keep_logits=False):
+    """keep_logits: the LM-head pass keeps its raw logits and the draw uses them; otherwise the stop rows
+    go through the LM head a second time."""
     bt = sd.Batch.of(w)
     st = sd.new_status()
     h, Wd = to_device(w.hidden), to_device(w.W)
@@ -447,13 +449,18 @@ def run_chain_q(w, tok, q, q_tok, inv_temp, u, wv):
     B, T = w.B, w.T_max
     ws = torch.zeros(sd.sd_workspace_bytes(bt, M, V), dtype=torch.uint8, device="cuda")
     lse = torch.zeros(M, dtype=torch.float32, device="cuda")
-    sd.sd_lmhead_stats(h, Wd, inv_temp, None, None, lse, ws, st)
+    logits = None
+    if keep_logits:
+        logits = torch.full((M, V), float("nan"), dtype=torch.float32, device="cuda")
+        sd.sd_lmhead_stats_logits(h, Wd, inv_temp, None, None, lse, logits, ws, st)
+    else:
+        sd.sd_lmhead_stats(h, Wd, inv_temp, None, None, lse, ws, st)
     n_acc = torch.full((B,), -9, dtype=torch.int32, device="cuda")
     path = torch.full((B, T), -9, dtype=torch.int32, device="cuda")
     out_tok = torch.full((B, T), -9, dtype=torch.int32, device="cuda")
     new_len = torch.full((B,), -9, dtype=torch.int32, device="cuda")
     sd.sd_accept_chain_sampled(bt, h, Wd, inv_temp, lse, to_device(tok), to_device(q_tok), to_device(q),
-                               to_device(u), to_device(wv), n_acc, path, out_tok, new_len, ws, st)
+                               to_device(u), to_device(wv), n_acc, path, out_tok, new_len, ws, st, logits=logits)
     torch.cuda.synchronize()
     return (n_acc.cpu().numpy(), path.cpu().numpy(), out_tok.cpu().numpy(), new_len.cpu().numpy(), int(st.item()))
 
@@ -500,7 +507,8 @@ def decisive_chain_inputs(w, tok, q, p64_of_row, g, floor=20 * WALK_CLOSE, floor
     ("chain11", dict(L=1, V=96, Hd=64, prefix=70), 1.5, 1.0),                # vocabulary below one 128-row tile
     ("chain11", dict(L=1, V=8192, Hd=512, prefix=100, B=16), 4.0, 0.4),      # 16 sequences
 ])
-def test_chain_acceptance_with_a_draft_distribution_against_the_reference(cfg, over, inv_temp, spread):
+@pytest.mark.parametrize("keep_logits", [False, True])
+def test_chain_acceptance_with_a_draft_distribution_against_the_reference(cfg, over, inv_temp, spread, keep_logits):
     w = wl.make(cfg, attention=False, hidden_gain=24.0, **over)
     B, T, V = w.B, w.T_max, w.W.shape[0]
     lg = oracle.logits(w.hidden, w.W)
@@ -510,7 +518,7 @@ def test_chain_acceptance_with_a_draft_distribution_against_the_reference(cfg, o
     moved = rejected = 0
     for rep in range(3):
         u, wv, ref_n, ref_out = decisive_chain_inputs(w, tok, q, lambda r: p64[r], g)
-        n_acc, path, out_tok, new_len, status = run_chain_q(w, tok, q, q_tok, inv_temp, u, wv)
+        n_acc, path, out_tok, new_len, status = run_chain_q(w, tok, q, q_tok, inv_temp, u, wv, keep_logits)
         assert status == 0
         np.testing.assert_array_equal(n_acc, ref_n)
         np.testing.assert_array_equal(out_tok, ref_out)
@@ -539,7 +547,7 @@ def test_chain_acceptance_draft_equal_to_the_target_accepts_everything():
         q_tok[b, 1:] = q[b, np.arange(T - 1), tok[b, 1:]]
     u = (g.random((B, T)) * 0.98).astype(np.float32)
     wv = g.random(B).astype(np.float32)
-    n_acc, path, out_tok, new_len, status = run_chain_q(w, tok, q, q_tok, inv_temp, u, wv)
+    n_acc, path, out_tok, new_len, status = run_chain_q(w, tok, q, q_tok, inv_temp, u, wv, keep_logits=True)
     assert status == 0
     np.testing.assert_array_equal(n_acc, w.n_nodes)
     for b in range(B):
@@ -559,7 +567,28 @@ def test_chain_acceptance_refuses_trees_that_branch():
     assert status == sd.SD_ERR_UNSUPPORTED and n_acc[0] == 0
 
 
-def test_chain_acceptance_full_vocabulary():
+def test_kept_logits_are_the_logits():
+    """sd_lmhead_stats_logits: every stored logit against the fp64 product (rows beyond one 32-column
+    chunk, a vocabulary with a ragged last tile), lse as without the logits."""
+    g = np.random.default_rng(31)
+    M, Hd, V = 45, 192, 1000
+    h = wl.f32_to_bf16_bits((g.standard_normal((M, Hd)) * 2).astype(np.float32))
+    W = wl.f32_to_bf16_bits((g.standard_normal((V, Hd)) / np.sqrt(Hd)).astype(np.float32))
+    hd, Wd = to_device(h), to_device(W)
+    lse = torch.zeros(M, dtype=torch.float32, device="cuda")
+    logits = torch.full((M, V), float("nan"), dtype=torch.float32, device="cuda")
+    ws = torch.empty(sd.sd_workspace_bytes(None, M, V), dtype=torch.uint8, device="cuda")
+    st = sd.new_status()
+    sd.sd_lmhead_stats_logits(hd, Wd, 1.3, None, None, lse, logits, ws, st)
+    torch.cuda.synchronize()
+    assert int(st.item()) == 0
+    lg = oracle.logits(h, W)
+    np.testing.assert_allclose(logits.cpu().numpy(), lg, rtol=0, atol=2e-5 * np.abs(lg).max())
+    np.testing.assert_allclose(lse.cpu().numpy(), smp.softmax_rows(lg, 1.3)[1], rtol=0, atol=3e-4)
+
+
+@pytest.mark.parametrize("keep_logits", [False, True])
+def test_chain_acceptance_full_vocabulary(keep_logits):
     """Root + 10 drafts, 8 sequences, vocabulary 152064, draft distributions of the full width."""
     w = wl.make("chain11", attention=False, hidden_gain=40.0)
     B, T, V = w.B, w.T_max, w.V
@@ -569,7 +598,7 @@ def test_chain_acceptance_full_vocabulary():
     q, tok, q_tok = drafted_chain(w, lg, inv_temp, 0.15, 9)
     g = np.random.default_rng(10)
     u, wv, ref_n, ref_out = decisive_chain_inputs(w, tok, q, lambda r: p64[r], g)
-    n_acc, path, out_tok, new_len, status = run_chain_q(w, tok, q, q_tok, inv_temp, u, wv)
+    n_acc, path, out_tok, new_len, status = run_chain_q(w, tok, q, q_tok, inv_temp, u, wv, keep_logits)
     assert status == 0
     np.testing.assert_array_equal(n_acc, ref_n)
     np.testing.assert_array_equal(out_tok, ref_out)
