@@ -30,6 +30,18 @@ residual_sample_q, verify_chain_q below):
     from the normalised positive part of p_i - q_i; if every draft was accepted emit one token from
     p_leaf.  Inverse CDF in vocabulary order with the uniform w, as above.
 
+For a TREE whose children were sampled (every child of node i drawn independently from the same draft
+distribution q_i; tokens may repeat) the rule is applied child after child, each rejection replacing
+the target distribution by its residual (verify_tree_q below):
+
+    at node i: r = p_i; for every child c of i in node order with token x:
+        accept c  iff  u[c] * q_i(x) < r(x)            (probability min(1, r/q)); continue at c
+        otherwise r <- normalised positive part of r - q_i
+    where no child is accepted: emit one token from r by inverse CDF with w.
+    Every r met this way has the form max(p_i - a q_i, 0) / b with scalars a, b (a = 0, b = 1 at the
+    start; a rejection makes a <- a + b and b <- sum_v max(p_i - a q_i, 0)), which the function below
+    does NOT use: it carries the vector r itself.
+
 Parity with the paper's own acceptance statistics is unpinned (they need the
 trained models).  The functions are pinned in tests/test_oracle_sampling.py:
 softmax_rows against torch's log_softmax / logsumexp in fp64, scipy's softmax
@@ -38,7 +50,9 @@ zero-temperature limit (the greedy rule), by the single-child case (the
 textbook accept test) and by numpy's cumsum/searchsorted for the inverse CDF;
 the general-q chain rule by Monte-Carlo frequencies against p, by the point-mass
 case (where it must reproduce verify_sequence), by q = p (everything accepted)
-and by a hand-computed case.
+and by a hand-computed case; the sampled-tree rule by Monte-Carlo frequencies
+with children drawn independently from q, by chains (where it must reproduce
+verify_chain_q) and by a hand-computed case.
 """
 from __future__ import annotations
 
@@ -176,3 +190,39 @@ def verify_chain_q(n_nodes, draft_tok, logits, inv_temp, q_rows, u, w):
     rejected = n_acc < n
     t, _, _ = residual_sample_q(p[stop], q_rows[stop] if rejected else None, w)
     return n_acc, [int(draft_tok[j]) for j in range(1, n_acc)] + [t]
+
+
+def verify_tree_q(parents, n_nodes, draft_tok, logits, inv_temp, q_rows, u, w):
+    """Whole rule for one tree whose children were sampled from q_rows[i] (the draft's distribution
+    behind node i), from the target's logits [T, V], fp64.  Returns (path, out_tok, walk_margin,
+    draw_margin, mass): the accepted root path, the emitted tokens, the smallest relative distance
+    |u q - r| / r over the accept tests made (infinity if none or r = 0 cases only), the distance of
+    the last draw's target from the nearer end of its CDF interval, and the mass it was normalised by
+    (before normalisation: the sum of the positive part carried so far, relative to p_i)."""
+    p, _ = softmax_rows(logits, inv_temp)
+    q_rows = np.asarray(q_rows, dtype=np.float64)
+    u = np.asarray(u, dtype=np.float64)
+    n = int(n_nodes)
+    cur, path = 0, [0]
+    walk_margin = np.inf
+    while True:
+        r = p[cur].copy()
+        q = q_rows[cur]
+        nxt = -1
+        for c in children_of(parents, n, cur):
+            x = int(draft_tok[c])
+            if r[x] > 0.0:
+                walk_margin = min(walk_margin, abs(u[c] * q[x] - r[x]) / r[x])
+            if u[c] * q[x] < r[x]:
+                nxt = c
+                break
+            r = np.maximum(r - q, 0.0)
+            tot = r.sum()
+            if tot > 0.0:
+                r = r / tot
+        if nxt < 0:
+            total = float(r.sum())
+            t, draw_margin = residual_sample(r, [], total, w)
+            return path, [int(draft_tok[j]) for j in path[1:]] + [t], walk_margin, draw_margin, total
+        cur = nxt
+        path.append(cur)

@@ -276,3 +276,106 @@ def test_chain_q_pins_catch_planted_mistakes():
                 mutant(use_q_after_full_accept=True)):                # residual applied although nothing was rejected
         with pytest.raises(AssertionError):
             chain_q_pins(bad)
+
+
+# ---------------------------------------------------------------------------------------------------
+# trees whose children were sampled independently from the draft distribution of their parent
+# ---------------------------------------------------------------------------------------------------
+def tree_q_pins(verify_tree_q):
+    g = np.random.default_rng(6)
+    V = 6
+    # (1) Monte Carlo on a fixed shape (root with three children, the first two with two children each);
+    # every child's token is drawn from its parent's q.  First emitted token ~ p_root; given that child c
+    # of the root was accepted, the second ~ p_c.
+    parents = np.array([-1, 0, 0, 0, 1, 1, 2, 2])
+    T = len(parents)
+    for spread in (1.5, 0.3):
+        logits = g.standard_normal((T, V)) * 1.5
+        p, _ = smp.softmax_rows(logits, 1.2)
+        q, _ = smp.softmax_rows(logits + g.standard_normal((T, V)) * spread, 1.0)
+        cdf = np.cumsum(q, axis=1)
+        first = np.zeros(V)
+        second = {1: np.zeros(V), 2: np.zeros(V), 3: np.zeros(V)}
+        for _ in range(60000):
+            tok = np.zeros(T, dtype=np.int64)
+            for j in range(1, T):
+                tok[j] = min(int(np.searchsorted(cdf[parents[j]], g.random(), side="right")), V - 1)
+            path, out, *_ = verify_tree_q(parents, T, tok, logits, 1.2, q, g.random(T), g.random())
+            first[out[0]] += 1
+            if len(path) >= 2:
+                second[path[1]][out[1]] += 1
+        checks = [(first, p[0])] + [(second[c], p[c]) for c in (1, 2, 3)]
+        for counts, target in checks:
+            n = counts.sum()
+            assert n > 500
+            sigma = np.sqrt(n * target * (1 - target))
+            assert (np.abs(counts - n * target) <= 5 * sigma + 1).all(), (spread, counts / n, target)
+    # (2) a chain is a tree: the chain rule, already pinned, must come out
+    for seed in range(30):
+        g2 = np.random.default_rng(200 + seed)
+        T2 = 5
+        logits = g2.standard_normal((T2, V)) * 2.0
+        q, _ = smp.softmax_rows(g2.standard_normal((T2, V)), 1.0)
+        tok = g2.integers(0, V, size=T2)
+        u, w = g2.random(T2), g2.random()
+        n_acc, out_ref = smp.verify_chain_q(T2, tok, logits, 1.3, q, u, w)
+        path, out, *_ = verify_tree_q(np.arange(-1, T2 - 1), T2, tok, logits, 1.3, q, u, w)
+        assert path == list(range(n_acc)) and out == out_ref, (seed, out, out_ref)
+    # (3) by hand: p = (0.5, 0.3, 0.2), q = (0.2, 0.7, 0.1), children of the root carry tokens 1 and 0.
+    #   child 1 (token 1): kept iff u < 3/7.  Rejected: r = (0.3, 0, 0.1) / 0.4 = (0.75, 0, 0.25).
+    #   child 2 (token 0): kept iff u * 0.2 < 0.75, i.e. always.  With tokens 1 and 1 instead: r(1) = 0, never.
+    #   Both rejected (tokens 1, 1): r <- max(r - q, 0) = (0.55, 0, 0.15) / 0.7: w = 0.78 -> token 0, 0.79 -> token 2.
+    logits = np.log(np.array([[0.5, 0.3, 0.2], [0.2, 0.2, 0.6], [0.1, 0.8, 0.1]]))
+    q = np.array([[0.2, 0.7, 0.1], [1 / 3, 1 / 3, 1 / 3], [1 / 3, 1 / 3, 1 / 3]])
+    par = np.array([-1, 0, 0])
+    assert verify_tree_q(par, 3, np.array([0, 1, 0]), logits, 1.0, q, [0, 0.43, 0.999], 0.05)[:2] == ([0, 2], [0, 0])
+    assert verify_tree_q(par, 3, np.array([0, 1, 0]), logits, 1.0, q, [0, 0.42, 0.999], 0.5)[:2] == ([0, 1], [1, 2])
+    assert verify_tree_q(par, 3, np.array([0, 1, 1]), logits, 1.0, q, [0, 0.43, 0.0001], 0.78)[:2] == ([0], [0])
+    assert verify_tree_q(par, 3, np.array([0, 1, 1]), logits, 1.0, q, [0, 0.43, 0.0001], 0.79)[:2] == ([0], [2])
+
+
+def test_tree_rule_with_sampled_children():
+    tree_q_pins(smp.verify_tree_q)
+
+
+def test_tree_q_pins_catch_planted_mistakes():
+    import pytest
+
+    def mutant(renormalise=True, subtract=lambda r, q: np.maximum(r - q, 0.0), reset=True,
+               accept=lambda u, qx, rx: u * qx < rx):
+        def f(parents, n_nodes, draft_tok, logits, inv_temp, q_rows, u, w):
+            p, _ = smp.softmax_rows(logits, inv_temp)
+            q_rows = np.asarray(q_rows, dtype=np.float64)
+            n = int(n_nodes)
+            cur, path = 0, [0]
+            r = p[0].copy()
+            while True:
+                if reset:
+                    r = p[cur].copy()
+                q = q_rows[cur]
+                nxt = -1
+                for c in smp.children_of(parents, n, cur):
+                    x = int(draft_tok[c])
+                    if accept(u[c], q[x], r[x]):
+                        nxt = c
+                        break
+                    r = subtract(r, q)
+                    if renormalise and r.sum() > 0:
+                        r = r / r.sum()
+                if nxt < 0:
+                    t, _ = smp.residual_sample(r, [], float(r.sum()), w)
+                    return path, [int(draft_tok[j]) for j in path[1:]] + [t], 0, 0, 0
+                cur = nxt
+                path.append(cur)
+                if not reset:
+                    r = p[cur].copy() * 0 + r       # (keeps the parent's residual: the planted mistake)
+        return f
+
+    tree_q_pins(mutant())                                                   # the harness itself is sound
+    for bad in (mutant(renormalise=False),                                  # residual not renormalised between siblings
+                mutant(subtract=lambda r, q: np.maximum(q - r, 0.0)),       # sign
+                mutant(subtract=lambda r, q: r),                            # no residual update
+                mutant(reset=False),                                        # the child starts from its parent's residual
+                mutant(accept=lambda u, qx, rx: u * rx < qx)):              # ratio upside down
+        with pytest.raises(AssertionError):
+            tree_q_pins(bad)
