@@ -368,10 +368,9 @@ sd_status sd_accept_tree_sampled(const sd_batch *batch, const void *hidden, cons
  * logits-sized data that reach memory).  A tree that branches stores SD_ERR_UNSUPPORTED, a bad tree
  * SD_ERR_INVALID_TREE, a draft token outside [0, V) SD_ERR_BOUNDS (through
  * *dev_status; n_acc[b] = 0 for the first two).  V > 1048576 returns SD_ERR_UNSUPPORTED
- * before anything is launched.  Drafted trees that branch AND were sampled from a
- * distribution are not covered (their rule renormalises over the vocabulary after
- * every rejected sibling); deterministic (top-k) trees go through
- * sd_accept_tree_sampled.
+ * before anything is launched.  Trees that branch and were sampled from a
+ * distribution go through sd_accept_tree_sampled_q, deterministic (top-k) trees
+ * through sd_accept_tree_sampled.
  */
 sd_status sd_accept_chain_sampled(const sd_batch *batch, const void *hidden, const void *W,
                                   int32_t Hd, int32_t V, float inv_temp, const float *lse,
@@ -381,6 +380,34 @@ sd_status sd_accept_chain_sampled(const sd_batch *batch, const void *hidden, con
                                   int32_t *n_acc, int32_t *path, int32_t *out_tok, int32_t *new_len,
                                   void *workspace, size_t workspace_bytes,
                                   int32_t *dev_status, void *stream);
+
+/*
+ * Acceptance at a sampling temperature for TREES whose children were sampled: every
+ * child of node i drawn independently from the draft's distribution q_i (Sec. 1,
+ * lossless validation; the cited rule applied child after child).  At node i, with
+ * r = p_i = softmax(logits_i * inv_temp):
+ *   for every child c of i in node order, x = draft_tok[c]:
+ *       accept c  iff  u[b][c] * q_i(x) < r(x);  continue at c with r = p_c
+ *       otherwise r <- normalised positive part of r - q_i
+ *   where no child is accepted one token is drawn from r: the first token, in
+ *   vocabulary order, at which the cumulative mass reaches w[b] times the total.
+ * Sibling tokens may repeat.  A chain is the special case of one child per node.
+ *   lse, logits : dev f32 [B * T_max] and [B * T_max][V] from sd_lmhead_stats_logits
+ *                 with the same inv_temp (row b * T_max + i = node i of sequence b)
+ *   q_rows      : dev f32 [B][T_max][V], row [b][i] = q_i (rows of nodes the walk visits are read)
+ *   u, w        : dev f32 [B][T_max] and [B], uniform numbers in [0, 1)
+ * Outputs as sd_accept_tree.  One cluster of eight CTAs per sequence keeps p_i and q_i
+ * of the current node in shared memory (V <= 163840, else SD_ERR_UNSUPPORTED before
+ * anything is launched); every rejection costs one reduction over the vocabulary.
+ * A bad tree stores SD_ERR_INVALID_TREE, a draft token outside [0, V) SD_ERR_BOUNDS
+ * (n_acc[b] = 0 in both cases).  Arithmetic: fp32, sums in a fixed order.
+ */
+sd_status sd_accept_tree_sampled_q(const sd_batch *batch, int32_t V, float inv_temp,
+                                   const float *lse, const float *logits,
+                                   const int32_t *draft_tok, const float *q_rows,
+                                   const float *u, const float *w,
+                                   int32_t *n_acc, int32_t *path, int32_t *out_tok, int32_t *new_len,
+                                   int32_t *dev_status, void *stream);
 
 /*
  * LM head, acceptance at a sampling temperature and compaction in one call (Sec. 1:

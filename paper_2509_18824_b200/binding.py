@@ -33,7 +33,7 @@ KERNELS_PER_SAMPLED_TAIL = 2       # sd_lmhead_accept_sampled_compact: LM-head t
 
 EXPORTS = ["sd_version", "sd_status_string", "sd_workspace_bytes", "sd_tree_prepare",
            "sd_verify_attention", "sd_verify_attention_layers", "sd_lmhead_argmax", "sd_lmhead_argmax_static", "sd_accept_tree",
-           "sd_compact_kv", "sd_lmhead_accept_compact", "sd_lmhead_stats", "sd_accept_tree_sampled", "sd_lmhead_accept_sampled_compact", "sd_accept_chain_sampled", "sd_lmhead_stats_logits",
+           "sd_compact_kv", "sd_lmhead_accept_compact", "sd_lmhead_stats", "sd_accept_tree_sampled", "sd_lmhead_accept_sampled_compact", "sd_accept_chain_sampled", "sd_lmhead_stats_logits", "sd_accept_tree_sampled_q",
            "sd_draft_feature_attention"]
 
 
@@ -94,6 +94,8 @@ def _load(path: str = LIB_PATH) -> C.CDLL:
                                            C.c_void_p, C.c_void_p, C.c_void_p, C.c_void_p,
                                            C.c_void_p, C.c_size_t, C.c_void_p, C.c_void_p]
     lib.sd_accept_chain_sampled.restype = C.c_int
+    lib.sd_accept_tree_sampled_q.restype = C.c_int
+    lib.sd_accept_tree_sampled_q.argtypes = [C.c_void_p, C.c_int32, C.c_float] + [C.c_void_p] * 12
     lib.sd_lmhead_stats_logits.restype = C.c_int
     lib.sd_lmhead_stats_logits.argtypes = [C.c_void_p, C.c_void_p, C.c_int32, C.c_int32, C.c_int32, C.c_float,
                                            C.c_void_p, C.c_void_p, C.c_void_p, C.c_void_p, C.c_void_p, C.c_size_t,
@@ -328,6 +330,18 @@ def sd_lmhead_stats_logits(hidden, W, inv_temp: float, argmax, maxlogit, lse, lo
     _check(lib.sd_lmhead_stats_logits(_ptr(hidden), _ptr(W), int(M), int(Hd), int(V), C.c_float(inv_temp), _ptr(argmax),
                                       _ptr(maxlogit), _ptr(lse), _ptr(logits), _ptr(workspace),
                                       workspace.numel() * workspace.element_size(), _ptr(status), _stream(stream)))
+
+
+def sd_accept_tree_sampled_q(batch: Batch, inv_temp: float, lse, logits, draft_tok, q_rows, u, w,
+                             n_acc, path, out_tok, new_len, status, stream=None) -> None:
+    """Acceptance at a sampling temperature for trees whose children were sampled from q_rows [B,T,V];
+    lse [M] and logits [M,V] from sd_lmhead_stats_logits (device f32)."""
+    M, V = logits.shape
+    assert M == batch.B * batch.T_max and tuple(q_rows.shape) == (batch.B, batch.T_max, V)
+    assert logits.dtype == torch.float32 and q_rows.dtype == torch.float32 and logits.is_contiguous() and q_rows.is_contiguous()
+    _check(lib.sd_accept_tree_sampled_q(batch.ref(), int(V), C.c_float(inv_temp), _ptr(lse), _ptr(logits), _ptr(draft_tok),
+                                        _ptr(q_rows), _ptr(u), _ptr(w), _ptr(n_acc), _ptr(path), _ptr(out_tok),
+                                        _ptr(new_len), _ptr(status), _stream(stream)))
 
 
 def sd_accept_chain_sampled(batch: Batch, hidden, W, inv_temp: float, lse, draft_tok, q_tok, q_rows, u, w,

@@ -224,6 +224,19 @@ sd_status sd_accept_chain_sampled(const sd_batch* batch, const void* hidden, con
                                        static_cast<cudaStream_t>(stream));
 }
 
+sd_status sd_accept_tree_sampled_q(const sd_batch* batch, int32_t V, float inv_temp, const float* lse, const float* logits,
+                                   const int32_t* draft_tok, const float* q_rows, const float* u, const float* w,
+                                   int32_t* n_acc, int32_t* path, int32_t* out_tok, int32_t* new_len,
+                                   int32_t* dev_status, void* stream) {
+    sd_status s = check_geometry(batch, true);
+    if (s != SD_OK) return s;
+    if (!lse || !logits || !draft_tok || !q_rows || !u || !w) return SD_ERR_INVALID_ARG;
+    if (!n_acc || !path || !out_tok || !new_len || !dev_status) return SD_ERR_INVALID_ARG;
+    if (V < 1 || !(inv_temp > 0.f)) return SD_ERR_INVALID_ARG;
+    return launch_accept_tree_sampled_q(*batch, V, inv_temp, lse, logits, draft_tok, q_rows, u, w, n_acc, path, out_tok,
+                                        new_len, dev_status, static_cast<cudaStream_t>(stream));
+}
+
 sd_status sd_lmhead_accept_sampled_compact(const sd_batch* batch, const void* hidden, const void* W, int32_t Hd, int32_t V,
                                            float inv_temp, const int32_t* draft_tok, const float* u, const float* w,
                                            const sd_kv_layer* layers, int32_t L,

@@ -88,6 +88,10 @@ sd_status launch_accept_chain_sampled(const sd_batch& bt, const void* hidden, co
                                       const float* q_rows, const float* u, const float* w, int32_t* n_acc, int32_t* path,
                                       int32_t* out_tok, int32_t* new_len, void* ws, size_t ws_bytes, int32_t* dev_status,
                                       cudaStream_t st);
+sd_status launch_accept_tree_sampled_q(const sd_batch& bt, int V, float inv_temp, const float* lse, const float* logits,
+                                       const int32_t* draft, const float* q_rows, const float* u, const float* w,
+                                       int32_t* n_acc, int32_t* path, int32_t* out_tok, int32_t* new_len,
+                                       int32_t* dev_status, cudaStream_t st);
 sd_status launch_lmhead_accept_sampled_compact(const sd_batch& bt, const void* hidden, const void* W, int Hd, int V,
                                                float inv_temp, const int32_t* draft, const float* u, const float* w,
                                                const sd_kv_layer* layers, int L, const void* const* kt, const void* const* vt,

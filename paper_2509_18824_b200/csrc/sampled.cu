@@ -626,6 +626,205 @@ sd_status launch_accept_chain_sampled(const sd_batch& bt, const void* hidden, co
 }
 
 // ---------------------------------------------------------------------------
+// Trees whose children were SAMPLED, every child of node i independently from the draft's distribution
+// q_i: the rule is applied child after child, and every rejection replaces the target distribution r
+// by the normalised positive part of r - q_i.  Every r met this way is max(p_i - a q_i, 0) / b with two
+// scalars (a = 0, b = 1 at a node's start; a rejection makes a <- a + b, b <- sum_v max(p_i - a q_i, 0)),
+// so a rejection costs one reduction over the vocabulary.  One cluster of eight CTAs per sequence:
+// every CTA keeps its eighth of p_i (from the logits the LM-head pass kept) and of q_i in shared
+// memory while the walk is at node i, sums its part in a fixed order, and the eight partial sums
+// are exchanged through remote stores and added in rank order, so that all eight CTAs take the same
+// decisions.  The last token is drawn from max(p - a q, 0) by inverse CDF in vocabulary order: the
+// CTA whose slice holds the crossing finds it.
+// ---------------------------------------------------------------------------
+constexpr int kTreeQCluster = 8;
+constexpr int kTreeQThreads = 256;
+constexpr int kTreeQMaxSlice = 20480;          // vocabulary entries per CTA: V <= 163840
+
+__global__ void __launch_bounds__(kTreeQThreads)
+tree_walk_q_kernel(sd_batch bt, int V, float inv_temp, const float* __restrict__ lse, const float* __restrict__ logits,
+                   const int32_t* __restrict__ draft, const float* __restrict__ q_rows, const float* __restrict__ u,
+                   const float* __restrict__ w, int32_t* n_acc, int32_t* path, int32_t* out_tok, int32_t* new_len,
+                   int32_t* status) {
+    extern __shared__ float s_pq[];                 // p slice, then q slice
+    __shared__ float s_part[kTreeQThreads];         // sums of the threads' runs
+    __shared__ float s_run[128];                    // one run, element by element (the last draw)
+    __shared__ float s_cta2[2][kTreeQCluster];      // the eight CTAs' sums, written by their owners; two sets in
+                                                    // turn: a CTA may start the next exchange while another still
+                                                    // reads this one (it cannot get two ahead: the barrier)
+    __shared__ int32_t s_path[kMaxT];
+    __shared__ float s_px, s_qx;
+    __shared__ int s_bad;
+    const int b = blockIdx.x / kTreeQCluster;
+    const int rank = (int)sm100::cluster_ctarank();
+    const int T = bt.T_max, tid = threadIdx.x, lane = tid & 31;
+    const int slice = (V + kTreeQCluster - 1) / kTreeQCluster;
+    const int v0 = min(V, rank * slice), v1 = min(V, v0 + slice), len = v1 - v0;
+    const int run = (slice + kTreeQThreads - 1) / kTreeQThreads;     // <= 80 entries per thread
+    float* s_p = s_pq;
+    float* s_q = s_pq + slice;
+    const int n = bt.n_nodes[b];
+    const int32_t* par = bt.parents + (size_t)b * T;
+    const int32_t* dt = draft + (size_t)b * T;
+    // the tree, checked by every CTA in the same way
+    if (tid == 0) s_bad = 0;
+    __syncthreads();
+    if (n < 1 || n > T) { if (tid == 0) s_bad = SD_ERR_INVALID_TREE; }
+    else
+        for (int i = tid; i < n; i += kTreeQThreads) {
+            const int p = par[i];
+            if (i == 0 ? (p != -1) : (p < 0 || p >= i)) s_bad = SD_ERR_INVALID_TREE;
+            else if (i > 0 && (dt[i] < 0 || dt[i] >= V)) atomicCAS(&s_bad, 0, (int)SD_ERR_BOUNDS);
+        }
+    __syncthreads();
+    if (s_bad != 0) {                               // (the same in every CTA: nobody reaches a cluster barrier)
+        if (rank == 0 && tid == 0) { set_status(status, s_bad); n_acc[b] = 0; }
+        return;
+    }
+    // sum over this CTA's slice of max(p - a q, 0), every thread a run of consecutive entries; the eight
+    // sums are exchanged; returns their total (rank order), the same bits in every CTA
+    int n_red = 0;
+    const float* s_cta = s_cta2[0];                 // the set of the latest exchange
+    auto reduce = [&](float a) -> float {
+        float* mine = s_cta2[n_red & 1];
+        ++n_red;
+        s_cta = mine;
+        const int i0 = min(len, tid * run), i1 = min(len, i0 + run);
+        float sum = 0.f;
+        for (int i = i0; i < i1; ++i) sum += fmaxf(s_p[i] - a * s_q[i], 0.f);
+        s_part[tid] = sum;
+        __syncthreads();
+        if (tid < 32) {
+            float total = 0.f;
+            warp_find_crossing(s_part, kTreeQThreads, INFINITY, &total, nullptr, lane);
+            if (lane < kTreeQCluster)
+                sm100::st_dsmem_f32(sm100::map_dsmem(sm100::smem_u32(&mine[rank]), (uint32_t)lane), total);
+        }
+        sm100::cluster_arrive_release();
+        sm100::cluster_wait_acquire();
+        float all = 0.f;
+#pragma unroll
+        for (int r = 0; r < kTreeQCluster; ++r) all += s_cta[r];
+        return all;
+    };
+    int cur = 0, na = 1;
+    float a = 0.f, bsum = 1.f;
+    if (tid == 0) s_path[0] = 0;
+    while (true) {
+        // this CTA's slice of p and q behind node cur
+        const int row = b * T + cur;
+        const float row_lse = lse[row];
+        const float* lrow = logits + (size_t)row * V + v0;
+        const float* qrow = q_rows + (size_t)row * V + v0;
+        for (int i = tid; i < len; i += kTreeQThreads) {
+            s_p[i] = __expf(__ldg(lrow + i) * inv_temp - row_lse);
+            s_q[i] = __ldg(qrow + i);
+        }
+        __syncthreads();
+        a = 0.f; bsum = 1.f;
+        int nxt = -1;
+        bool summed = false;                         // the partial sums on hand belong to this node and this a
+        for (int c = cur + 1; c < n; ++c) {          // children of cur in node order (the same walk in every CTA)
+            if (par[c] != cur) continue;
+            const int x = dt[c];
+            if (tid == 0) {
+                s_px = __expf(__ldg(logits + (size_t)row * V + x) * inv_temp - row_lse);
+                s_qx = __ldg(q_rows + (size_t)row * V + x);
+            }
+            __syncthreads();
+            const float num = fmaxf(s_px - a * s_qx, 0.f);
+            const bool keep = u[(size_t)b * T + c] * bsum * s_qx < num;
+            __syncthreads();                        // (s_px, s_qx are rewritten for the next child)
+            if (keep) { nxt = c; break; }
+            a += bsum;
+            bsum = reduce(a);
+            summed = true;
+        }
+        if (nxt < 0) {
+            if (!summed) bsum = reduce(a);           // the sums the draw walks over (nothing rejected here: all of p)
+            break;
+        }
+        if (tid == 0) s_path[na] = nxt;
+        cur = nxt;
+        ++na;
+        __syncthreads();
+    }
+    // outputs of the walk
+    if (rank == 0) {
+        for (int k = tid; k < T; k += kTreeQThreads) {
+            path[(size_t)b * T + k] = k < na ? s_path[k] : -1;
+            if (k != na - 1) out_tok[(size_t)b * T + k] = k + 1 < na ? dt[s_path[k + 1]] : -1;
+        }
+        if (tid == 0) { n_acc[b] = na; new_len[b] = bt.len[b] + na; }
+    }
+    // the last token: which CTA's slice holds the crossing of w * (total mass), then which run, then which entry
+    const float target = w[b] * bsum;
+    float before = 0.f;
+    int owner = -1, last_with_mass = -1;
+    for (int r = 0; r < kTreeQCluster; ++r) {
+        if (s_cta[r] > 0.f) last_with_mass = r;
+        if (owner < 0 && s_cta[r] > 0.f && before + s_cta[r] >= target) owner = r;
+        if (owner < 0) before += s_cta[r];
+    }
+    if (owner < 0) {                                 // rounding left the sum short: the last slice with mass
+        owner = last_with_mass;
+        if (owner >= 0) before -= s_cta[owner];
+    }
+    if (owner < 0) {                                 // no mass at all (inputs not finite, or r vanished by rounding)
+        if (rank == 0 && tid == 0) { set_status(status, SD_ERR_BOUNDS); out_tok[(size_t)b * T + na - 1] = 0; }
+        return;
+    }
+    if (rank != owner) return;
+    __shared__ float s_acc;
+    __shared__ int s_t, s_pick;
+    if (tid < 32) {
+        float acc = before;
+        int lastp = -1;
+        int t = warp_find_crossing(s_part, kTreeQThreads, target, &acc, &lastp, lane);
+        if (t < 0) { t = max(lastp, 0); acc -= s_part[t]; }
+        if (lane == 0) { s_acc = acc; s_t = t; }
+    }
+    __syncthreads();
+    const int i0 = min(len, s_t * run), i1 = min(len, i0 + run);
+    if (tid < i1 - i0) s_run[tid] = fmaxf(s_p[i0 + tid] - a * s_q[i0 + tid], 0.f);
+    __syncthreads();
+    if (tid < 32) {
+        float acc = s_acc;
+        int lastp = -1;
+        int k = warp_find_crossing(s_run, i1 - i0, target, &acc, &lastp, lane);
+        if (k < 0) k = max(lastp, 0);
+        if (lane == 0) out_tok[(size_t)b * T + na - 1] = v0 + i0 + k;
+    }
+}
+
+sd_status launch_accept_tree_sampled_q(const sd_batch& bt, int V, float inv_temp, const float* lse, const float* logits,
+                                       const int32_t* draft, const float* q_rows, const float* u, const float* w,
+                                       int32_t* n_acc, int32_t* path, int32_t* out_tok, int32_t* new_len,
+                                       int32_t* dev_status, cudaStream_t st) {
+    const int slice = (V + kTreeQCluster - 1) / kTreeQCluster;
+    if (slice > kTreeQMaxSlice) return SD_ERR_UNSUPPORTED;
+    const size_t dyn = (size_t)slice * 2 * sizeof(float);
+    if (cudaFuncSetAttribute(tree_walk_q_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)dyn) != cudaSuccess)
+        return SD_ERR_CUDA;
+    cudaLaunchConfig_t cfg = {};
+    cfg.gridDim = dim3(bt.B * kTreeQCluster);
+    cfg.blockDim = dim3(kTreeQThreads);
+    cfg.dynamicSmemBytes = dyn;
+    cfg.stream = st;
+    cudaLaunchAttribute attr[1];
+    attr[0].id = cudaLaunchAttributeClusterDimension;
+    attr[0].val.clusterDim.x = kTreeQCluster;
+    attr[0].val.clusterDim.y = 1;
+    attr[0].val.clusterDim.z = 1;
+    cfg.attrs = attr;
+    cfg.numAttrs = 1;
+    if (cudaLaunchKernelEx(&cfg, tree_walk_q_kernel, bt, V, inv_temp, lse, logits, draft, q_rows, u, w, n_acc, path, out_tok,
+                           new_len, dev_status) != cudaSuccess)
+        return SD_ERR_CUDA;
+    return SD_OK;
+}
+
+// ---------------------------------------------------------------------------
 // Tail of a verify step at a sampling temperature, behind the LM-head tiles of a statistics pass: one
 // cluster of eight CTAs per sequence.
 //   1. every CTA merges the per-CTA soft-max partials of eight of the sequence's LM-head rows -> lse

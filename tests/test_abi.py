@@ -110,6 +110,11 @@ def test_host_side_refusals_come_before_any_launch():
     assert chain(1000, ok, 16) == b.SD_ERR_WORKSPACE
     assert L.sd_lmhead_stats_logits(ok, ok, 8, 128, 100, f(1.0), None, None, ok, None, ok, 1 << 30, ok, None) == b.SD_ERR_INVALID_ARG
     assert L.sd_lmhead_stats_logits(ok, ok, 8, 100, 100, f(1.0), None, None, ok, ok, ok, 1 << 30, ok, None) == b.SD_ERR_UNSUPPORTED
+    # sampled trees: the vocabulary must fit eight shared-memory slices
+    assert L.sd_accept_tree_sampled_q(ctypes.byref(bt), 8 * 20480 + 1, f(1.0), ok, ok, ok, ok, ok, ok, ok, ok, ok, ok, ok,
+                                      None) == b.SD_ERR_UNSUPPORTED
+    assert L.sd_accept_tree_sampled_q(ctypes.byref(bt), 1000, f(1.0), ok, None, ok, ok, ok, ok, ok, ok, ok, ok, ok,
+                                      None) == b.SD_ERR_INVALID_ARG
     # the fused call at a temperature: the same vocabulary limit, the group table is required, workspace
     fused = lambda V, gs, ws_bytes: L.sd_lmhead_accept_sampled_compact(
         ctypes.byref(bt), ok, ok, 128, V, f(1.0), ok, ok, ok, ctypes.byref(cache), 1, ptrs, ptrs, ok, gs,

@@ -646,3 +646,173 @@ def test_chain_acceptance_gpu_output_frequencies_follow_the_target_distribution(
     n = B * reps
     sigma = np.sqrt(n * p[0] * (1 - p[0]))
     assert (np.abs(counts - n * p[0]) <= 5 * sigma + 1).all(), (counts / n, p[0])
+
+
+# ---------------------------------------------------------------------------------------------------
+# trees whose children were sampled from their parent's draft distribution: sd_accept_tree_sampled_q
+# ---------------------------------------------------------------------------------------------------
+def drafted_tree(w, lg, inv_temp, spread, seed):
+    """q[b][i] = softmax of the target's logits behind node i plus noise (float32, read by both sides);
+    every child of node i carries a token drawn from q[b][i], independently of its siblings."""
+    g = np.random.default_rng(seed)
+    B, T, V = w.B, w.T_max, lg.shape[1]
+    q64, _ = smp.softmax_rows(lg + g.standard_normal(lg.shape) * spread, inv_temp * 0.8)
+    q = np.ascontiguousarray(q64.astype(np.float32).reshape(B, T, V))
+    tok = np.zeros((B, T), dtype=np.int32)
+    for b in range(B):
+        cdfs = {}
+        for j in range(1, int(w.n_nodes[b])):
+            i = int(w.parents[b][j])
+            if i not in cdfs:
+                cdfs[i] = np.cumsum(q[b, i].astype(np.float64))
+            tok[b, j] = min(int(np.searchsorted(cdfs[i], g.random() * cdfs[i][-1], side="right")), V - 1)
+    return q, tok
+
+
+def run_tree_q(w, tok, q, inv_temp, u, wv):
+    bt = sd.Batch.of(w)
+    st = sd.new_status()
+    h, Wd = to_device(w.hidden), to_device(w.W)
+    M, V = w.hidden.shape[0], w.W.shape[0]
+    B, T = w.B, w.T_max
+    ws = torch.zeros(sd.sd_workspace_bytes(bt, M, V), dtype=torch.uint8, device="cuda")
+    lse = torch.zeros(M, dtype=torch.float32, device="cuda")
+    logits = torch.full((M, V), float("nan"), dtype=torch.float32, device="cuda")
+    sd.sd_lmhead_stats_logits(h, Wd, inv_temp, None, None, lse, logits, ws, st)
+    n_acc = torch.full((B,), -9, dtype=torch.int32, device="cuda")
+    path = torch.full((B, T), -9, dtype=torch.int32, device="cuda")
+    out_tok = torch.full((B, T), -9, dtype=torch.int32, device="cuda")
+    new_len = torch.full((B,), -9, dtype=torch.int32, device="cuda")
+    sd.sd_accept_tree_sampled_q(bt, inv_temp, lse, logits, to_device(tok), to_device(q), to_device(u), to_device(wv),
+                                n_acc, path, out_tok, new_len, st)
+    torch.cuda.synchronize()
+    return (n_acc.cpu().numpy(), path.cpu().numpy(), out_tok.cpu().numpy(), new_len.cpu().numpy(), int(st.item()))
+
+
+def decisive_tree_inputs(w, tok, q, lg, inv_temp, g, floor=20 * WALK_CLOSE, floor_w=2e-3):
+    """Uniforms under which the fp64 rule makes no close call (accept tests further than `floor`, relative,
+    from equality; the last draw further than floor_w of the mass from a CDF step), and its results."""
+    B, T = w.B, w.T_max
+    u = np.zeros((B, T), np.float32)
+    wv = np.zeros(B, np.float32)
+    ref_n, ref_path, ref_out = np.zeros(B, np.int32), np.full((B, T), -1, np.int32), np.full((B, T), -1, np.int32)
+    rejections = 0
+    for b in range(B):
+        n = int(w.n_nodes[b])
+        rows = slice(b * T, b * T + T)
+        for _ in range(400):
+            u[b] = g.random(T).astype(np.float32)
+            wv[b] = np.float32(g.random())
+            path, out, walk_margin, draw_margin, total = smp.verify_tree_q(
+                w.parents[b], n, tok[b], lg[rows], inv_temp, q[b], u[b].astype(np.float64), float(wv[b]))
+            if walk_margin > floor and draw_margin > floor_w * total:
+                break
+        else:
+            raise AssertionError("no decisive uniforms found")
+        ref_n[b] = len(path)
+        ref_path[b, :len(path)] = path
+        ref_out[b, :len(out)] = out
+        rejections += sum(1 for c in range(1, n) if int(w.parents[b][c]) in path and c not in path)
+    return u, wv, ref_n, ref_path, ref_out, rejections
+
+
+@pytest.mark.parametrize("cfg,over,inv_temp,spread", [
+    ("c1", dict(), 2.0, 0.8),
+    ("c1", dict(V=96, Hd=64), 1.5, 1.0),                                     # slices of 12 vocabulary entries
+    ("c5", dict(L=1, V=8192, Hd=512, prefix=100), 4.0, 0.5),                 # 60-node trees: up to ten siblings
+    ("c5", dict(L=1, V=8192, Hd=512, prefix=100), 4.0, 0.05),                # a drafter very close to the target
+    ("c4", dict(L=1, V=4099, Hd=256, prefix_range=(40, 300)), 3.0, 0.6),     # 16 ragged trees, odd vocabulary
+    ("chain11", dict(L=1, V=3000, Hd=128, prefix=70), 2.5, 0.6),
+])
+def test_tree_acceptance_with_sampled_children_against_the_reference(cfg, over, inv_temp, spread):
+    w = wl.make(cfg, attention=False, hidden_gain=24.0, **over)
+    B, T, V = w.B, w.T_max, w.W.shape[0]
+    lg = oracle.logits(w.hidden, w.W)
+    q, tok = drafted_tree(w, lg, inv_temp, spread, 13)
+    g = np.random.default_rng(14)
+    moved = rejected = 0
+    for rep in range(3 if B > 1 else 12):
+        u, wv, ref_n, ref_path, ref_out, rej = decisive_tree_inputs(w, tok, q, lg, inv_temp, g)
+        n_acc, path, out_tok, new_len, status = run_tree_q(w, tok, q, inv_temp, u, wv)
+        assert status == 0
+        np.testing.assert_array_equal(n_acc, ref_n)
+        np.testing.assert_array_equal(path, ref_path)
+        np.testing.assert_array_equal(out_tok, ref_out)
+        np.testing.assert_array_equal(new_len, w.len + ref_n)
+        moved += int((ref_n > 1).sum())
+        rejected += rej
+    assert moved > 0 and rejected > 0
+
+
+def test_tree_acceptance_with_sampled_children_full_vocabulary():
+    """One 60-node tree over the vocabulary of 152064 (slices of 19008 entries per CTA)."""
+    w = wl.make("c2", attention=False, hidden_gain=40.0)
+    lg = oracle.logits(w.hidden, w.W)
+    inv_temp = 6.0
+    q, tok = drafted_tree(w, lg, inv_temp, 0.15, 15)
+    g = np.random.default_rng(16)
+    total_rej = 0
+    for rep in range(4):
+        u, wv, ref_n, ref_path, ref_out, rej = decisive_tree_inputs(w, tok, q, lg, inv_temp, g)
+        n_acc, path, out_tok, new_len, status = run_tree_q(w, tok, q, inv_temp, u, wv)
+        assert status == 0
+        np.testing.assert_array_equal(n_acc, ref_n)
+        np.testing.assert_array_equal(path, ref_path)
+        np.testing.assert_array_equal(out_tok, ref_out)
+        total_rej += rej
+    assert total_rej > 0
+
+
+def test_tree_acceptance_with_sampled_children_reports_bad_inputs():
+    w = wl.make("c1", attention=False, hidden_gain=16.0)
+    V = w.W.shape[0]
+    q = np.full((1, 8, V), 1.0 / V, np.float32)
+    half, wv = np.full((1, 8), 0.5, np.float32), np.full(1, 0.5, np.float32)
+    tok = np.arange(8, dtype=np.int32)[None].copy(); tok[0, 3] = V + 5
+    n_acc, *_, status = run_tree_q(w, tok, q, 1.0, half, wv)
+    assert status == sd.SD_ERR_BOUNDS and n_acc[0] == 0
+    w.parents = w.parents.copy(); w.parents[0, 3] = 6
+    n_acc, *_, status = run_tree_q(w, np.arange(8, dtype=np.int32)[None], q, 1.0, half, wv)
+    assert status == sd.SD_ERR_INVALID_TREE and n_acc[0] == 0
+
+
+def test_tree_acceptance_with_sampled_children_gpu_frequencies():
+    """Losslessness on the GPU path: 16 identical trees (root with three children, the first with two),
+    children redrawn from q 300 times; the first emitted token must be distributed as p at the root."""
+    B, T, Hd, V, inv_temp, reps = 16, 6, 64, 16, 1.2, 300
+    g = np.random.default_rng(23)
+    bf = lambda a: wl.f32_to_bf16_bits(a.astype(np.float32))
+    hid_one = bf(g.standard_normal((T, Hd)))
+    W = bf(g.standard_normal((V, Hd)) * 0.25)
+
+    class Geo:
+        pass
+    w = Geo()
+    w.B, w.T_max, w.Hq, w.Hkv, w.D = B, T, 4, 1, 128
+    w.block_table = np.arange(B, dtype=np.int32).reshape(B, 1)
+    w.len = np.full(B, 5, np.int32)
+    w.n_nodes = np.full(B, T, np.int32)
+    par = np.array([-1, 0, 0, 0, 1, 1], np.int32)
+    w.parents = np.tile(par, (B, 1))
+    w.hidden = np.tile(hid_one, (B, 1))
+    w.W = W
+    lg = oracle.logits(hid_one, W)
+    p, _ = smp.softmax_rows(lg, inv_temp)
+    q_one, _ = smp.softmax_rows(lg + g.standard_normal(lg.shape) * 0.8, 1.0)
+    q = np.ascontiguousarray(np.tile(q_one.astype(np.float32)[None], (B, 1, 1)))
+    cdf = np.cumsum(q_one.astype(np.float32).astype(np.float64), axis=1)
+    counts = np.zeros(V)
+    for rep in range(reps):
+        tok = np.zeros((B, T), np.int32)
+        for b in range(B):
+            for j in range(1, T):
+                i = par[j]
+                tok[b, j] = min(int(np.searchsorted(cdf[i], g.random() * cdf[i, -1], side="right")), V - 1)
+        u = g.random((B, T)).astype(np.float32)
+        wv = g.random(B).astype(np.float32)
+        n_acc, path, out_tok, new_len, status = run_tree_q(w, tok, q, inv_temp, u, wv)
+        assert status == 0
+        np.add.at(counts, out_tok[:, 0], 1)
+    n = B * reps
+    sigma = np.sqrt(n * p[0] * (1 - p[0]))
+    assert (np.abs(counts - n * p[0]) <= 5 * sigma + 1).all(), (counts / n, p[0])
