@@ -203,6 +203,34 @@ def chain_sampled(inv_temp=1.0):
                       "second_pass_weight_stream_gbs": V * w.Hd * 2 / ms_acc / 1e6, "status": int(st.item())}))
 
 
+def tree_sampled_q(inv_temp=1.0):
+    """sd_lmhead_stats_logits + sd_accept_tree_sampled_q on the bench's shapes (8 trees of 60 nodes,
+    vocabulary 152064).  Random q and tokens: nearly every child is rejected, the expensive case."""
+    from .step import VerifyStep
+    w = wl.make("c5", attention=False, L=1)
+    wl.fill_attention(w, [0])
+    vs = VerifyStep(w)
+    B, T, M, V = w.B, w.T_max, w.B * w.T_max, w.V
+    g = torch.Generator(device="cuda"); g.manual_seed(0)
+    u = torch.rand((B, T), device="cuda", generator=g)
+    wv = torch.rand((B,), device="cuda", generator=g)
+    q = torch.rand((B, T, V), device="cuda", generator=g)
+    q /= q.sum(dim=-1, keepdim=True)
+    lse = torch.zeros(M, dtype=torch.float32, device="cuda")
+    logits = torch.empty((M, V), dtype=torch.float32, device="cuda")
+    ws = torch.empty(sd.sd_workspace_bytes(vs.batch, M, V), dtype=torch.uint8, device="cuda")
+    st = vs.status
+    ms_stats = _time(lambda: sd.sd_lmhead_stats_logits(vs.hidden, vs.W, inv_temp, None, None, lse, logits, ws, st), 10)
+    res = {}
+    for name, uu in (("all_rejected", torch.full((B, T), 0.999, device="cuda")), ("random", u),
+                     ("all_accepted", torch.zeros((B, T), device="cuda"))):
+        res[name] = _time(lambda: sd.sd_accept_tree_sampled_q(vs.batch, inv_temp, lse, logits, vs.draft_tok, q, uu, wv,
+                                                              vs.n_acc, vs.path, vs.out_tok, vs.new_len, st), 10) * 1e3
+    print(json.dumps({"call": "sd_accept_tree_sampled_q", "workload": "c5", "rows": M,
+                      "sd_lmhead_stats_logits_us": ms_stats * 1e3, "sd_accept_tree_sampled_q_us": res,
+                      "logits_bytes": M * V * 4, "status": int(st.item())}))
+
+
 def draft(S=4096, L=28, Q=4, H=28):
     """Draft-side feature aggregation on a 7B-shaped prefill: S tokens x 28 layer features of width 3584."""
     hbm, _, src = _peaks()
@@ -266,6 +294,7 @@ if __name__ == "__main__":
     if "sampled" in what:
         sampled()
         chain_sampled()
+        tree_sampled_q()
     if "draft" in what:
         draft()
     if "compact" in what:
