@@ -213,17 +213,21 @@ __device__ __forceinline__ void epi_tile(const LmParams& p, EpiState& e, uint32_
                 continue;
             }
             if (stats) {
+                if (p.logit_out && v_ok) {             // the raw logits, one running address (few rows: chain decoding)
+                    float* dst = p.logit_out + (size_t)(p.row0 + c * 32) * p.V + v_base + lane;
+                    const int lim = p.rows - c * 32;
+#pragma unroll
+                    for (int j = 0; j < 32; ++j) {
+                        if (j < lim) *dst = __uint_as_float(r[j]);
+                        dst += p.V;
+                    }
+                }
                 float cs;
                 column_argmax_stats32(r, v_ok, v_base, lane, p.c2, cv, ci, cs);
                 merge_sumexp(e.run_ref[h], e.run_sum[h], cv, cs, p.c2);
                 if (p.group_stats && v_base < p.V && c * 32 + lane < p.rows)
                     p.group_stats[(size_t)(v_base >> 5) * p.M_total + p.row0 + c * 32 + lane] = make_float2(cv, cs);
-                if (p.logit_out && v_ok) {
-#pragma unroll
-                    for (int j = 0; j < 32; ++j)
-                        if (c * 32 + j < p.rows)
-                            p.logit_out[(size_t)(p.row0 + c * 32 + j) * p.V + v_base + lane] = __uint_as_float(r[j]);
-                }
+
             } else {
                 column_argmax32(r, v_ok, v_base, lane, cv, ci);
             }
